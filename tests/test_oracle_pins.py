@@ -1,0 +1,587 @@
+"""Pins for the CPU oracle: it is checked against what the paper prints and what mathematics
+fixes (printed extremes and worked example, library conversions on the ranges where they
+coincide, exact-rational restatements on tiny inputs, closed forms, known-answer vectors),
+never against itself or against the CUDA path."""
+import math
+import os
+from fractions import Fraction as Fr
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from conftest import GOLDEN
+
+E2M1_MAGS = [Fr(0), Fr(1, 2), Fr(1), Fr(3, 2), Fr(2), Fr(3), Fr(4), Fr(6)]
+
+
+def f32(x):
+    return np.float32(x)
+
+
+def bf16_bits(a):
+    return torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).view(torch.uint16).numpy()
+
+
+# ------------------------------------------------------------------------------------------
+# Codebooks (Section 1, Section 4.1, Table 2)
+# ------------------------------------------------------------------------------------------
+def test_e2m1_codebook(printed):
+    vals = [oracle.e2m1_value(c) for c in range(16)]
+    assert max(vals) == printed["e2m1_max"] and min(vals) == -printed["e2m1_max"]
+    assert [Fr(v) for v in vals[:8]] == E2M1_MAGS
+    assert [Fr(v) for v in vals[8:]] == [-m for m in E2M1_MAGS]
+    assert math.copysign(1.0, vals[8]) == -1.0       # code 0x8 is negative zero
+    # one fraction bit: every magnitude has at most two significant bits
+    for v in vals[1:8]:
+        m, _ = math.frexp(v)
+        assert (m * 4).is_integer()
+
+
+def test_e2m1_matches_library_dtype():
+    ml = pytest.importorskip("ml_dtypes")
+    table = np.arange(16, dtype=np.uint8).view(ml.float4_e2m1fn).astype(np.float32)
+    assert [oracle.e2m1_value(c) for c in range(16)] == [float(v) for v in table]
+
+
+def test_ue5m3_codebook_extremes(printed):
+    vals = [oracle.ue5m3_value(c) for c in range(256)]
+    finite = [v for v in vals if math.isfinite(v)]
+    assert len(finite) == 248
+    assert max(finite) == printed["ue5m3_max"]
+    assert max(finite) == printed["ue5m3_max_significand"] * 2.0 ** printed["ue5m3_max_exponent"]
+    positive = [v for v in finite if v > 0]
+    assert min(positive) == 2.0 ** printed["ue5m3_min_subnormal_log2"]
+    # smallest normal: first value from which the spacing is relative (8 steps per binade)
+    assert vals[0x08] == 2.0 ** printed["ue5m3_min_normal_log2"]
+    assert vals[0x07] == 7 * 2.0 ** -17 and vals[0x09] == 9 * 2.0 ** -17
+    assert vals[0] == 0.0
+    assert all(b > a for a, b in zip(finite, finite[1:]))       # code order is value order
+    assert math.isinf(vals[0xF8]) and all(math.isnan(v) for v in vals[0xF9:])
+    # comparisons with E4M3 printed in Section 4.1 / Table 2
+    assert round(max(finite) / printed["e4m3_max"]) == printed["max_ratio_ue5m3_over_e4m3"]
+    assert 2.0 ** printed["e4m3_min_subnormal_log2"] / min(positive) == printed["min_ratio_e4m3_over_ue5m3"]
+    # landmarks used elsewhere
+    assert vals[0x78] == 1.0 and vals[0xBE] == 448.0 and vals[0xD0] == 2048.0 and vals[0xF7] == 61440.0
+    # three fraction bits: at most 4 significant bits
+    for v in positive:
+        m, _ = math.frexp(v)
+        assert (m * 16).is_integer()
+
+
+def test_ue5m3_same_spacing_as_e4m3_where_they_overlap():
+    """Section 4.1: at a fixed exponent E4M3 and UE5M3 have the same spacing.  The positive normal
+    E4M3 values (library dtype) are therefore all UE5M3 values."""
+    ml = pytest.importorskip("ml_dtypes")
+    e4 = np.arange(0x08, 0x7F, dtype=np.uint8).view(ml.float8_e4m3fn).astype(np.float64)
+    ue = {oracle.ue5m3_value(c) for c in range(0xF8)}
+    assert all(v in ue for v in e4)
+
+
+# ------------------------------------------------------------------------------------------
+# Encoders
+# ------------------------------------------------------------------------------------------
+def test_ue5m3_encode_roundtrip_ties_saturation():
+    vals = [oracle.ue5m3_value(c) for c in range(0xF8)]
+    for c, v in enumerate(vals):
+        assert oracle.ue5m3_encode(v) == c
+    for c in range(0xF7):
+        mid = 0.5 * (vals[c] + vals[c + 1])           # exact in float32 (5 significant bits)
+        assert float(f32(mid)) == mid
+        even = c if c % 2 == 0 else c + 1
+        assert oracle.ue5m3_encode(mid) == even
+        assert oracle.ue5m3_encode(np.nextafter(f32(mid), f32(0))) == c
+        assert oracle.ue5m3_encode(np.nextafter(f32(mid), f32(1e9))) == c + 1
+    for big in (61440.0, 61441.0, 63488.0, 65536.0, 1e30, np.inf):
+        assert oracle.ue5m3_encode(big) == 0xF7
+    assert oracle.ue5m3_encode(0.0) == 0
+    assert oracle.ue5m3_encode(2.0 ** -18) == 0                     # tie between 0 and 2^-17 -> even
+    assert oracle.ue5m3_encode(np.nextafter(f32(2.0 ** -18), f32(1))) == 1
+
+
+def test_ue5m3_encode_equals_library_e4m3_rounding_on_shared_range():
+    """On [2^-6, 448] the two formats have the same grid, so RNE must agree with the library's
+    float32 -> E4M3 conversion."""
+    ml = pytest.importorskip("ml_dtypes")
+    rng = np.random.default_rng(1)
+    u = np.exp(rng.uniform(math.log(2.0 ** -6), math.log(448.0), 20000)).astype(np.float32)
+    grid = np.arange(0x08, 0x7F, dtype=np.uint8).view(ml.float8_e4m3fn).astype(np.float32)
+    mids = (grid[:-1] + grid[1:]) / 2
+    u = np.concatenate([u, grid, mids, np.nextafter(mids, np.float32(0)), np.nextafter(mids, np.float32(1e9))])
+    u = u[(u >= 2.0 ** -6) & (u <= 448.0)]
+    lib = u.astype(ml.float8_e4m3fn).astype(np.float64)
+    mine = np.array([oracle.ue5m3_value(oracle.ue5m3_encode(v)) for v in u])
+    assert np.array_equal(lib, mine)
+
+
+def test_ue5m3_encode_is_nearest_everywhere():
+    vals = np.array([oracle.ue5m3_value(c) for c in range(0xF8)])
+    rng = np.random.default_rng(2)
+    u = np.exp(rng.uniform(math.log(2.0 ** -20), math.log(70000.0), 20000)).astype(np.float32)
+    for v in u:
+        c = oracle.ue5m3_encode(v)
+        err = np.abs(vals - np.float64(v))
+        assert err[c] == err.min()
+
+
+def test_e2m1_rne_matches_library_and_argmin():
+    ml = pytest.importorskip("ml_dtypes")
+    rng = np.random.default_rng(3)
+    z = np.concatenate([
+        rng.uniform(-7, 7, 40000), rng.normal(0, 0.3, 20000),
+        [0.0, -0.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 6.5, 100.0, np.inf, -np.inf],
+    ]).astype(np.float32)
+    thr = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0], dtype=np.float32)
+    for t in thr:                                       # every float32 next to each decision point
+        z = np.concatenate([z, [np.nextafter(t, np.float32(0)), np.nextafter(t, np.float32(9))],
+                            [-np.nextafter(t, np.float32(0)), -t]]).astype(np.float32)
+    lib = z.astype(ml.float4_e2m1fn).view(np.uint8) & 0xF
+    mine = np.array([oracle.e2m1_encode_rne(v) for v in z], dtype=np.uint8)
+    assert np.array_equal(lib, mine)
+    # definition: nearest magnitude, sign kept, saturating
+    mags = np.array([float(m) for m in E2M1_MAGS])
+    for v, c in zip(z, mine):
+        a = min(abs(float(v)), 6.0)
+        assert abs(mags[c & 7] - a) == np.abs(mags - a).min()
+        assert (c >> 3) == (1 if np.signbit(v) else 0)
+    assert oracle.e2m1_encode_rne(np.nan) == 0x7
+    # ties go to the code with a zero fraction bit
+    assert [oracle.e2m1_encode_rne(t) for t in (0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0)] == [0, 2, 2, 4, 4, 6, 6]
+
+
+# ------------------------------------------------------------------------------------------
+# Tensor reference, scale target (Section 5.1, 5.2, Table 3, Proposition 1)
+# ------------------------------------------------------------------------------------------
+def test_tensor_constants_exact_cases():
+    for k in range(-8, 9):
+        for T in (448.0, 2048.0):
+            g = T * 2.0 ** k
+            ge, S, G, d = oracle.tensor_constants(g, T)
+            assert (ge, S, G) == (g, 2.0 ** -k, 6.0 * 2.0 ** -k)
+            assert float(d) == float(f32(2.0 ** k) / f32(6.0))
+    # correctly rounded single divisions
+    ge, S, G, d = oracle.tensor_constants(100.0, 448.0)
+    assert S == f32(448.0) / f32(100.0) and G == f32(2688.0) / f32(100.0) and d == f32(100.0) / f32(2688.0)
+    assert abs(Fr(float(G)) - Fr(2688, 100)) <= Fr(2688, 100) * Fr(1, 2 ** 24)
+    # unusable references fall back to 1.0; tiny ones are floored at 2^-60
+    for bad in (0.0, -3.0, np.inf, np.nan):
+        assert oracle.tensor_constants(bad, 448.0)[0] == 1.0
+    assert oracle.tensor_constants(1e-30, 448.0)[0] == 2.0 ** -60
+
+
+def _one_block(values, g, T, rounding=oracle.ROUND_RNE, seed=0):
+    x = np.zeros((16, 16), np.float32)
+    x[0, :] = values
+    return oracle.quantize(x, oracle.LAYOUT_1D_ROW, rounding, g, T, seed)
+
+
+def test_worked_example_table3(printed):
+    g = printed["t3_g"]
+    U = printed["ue5m3_max"]
+    for T, tag in ((448.0, "T448"), (2048.0, "T2048")):
+        # a block as large as g lands on the code whose value is T
+        q = _one_block([g] + [0.0] * 15, g, T)
+        assert oracle.ue5m3_value(q["scales"][0, 0]) == printed[f"t3_{tag}_code_for_block_eq_g"]
+        # window edges implied by the smallest nonzero code and the largest code
+        lo = 2.0 ** printed["ue5m3_min_subnormal_log2"] * g / T
+        hi = U * g / T
+        assert float(f"{lo:.1e}") == printed[f"t3_{tag}_smallest_nonzero"]
+        assert int(hi) == printed[f"t3_{tag}_largest"]
+        assert int(hi / g) == printed[f"t3_{tag}_growth"]
+        # and the oracle's encoder places those block maxima on exactly those codes
+        q = _one_block([f32(lo)] + [0.0] * 15, g, T)
+        assert q["scales"][0, 0] == 0x01 and q["stats"]["zero_repaired"] == 15
+        q = _one_block([f32(hi * 0.999)] + [0.0] * 15, g, T)
+        assert q["scales"][0, 0] == 0xF7 and q["stats"]["scale_saturated"] == 0
+        q = _one_block([f32(hi * 1.001)] + [0.0] * 15, g, T)
+        assert q["scales"][0, 0] == 0xF7 and q["stats"]["scale_saturated"] == 1
+    assert round(printed["override_target"] / printed["default_target"], 1) == printed["target_ratio"]
+
+
+def test_block_equal_to_reference_gets_code_T_on_random_tensors():
+    """Eq. "scale-target": a_B = g gives u_B = T exactly -- holds for any g because
+    RN32(g * RN32(T/g)) stays within half a UE5M3 step of T."""
+    rng = np.random.default_rng(5)
+    for T, code in ((448.0, 0xBE), (2048.0, 0xD0)):
+        for _ in range(50):
+            x = rng.normal(0, rng.uniform(1e-3, 1e3), (16, 64)).astype(np.float32)
+            g = np.abs(x).max()
+            q = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, T)
+            r, c = np.unravel_index(np.abs(x).argmax(), x.shape)
+            assert q["scales"][r, c // 16] == code
+            assert (q["payload"][r, c // 2] >> (4 * (c % 2))) & 7 == 7      # the maximum itself maps to 6
+
+
+def test_proposition1_saturation_boundary():
+    """A block avoids scale saturation exactly when a_B <= U g / T (g = T 2^k keeps u exact)."""
+    U = 61440.0
+    for T in (448.0, 2048.0):
+        for k in (-3, 0, 5):
+            g = T * 2.0 ** k
+            edge = f32(U * g / T)                         # = 61440 * 2^k, exact
+            cands = [edge, np.nextafter(edge, f32(0)), np.nextafter(edge, f32(np.inf)), edge * f32(0.5), edge * f32(2)]
+            x = np.zeros((16, 16 * len(cands)), np.float32)
+            for i, a in enumerate(cands):
+                x[3, 16 * i + 5] = -a
+            q = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, T)
+            want = sum(1 for a in cands if Fr(float(a)) > Fr(U) * Fr(g) / Fr(T))
+            assert q["stats"]["scale_saturated"] == want == 2
+            assert all(q["scales"][3, i] == 0xF7 for i in (0, 2, 4))
+            assert q["scales"][3, 1] == 0xF7 or oracle.ue5m3_value(q["scales"][3, 1]) < U
+
+
+def test_zero_scale_rule():
+    """A block-scale code that rounds to zero is replaced with the value 1 (byte 0x78)."""
+    g, T = 448.0, 448.0                                   # S = 1, G = 6
+    x = np.zeros((16, 48), np.float32)
+    x[0, 16:32] = 2.0 ** -19                              # u_B = 2^-19 < 2^-18 -> code 0
+    x[0, 17] = -(2.0 ** -19)
+    x[0, 32] = 2.0 ** -17                                 # smallest nonzero code, not repaired
+    q = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, T)
+    assert list(q["scales"][0]) == [0x78, 0x78, 0x01]
+    assert q["stats"]["zero_repaired"] == 2 + 15 * 3
+    nib = lambda k: (q["payload"][0, k // 2] >> (4 * (k % 2))) & 0xF
+    assert [nib(k) for k in range(16)] == [0] * 16
+    assert nib(16) == 0 and nib(17) == 8                  # signed zeros
+    assert nib(32) == 7                                   # 2^-17 / 2^-17 * 6 = 6
+
+
+def test_amax_and_hold_schedule(printed):
+    rng = np.random.default_rng(7)
+    x = rng.normal(0, 3, (48, 80)).astype(np.float32)
+    x[5, 7] = np.nan
+    assert oracle.amax(x) == np.nanmax(np.abs(x))
+    view = x[:, :64]                                      # leading dimension larger than cols
+    assert oracle.amax(view) == np.nanmax(np.abs(view))
+    xb = bf16_bits(rng.normal(0, 3, (32, 32)))
+    ref = torch.from_numpy(xb).view(torch.bfloat16).float().abs().max().item()
+    assert oracle.amax(xb) == ref
+    D = int(printed["refresh_interval"])
+    assert oracle.hold_schedule(200, D) == [0, 50, 100, 150]
+    assert oracle.hold_schedule(5, 1) == [0, 1, 2, 3, 4]
+
+
+# ------------------------------------------------------------------------------------------
+# Whole quantizer against the textbook statement in exact rationals (Eq. "microscaling")
+# ------------------------------------------------------------------------------------------
+def _blocks(rows, cols, layout):
+    """Block membership written independently of the oracle: lists of (r, c) plus where the codes go."""
+    out = []
+    if layout == oracle.LAYOUT_1D_ROW:
+        for r in range(rows):
+            for kb in range(cols // 16):
+                out.append(([(r, 16 * kb + j) for j in range(16)], (r, kb)))
+    elif layout == oracle.LAYOUT_1D_COL:
+        for c in range(cols):
+            for rb in range(rows // 16):
+                out.append(([(16 * rb + j, c) for j in range(16)], (c, rb)))
+    else:
+        for rb in range(rows // 16):
+            for cb in range(cols // 16):
+                out.append(([(16 * rb + i, 16 * cb + j) for i in range(16) for j in range(16)], (rb, cb)))
+    return out
+
+
+def _nearest_ue5m3(u):
+    vals = [Fr(oracle.ue5m3_value(c)) for c in range(0xF8)]
+    best = min(range(0xF8), key=lambda c: (abs(vals[c] - u), c % 2))
+    return best
+
+
+@pytest.mark.parametrize("layout", [oracle.LAYOUT_1D_ROW, oracle.LAYOUT_1D_COL, oracle.LAYOUT_2D])
+@pytest.mark.parametrize("as_bf16", [False, True])
+def test_quantizer_equals_rational_microscaling(layout, as_bf16):
+    """With g = T 2^k the tensor multiplier is exact, so q_i must be the E2M1 value nearest to the
+    exact rational x_i T F / (g s_hat), s_hat the UE5M3 value nearest to a_B T / g."""
+    rng = np.random.default_rng(11 + layout)
+    rows, cols = 32, 48
+    xf = (rng.normal(0, 1, (rows, cols)) * 10.0 ** rng.uniform(-2, 2, (rows, 1))).astype(np.float32)
+    xf[4, 9] = 0.0
+    xf[:16, :16] *= 1e-9                                   # a tile that needs the zero-scale rule
+    xf = torch.from_numpy(xf).to(torch.bfloat16).float().numpy()
+    x = bf16_bits(xf) if as_bf16 else xf
+    T = 448.0
+    g = T * 2.0 ** -1                                      # 224: stale reference, several blocks clip
+    q = oracle.quantize(x, layout, oracle.ROUND_RNE, g, T, want_t=True)
+    assert q["decode"] == f32(g) / f32(6 * T)
+    n_checked = n_skipped = clip = repaired = 0
+    for members, (orow, ocol) in _blocks(rows, cols, layout):
+        aB = max(abs(Fr(float(xf[r, c]))) for r, c in members)
+        code = _nearest_ue5m3(aB * Fr(T) / Fr(g))
+        if code == 0:
+            code = 0x78
+            repaired += 1
+        assert q["scales"][orow, ocol] == code
+        s_hat = Fr(oracle.ue5m3_value(code))
+        for r, c in members:
+            z = Fr(float(xf[r, c])) * 6 * Fr(T) / (Fr(g) * s_hat)
+            a = min(abs(z), Fr(6))
+            if layout == oracle.LAYOUT_1D_COL:
+                byte = q["payload"][c, r // 2]; sh = 4 * (r % 2)
+            else:
+                byte = q["payload"][r, c // 2]; sh = 4 * (c % 2)
+            got = (byte >> sh) & 0xF
+            if layout == oracle.LAYOUT_2D:
+                assert (q["payload_t"][c, r // 2] >> (4 * (r % 2))) & 0xF == got
+            d = sorted(abs(m - a) for m in E2M1_MAGS)
+            if d[1] - d[0] < Fr(1, 2 ** 18) or abs(abs(z) - 6) < Fr(1, 2 ** 18):
+                n_skipped += 1                              # within float32 rounding of a decision point
+                continue
+            n_checked += 1
+            assert abs(E2M1_MAGS[got & 7] - a) == d[0]
+            assert (got >> 3) == (1 if xf[r, c] < 0 or (xf[r, c] == 0 and np.signbit(xf[r, c])) else 0)
+            clip += abs(z) > 6
+    if layout == oracle.LAYOUT_2D:
+        assert np.array_equal(q["scales_t"], q["scales"].T)
+    assert n_checked > 0.98 * rows * cols and n_skipped < 0.02 * rows * cols
+    assert abs(q["stats"]["payload_clipped"] - clip) <= n_skipped
+    assert q["stats"]["zero_repaired"] == repaired and repaired >= 1
+
+
+def test_roundtrip_error_bound_and_rms():
+    """Unsaturated block: |x - d s_hat q| <= d s_hat h(|q|) with h the half step of the E2M1 grid
+    (clipping above 6 adds at most 6/16 because s_hat rounds down by at most 1/16)."""
+    rng = np.random.default_rng(13)
+    x = rng.normal(0, 1, (64, 256)).astype(np.float32)
+    g = np.abs(x).max()
+    q = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, 448.0)
+    assert q["stats"]["scale_saturated"] == 0 and q["stats"]["zero_repaired"] == 0
+    xh = oracle.dequantize(q["payload"], q["scales"], False, q["decode"])
+    s = np.repeat(np.array([[oracle.ue5m3_value(c) for c in row] for row in q["scales"]]), 16, axis=1) * float(q["decode"])
+    qa = np.abs(xh) / s
+    half = np.where(qa < 2, 0.25, np.where(qa < 4, 0.5, 1.0))
+    assert np.all(np.abs(xh - x) <= s * half * (1 + 1e-5))
+    rel_rms = np.sqrt(np.mean((xh - x) ** 2) / np.mean(x ** 2))
+    assert 0.05 < rel_rms < 0.15                           # 4-bit payload: about one tenth
+    # x_hat = g s_hat q / (T F): the block maximum is recovered to within the UE5M3 step
+    bm = np.abs(x).reshape(64, 16, 16).max(axis=2)
+    bmh = np.abs(xh).reshape(64, 16, 16).max(axis=2)
+    assert np.all(np.abs(bmh - bm) <= bm / 16 * (1 + 1e-5))
+
+
+def test_dot_product_error_is_in_the_band_the_paper_reports(printed):
+    """Appendix C: input quantization contributes 1.24-1.83 % relative RMS error to correlated
+    (rho = 0.25) K = 4096 dot products.  Distribution families as listed there."""
+    rng = np.random.default_rng(17)
+    n, K, rho = 256, 4096, 0.25
+
+    def draw(kind):
+        if kind == "gauss":
+            return rng.normal(0, 1, (n, K))
+        if kind == "laplace":
+            return rng.laplace(0, 1 / math.sqrt(2), (n, K))
+        t = rng.standard_t(3, (n, K))
+        return t / math.sqrt(3.0)
+
+    seen = []
+    for kind in ("gauss", "laplace", "student"):
+        a = draw(kind)
+        b = rho * a + math.sqrt(1 - rho ** 2) * draw(kind)
+        a32, b32 = a.astype(np.float32), b.astype(np.float32)
+        qa = oracle.quantize(a32, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, np.abs(a32).max(), 448.0)
+        qb = oracle.quantize(b32, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, np.abs(b32).max(), 448.0)
+        idx = np.arange(n)
+        y, _ = oracle.gemm_cells(qa["payload"], qa["scales"], False, qa["decode"],
+                                 qb["payload"], qb["scales"], False, qb["decode"], idx, idx)
+        exact = np.einsum("ik,ik->i", a32.astype(np.float64), b32.astype(np.float64))
+        seen.append(100 * np.sqrt(np.mean((y - exact) ** 2) / np.mean(exact ** 2)))
+    lo, hi = printed["dot_rel_rms_low_percent"], printed["dot_rel_rms_high_percent"]
+    assert lo * 0.8 <= min(seen) and max(seen) <= hi * 1.25, seen
+
+
+# ------------------------------------------------------------------------------------------
+# Stochastic rounding (Eq. "sr") and its random bits
+# ------------------------------------------------------------------------------------------
+def test_philox_known_answers():
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        w = [int(v, 16) for v in r]
+        assert list(oracle.philox4x32_10(w[0:4], w[4:6])) == w[6:10]
+
+
+def test_sr_bits_indexing():
+    seed = 0x0123456789ABCDEF
+    for i in (0, 5, 8, 1023, 2 ** 35 + 3):
+        w = oracle.philox4x32_10([(i >> 3) & 0xFFFFFFFF, (i >> 3) >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32])
+        j = i & 7
+        assert oracle.sr_bits(seed, i) == (int(w[j >> 1]) >> (16 * (j & 1))) & 0xFFFF
+    draws = np.array([oracle.sr_bits(3, i) for i in range(1 << 14)])
+    assert abs(draws.mean() / 65535 - 0.5) < 0.01 and len(set(draws.tolist())) > 14000
+
+
+def test_sr_fixed_points_neighbours_and_exact_upcount():
+    mags = [float(m) for m in E2M1_MAGS]
+    for s in (1.0, -1.0):
+        for c, m in enumerate(mags):
+            for r in (0, 1, 0x7FFF, 0xFFFF):
+                assert oracle.e2m1_encode_sr(s * m, r) == (8 if s < 0 else 0) | c
+    assert oracle.e2m1_encode_sr(-0.0, 0xFFFF) == 8
+    for big in (6.5, 1e9, np.inf, np.nan):
+        assert oracle.e2m1_encode_sr(big, 0xFFFF) == 7
+    assert oracle.e2m1_encode_sr(-np.inf, 0) == 0xF
+    rng = np.random.default_rng(19)
+    for z in np.concatenate([rng.uniform(0, 6, 24), [1e-3, 0.4999, 0.5001, 1.9999, 3.9999, 5.9999]]).astype(np.float32):
+        lo = max(i for i, m in enumerate(mags) if m <= z)
+        hi = lo + 1
+        ups = 0
+        for r in range(0, 65536):
+            c = oracle.e2m1_encode_sr(z, r)
+            assert c in (lo, hi)
+            ups += c == hi
+        # Eq. "sr": P(up) = (z - q-)/(q+ - q-); 16 centred bits realise it to within 2^-17 (+ one
+        # float32 rounding of z + 1 below 1)
+        p = (Fr(float(z)) - Fr(mags[lo])) / (Fr(mags[hi]) - Fr(mags[lo]))
+        assert abs(Fr(ups, 65536) - p) <= Fr(1, 2 ** 17) + Fr(1, 2 ** 22)
+        # monotone in the draw: once it rounds up it stays up
+        flips = [oracle.e2m1_encode_sr(z, r) for r in (0, 16384, 32768, 49152, 65535)]
+        assert flips == sorted(flips)
+        # negative side mirrors
+        assert oracle.e2m1_encode_sr(-z, 12345) == 8 | oracle.e2m1_encode_sr(z, 12345)
+
+
+def test_sr_is_unbiased_through_the_quantizer_and_leaves_scales_alone():
+    rng = np.random.default_rng(23)
+    x = rng.normal(0, 1, (16, 64)).astype(np.float32)
+    g = np.abs(x).max()
+    rne = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, 448.0)
+    acc = np.zeros_like(x, dtype=np.float64)
+    n = 400
+    differs = 0
+    for seed in range(n):
+        sr = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_SR, g, 448.0, seed=seed)
+        assert np.array_equal(sr["scales"], rne["scales"])          # SR touches the payload only
+        differs += not np.array_equal(sr["payload"], rne["payload"])
+        acc += oracle.dequantize(sr["payload"], sr["scales"], False, sr["decode"])
+    assert differs == n
+    mean = acc / n
+    s = np.repeat(np.array([[oracle.ue5m3_value(c) for c in row] for row in rne["scales"]]), 16, axis=1) * float(rne["decode"])
+    clipped = np.abs(x) > 6 * s
+    # per-element std of one draw is at most step/2 <= s; mean of n draws within 5 sigma
+    assert np.all(np.abs(mean - x)[~clipped] <= 5 * s[~clipped] / math.sqrt(n))
+    # and in aggregate the bias is far below the RNE error
+    assert abs(np.mean((mean - x)[~clipped] / s[~clipped])) < 0.01
+    # the draw for an element depends on its index in the source, not on the layout
+    a = oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_SR, g, 448.0, seed=9)
+    assert not np.array_equal(a["payload"], oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_SR, g, 448.0, seed=10)["payload"])
+
+
+def test_sr_col_layout_uses_source_indices():
+    """1D_COL output describes x^T; with one value everywhere and a power-of-two scale every
+    element has the same z, so nibble (c, r) must equal the scalar rule fed with bits of r*cols+c."""
+    rows, cols = 32, 16
+    x = np.full((rows, cols), 0.8125, np.float32)           # z = 0.8125 * 6 / 1 ... see below
+    g, T = 448.0, 448.0                                     # S = 1, G = 6; a_B = .8125 -> s_hat = .8125 (code 0x75)
+    q = oracle.quantize(x, oracle.LAYOUT_1D_COL, oracle.ROUND_SR, g, T, seed=77)
+    assert np.all(q["scales"] == oracle.ue5m3_encode(0.8125))
+    inv = f32(1) / f32(0.8125)
+    z = f32(0.8125) * (f32(6) * inv)
+    for r in range(rows):
+        for c in range(cols):
+            want = oracle.e2m1_encode_sr(z, oracle.sr_bits(77, r * cols + c))
+            assert (q["payload"][c, r // 2] >> (4 * (r % 2))) & 0xF == want
+
+
+# ------------------------------------------------------------------------------------------
+# GEMM (Section 5.3 / 6.1: plain sums over the decoded operands)
+# ------------------------------------------------------------------------------------------
+def _rand_operand(rng, R, Kc, scale2d):
+    payload = rng.integers(0, 256, (R, Kc // 2), dtype=np.uint8)
+    shape = (R // 16, Kc // 16) if scale2d else (R, Kc // 16)
+    scales = rng.integers(0, 0xF8, shape, dtype=np.uint8)
+    return payload, scales
+
+
+def _decode_fr(payload, scales, scale2d, r, k):
+    nib = (int(payload[r, k // 2]) >> (4 * (k % 2))) & 0xF
+    sc = int(scales[r // 16 if scale2d else r, k // 16])
+    return Fr(oracle.ue5m3_value(sc)) * Fr(oracle.e2m1_value(nib))
+
+
+@pytest.mark.parametrize("a2d,b2d", [(False, False), (False, True), (True, False)])
+def test_gemm_is_exact_against_rational_brute_force(a2d, b2d):
+    rng = np.random.default_rng(29)
+    Mo, No, Kc = 16, 32, 48
+    ap, asc = _rand_operand(rng, Mo, Kc, a2d)
+    bp, bsc = _rand_operand(rng, No, Kc, b2d)
+    dA, dB = f32(0.37), f32(1.0 / 2688.0)
+    y, sa = oracle.gemm(ap, asc, a2d, dA, bp, bsc, b2d, dB)
+    alpha = Fr(float(dA)) * Fr(float(dB))
+    for i in range(Mo):
+        for j in range(0, No, 5):
+            prods = [_decode_fr(ap, asc, a2d, i, k) * _decode_fr(bp, bsc, b2d, j, k) for k in range(Kc)]
+            exact = alpha * sum(prods)
+            exact_abs = alpha * sum(abs(p) for p in prods)
+            assert abs(Fr(float(y[i, j])) - exact) <= abs(exact) * Fr(1, 2 ** 50)
+            assert abs(Fr(float(sa[i, j])) - exact_abs) <= exact_abs * Fr(1, 2 ** 50)
+    ci, cj = np.array([3, 15, 0]), np.array([31, 2, 0])
+    yc, sc = oracle.gemm_cells(ap, asc, a2d, dA, bp, bsc, b2d, dB, ci, cj)
+    assert np.array_equal(yc, y[ci, cj]) and np.array_equal(sc, sa[ci, cj])
+
+
+def test_gemm_small_integer_case_equals_library_matmul():
+    """All scales 1.0 and payloads in {0, +-1, +-2, +-4}: the GEMM is an integer matrix product."""
+    rng = np.random.default_rng(31)
+    code_of = {0: 0, 1: 2, 2: 4, 4: 6, -1: 10, -2: 12, -4: 14}
+    ints = np.array([0, 1, 2, 4, -1, -2, -4])
+    Mo, No, Kc = 32, 48, 64
+    A = rng.choice(ints, (Mo, Kc))
+    B = rng.choice(ints, (No, Kc))
+    pack = lambda M: np.array([[code_of[int(M[r, 2 * p])] | (code_of[int(M[r, 2 * p + 1])] << 4)
+                                for p in range(M.shape[1] // 2)] for r in range(M.shape[0])], dtype=np.uint8)
+    ones = lambda R: np.full((R, Kc // 16), 0x78, np.uint8)
+    y, sa = oracle.gemm(pack(A), ones(Mo), False, 1.0, pack(B), ones(No), False, 1.0)
+    assert np.array_equal(y, (A @ B.T).astype(np.float64))
+    assert np.array_equal(sa, (np.abs(A) @ np.abs(B).T).astype(np.float64))
+    # alpha = product of the decode factors, which is 1 when g = 6 T on both sides
+    d = oracle.tensor_constants(6 * 448.0, 448.0)[3]
+    assert d == 1.0
+
+
+def test_gemm_2d_scales_equal_expanded_1d_scales_and_transpose_view():
+    rng = np.random.default_rng(37)
+    W = rng.normal(0, 0.02, (64, 96)).astype(np.float32)
+    X = rng.normal(0, 1, (32, 96)).astype(np.float32)
+    dY = rng.normal(0, 1e-3, (32, 64)).astype(np.float32)
+    qw = oracle.quantize(W, oracle.LAYOUT_2D, oracle.ROUND_RNE, np.abs(W).max(), 448.0, want_t=True)
+    qx = oracle.quantize(X, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, np.abs(X).max(), 448.0)
+    qg = oracle.quantize(dY, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, np.abs(dY).max(), 448.0)
+    y2, _ = oracle.gemm(qx["payload"], qx["scales"], False, qx["decode"], qw["payload"], qw["scales"], True, qw["decode"])
+    y1, _ = oracle.gemm(qx["payload"], qx["scales"], False, qx["decode"],
+                        qw["payload"], np.repeat(qw["scales"], 16, axis=0), False, qw["decode"])
+    assert np.array_equal(y1, y2)
+    # fprop equals the float64 product of the reconstructions (Eq. "microscaling")
+    Xh = oracle.dequantize(qx["payload"], qx["scales"], False, qx["decode"])
+    Wh = oracle.dequantize(qw["payload"], qw["scales"], True, qw["decode"])
+    assert np.allclose(y2, Xh @ Wh.T, rtol=1e-12, atol=1e-300)
+    # 2D scaling: the transposed view decodes to the transpose, so dgrad dX = dY W uses the same W_hat
+    Wth = oracle.dequantize(qw["payload_t"], qw["scales_t"], True, qw["decode"])
+    assert np.array_equal(Wth, Wh.T)
+    dx, _ = oracle.gemm(qg["payload"], qg["scales"], False, qg["decode"], qw["payload_t"], qw["scales_t"], True, qw["decode"])
+    Gh = oracle.dequantize(qg["payload"], qg["scales"], False, qg["decode"])
+    assert np.allclose(dx, Gh @ Wh, rtol=1e-12, atol=1e-300)
+    # wgrad dW = dY^T X from the two column-layout quantizations
+    qgc = oracle.quantize(dY, oracle.LAYOUT_1D_COL, oracle.ROUND_RNE, np.abs(dY).max(), 448.0)
+    qxc = oracle.quantize(X, oracle.LAYOUT_1D_COL, oracle.ROUND_RNE, np.abs(X).max(), 448.0)
+    dw, _ = oracle.gemm(qgc["payload"], qgc["scales"], False, qgc["decode"], qxc["payload"], qxc["scales"], False, qxc["decode"])
+    Gch = oracle.dequantize(qgc["payload"], qgc["scales"], False, qgc["decode"])      # [N, M]
+    Xch = oracle.dequantize(qxc["payload"], qxc["scales"], False, qxc["decode"])      # [K, M]
+    assert dw.shape == (64, 96) and np.allclose(dw, Gch @ Xch.T, rtol=1e-12, atol=1e-300)
+    # a column-layout quantization is the row-layout quantization of the transpose
+    qxt = oracle.quantize(np.ascontiguousarray(X.T), oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, np.abs(X).max(), 448.0)
+    assert np.array_equal(qxt["payload"], qxc["payload"]) and np.array_equal(qxt["scales"], qxc["scales"])
+
+
+def test_bf16_rne_matches_library_conversion():
+    rng = np.random.default_rng(41)
+    v = np.concatenate([rng.normal(0, 1, 5000) * 10.0 ** rng.uniform(-42, 38, 5000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e38, 1e-40, 9.18e-41, np.inf, -np.inf]])
+    v32 = v.astype(np.float32)
+    lib = torch.from_numpy(v32).to(torch.bfloat16).view(torch.uint16).numpy()
+    mine = np.array([oracle.bf16_rne(float(x)) for x in v32], dtype=np.uint16)
+    assert np.array_equal(lib, mine)
+    # a binary64 value just above a BF16 tie must round up even though its float32 rounding is the tie
+    tie = 1.0 + 2.0 ** -8
+    assert oracle.bf16_rne(tie) == 0x3F80 and oracle.bf16_rne(tie + 2.0 ** -40) == 0x3F81
