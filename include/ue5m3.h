@@ -1,0 +1,172 @@
+/*
+ * ue5m3.h -- C ABI of the UE5M3-FP4 quantize-and-multiply library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-linear hot path of the UE5M3 FP4 pretraining recipe: operands
+ * are stored as packed E2M1 payloads (4 bits) with one unsigned E5M3 block scale per 16 values
+ * and one FP32 tensor reference per operand, and the three GEMMs of a linear layer are computed
+ * on those operands.
+ *
+ * General rules for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller.  Nothing is allocated, nothing
+ *     is kept between calls, the host is never synchronised.  Work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*, NULL = the legacy default stream).
+ *   - Return value: 0 (UE5M3_OK) or one of the UE5M3_ERR_* codes below.  Argument errors are found
+ *     on the host before anything is enqueued.  There is no CPU fallback.
+ *   - Matrices are row-major.  "K-major operand [R, Kc]" means R rows, each holding the Kc values
+ *     of the GEMM contraction dimension contiguously.
+ *
+ * Storage formats
+ *   E2M1 payload   code = s<<3 | e<<1 | m, bias 1: magnitudes {0, 0.5, 1, 1.5, 2, 3, 4, 6}
+ *                  (paper, Section 1 and Section 5.2: largest magnitude F = 6).  Byte p of a row
+ *                  holds element 2p in bits 3:0 and element 2p+1 in bits 7:4.  A row of a K-major
+ *                  operand is Kc/2 bytes.
+ *   UE5M3 scale    code = e<<3 | m, bias 15: e = 0 -> m * 2^-17, 1 <= e <= 30 -> (1 + m/8) * 2^(e-15);
+ *                  largest value 61440 = 0xF7, smallest normal 2^-14, smallest subnormal 2^-17
+ *                  (Section 4.1, equation for U_max, and Table 2).  Codes 0xF8..0xFF are not finite
+ *                  and are never produced; the GEMM requires that they do not occur.
+ *   scale layouts  UE5M3_SCALES_ROWMAJOR: [R, Kc/16] bytes (1D blocks) or [R/16, Kc/16] (2D tiles).
+ *                  UE5M3_SCALES_TILED (1D blocks only): the row-major matrix cut into tiles of
+ *                  128 rows x 16 block columns, each tile stored contiguously (2048 bytes, byte
+ *                  (r % 128) * 16 + (kb % 16)), tiles ordered [ceil(R/128)][ceil(Kc/256)].
+ */
+#ifndef UE5M3_H_
+#define UE5M3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    UE5M3_OK = 0,
+    UE5M3_ERR_INVALID_ARG = 1,  /* null pointer, unknown enum value, non-positive size, bad target */
+    UE5M3_ERR_SHAPE = 2,        /* a dimension is not a multiple of what the call requires */
+    UE5M3_ERR_ALIGN = 3,        /* a pointer or leading dimension breaks the stated alignment */
+    UE5M3_ERR_UNSUPPORTED = 4,  /* valid request this build does not implement, or not an sm_100 device */
+    UE5M3_ERR_CUDA = 5,         /* the CUDA runtime or driver reported an error while enqueueing */
+    UE5M3_ERR_TIMEOUT = 6       /* a device-side wait gave up (reported by ue5m3_last_device_status) */
+};
+
+enum { UE5M3_F32 = 0, UE5M3_BF16 = 1 };                                   /* element types */
+enum { UE5M3_LAYOUT_1D_ROW = 0, UE5M3_LAYOUT_1D_COL = 1, UE5M3_LAYOUT_2D = 2 };
+enum { UE5M3_ROUND_RNE = 0, UE5M3_ROUND_SR = 1 };
+enum { UE5M3_SCALES_ROWMAJOR = 0, UE5M3_SCALES_TILED = 1 };
+enum { UE5M3_SCALE_1D = 0, UE5M3_SCALE_1D_TILED = 1, UE5M3_SCALE_2D = 2 };  /* how a GEMM operand's scales are stored */
+enum { UE5M3_FPROP = 0, UE5M3_DGRAD = 1, UE5M3_WGRAD = 2 };
+
+/*
+ * Tensor maximum a = max_i |x_i| (paper, Section 5.1, first equation).  Run only on the steps
+ * at which the sample-and-hold rule refreshes the cached reference (every D = 50 steps).
+ *   x        device, [rows, cols] with leading dimension ld (elements), dtype UE5M3_F32 / UE5M3_BF16;
+ *            16-byte aligned, ld * element size a multiple of 16 bytes, cols a multiple of 8.
+ *   amax_out device, 1 float; overwritten (the call clears it first).  NaNs are ignored;
+ *            +-Inf yields +Inf.  The result does not depend on launch geometry.
+ */
+int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                      float* amax_out, void* stream);
+
+/*
+ * Fused quantizer (paper, Section 3.2 microscaling equation, Section 5.2 scale-target equation,
+ * Section 5.3 rounding assignment, Section 5.4 zero-scale rule).
+ *
+ * With g the held tensor reference read from *amax_held, T the scale target and F = 6:
+ *   g_eff = g if finite and > 0 (raised to at least 2^-60), else 1;
+ *   S = T / g_eff, G = 6T / g_eff, d = g_eff / (6T)              (one binary32 division each)
+ *   per block B:  a_B = max |x_i| (NaN ignored);  u_B = a_B * S;
+ *                 code = UE5M3(u_B), round to nearest even, saturating at 0xF7;
+ *                 a code of 0 is replaced by 0x78 (the value 1);
+ *                 r_B = G * (1 / s_hat_B)                          (binary32, each step rounded)
+ *   per element:  z = x_i * r_B;  q_i = E2M1(z), clamped to +-6, sign of z kept, NaN -> +6;
+ *                 round to nearest even (UE5M3_ROUND_RNE) or stochastic rounding (UE5M3_ROUND_SR).
+ * The reconstruction is x_i ~ d * s_hat_B * q_i.
+ *
+ * Stochastic rounding rounds |z| up to the next E2M1 magnitude with probability equal to its
+ * relative position between the two neighbours, resolved to 16 bits: the 16 random bits of source
+ * element i = row * cols + col are taken from Philox4x32-10 with key = (seed low, seed high) and
+ * counter = (low32(i>>3), high32(i>>3), 0, 0): element lane j = i & 7 uses half (j & 1) of output
+ * word j >> 1.  Block scales are never rounded stochastically.
+ *
+ *   x          device, [rows, cols], leading dimension ld (elements), UE5M3_F32 or UE5M3_BF16;
+ *              16-byte aligned, ld * element size a multiple of 16 bytes.
+ *              rows and cols must be multiples of 16 (UE5M3_ERR_SHAPE otherwise).
+ *   layout     UE5M3_LAYOUT_1D_ROW  blocks of 16 along cols (the contraction dimension is cols):
+ *                                   payload [rows, cols/2], scales [rows, cols/16].
+ *              UE5M3_LAYOUT_1D_COL  blocks of 16 along rows; the outputs describe x^T as a K-major
+ *                                   operand: payload [cols, rows/2], scales [cols, rows/16].
+ *              UE5M3_LAYOUT_2D      one scale per 16x16 tile: payload [rows, cols/2],
+ *                                   scales [rows/16, cols/16]; if payload_t and scales_t are both
+ *                                   non-null they receive the same codes for x^T:
+ *                                   payload_t [cols, rows/2], scales_t [cols/16, rows/16].
+ *   amax_held  device, 1 float (g).        target_T  integer-valued, 0 < T <= 61440 (448 or 2048).
+ *   seed       used only for UE5M3_ROUND_SR.
+ *   payload, scales       device outputs, 16-byte aligned (payload) / any alignment (scales).
+ *   payload_t, scales_t   2D only, both null or both non-null; must be null for 1D layouts.
+ *   decode_out device, 1 float, receives d; may be null.
+ *   stats      device, 4 x uint64, may be null.  The call ADDS to: [0] blocks with u_B > 61440
+ *              (scale saturated, Proposition 1), [1] blocks whose code was 0 and was replaced,
+ *              [2] elements with |z| > 6 (payload clipped), [3] non-finite input elements.
+ *   scale_layout  UE5M3_SCALES_ROWMAJOR, or UE5M3_SCALES_TILED (1D layouts only; the buffer must
+ *              hold ue5m3_scales_bytes(...) bytes; padding bytes are left untouched).
+ */
+int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                   int layout, int rounding,
+                   const float* amax_held, float target_T, uint64_t seed,
+                   uint8_t* payload, uint8_t* scales,
+                   uint8_t* payload_t, uint8_t* scales_t,
+                   float* decode_out, uint64_t* stats,
+                   int scale_layout, void* stream);
+
+/*
+ * Block-scaled GEMM on quantized operands (paper, Section 5.3: Y = X W^T, dX = dY W,
+ * dW = dY^T X; Section 6.1: y = sum_k a_k b_k on the decoded operands, the tensor-scale product
+ * applied after accumulation):
+ *     C[Mo, No] = (d_A * d_B) * sum_k (s_hat q)_A[m, k] * (s_hat q)_B[n, k]
+ * Both operands are K-major.  Every E2M1 x UE5M3 product is exact in BF16; products of two such
+ * values are accumulated in FP32 on the tensor cores.  `op` only names the role of the call:
+ *     FPROP  A = X  (1D_ROW),        B = W   (2D payload, scales)          Mo = tokens, No = out, Kc = in
+ *     DGRAD  A = dY (1D_ROW, SR),    B = W^T (2D payload_t, scales_t)      Mo = tokens, No = in,  Kc = out
+ *     WGRAD  A = dY^T (1D_COL, SR),  B = X^T (1D_COL)                      Mo = out,    No = in,  Kc = tokens
+ *   Mo, No multiples of 128, Kc a multiple of 256 (UE5M3_ERR_SHAPE otherwise).
+ *   a_payload [Mo, Kc/2], b_payload [No, Kc/2]   device, 16-byte aligned.
+ *   a_scales, b_scales   device, 16-byte aligned; a_scale_mode / b_scale_mode say how they are
+ *                        stored: UE5M3_SCALE_1D ([R, Kc/16] row-major), UE5M3_SCALE_1D_TILED,
+ *                        UE5M3_SCALE_2D ([R/16, Kc/16] row-major).  No code >= 0xF8.
+ *   a_decode, b_decode   device, 1 float each (the d written by ue5m3_quantize).
+ *   out        device, [Mo, No] with leading dimension ldo (elements), out_dtype UE5M3_F32 or
+ *              UE5M3_BF16 (rounded to nearest even from the FP32 result); 16-byte aligned rows.
+ * Device-side waits are bounded; if one gives up the tile is abandoned and the status word read by
+ * ue5m3_last_device_status becomes UE5M3_ERR_TIMEOUT.
+ */
+int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
+               const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
+               const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
+               void* out, int out_dtype, int64_t ldo, void* stream);
+
+/*
+ * Bytes a scale buffer needs.  rows/cols are those of the SOURCE tensor given to ue5m3_quantize.
+ * (Section 3.2: one scale per block of B = 16; Section 3.3: one per 16x16 weight tile.)
+ * Returns 0 for invalid arguments.
+ */
+size_t ue5m3_scales_bytes(int64_t rows, int64_t cols, int layout, int scale_layout);
+
+/*
+ * Rewrite tiled scales as row-major [R, kblocks] (for inspection and parity checks).
+ * in: device, tiled buffer for R rows x kblocks block columns; out: device, R * kblocks bytes.
+ */
+int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream);
+
+/*
+ * Synchronises the current device and reports the sticky device-side status word
+ * (UE5M3_OK or UE5M3_ERR_TIMEOUT) of the current device, then clears it.
+ */
+int ue5m3_last_device_status(void);
+
+/* Static, human-readable name of a status code. */
+const char* ue5m3_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UE5M3_H_ */

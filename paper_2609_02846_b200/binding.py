@@ -1,0 +1,253 @@
+"""ctypes binding of ``libue5m3.so``: same names as the C ABI, argument marshalling only.
+
+Every function takes torch CUDA tensors, passes their device pointers and the current CUDA stream
+to the library and returns torch tensors that wrap the caller-visible outputs.  Nothing is computed
+here.  The library is required: a missing or unloadable ``libue5m3.so`` raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+F32, BF16 = 0, 1
+LAYOUT_1D_ROW, LAYOUT_1D_COL, LAYOUT_2D = 0, 1, 2
+ROUND_RNE, ROUND_SR = 0, 1
+SCALES_ROWMAJOR, SCALES_TILED = 0, 1
+SCALE_1D, SCALE_1D_TILED, SCALE_2D = 0, 1, 2
+FPROP, DGRAD, WGRAD = 0, 1, 2
+
+SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_gemm", "ue5m3_scales_bytes",
+           "ue5m3_unswizzle_scales", "ue5m3_last_device_status", "ue5m3_status_string")
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libue5m3.so")
+_lib = None
+
+
+class Ue5m3Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise FileNotFoundError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2609_02846_b200.build` "
+                "(there is no fallback implementation)")
+        L = C.CDLL(_LIB_PATH)
+        i64, u64, vp, ci, f32 = C.c_int64, C.c_uint64, C.c_void_p, C.c_int, C.c_float
+        L.ue5m3_sample_amax.restype = ci
+        L.ue5m3_sample_amax.argtypes = [vp, ci, i64, i64, i64, vp, vp]
+        L.ue5m3_quantize.restype = ci
+        L.ue5m3_quantize.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, f32, u64, vp, vp, vp, vp, vp, vp, ci, vp]
+        L.ue5m3_gemm.restype = ci
+        L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
+        L.ue5m3_scales_bytes.restype = C.c_size_t
+        L.ue5m3_scales_bytes.argtypes = [i64, i64, ci, ci]
+        L.ue5m3_unswizzle_scales.restype = ci
+        L.ue5m3_unswizzle_scales.argtypes = [vp, vp, i64, i64, vp]
+        L.ue5m3_last_device_status.restype = ci
+        L.ue5m3_last_device_status.argtypes = []
+        L.ue5m3_status_string.restype = C.c_char_p
+        L.ue5m3_status_string.argtypes = [ci]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return _load().ue5m3_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise Ue5m3Error(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: the library takes float32 or bfloat16")
+
+
+def _dev_ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("the library takes device tensors only")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(t: torch.Tensor):
+    return C.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def _matrix(x: torch.Tensor):
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("expected a 2-D tensor whose rows are contiguous")
+    return x.shape[0], x.shape[1], x.stride(0)
+
+
+# ---------------------------------------------------------------------------------------------
+def sample_amax(x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """max |x| as a 1-element float32 device tensor (no host synchronisation)."""
+    rows, cols, ld = _matrix(x)
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(_load().ue5m3_sample_amax(_dev_ptr(x), _dtype_code(x), rows, cols, ld, _dev_ptr(out), _stream(x)),
+               "ue5m3_sample_amax")
+    return out
+
+
+def scales_bytes(rows: int, cols: int, layout: int, scale_layout: int = SCALES_ROWMAJOR) -> int:
+    return int(_load().ue5m3_scales_bytes(rows, cols, layout, scale_layout))
+
+
+@dataclass
+class QuantizedOperand:
+    """A K-major GEMM operand [R, Kc]: packed E2M1 payload, UE5M3 scales, tensor decode factor."""
+    payload: torch.Tensor                 # uint8 [R, Kc/2]
+    scales: torch.Tensor                  # uint8, row-major [R, Kc/16] / [R/16, Kc/16], or flat tiled buffer
+    decode: torch.Tensor                  # float32 [1]
+    scale_mode: int                       # SCALE_1D, SCALE_1D_TILED or SCALE_2D
+    payload_t: Optional[torch.Tensor] = None   # 2D only: the same codes for the transpose [Kc, R/2]
+    scales_t: Optional[torch.Tensor] = None    # 2D only: [Kc/16, R/16]
+
+    @property
+    def R(self) -> int:
+        return self.payload.shape[0]
+
+    @property
+    def Kc(self) -> int:
+        return self.payload.shape[1] * 2
+
+    def transposed(self) -> "QuantizedOperand":
+        if self.payload_t is None:
+            raise ValueError("this operand was quantized without its transposed copy")
+        return QuantizedOperand(self.payload_t, self.scales_t, self.decode, SCALE_2D, self.payload, self.scales)
+
+
+def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tensor, target_T: float = 448.0,
+             seed: int = 0, want_transpose: bool = False, stats: Optional[torch.Tensor] = None,
+             scale_layout: int = SCALES_ROWMAJOR, out: Optional[QuantizedOperand] = None) -> QuantizedOperand:
+    """ue5m3_quantize.  `stats` (int64[4], device) is accumulated into when given."""
+    rows, cols, ld = _matrix(x)
+    dev = x.device
+    u8 = dict(dtype=torch.uint8, device=dev)
+    if out is None:
+        nbytes = scales_bytes(rows, cols, layout, scale_layout)
+        if nbytes == 0:
+            _check(2, "ue5m3_quantize (rows and cols must be positive multiples of 16)")
+        if layout == LAYOUT_1D_ROW:
+            payload = torch.empty((rows, cols // 2), **u8)
+            sshape = (rows, cols // 16)
+        elif layout == LAYOUT_1D_COL:
+            payload = torch.empty((cols, rows // 2), **u8)
+            sshape = (cols, rows // 16)
+        else:
+            payload = torch.empty((rows, cols // 2), **u8)
+            sshape = (rows // 16, cols // 16)
+        if scale_layout == SCALES_TILED:
+            scales = torch.zeros(nbytes, **u8)
+        else:
+            scales = torch.empty(sshape, **u8)
+        payload_t = scales_t = None
+        if layout == LAYOUT_2D and want_transpose:
+            payload_t = torch.empty((cols, rows // 2), **u8)
+            scales_t = torch.empty((cols // 16, rows // 16), **u8)
+        mode = SCALE_2D if layout == LAYOUT_2D else (SCALE_1D_TILED if scale_layout == SCALES_TILED else SCALE_1D)
+        out = QuantizedOperand(payload, scales, torch.empty(1, dtype=torch.float32, device=dev), mode, payload_t, scales_t)
+    if stats is not None and (stats.dtype != torch.int64 or stats.numel() != 4):
+        raise ValueError("stats must be an int64 tensor with 4 elements")
+    with torch.cuda.device(dev):
+        _check(_load().ue5m3_quantize(
+            _dev_ptr(x), _dtype_code(x), rows, cols, ld, layout, rounding, _dev_ptr(amax_held),
+            C.c_float(target_T), C.c_uint64(int(seed) & (2 ** 64 - 1)),
+            _dev_ptr(out.payload), _dev_ptr(out.scales), _dev_ptr(out.payload_t), _dev_ptr(out.scales_t),
+            _dev_ptr(out.decode), _dev_ptr(stats), scale_layout, _stream(x)), "ue5m3_quantize")
+    return out
+
+
+def unswizzle_scales(tiled: torch.Tensor, R: int, kblocks: int) -> torch.Tensor:
+    out = torch.empty((R, kblocks), dtype=torch.uint8, device=tiled.device)
+    with torch.cuda.device(tiled.device):
+        _check(_load().ue5m3_unswizzle_scales(_dev_ptr(tiled), _dev_ptr(out), R, kblocks, _stream(tiled)),
+               "ue5m3_unswizzle_scales")
+    return out
+
+
+def gemm(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
+         out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """C[Mo, No] = d_A d_B * A[Mo, Kc] B[No, Kc]^T on the quantized operands (ue5m3_gemm)."""
+    Mo, No, Kc = a.R, b.R, a.Kc
+    if b.Kc != Kc:
+        raise ValueError(f"contraction sizes differ: {Kc} vs {b.Kc}")
+    if out is None:
+        out = torch.empty((Mo, No), dtype=out_dtype, device=a.payload.device)
+    with torch.cuda.device(out.device):
+        _check(_load().ue5m3_gemm(op, Mo, No, Kc,
+                                  _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
+                                  _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
+                                  _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)), "ue5m3_gemm")
+    return out
+
+
+def last_device_status() -> int:
+    return int(_load().ue5m3_last_device_status())
+
+
+# ---------------------------------------------------------------------------------------------
+class AmaxCache:
+    """Sample-and-hold tensor reference of one operand: the maximum is re-sampled when the cache is
+    empty or `interval` steps old and held in between (not a window maximum).  The held value stays
+    on the device, so holding costs nothing and refreshing costs one ue5m3_sample_amax launch."""
+
+    def __init__(self, interval: int = 50):
+        self.interval = int(interval)
+        self.last_refresh: Optional[int] = None
+        self.held: Optional[torch.Tensor] = None
+
+    def refreshes_at(self, step: int) -> bool:
+        return self.last_refresh is None or step - self.last_refresh >= self.interval
+
+    def get(self, x: torch.Tensor, step: int) -> torch.Tensor:
+        if self.refreshes_at(step):
+            self.held = sample_amax(x, self.held)
+            self.last_refresh = step
+        return self.held
+
+
+def linear_forward(x: torch.Tensor, w: torch.Tensor, amax_x: torch.Tensor, amax_w: torch.Tensor,
+                   target_T: float = 448.0, out_dtype: torch.dtype = torch.bfloat16,
+                   scale_layout: int = SCALES_ROWMAJOR):
+    """Y = X W^T: quantize X (1D along K, RNE) and W (2D tiles, RNE, with transposed copy), multiply.
+    Returns (Y, qx, qw); qw carries the transposed view the backward pass needs."""
+    qx = quantize(x, LAYOUT_1D_ROW, ROUND_RNE, amax_x, target_T, scale_layout=scale_layout)
+    qw = quantize(w, LAYOUT_2D, ROUND_RNE, amax_w, target_T, want_transpose=True)
+    return gemm(FPROP, qx, qw, out_dtype), qx, qw
+
+
+def linear_backward(dy: torch.Tensor, x: torch.Tensor, qw: QuantizedOperand, amax_dy: torch.Tensor,
+                    amax_x: torch.Tensor, seed: int, target_T: float = 448.0, target_T_wgrad_dy: float = 448.0,
+                    out_dtype: torch.dtype = torch.bfloat16, scale_layout: int = SCALES_ROWMAJOR):
+    """dX = dY W and dW = dY^T X.  dY is rounded stochastically, once per GEMM with seeds 4*seed and
+    4*seed + 1; the saved activation X is re-quantized along the token dimension with RNE."""
+    qdy = quantize(dy, LAYOUT_1D_ROW, ROUND_SR, amax_dy, target_T, seed=4 * seed, scale_layout=scale_layout)
+    dx = gemm(DGRAD, qdy, qw.transposed(), out_dtype)
+    qdy_t = quantize(dy, LAYOUT_1D_COL, ROUND_SR, amax_dy, target_T_wgrad_dy, seed=4 * seed + 1, scale_layout=scale_layout)
+    qx_t = quantize(x, LAYOUT_1D_COL, ROUND_RNE, amax_x, target_T, scale_layout=scale_layout)
+    dw = gemm(WGRAD, qdy_t, qx_t, out_dtype)
+    return dx, dw

@@ -1,0 +1,138 @@
+// C ABI of the UE5M3-FP4 library: argument checks on the host, then kernel launches.
+#include <cuda_runtime.h>
+#include <cstdint>
+#include "../../include/ue5m3.h"
+#include "launch.h"
+
+namespace ue5m3 {
+
+struct DeviceInfo { int ok; int sms; int major; };
+
+static DeviceInfo device_info() {
+    // one entry per device ordinal; filled on first use with that device current
+    static DeviceInfo cache[64];
+    static bool known[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DeviceInfo{0, 0, 0};
+    if (!known[dev]) {
+        cudaDeviceProp p;
+        if (cudaGetDeviceProperties(&p, dev) != cudaSuccess) return DeviceInfo{0, 0, 0};
+        cache[dev] = DeviceInfo{1, p.multiProcessorCount, p.major};
+        known[dev] = true;
+    }
+    return cache[dev];
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace ue5m3
+
+using namespace ue5m3;
+
+extern "C" {
+
+const char* ue5m3_status_string(int status) {
+    switch (status) {
+        case UE5M3_OK: return "UE5M3_OK";
+        case UE5M3_ERR_INVALID_ARG: return "UE5M3_ERR_INVALID_ARG: null pointer, unknown enum value or non-positive size";
+        case UE5M3_ERR_SHAPE: return "UE5M3_ERR_SHAPE: a dimension is not a multiple of what the call requires";
+        case UE5M3_ERR_ALIGN: return "UE5M3_ERR_ALIGN: pointer or leading dimension not 16-byte aligned";
+        case UE5M3_ERR_UNSUPPORTED: return "UE5M3_ERR_UNSUPPORTED: not implemented for these arguments or this device";
+        case UE5M3_ERR_CUDA: return "UE5M3_ERR_CUDA: the CUDA runtime reported an error";
+        case UE5M3_ERR_TIMEOUT: return "UE5M3_ERR_TIMEOUT: a device-side wait gave up";
+        default: return "unknown UE5M3 status";
+    }
+}
+
+size_t ue5m3_scales_bytes(int64_t rows, int64_t cols, int layout, int scale_layout) {
+    if (rows <= 0 || cols <= 0 || (rows % 16) || (cols % 16)) return 0;
+    if (layout == UE5M3_LAYOUT_2D) {
+        if (scale_layout != UE5M3_SCALES_ROWMAJOR) return 0;
+        return (size_t)(rows / 16) * (size_t)(cols / 16);
+    }
+    int64_t R, kb;
+    if (layout == UE5M3_LAYOUT_1D_ROW) { R = rows; kb = cols / 16; }
+    else if (layout == UE5M3_LAYOUT_1D_COL) { R = cols; kb = rows / 16; }
+    else return 0;
+    if (scale_layout == UE5M3_SCALES_ROWMAJOR) return (size_t)R * (size_t)kb;
+    if (scale_layout == UE5M3_SCALES_TILED) return (size_t)((R + 127) / 128) * (size_t)((kb + 15) / 16) * 2048;
+    return 0;
+}
+
+int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* amax_out, void* stream) {
+    if (!x || !amax_out || rows <= 0 || cols <= 0 || ld < cols) return UE5M3_ERR_INVALID_ARG;
+    if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
+    if (cols % 8) return UE5M3_ERR_SHAPE;
+    const int64_t esz = dtype == UE5M3_F32 ? 4 : 2;
+    if (!aligned16(x) || ((ld * esz) % 16) || (reinterpret_cast<uintptr_t>(amax_out) & 3u)) return UE5M3_ERR_ALIGN;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    return launch_amax(x, dtype, rows, cols, ld, amax_out, di.sms, (cudaStream_t)stream) == cudaSuccess ? UE5M3_OK
+                                                                                                        : UE5M3_ERR_CUDA;
+}
+
+int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int layout, int rounding,
+                   const float* amax_held, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
+                   uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
+                   void* stream) {
+    if (!x || !amax_held || !payload || !scales || rows <= 0 || cols <= 0 || ld < cols) return UE5M3_ERR_INVALID_ARG;
+    if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
+    if (layout != UE5M3_LAYOUT_1D_ROW && layout != UE5M3_LAYOUT_1D_COL && layout != UE5M3_LAYOUT_2D) return UE5M3_ERR_INVALID_ARG;
+    if (rounding != UE5M3_ROUND_RNE && rounding != UE5M3_ROUND_SR) return UE5M3_ERR_INVALID_ARG;
+    if (scale_layout != UE5M3_SCALES_ROWMAJOR && scale_layout != UE5M3_SCALES_TILED) return UE5M3_ERR_INVALID_ARG;
+    if (!(target_T > 0.0f) || target_T > 61440.0f || target_T != (float)(int)target_T) return UE5M3_ERR_INVALID_ARG;
+    if ((payload_t == nullptr) != (scales_t == nullptr)) return UE5M3_ERR_INVALID_ARG;
+    if (layout != UE5M3_LAYOUT_2D && payload_t) return UE5M3_ERR_INVALID_ARG;
+    if (layout == UE5M3_LAYOUT_2D && scale_layout != UE5M3_SCALES_ROWMAJOR) return UE5M3_ERR_INVALID_ARG;
+    if ((rows % 16) || (cols % 16)) return UE5M3_ERR_SHAPE;
+    const int64_t esz = dtype == UE5M3_F32 ? 4 : 2;
+    if (!aligned16(x) || ((ld * esz) % 16) || !aligned16(payload) || !aligned16(scales)) return UE5M3_ERR_ALIGN;
+    if (payload_t && (!aligned16(payload_t) || !aligned16(scales_t))) return UE5M3_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(amax_held) & 3u) || (reinterpret_cast<uintptr_t>(decode_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(stats) & 7u))
+        return UE5M3_ERR_ALIGN;
+    if (rows * (cols / 16) >= ((int64_t)1 << 31) * 256) return UE5M3_ERR_UNSUPPORTED;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    QuantArgs a{x, rows, cols, ld, amax_held, target_T, seed, payload, scales, payload_t, scales_t, decode_out,
+                reinterpret_cast<unsigned long long*>(stats)};
+    return launch_quantize(a, dtype, layout, rounding, scale_layout == UE5M3_SCALES_TILED, (cudaStream_t)stream) == cudaSuccess
+               ? UE5M3_OK
+               : UE5M3_ERR_CUDA;
+}
+
+int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+               int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+               int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
+    if (op != UE5M3_FPROP && op != UE5M3_DGRAD && op != UE5M3_WGRAD) return UE5M3_ERR_INVALID_ARG;
+    if (!a_payload || !a_scales || !a_decode || !b_payload || !b_scales || !b_decode || !out) return UE5M3_ERR_INVALID_ARG;
+    if (Mo <= 0 || No <= 0 || Kc <= 0 || ldo < No) return UE5M3_ERR_INVALID_ARG;
+    if (out_dtype != UE5M3_F32 && out_dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
+    for (int m : {a_scale_mode, b_scale_mode})
+        if (m != UE5M3_SCALE_1D && m != UE5M3_SCALE_1D_TILED && m != UE5M3_SCALE_2D) return UE5M3_ERR_INVALID_ARG;
+    if ((Mo % 128) || (No % 128) || (Kc % 256)) return UE5M3_ERR_SHAPE;
+    const int64_t osz = out_dtype == UE5M3_F32 ? 4 : 2;
+    if (!aligned16(a_payload) || !aligned16(b_payload) || !aligned16(a_scales) || !aligned16(b_scales) || !aligned16(out) ||
+        ((ldo * osz) % 16))
+        return UE5M3_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(a_decode) & 3u) || (reinterpret_cast<uintptr_t>(b_decode) & 3u)) return UE5M3_ERR_ALIGN;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
+               out, out_dtype, ldo};
+    return launch_gemm(g, di.sms, (cudaStream_t)stream);
+}
+
+int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream) {
+    if (!in || !out || R <= 0 || kblocks <= 0) return UE5M3_ERR_INVALID_ARG;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    return launch_unswizzle(in, out, R, kblocks, (cudaStream_t)stream) == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
+}
+
+int ue5m3_last_device_status(void) { return read_and_clear_device_status(); }
+
+}  // extern "C"

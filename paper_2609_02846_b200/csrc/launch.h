@@ -1,0 +1,36 @@
+// Host-side launch interface between the C ABI (api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace ue5m3 {
+
+struct QuantArgs {
+    const void* x;
+    int64_t rows, cols, ld;
+    const float* amax_held;
+    float T;
+    uint64_t seed;
+    uint8_t* payload;
+    uint8_t* scales;
+    uint8_t* payload_t;
+    uint8_t* scales_t;
+    float* decode_out;
+    unsigned long long* stats;
+};
+
+struct GemmArgs {
+    int64_t Mo, No, Kc;
+    const uint8_t* a_payload; const uint8_t* a_scales; int a_scale_mode; const float* a_decode;
+    const uint8_t* b_payload; const uint8_t* b_scales; int b_scale_mode; const float* b_decode;
+    void* out; int out_dtype; int64_t ldo;
+};
+
+cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, cudaStream_t st);
+cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* out, int num_sms,
+                        cudaStream_t st);
+cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, cudaStream_t st);
+int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st);   // returns a UE5M3_* status
+int read_and_clear_device_status();                                  // synchronises the device
+
+}  // namespace ue5m3

@@ -1,0 +1,170 @@
+"""Parity of the CUDA quantizer and tensor maximum with the CPU oracle: every payload byte, scale
+byte, decode factor, stochastic-rounding draw and counter must be identical."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_same_quantization, lib_quantize, oracle_quantize
+import synth_inputs as si
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+LAYOUTS = [oracle.LAYOUT_1D_ROW, oracle.LAYOUT_1D_COL, oracle.LAYOUT_2D]
+ROUNDINGS = [oracle.ROUND_RNE, oracle.ROUND_SR]
+
+
+def _amax(x):
+    return float(x.float().abs().max().item())
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("rounding", ROUNDINGS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("shape", [(16, 16), (256, 256), (272, 4112), (1040, 208)])
+def test_quantize_matches_oracle(layout, rounding, dtype, shape):
+    rows, cols = shape
+    x = si.channel_scaled_activation(rows, cols, seed=rows + cols, device=DEV, dtype=dtype)
+    x[0, 0] = 0.0
+    x[rows - 1, cols - 1] = -0.0
+    g = _amax(x) * 0.37                                  # stale reference: some payloads clip
+    want_t = layout == oracle.LAYOUT_2D
+    _, got = lib_quantize(x, layout, rounding, g, 448.0, seed=0xC0FFEE12345, want_t=want_t)
+    want = oracle_quantize(x, layout, rounding, g, 448.0, seed=0xC0FFEE12345, want_t=want_t)
+    assert_same_quantization(got, want)
+    assert want["stats"]["payload_clipped"] > 0
+
+
+@pytest.mark.parametrize("layout", [oracle.LAYOUT_1D_ROW, oracle.LAYOUT_1D_COL])
+@pytest.mark.parametrize("rounding", ROUNDINGS)
+def test_tiled_scale_layout_holds_the_same_scales(layout, rounding):
+    x = si.heavy_tailed_gradient(400, 528, seed=5, device=DEV)
+    g = _amax(x)
+    _, got = lib_quantize(x, layout, rounding, g, 2048.0, seed=9, scale_layout=1)
+    want = oracle_quantize(x, layout, rounding, g, 2048.0, seed=9)
+    assert_same_quantization(got, want)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_strided_input_and_no_transpose_request(layout):
+    big = si.row_scaled_tensor(320, 640, seed=3, device=DEV)
+    x = big[:, 64:64 + 512]                              # ld = 640 > cols = 512, offset keeps 16-byte alignment
+    g = _amax(x)
+    _, got = lib_quantize(x, layout, oracle.ROUND_SR, g, seed=77, want_t=False)
+    want = oracle.quantize(si.to_numpy_bits(big)[:, 64:64 + 512], layout, oracle.ROUND_SR, g, 448.0, 77, False)
+    assert_same_quantization(got, want)
+
+
+def test_every_e2m1_decision_point_and_sign():
+    """g = 6T and a 6.0 in every block make the element multiplier exactly 1, so z = x."""
+    thr = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0], dtype=np.float32)
+    probes = [0.0, -0.0, 1e-30, -1e-30, 6.0, -6.0]
+    for t in thr:
+        for v in (t, np.nextafter(t, np.float32(0)), np.nextafter(t, np.float32(9))):
+            probes += [float(v), -float(v)]
+    probes = np.array(probes, dtype=np.float32)
+    n = len(probes)
+    blocks = (n + 14) // 15
+    x = np.zeros((16, blocks * 16), np.float32)
+    for b in range(blocks):
+        x[0, 16 * b] = 6.0
+        chunk = probes[15 * b:15 * b + 15]
+        x[0, 16 * b + 1:16 * b + 1 + len(chunk)] = chunk
+    xt = torch.from_numpy(x).to(DEV)
+    for rounding in ROUNDINGS:
+        _, got = lib_quantize(xt, oracle.LAYOUT_1D_ROW, rounding, 2688.0, seed=3)
+        want = oracle_quantize(xt, oracle.LAYOUT_1D_ROW, rounding, 2688.0, seed=3)
+        assert np.all(want["scales"][0] == 0x78)
+        assert_same_quantization(got, want)
+
+
+def test_every_ue5m3_decision_point():
+    """g = T makes u_B = a_B, so block maxima placed on and next to every code midpoint exercise the
+    scale encoder's rounding, its subnormal range, saturation and the zero-scale rule."""
+    vals = np.array([oracle.ue5m3_value(c) for c in range(0xF8)], dtype=np.float64)
+    mids = ((vals[:-1] + vals[1:]) / 2).astype(np.float32)
+    cand = np.concatenate([vals.astype(np.float32), mids, np.nextafter(mids, np.float32(0)),
+                           np.nextafter(mids, np.float32(1e9)),
+                           np.array([0.0, 1e-8, 2.0 ** -18, 61441.0, 63488.0, 65536.0, 1e30, np.inf], np.float32)])
+    x = np.zeros((16, 16 * len(cand)), np.float32)
+    x[3, 5::16] = -cand
+    xt = torch.from_numpy(x).to(DEV)
+    _, got = lib_quantize(xt, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, 448.0)
+    want = oracle_quantize(xt, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, 448.0)
+    assert_same_quantization(got, want)
+    assert want["stats"]["scale_saturated"] >= 4 and want["stats"]["zero_repaired"] > 0
+    assert want["stats"]["nonfinite"] == 1
+
+
+@pytest.mark.parametrize("g", [0.0, -1.0, float("inf"), float("nan"), 1e-30, 3e38, 1e-12])
+def test_degenerate_references(g):
+    x = si.weight(64, 64, seed=1, device=DEV)
+    for layout in LAYOUTS:
+        _, got = lib_quantize(x, layout, oracle.ROUND_RNE, g)
+        want = oracle_quantize(x, layout, oracle.ROUND_RNE, g)
+        assert_same_quantization(got, want)
+
+
+def test_all_zero_and_nonfinite_inputs():
+    x = torch.zeros(32, 64, dtype=torch.bfloat16, device=DEV)
+    x[0, 1] = -0.0
+    for layout in LAYOUTS:
+        for rounding in ROUNDINGS:
+            _, got = lib_quantize(x, layout, rounding, 1.0, seed=1)
+            want = oracle_quantize(x, layout, rounding, 1.0, seed=1)
+            assert_same_quantization(got, want)
+            assert np.all(want["scales"] == 0x78)
+    y = si.weight(32, 64, seed=2, device=DEV, dtype=torch.float32)
+    y[3, 3] = float("nan"); y[4, 40] = float("inf"); y[20, 17] = float("-inf"); y[31, 63] = float("nan")
+    for layout in LAYOUTS:
+        for rounding in ROUNDINGS:
+            _, got = lib_quantize(y, layout, rounding, 0.1, seed=1)
+            want = oracle_quantize(y, layout, rounding, 0.1, seed=1)
+            assert_same_quantization(got, want)
+            assert want["stats"]["nonfinite"] == 4
+
+
+def test_sr_scales_equal_rne_scales_and_draws_differ_by_seed():
+    x = si.heavy_tailed_gradient(256, 512, seed=8, device=DEV)
+    g = _amax(x)
+    _, rne = lib_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g)
+    _, s1 = lib_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_SR, g, seed=4)
+    _, s2 = lib_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_SR, g, seed=5)
+    assert np.array_equal(rne["scales"], s1["scales"]) and np.array_equal(rne["scales"], s2["scales"])
+    assert not np.array_equal(s1["payload"], s2["payload"]) and not np.array_equal(s1["payload"], rne["payload"])
+    _, s1b = lib_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_SR, g, seed=4)
+    assert np.array_equal(s1["payload"], s1b["payload"])          # same seed, same bytes
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("shape", [(16, 16), (300, 520), (2048, 4096)])
+def test_sample_amax(dtype, shape):
+    import paper_2609_02846_b200 as lib
+    x = si.outlier_activation(shape[0], shape[1], seed=4, device=DEV, dtype=dtype)
+    want = oracle.amax(si.to_numpy_bits(x))
+    assert lib.sample_amax(x).item() == want
+    x[shape[0] // 2, 3] = float("nan")
+    assert lib.sample_amax(x).item() == want
+    view = x[:, 8:shape[1]]                              # strided, 16-byte aligned start
+    assert lib.sample_amax(view).item() == oracle.amax(si.to_numpy_bits(x)[:, 8:shape[1]])
+    x[1, 9] = float("-inf")
+    assert lib.sample_amax(x).item() == float("inf")
+    assert lib.sample_amax(torch.zeros(16, 16, dtype=dtype, device=DEV)).item() == 0.0
+
+
+def test_argument_errors_are_reported_not_executed():
+    import paper_2609_02846_b200 as lib
+    x = torch.zeros(32, 40, dtype=torch.bfloat16, device=DEV)
+    g = torch.ones(1, device=DEV)
+    with pytest.raises(lib.Ue5m3Error) as e:
+        lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
+    assert e.value.status == 2
+    x = torch.zeros(32, 64, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(lib.Ue5m3Error) as e:
+        lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g, target_T=0.0)
+    assert e.value.status == 1
+    with pytest.raises(lib.Ue5m3Error) as e:
+        lib.quantize(x[:, 1:33], lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
+    assert e.value.status == 3
+    with pytest.raises(TypeError):
+        lib.quantize(x.half(), lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
