@@ -35,6 +35,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define UE5M3_API __attribute__((visibility("default")))
+#else
+#define UE5M3_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -64,7 +70,7 @@ enum { UE5M3_FPROP = 0, UE5M3_DGRAD = 1, UE5M3_WGRAD = 2 };
  *   amax_out device, 1 float; overwritten (the call clears it first).  NaNs are ignored;
  *            +-Inf yields +Inf.  The result does not depend on launch geometry.
  */
-int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+UE5M3_API int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
                       float* amax_out, void* stream);
 
 /*
@@ -101,7 +107,7 @@ int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int6
  *                                   payload_t [cols, rows/2], scales_t [cols/16, rows/16].
  *   amax_held  device, 1 float (g).        target_T  integer-valued, 0 < T <= 61440 (448 or 2048).
  *   seed       used only for UE5M3_ROUND_SR.
- *   payload, scales       device outputs, 16-byte aligned (payload) / any alignment (scales).
+ *   payload, scales       device outputs, both 16-byte aligned.
  *   payload_t, scales_t   2D only, both null or both non-null; must be null for 1D layouts.
  *   decode_out device, 1 float, receives d; may be null.
  *   stats      device, 4 x uint64, may be null.  The call ADDS to: [0] blocks with u_B > 61440
@@ -110,7 +116,7 @@ int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int6
  *   scale_layout  UE5M3_SCALES_ROWMAJOR, or UE5M3_SCALES_TILED (1D layouts only; the buffer must
  *              hold ue5m3_scales_bytes(...) bytes; padding bytes are left untouched).
  */
-int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+UE5M3_API int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
                    int layout, int rounding,
                    const float* amax_held, float target_T, uint64_t seed,
                    uint8_t* payload, uint8_t* scales,
@@ -139,7 +145,7 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
  * Device-side waits are bounded; if one gives up the tile is abandoned and the status word read by
  * ue5m3_last_device_status becomes UE5M3_ERR_TIMEOUT.
  */
-int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
+UE5M3_API int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
                const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
                const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
                void* out, int out_dtype, int64_t ldo, void* stream);
@@ -149,22 +155,22 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
  * (Section 3.2: one scale per block of B = 16; Section 3.3: one per 16x16 weight tile.)
  * Returns 0 for invalid arguments.
  */
-size_t ue5m3_scales_bytes(int64_t rows, int64_t cols, int layout, int scale_layout);
+UE5M3_API size_t ue5m3_scales_bytes(int64_t rows, int64_t cols, int layout, int scale_layout);
 
 /*
  * Rewrite tiled scales as row-major [R, kblocks] (for inspection and parity checks).
  * in: device, tiled buffer for R rows x kblocks block columns; out: device, R * kblocks bytes.
  */
-int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream);
+UE5M3_API int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream);
 
 /*
  * Synchronises the current device and reports the sticky device-side status word
  * (UE5M3_OK or UE5M3_ERR_TIMEOUT) of the current device, then clears it.
  */
-int ue5m3_last_device_status(void);
+UE5M3_API int ue5m3_last_device_status(void);
 
 /* Static, human-readable name of a status code. */
-const char* ue5m3_status_string(int status);
+UE5M3_API const char* ue5m3_status_string(int status);
 
 #ifdef __cplusplus
 }

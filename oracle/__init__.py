@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
         L.oracle_gemm_cells.argtypes = [i64, vp, vp, C.c_int, f32, vp, vp, C.c_int, f32, i64, vp, vp, vp, vp]
         L.oracle_bf16_rne.restype = C.c_uint16
         L.oracle_bf16_rne.argtypes = [f64]
+        L.oracle_bf16_rne_array.restype = None
+        L.oracle_bf16_rne_array.argtypes = [vp, i64, vp]
         L.oracle_num_threads.restype = C.c_int
         L.oracle_set_num_threads.argtypes = [C.c_int]
         _lib = L
@@ -126,6 +128,13 @@ def sr_bits(seed: int, index: int) -> int:
 
 def bf16_rne(v: float) -> int:
     return lib().oracle_bf16_rne(float(v))
+
+
+def bf16_rne_array(v: np.ndarray) -> np.ndarray:
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    out = np.zeros(v.shape, np.uint16)
+    lib().oracle_bf16_rne_array(_ptr(v), v.size, _ptr(out))
+    return out
 
 
 # ---- tensor reference -------------------------------------------------------------------

@@ -465,3 +465,9 @@ ORACLE_API void oracle_set_num_threads(int n) { omp_set_num_threads(n); }
 ORACLE_API int oracle_num_threads(void) { return 1; }
 ORACLE_API void oracle_set_num_threads(int n) { (void)n; }
 #endif
+
+/* oracle_bf16_rne over an array. */
+ORACLE_API void oracle_bf16_rne_array(const double *v, int64_t n, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_bf16_rne(v[i]);
+}

@@ -1,0 +1,125 @@
+"""Parity of the CUDA block-scaled GEMM with the exact-integer oracle.
+FP32 outputs: |y - y*| <= 1e-5 * sum_k |a_k b_k| + 1e-30.  BF16 outputs: within 1 ulp."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_02846_b200 as lib
+import synth_inputs as si
+from helpers import assert_same_quantization, check_gemm_output, lib_quantize, oracle_quantize
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _operand(rng, R, Kc, mode, lo_code=0, hi_code=0xF8, dec=1.0):
+    """Random payload/scale bytes straight into a QuantizedOperand (every code < 0xF8 is legal input)."""
+    payload = rng.integers(0, 256, (R, Kc // 2), dtype=np.uint8)
+    shape = (R // 16, Kc // 16) if mode == lib.SCALE_2D else (R, Kc // 16)
+    scales = rng.integers(lo_code, hi_code, shape, dtype=np.uint8)
+    dev_scales = torch.from_numpy(scales).to(DEV)
+    if mode == lib.SCALE_1D_TILED:
+        kb = Kc // 16
+        buf = np.zeros(((R + 127) // 128) * ((kb + 15) // 16) * 2048, np.uint8)
+        r, k = np.meshgrid(np.arange(R), np.arange(kb), indexing="ij")
+        off = ((r >> 7) * ((kb + 15) // 16) + (k >> 4)) * 2048 + (r & 127) * 16 + (k & 15)
+        buf[off.ravel()] = scales.ravel()
+        dev_scales = torch.from_numpy(buf).to(DEV)
+    q = lib.QuantizedOperand(torch.from_numpy(payload).to(DEV), dev_scales,
+                             torch.tensor([dec], dtype=torch.float32, device=DEV), mode)
+    return q, payload, scales
+
+
+@pytest.mark.parametrize("shape", [(128, 128, 256), (256, 384, 512), (384, 640, 1024)])
+@pytest.mark.parametrize("modes", [(0, 0), (0, 2), (1, 1), (2, 0), (1, 2)])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_gemm_random_codes(shape, modes, out_dtype):
+    Mo, No, Kc = shape
+    rng = np.random.default_rng(Mo + No + Kc + 7 * modes[0] + modes[1])
+    # scale codes around 1.0 keep sums of ~1e3 products comfortably inside FP32/BF16 range
+    qa, ap, asc = _operand(rng, Mo, Kc, modes[0], 0x40, 0xB0, dec=0.37)
+    qb, bp, bsc = _operand(rng, No, Kc, modes[1], 0x40, 0xB0, dec=1.0 / 2688.0)
+    out = lib.gemm(lib.FPROP, qa, qb, out_dtype)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    y, sa = oracle.gemm(ap, asc, modes[0] == 2, 0.37, bp, bsc, modes[1] == 2, np.float32(1.0 / 2688.0))
+    check_gemm_output(out, y, sa)
+
+
+def test_gemm_whole_code_range_including_subnormal_and_zero_scales():
+    rng = np.random.default_rng(5)
+    Mo, No, Kc = 128, 256, 256
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x00, 0xF8)
+    qb, bp, bsc = _operand(rng, No, Kc, 0, 0x00, 0x30)       # B small, so products stay finite
+    out = lib.gemm(lib.FPROP, qa, qb, torch.float32)
+    y, sa = oracle.gemm(ap, asc, False, 1.0, bp, bsc, False, 1.0)
+    check_gemm_output(out, y, sa)
+    # exactness of the BF16 reconstruction: one nonzero product per output
+    ap2 = np.zeros_like(ap); bp2 = np.zeros_like(bp)
+    ap2[:, 0] = rng.integers(0, 256, Mo, dtype=np.uint8) & 0x0F
+    bp2[:, 0] = rng.integers(0, 256, No, dtype=np.uint8) & 0x0F
+    qa.payload.copy_(torch.from_numpy(ap2)); qb.payload.copy_(torch.from_numpy(bp2))
+    out = lib.gemm(lib.FPROP, qa, qb, torch.float32)
+    y, _ = oracle.gemm(ap2, asc, False, 1.0, bp2, bsc, False, 1.0)
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), y)       # a single product has no rounding at all
+
+
+def test_small_forward_linear_fp32():
+    """M = N = K = 256 forward linear in FP32 with outlier activations and current-amax scales."""
+    X = si.outlier_activation(256, 256, seed=0, device=DEV)
+    W = si.weight(256, 256, seed=1, device=DEV, dtype=torch.float32)
+    ax, aw = lib.sample_amax(X), lib.sample_amax(W)
+    y, qx, qw = lib.linear_forward(X, W, ax, aw, 448.0, torch.float32)
+    torch.cuda.synchronize()
+    ox = oracle_quantize(X, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, oracle.amax(si.to_numpy_bits(X)))
+    ow = oracle_quantize(W, oracle.LAYOUT_2D, oracle.ROUND_RNE, oracle.amax(si.to_numpy_bits(W)), want_t=True)
+    assert np.array_equal(qx.payload.cpu().numpy(), ox["payload"]) and np.array_equal(qx.scales.cpu().numpy(), ox["scales"])
+    assert np.array_equal(qw.payload.cpu().numpy(), ow["payload"]) and np.array_equal(qw.scales.cpu().numpy(), ow["scales"])
+    r, c = np.unravel_index(np.abs(X.cpu().numpy()).argmax(), (256, 256))
+    assert ox["scales"][r, c // 16] == 0xBE                   # the block holding max|X| sits on the target 448
+    yr, sa = oracle.gemm(ox["payload"], ox["scales"], False, ox["decode"], ow["payload"], ow["scales"], True, ow["decode"])
+    check_gemm_output(y, yr, sa)
+    # and the quantized product is a fair approximation of the real one
+    exact = X.double().cpu().numpy() @ W.double().cpu().numpy().T
+    assert np.sqrt(np.mean((yr - exact) ** 2) / np.mean(exact ** 2)) < 0.25
+
+
+@pytest.mark.parametrize("scale_layout", [0, 1])
+def test_linear_forward_backward_small(scale_layout):
+    """fprop, dgrad and wgrad wiring on M = 512 tokens, K = 768, N = 384 (BF16, SR on dY)."""
+    M, K, N = 512, 768, 384
+    X = si.channel_scaled_activation(M, K, seed=2, device=DEV)
+    W = si.weight(N, K, seed=3, device=DEV)
+    dY = si.heavy_tailed_gradient(M, N, seed=4, device=DEV)
+    ax, aw, ag = lib.sample_amax(X), lib.sample_amax(W), lib.sample_amax(dY)
+    y, qx, qw = lib.linear_forward(X, W, ax, aw, scale_layout=scale_layout)
+    dx, dw = lib.linear_backward(dY, X, qw, ag, ax, seed=11, scale_layout=scale_layout)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    gx, gw, gg = (float(t.item()) for t in (ax, aw, ag))
+    ox = oracle_quantize(X, 0, 0, gx); ow = oracle_quantize(W, 2, 0, gw, want_t=True)
+    og = oracle_quantize(dY, 0, 1, gg, seed=44); ogt = oracle_quantize(dY, 1, 1, gg, seed=45); oxt = oracle_quantize(X, 1, 0, gx)
+    yr, sa = oracle.gemm(ox["payload"], ox["scales"], False, ox["decode"], ow["payload"], ow["scales"], True, ow["decode"])
+    check_gemm_output(y, yr, sa)
+    yr, sa = oracle.gemm(og["payload"], og["scales"], False, og["decode"], ow["payload_t"], ow["scales_t"], True, ow["decode"])
+    assert dx.shape == (M, K)
+    check_gemm_output(dx, yr, sa)
+    yr, sa = oracle.gemm(ogt["payload"], ogt["scales"], False, ogt["decode"], oxt["payload"], oxt["scales"], False, oxt["decode"])
+    assert dw.shape == (N, K)
+    check_gemm_output(dw, yr, sa)
+
+
+def test_gemm_rejects_bad_shapes():
+    rng = np.random.default_rng(1)
+    qa, *_ = _operand(rng, 128, 256, 0)
+    qb, *_ = _operand(rng, 128, 256, 0)
+    bad = lib.QuantizedOperand(qa.payload[:64], qa.scales[:64], qa.decode, 0)
+    with pytest.raises(lib.Ue5m3Error) as e:
+        lib.gemm(lib.FPROP, bad, qb)
+    assert e.value.status == 2
+    qc, *_ = _operand(rng, 128, 128, 0)
+    qd, *_ = _operand(rng, 128, 128, 0)
+    with pytest.raises(lib.Ue5m3Error) as e:
+        lib.gemm(lib.FPROP, qc, qd)
+    assert e.value.status == 2
