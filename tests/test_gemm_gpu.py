@@ -87,8 +87,8 @@ def test_small_forward_linear_fp32():
 
 @pytest.mark.parametrize("scale_layout", [0, 1])
 def test_linear_forward_backward_small(scale_layout):
-    """fprop, dgrad and wgrad wiring on M = 512 tokens, K = 768, N = 384 (BF16, SR on dY)."""
-    M, K, N = 512, 768, 384
+    """fprop, dgrad and wgrad wiring on M = 512 tokens, K = 768, N = 512 (BF16, SR on dY)."""
+    M, K, N = 512, 768, 512
     X = si.channel_scaled_activation(M, K, seed=2, device=DEV)
     W = si.weight(N, K, seed=3, device=DEV)
     dY = si.heavy_tailed_gradient(M, N, seed=4, device=DEV)
