@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the UE5M3-FP4 per-linear hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic input shaped like the
+8B-hybrid linears: tokens M = 8192, in-features K = 4096, out-features N = 16384, BF16:
+    quantize X (1D rows, RNE), W (2D tiles + transposed copy, RNE), dY (1D rows, SR), dY (1D columns, SR),
+    X (1D columns, RNE);  GEMMs fprop Y = X W^T, dgrad dX = dY W, wgrad dW = dY^T X;
+    tensor maxima are sampled at step 0 and held (re-sampled every 50 steps).
+The reported value is the whole-step rate in TFLOP/s (GEMM flops only: 3 * 2 M K N per step, the
+quantization time is inside the step).  The roofline object covers the dominant kernel (the GEMM);
+the `quantizer` object reports the streaming kernels against the HBM roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--sweep]
+
+With N > 1 (launched by torchrun) every rank runs the same workload on its own tokens: the path
+shards over tokens without any exchange, so scaling is "weak" and no collective is on the data path.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+`--sweep` prints the quantizer bandwidth sweep (2^20 .. 2^30 elements) instead of the step benchmark.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+M_TOK, K_IN, N_OUT = 8192, 4096, 16384
+WORKLOAD = "linear fwd+bwd M=8192 K=4096 N=16384 bf16 (fprop+dgrad+wgrad, 5 quantizations, SR on dY)"
+METRIC = "fwd+bwd block-scaled linear throughput (quantize + 3 GEMMs)"
+UNIT = "TFLOP/s"
+FLOPS_PER_STEP = 3 * 2 * M_TOK * K_IN * N_OUT
+
+
+def set_shape(m, k, n):
+    """Profiling aid: run the same step on another linear shape (the JSON line then names it)."""
+    global M_TOK, K_IN, N_OUT, WORKLOAD, FLOPS_PER_STEP, GEMM_FLOPS, KERNEL_BYTES
+    M_TOK, K_IN, N_OUT = m, k, n
+    WORKLOAD = f"NON-DEFAULT profiling shape: linear fwd+bwd M={m} K={k} N={n} bf16"
+    FLOPS_PER_STEP = 3 * 2 * m * k * n
+    GEMM_FLOPS = 2 * m * k * n
+    KERNEL_BYTES = kernel_bytes()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (the benchmark's cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+SAMPLE_M, SAMPLE_N = 256, 1024
+SAMPLE_DESC = (f"same linear cut to M={SAMPLE_M} tokens, K={K_IN}, N={SAMPLE_N}: 5 oracle quantizations + 3 exact "
+               "oracle GEMMs, all host threads")
+
+
+def oracle_sample_inputs():
+    import synth_inputs as si
+    X = si.to_numpy_bits(si.channel_scaled_activation(SAMPLE_M, K_IN, seed=1))
+    W = si.to_numpy_bits(si.weight(SAMPLE_N, K_IN, seed=2))
+    dY = si.to_numpy_bits(si.heavy_tailed_gradient(SAMPLE_M, SAMPLE_N, seed=3))
+    return X, W, dY
+
+
+def oracle_step(X, W, dY, g, seed):
+    import oracle
+    qx = oracle.quantize(X, 0, 0, g[0])
+    qw = oracle.quantize(W, 2, 0, g[1], want_t=True)
+    qg = oracle.quantize(dY, 0, 1, g[2], seed=4 * seed)
+    qgt = oracle.quantize(dY, 1, 1, g[2], seed=4 * seed + 1)
+    qxt = oracle.quantize(X, 1, 0, g[0])
+    oracle.gemm(qx["payload"], qx["scales"], False, qx["decode"], qw["payload"], qw["scales"], True, qw["decode"])
+    oracle.gemm(qg["payload"], qg["scales"], False, qg["decode"], qw["payload_t"], qw["scales_t"], True, qw["decode"])
+    oracle.gemm(qgt["payload"], qgt["scales"], False, qgt["decode"], qxt["payload"], qxt["scales"], False, qxt["decode"])
+
+
+def time_oracle(steps: int, warmup: int):
+    import oracle
+    X, W, dY = oracle_sample_inputs()
+    g = (oracle.amax(X), oracle.amax(W), oracle.amax(dY))
+    for s in range(warmup):
+        oracle_step(X, W, dY, g, s)
+    t0 = time.perf_counter()
+    for s in range(steps):
+        oracle_step(X, W, dY, g, warmup + s)
+    dt = (time.perf_counter() - t0) / steps
+    flops = 3 * 2 * SAMPLE_M * K_IN * SAMPLE_N
+    return flops / dt / 1e12, dt, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 3))
+    warmup = min(args.warmup, 1)
+    val, dt, cores = time_oracle(steps, warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int128 exact sum / f32 stepwise quantizer", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": SAMPLE_DESC},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": SAMPLE_DESC},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of this rank's GPU while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        import torch
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            self.gpu_id = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            self.gpu_id = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            cmd = ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.gpu_id:
+                cmd += ["-i", self.gpu_id]
+            self.proc = subprocess.Popen(cmd, stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    c = [v.strip() for v in line.split(",")]
+                    if len(c) < 7:
+                        continue
+                    try:
+                        sm.append(float(c[0])); mx.append(float(c[1])); pw.append(float(c[2]))
+                    except ValueError:
+                        continue
+                    for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[3:7]):
+                        if v.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(pw), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+class LinearStep:
+    """Pre-allocated buffers and the launch sequence of one fwd+bwd step."""
+    KERNELS = ("q_x_row", "q_w_2d", "gemm_fprop", "q_dy_row_sr", "gemm_dgrad", "q_dy_col_sr", "q_x_col", "gemm_wgrad")
+
+    def __init__(self, device, seed=0, scale_layout=0):
+        import torch
+        import paper_2609_02846_b200 as lib
+        import synth_inputs as si
+        self.torch, self.lib, self.dev = torch, lib, device
+        self.X = si.channel_scaled_activation(M_TOK, K_IN, seed=seed * 3 + 1, device=device)
+        self.W = si.weight(N_OUT, K_IN, seed=seed * 3 + 2, device=device)
+        self.dY = si.heavy_tailed_gradient(M_TOK, N_OUT, seed=seed * 3 + 3, device=device)
+        self.cx, self.cw, self.cg = lib.AmaxCache(50), lib.AmaxCache(50), lib.AmaxCache(50)
+        self.scale_layout = scale_layout
+        self.q = {}
+        self.Y = torch.empty((M_TOK, N_OUT), dtype=torch.bfloat16, device=device)
+        self.dX = torch.empty((M_TOK, K_IN), dtype=torch.bfloat16, device=device)
+        self.dW = torch.empty((N_OUT, K_IN), dtype=torch.bfloat16, device=device)
+        self.launches = 0
+
+    def _timed(self, name, fn, ev):
+        if ev is None:
+            return fn()
+        a, b = self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+        a.record()
+        r = fn()
+        b.record()
+        ev.setdefault(name, []).append((a, b))
+        return r
+
+    def run(self, step, ev=None):
+        lib = self.lib
+        refresh = self.cx.refreshes_at(step)
+        gx, gw, gg = self.cx.get(self.X, step), self.cw.get(self.W, step), self.cg.get(self.dY, step)
+        self.launches += 3 if refresh else 0
+        sl = self.scale_layout
+        q = self.q
+        q["x"] = self._timed("q_x_row", lambda: lib.quantize(self.X, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, gx, 448.0,
+                                                             scale_layout=sl, out=q.get("x")), ev)
+        q["w"] = self._timed("q_w_2d", lambda: lib.quantize(self.W, lib.LAYOUT_2D, lib.ROUND_RNE, gw, 448.0,
+                                                            want_transpose=True, out=q.get("w")), ev)
+        self._timed("gemm_fprop", lambda: lib.gemm(lib.FPROP, q["x"], q["w"], out=self.Y), ev)
+        q["g"] = self._timed("q_dy_row_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_ROW, lib.ROUND_SR, gg, 448.0,
+                                                                 seed=4 * step, scale_layout=sl, out=q.get("g")), ev)
+        self._timed("gemm_dgrad", lambda: lib.gemm(lib.DGRAD, q["g"], q["w"].transposed(), out=self.dX), ev)
+        q["gt"] = self._timed("q_dy_col_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, 448.0,
+                                                                  seed=4 * step + 1, scale_layout=sl, out=q.get("gt")), ev)
+        q["xt"] = self._timed("q_x_col", lambda: lib.quantize(self.X, lib.LAYOUT_1D_COL, lib.ROUND_RNE, gx, 448.0,
+                                                              scale_layout=sl, out=q.get("xt")), ev)
+        self._timed("gemm_wgrad", lambda: lib.gemm(lib.WGRAD, q["gt"], q["xt"], out=self.dW), ev)
+        self.launches += 8
+
+
+# algorithmic bytes of each streaming kernel per launch (BF16 in, payload + scales out)
+def _quant_bytes(rows, cols, layout, transposed_copy=False):
+    n = rows * cols
+    if layout == 2:
+        return n * 2 + n // 2 * (2 if transposed_copy else 1) + n // 256 * (2 if transposed_copy else 1)
+    return n * 2 + n // 2 + n // 16
+
+
+def kernel_bytes():
+    return {
+        "q_x_row": _quant_bytes(M_TOK, K_IN, 0), "q_x_col": _quant_bytes(M_TOK, K_IN, 1),
+        "q_w_2d": _quant_bytes(N_OUT, K_IN, 2, True),
+        "q_dy_row_sr": _quant_bytes(M_TOK, N_OUT, 0), "q_dy_col_sr": _quant_bytes(M_TOK, N_OUT, 1),
+    }
+
+
+KERNEL_BYTES = kernel_bytes()
+GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    import paper_2609_02846_b200 as lib
+    peaks = measured_peaks()
+    step = LinearStep(dev, seed=rank, scale_layout=args.scale_layout)
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    for s in range(Wm):
+        step.run(s)
+    barrier()
+    launches0 = step.launches
+    sampler = ClockSampler(dev)
+    sampler.start()
+    ev = {}
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0.record()
+    for s in range(K):
+        step.run(Wm + s, ev)
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t0.elapsed_time(t1)
+    status = lib.last_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {lib.status_string(status)}")
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    value = world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e12
+    gpu_launches = step.launches - launches0
+
+    per_kernel = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in ev.items()}
+    gemm_ms = statistics.mean(per_kernel[k] for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad"))
+    gemm_tflops = GEMM_FLOPS / (gemm_ms * 1e-3) / 1e12
+    quant = {}
+    qbytes = qms = 0.0
+    for k, nbytes in KERNEL_BYTES.items():
+        gbs = nbytes / (per_kernel[k] * 1e-3) / 1e9
+        quant[k] = {"ms": round(per_kernel[k], 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+        qbytes += nbytes
+        qms += per_kernel[k]
+    quant["all"] = {"ms": round(qms, 4), "GB/s": round(qbytes / (qms * 1e-3) / 1e9, 1),
+                    "frac_of_measured_hbm": round(qbytes / (qms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
+
+    # ---- end to end: host buffers in, results back to the host, every step ----
+    e2e = None
+    if rank == 0 or world > 1:
+        Xh, Wh, dYh = (t.cpu().pin_memory() for t in (step.X, step.W, step.dY))
+        Yh, dXh, dWh = (torch.empty_like(t, device="cpu").pin_memory() for t in (step.Y, step.dX, step.dW))
+        n_e2e = max(1, min(K, 5))
+
+        def e2e_step(s):
+            step.X.copy_(Xh, non_blocking=True); step.W.copy_(Wh, non_blocking=True); step.dY.copy_(dYh, non_blocking=True)
+            step.run(s)
+            Yh.copy_(step.Y, non_blocking=True); dXh.copy_(step.dX, non_blocking=True); dWh.copy_(step.dW, non_blocking=True)
+
+        e2e_step(Wm + K)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for s in range(n_e2e):
+            e2e_step(Wm + K + 1 + s)
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e_ms /= n_e2e
+        h2d = sum(t.numel() * t.element_size() for t in (Xh, Wh, dYh))
+        d2h = sum(t.numel() * t.element_size() for t in (Yh, dXh, dWh))
+        e2e = {"value": world * FLOPS_PER_STEP / (e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e_ms, "steps": n_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            v, dt, cores = time_oracle(1, 0)
+            cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": SAMPLE_DESC, "seconds": round(dt, 2)}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_gpu": M_TOK, "l2": f"inputs ({2 * (M_TOK * K_IN + N_OUT * K_IN + M_TOK * N_OUT) >> 20} MiB per step) exceed the 126 MB L2",
+                       "scale_layout": "tiled" if args.scale_layout else "rowmajor", "amax": "sampled at step 0, held 50 steps"},
+            "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": gemm_tflops,
+                         "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": gemm_tflops / peaks["bf16_tflops_sustained"],
+                         "frac_of_burst_peak": gemm_tflops / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained)",
+                         "avg_launch_ms": gemm_ms, "traffic": None,
+                         "per_gemm_ms": {k: round(per_kernel[k], 4) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}},
+            "quantizer": quant,
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_sweep(args):
+    """Quantizer-only bandwidth sweep: BF16 [rows, 4096], 2^20 .. 2^30 elements, {1D, 2D} x {RNE, SR} + amax."""
+    import torch
+    import paper_2609_02846_b200 as lib
+    import synth_inputs as si
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = []
+    for log2n in range(20, 31, args.sweep_stride):
+        rows = (1 << log2n) // 4096
+        x = si.row_scaled_tensor(rows, 4096, seed=log2n, device=dev)
+        g = lib.sample_amax(x)
+        cells = {"amax": (lambda: lib.sample_amax(x, g), rows * 4096 * 2)}
+        for lname, layout in (("1d_row", 0), ("1d_col", 1), ("2d", 2)):
+            for rname, rnd in (("rne", 0), ("sr", 1)):
+                q = lib.quantize(x, layout, rnd, g, seed=1)
+                cells[f"{lname}_{rname}"] = ((lambda layout=layout, rnd=rnd, q=q: lib.quantize(x, layout, rnd, g, seed=1, out=q)),
+                                             _quant_bytes(rows, 4096, layout))
+        row = {"log2_elements": log2n}
+        for name, (fn, nbytes) in cells.items():
+            for _ in range(3):
+                fn()
+            ts = []
+            for _ in range(args.sweep_iters):
+                if nbytes < (256 << 20):
+                    flush.zero_()                      # inputs that fit in L2: flush it between timed launches
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            ms = statistics.median(ts)
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+        out.append(row)
+        print(json.dumps(row), flush=True)
+        del x
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scale-layout", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sweep-iters", type=int, default=20)
+    ap.add_argument("--sweep-stride", type=int, default=2)
+    ap.add_argument("--shape", default=None, help="M,K,N override for profiling runs (not the benchmark workload)")
+    args = ap.parse_args()
+    if args.shape:
+        set_shape(*(int(v) for v in args.shape.split(",")))
+    if args.impl == "reference":
+        run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
