@@ -92,7 +92,7 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
     if ((reinterpret_cast<uintptr_t>(amax_held) & 3u) || (reinterpret_cast<uintptr_t>(decode_out) & 3u) ||
         (reinterpret_cast<uintptr_t>(stats) & 7u))
         return UE5M3_ERR_ALIGN;
-    if (rows * (cols / 16) >= ((int64_t)1 << 31) * 256) return UE5M3_ERR_UNSUPPORTED;
+    if (rows * (cols / 16) >= ((int64_t)1 << 32) - 256) return UE5M3_ERR_UNSUPPORTED;   // 32-bit block index
     const DeviceInfo di = device_info();
     if (!di.ok) return UE5M3_ERR_CUDA;
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;

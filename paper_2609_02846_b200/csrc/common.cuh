@@ -66,18 +66,23 @@ __device__ __forceinline__ uint32_t e2m1x2_rne(float lo, float hi) {
     return (uint32_t)p;
 }
 
-// Stochastic rounding of one value with a 16-bit draw (Eq. "sr").  |z| is clamped to 6 (NaN -> +6),
-// [0,1) is moved to [1,2) so that on every binade exactly the top fraction bit is kept, the draw is
-// added below that bit (centred by 32) and the rest is truncated.
-__device__ __forceinline__ uint32_t e2m1_sr(float z, uint32_t r16) {
-    const float zc = fmaxf(fminf(z, 6.0f), -6.0f);
-    const float a = fabsf(zc);
-    const bool sub = a < 1.0f;
-    const float b = sub ? __fadd_rn(a, 1.0f) : a;
-    const uint32_t Bp = __float_as_uint(b) + (r16 << 6) + 32u;
-    const uint32_t mag = (Bp >> 22) - (sub ? 0xFEu : 0xFCu);
-    return ((__float_as_uint(zc) >> 28) & 8u) | mag;
+// Stochastic rounding with a 16-bit draw per value (Eq. "sr").  |z| is clamped to 6 (NaN -> +6).  On
+// every binade of [1,8) the E2M1 grid keeps exactly the top fraction bit; [0,1) has the same step as
+// [1,2) and is folded onto the binade [1/2,1) by b = a/2 + 1/2 (one rounding, the same bits as a + 1 one
+// exponent lower), so that in all cases  code = (bits(b) + draw * 2^6 + 2^5) >> 22  minus one common
+// offset.  sr_accumulate adds element j (0..7) of a group to the packed magnitude and sign words.
+__device__ __forceinline__ void sr_accumulate(float z, uint32_t word, int j, uint32_t& mags, uint32_t& signs) {
+    const float t = fminf(z, 6.0f);                       // NaN -> +6, sign of everything else kept
+    const float a = fminf(fabsf(t), 6.0f);
+    const float b = (a < 1.0f) ? __fmaf_rn(a, 0.5f, 0.5f) : a;
+    const uint32_t r = (j & 1) ? (word >> 10) : (word << 6);           // draw * 2^6 ...
+    const uint32_t Bp = __float_as_uint(b) + ((r & 0x3FFFC0u) | 32u);  // ... + 2^5, added below the kept bit
+    // bits 24:22 of Bp are the magnitude code plus 4 (mod 8); bit 31 of t is the sign
+    const uint32_t m = (22 - 4 * j >= 0) ? (Bp >> (22 - 4 * j)) : (Bp << (4 * j - 22));
+    mags |= m & (7u << (4 * j));
+    signs |= (__float_as_uint(t) >> (28 - 4 * j)) & (8u << (4 * j));
 }
+__device__ __forceinline__ uint32_t sr_finish(uint32_t mags, uint32_t signs) { return (mags ^ 0x44444444u) | signs; }
 
 // Philox4x32-10 (Salmon et al. 2011).
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
@@ -99,9 +104,6 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 // Random bits of the 8 source elements whose logical index i has i >> 3 == group.
 __device__ __forceinline__ void sr_bits8(uint64_t seed, uint64_t group, uint32_t w[4]) {
     philox4x32_10((uint32_t)group, (uint32_t)(group >> 32), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), w);
-}
-__device__ __forceinline__ uint32_t sr_lane(const uint32_t w[4], int j) {   // j = i & 7
-    return (w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
 }
 
 // ---------------------------------------------------------------------------------------

@@ -44,8 +44,10 @@ __device__ __forceinline__ uint32_t encode8(const float f[8], float rB, const ui
     for (int j = 0; j < 8; ++j) clip += (fabsf(z[j]) > 6.0f) ? 1u : 0u;
     uint32_t out = 0;
     if (SR) {
+        uint32_t mags = 0, signs = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) out |= e2m1_sr(z[j], sr_lane(w, j)) << (4 * j);
+        for (int j = 0; j < 8; ++j) sr_accumulate(z[j], w[j >> 1], j, mags, signs);
+        out = sr_finish(mags, signs);
     } else {
 #pragma unroll
         for (int j = 0; j < 4; ++j) out |= e2m1x2_rne(z[2 * j], z[2 * j + 1]) << (8 * j);
@@ -56,22 +58,31 @@ __device__ __forceinline__ uint32_t encode8(const float f[8], float rB, const ui
 // ---------------------------------------------------------------------------------------
 // 1D blocks along the contiguous dimension
 // ---------------------------------------------------------------------------------------
+// Tensor constants are computed once per CTA (three IEEE divisions) and broadcast through shared memory.
+__device__ __forceinline__ TensorConsts cta_tensor_consts(const float* amax_held, float T) {
+    __shared__ TensorConsts s_tc;
+    if (threadIdx.x == 0) s_tc = tensor_consts(__ldg(amax_held), T);
+    __syncthreads();
+    return s_tc;
+}
+
 template <bool IS_BF16, bool SR, bool STATS, bool TILED>
-__global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a) {
-    const TensorConsts tc = tensor_consts(__ldg(a.amax_held), a.T);
+__global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a, int kb_shift) {
+    const TensorConsts tc = cta_tensor_consts(a.amax_held, a.T);
     const uint32_t kbpr = (uint32_t)(a.cols >> 4);
-    const uint64_t nblocks = (uint64_t)a.rows * kbpr;
-    const uint64_t idx = (uint64_t)blockIdx.x * kRowThreads + threadIdx.x;
+    const uint32_t nblocks = (uint32_t)a.rows * kbpr;          // the launcher guarantees < 2^32 blocks
+    const uint32_t idx = blockIdx.x * kRowThreads + threadIdx.x;
     if (idx == 0 && a.decode_out) *a.decode_out = tc.d;
     const bool live = idx < nblocks;
-    const uint64_t idc = live ? idx : 0;
-    const uint64_t row = idc / kbpr;
-    const uint32_t kb = (uint32_t)(idc - row * kbpr);
+    const uint32_t idc = live ? idx : 0;
+    // blocks per row is a power of two for the usual widths: shift instead of divide
+    const uint32_t row = (kb_shift >= 0) ? (idc >> kb_shift) : (idc / kbpr);
+    const uint32_t kb = idc - row * kbpr;
 
     float f[16];
     float aB = 0.0f;
     if (IS_BF16) {
-        const uint16_t* p = reinterpret_cast<const uint16_t*>(a.x) + row * a.ld + (uint64_t)kb * 16;
+        const uint16_t* p = reinterpret_cast<const uint16_t*>(a.x) + (int64_t)row * a.ld + kb * 16;
         const uint4 v0 = ldg_nc_v4(p), v1 = ldg_nc_v4(p + 8);
         uint32_t m = bf16x2_absmax(0u, v0.x);
         m = bf16x2_absmax(m, v0.y); m = bf16x2_absmax(m, v0.z); m = bf16x2_absmax(m, v0.w);
@@ -80,7 +91,7 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a) 
         unpack_bf16x8(v0, f);
         unpack_bf16x8(v1, f + 8);
     } else {
-        const float* p = reinterpret_cast<const float*>(a.x) + row * a.ld + (uint64_t)kb * 16;
+        const float* p = reinterpret_cast<const float*>(a.x) + (int64_t)row * a.ld + kb * 16;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint4 v = ldg_nc_v4(p + 4 * q);
@@ -97,7 +108,7 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a) 
 
     uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};
     if (SR) {
-        const uint64_t g0 = (row * (uint64_t)a.cols + (uint64_t)kb * 16) >> 3;
+        const uint64_t g0 = ((uint64_t)row * (uint64_t)a.cols + (uint64_t)kb * 16) >> 3;
         sr_bits8(a.seed, g0, w0);
         sr_bits8(a.seed, g0 + 1, w1);
     }
@@ -106,7 +117,7 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a) 
     out.x = encode8<SR>(f, rB, w0, clip);
     out.y = encode8<SR>(f + 8, rB, w1, clip);
 
-    if (live) *reinterpret_cast<uint2*>(a.payload + idx * 8) = out;
+    if (live) *reinterpret_cast<uint2*>(a.payload + (uint64_t)idx * 8) = out;
 
     if (TILED) {
         if (live) a.scales[tiled_scale_offset((int64_t)row, kb, kbpr)] = (uint8_t)code;
@@ -154,7 +165,7 @@ template <bool IS_BF16, bool SR, bool STATS, int MODE, bool TILED, bool WANT_T>
 __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a) {
     __shared__ __align__(16) uint8_t s_t[(MODE == 1 && WANT_T) ? kTileCols * (kTileRows / 2) : 16];
 
-    const TensorConsts tc = tensor_consts(__ldg(a.amax_held), a.T);
+    const TensorConsts tc = cta_tensor_consts(a.amax_held, a.T);
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tc.d;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -240,8 +251,10 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
         for (int j = 0; j < 8; ++j) clip += (fabsf(z[j]) > 6.0f) ? 1u : 0u;
         uint32_t o = 0;
         if (SR) {
+            uint32_t mags = 0, signs = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) o |= e2m1_sr(z[j], sr_lane(w, j)) << (4 * j);
+            for (int j = 0; j < 8; ++j) sr_accumulate(z[j], w[j >> 1], j, mags, signs);
+            o = sr_finish(mags, signs);
         } else {
 #pragma unroll
             for (int j = 0; j < 4; ++j) o |= e2m1x2_rne(z[2 * j], z[2 * j + 1]) << (8 * j);
@@ -389,8 +402,11 @@ template <bool IS_BF16, bool SR, bool STATS>
 static cudaError_t launch_row(const QuantArgs& a, bool tiled, cudaStream_t st) {
     const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
     const unsigned grid = (unsigned)((nblocks + kRowThreads - 1) / kRowThreads);
-    if (tiled) quantize_row_kernel<IS_BF16, SR, STATS, true><<<grid, kRowThreads, 0, st>>>(a);
-    else       quantize_row_kernel<IS_BF16, SR, STATS, false><<<grid, kRowThreads, 0, st>>>(a);
+    const uint64_t kbpr = (uint64_t)(a.cols >> 4);
+    int kb_shift = -1;
+    if ((kbpr & (kbpr - 1)) == 0) { kb_shift = 0; while ((1ull << kb_shift) < kbpr) ++kb_shift; }
+    if (tiled) quantize_row_kernel<IS_BF16, SR, STATS, true><<<grid, kRowThreads, 0, st>>>(a, kb_shift);
+    else       quantize_row_kernel<IS_BF16, SR, STATS, false><<<grid, kRowThreads, 0, st>>>(a, kb_shift);
     return cudaGetLastError();
 }
 
