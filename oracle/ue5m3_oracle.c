@@ -253,7 +253,11 @@ static void put_nibble(uint8_t *payload, int64_t row_bytes, int64_t r, int64_t k
 /* One block: members are source positions (r0 + i*dr_i..., see callers). */
 typedef struct { int64_t r, c; } pos_t;
 
-static void quantize_block(const void *x, int dtype, int64_t cols, int64_t ld,
+/* A call may describe a WINDOW of a larger logical tensor: the window's element (r, c) is element
+ * (row0 + r, col0 + c) of a tensor with full_cols columns.  Only the stochastic-rounding index sees this. */
+typedef struct { int64_t full_cols, row0, col0; } window_t;
+
+static void quantize_block(const void *x, int dtype, window_t win, int64_t ld,
                            const pos_t *mem, int n, float S, float G, int rounding, uint64_t seed,
                            int *codes_out, int *scale_code_out, uint64_t stats[4])
 {
@@ -278,7 +282,7 @@ static void quantize_block(const void *x, int dtype, int64_t cols, int64_t ld,
         float z = v * rB;                               /* x_i / (g s_hat), with G = TF/g folded in */
         if (fabsf(z) > 6.0f) stats[STAT_PAYLOAD_CLIPPED]++;
         if (rounding == ROUND_SR) {
-            uint64_t idx = (uint64_t)mem[i].r * (uint64_t)cols + (uint64_t)mem[i].c;
+            uint64_t idx = (uint64_t)(win.row0 + mem[i].r) * (uint64_t)win.full_cols + (uint64_t)(win.col0 + mem[i].c);
             codes_out[i] = oracle_e2m1_encode_sr(z, oracle_sr_bits(seed, idx));
         } else {
             codes_out[i] = oracle_e2m1_encode_rne(z);
@@ -297,13 +301,16 @@ static void quantize_block(const void *x, int dtype, int64_t cols, int64_t ld,
  *                payload_t [cols, rows/2], scales_t [cols/16, rows/16].
  * Returns 0, or -1 for shapes that are not multiples of 16.
  */
-ORACLE_API int oracle_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
-                               int layout, int rounding, float g, float T, uint64_t seed,
-                               uint8_t *payload, uint8_t *scales,
-                               uint8_t *payload_t, uint8_t *scales_t,
-                               float *decode_out, uint64_t *stats_out)
+ORACLE_API int oracle_quantize_window(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                                      int layout, int rounding, float g, float T, uint64_t seed,
+                                      int64_t full_cols, int64_t row0, int64_t col0,
+                                      uint8_t *payload, uint8_t *scales,
+                                      uint8_t *payload_t, uint8_t *scales_t,
+                                      float *decode_out, uint64_t *stats_out)
 {
     if (rows <= 0 || cols <= 0 || (rows % 16) || (cols % 16)) return -1;
+    if ((row0 % 16) || (col0 % 16) || row0 < 0 || col0 < 0 || col0 + cols > full_cols) return -1;
+    window_t win = { full_cols, row0, col0 };
     float g_eff, S, G, d;
     oracle_tensor_constants(g, T, &g_eff, &S, &G, &d);
     if (decode_out) *decode_out = d;
@@ -317,7 +324,7 @@ ORACLE_API int oracle_quantize(const void *x, int dtype, int64_t rows, int64_t c
             for (int64_t kb = 0; kb < cols / 16; ++kb) {
                 pos_t mem[16]; int codes[16]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
                 for (int j = 0; j < 16; ++j) { mem[j].r = r; mem[j].c = 16 * kb + j; }
-                quantize_block(x, dtype, cols, ld, mem, 16, S, G, rounding, seed, codes, &sc, stats);
+                quantize_block(x, dtype, win, ld, mem, 16, S, G, rounding, seed, codes, &sc, stats);
                 s0 += stats[0]; s1 += stats[1]; s2 += stats[2]; s3 += stats[3];
                 scales[r * (cols / 16) + kb] = (uint8_t)sc;
                 for (int j = 0; j < 16; ++j) put_nibble(payload, cols / 2, r, 16 * kb + j, codes[j]);
@@ -328,7 +335,7 @@ ORACLE_API int oracle_quantize(const void *x, int dtype, int64_t rows, int64_t c
             for (int64_t rb = 0; rb < rows / 16; ++rb) {
                 pos_t mem[16]; int codes[16]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
                 for (int j = 0; j < 16; ++j) { mem[j].r = 16 * rb + j; mem[j].c = c; }
-                quantize_block(x, dtype, cols, ld, mem, 16, S, G, rounding, seed, codes, &sc, stats);
+                quantize_block(x, dtype, win, ld, mem, 16, S, G, rounding, seed, codes, &sc, stats);
                 s0 += stats[0]; s1 += stats[1]; s2 += stats[2]; s3 += stats[3];
                 scales[c * (rows / 16) + rb] = (uint8_t)sc;
                 for (int j = 0; j < 16; ++j) put_nibble(payload, rows / 2, c, 16 * rb + j, codes[j]);
@@ -340,7 +347,7 @@ ORACLE_API int oracle_quantize(const void *x, int dtype, int64_t rows, int64_t c
                 pos_t mem[256]; int codes[256]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
                 for (int i = 0; i < 16; ++i)
                     for (int j = 0; j < 16; ++j) { mem[16 * i + j].r = 16 * rb + i; mem[16 * i + j].c = 16 * cb + j; }
-                quantize_block(x, dtype, cols, ld, mem, 256, S, G, rounding, seed, codes, &sc, stats);
+                quantize_block(x, dtype, win, ld, mem, 256, S, G, rounding, seed, codes, &sc, stats);
                 s0 += stats[0]; s1 += stats[1]; s2 += stats[2]; s3 += stats[3];
                 scales[rb * (cols / 16) + cb] = (uint8_t)sc;
                 if (scales_t) scales_t[cb * (rows / 16) + rb] = (uint8_t)sc;
@@ -355,6 +362,17 @@ ORACLE_API int oracle_quantize(const void *x, int dtype, int64_t rows, int64_t c
     }
     if (stats_out) { stats_out[0] = s0; stats_out[1] = s1; stats_out[2] = s2; stats_out[3] = s3; }
     return 0;
+}
+
+/* The whole tensor is the window at (0, 0). */
+ORACLE_API int oracle_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                               int layout, int rounding, float g, float T, uint64_t seed,
+                               uint8_t *payload, uint8_t *scales,
+                               uint8_t *payload_t, uint8_t *scales_t,
+                               float *decode_out, uint64_t *stats_out)
+{
+    return oracle_quantize_window(x, dtype, rows, cols, ld, layout, rounding, g, T, seed, cols, 0, 0,
+                                  payload, scales, payload_t, scales_t, decode_out, stats_out);
 }
 
 /* Reconstruction x_hat = d * s_hat * q (Eq. "microscaling" with the tensor

@@ -14,7 +14,7 @@
 //   warp 2        tensor-memory allocation
 //   warps 4-7     epilogue: tcgen05.ld, scale, convert, store (overlaps the next tile's main loop
 //                 through two 256-column accumulators)
-//   warps 8-15    dequantizers: packed smem -> BF16 smem in the 128B-swizzled K-major UMMA layout
+//   warps 8-23    dequantizers: packed smem -> BF16 smem in the 128B-swizzled K-major UMMA layout
 // Every wait is bounded; a wait that gives up sets the device status word and the CTA drains.
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -32,8 +32,9 @@ constexpr int BM = 128, BN = 256;
 constexpr int KCHUNK = 256;                 // K per packed stage
 constexpr int KSUB = 64;                    // K per BF16 stage (one 128-byte swizzle row)
 constexpr int PK_STAGES = 2, BF_STAGES = 2;
-constexpr int NUM_THREADS = 512;
-constexpr int DEQ_WARP0 = 8, DEQ_WARPS = 8, EPI_WARP0 = 4;
+constexpr int DEQ_WARP0 = 8, DEQ_WARPS = 16, EPI_WARP0 = 4;
+constexpr int NUM_THREADS = 32 * (DEQ_WARP0 + DEQ_WARPS);
+constexpr int DEQ_TASKS = 48 / DEQ_WARPS;      // 8-row groups (16 of A, 32 of B) per dequantizer warp and 64-wide slice
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;        // 16384
 constexpr int PK_B_BYTES = BN * KCHUNK / 2;        // 32768
@@ -352,12 +353,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const uint8_t* st = smem_gen + ps * PK_STAGE_BYTES;
 #pragma unroll 1
                 for (int sub = 0; sub < KCHUNK / KSUB; ++sub, ++it_bf) {
-                    // gather this thread's six blocks of the 64-wide slice
-                    uint2 pay[6];
-                    uint32_t code[6];
+                    // gather this thread's blocks of the 64-wide slice
+                    uint2 pay[DEQ_TASKS];
+                    uint32_t code[DEQ_TASKS];
 #pragma unroll
-                    for (int t = 0; t < 6; ++t) {
-                        const int rg = dw + 8 * t;                  // 8-row group: 0..15 are A, 16..47 are B
+                    for (int t = 0; t < DEQ_TASKS; ++t) {
+                        const int rg = dw + DEQ_WARPS * t;          // 8-row group: 0..15 are A, 16..47 are B
                         const bool isA = rg < 16;
                         const int row = (isA ? rg : rg - 16) * 8 + r7;
                         const uint8_t* pk = st + (isA ? 0 : PK_A_BYTES) + row * 128 + ((((sub << 1) | (j >> 1)) ^ r7) << 4) + ((j & 1) << 3);
@@ -369,8 +370,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     if (!mbar_wait(bf_empty + 8 * bs, bph ^ 1, abort_flag)) { ok = false; break; }
                     uint8_t* bf = smem_gen + PK_STAGES * PK_STAGE_BYTES + bs * BF_STAGE_BYTES;
 #pragma unroll
-                    for (int t = 0; t < 6; ++t) {
-                        const int rg = dw + 8 * t;
+                    for (int t = 0; t < DEQ_TASKS; ++t) {
+                        const int rg = dw + DEQ_WARPS * t;
                         const bool isA = rg < 16;
                         const int row = (isA ? rg : rg - 16) * 8 + r7;
                         const uint32_t m = scale_pair(code[t]);

@@ -585,3 +585,24 @@ def test_bf16_rne_matches_library_conversion():
     # a binary64 value just above a BF16 tie must round up even though its float32 rounding is the tie
     tie = 1.0 + 2.0 ** -8
     assert oracle.bf16_rne(tie) == 0x3F80 and oracle.bf16_rne(tie + 2.0 ** -40) == 0x3F81
+
+
+def test_window_calls_reproduce_the_full_tensor():
+    """A window of a larger tensor draws the SR bits of its own source indices, so quantizing windows
+    must reproduce the corresponding bytes of the full-tensor call in every layout."""
+    rng = np.random.default_rng(43)
+    x = rng.normal(0, 1, (64, 96)).astype(np.float32)
+    g = np.abs(x).max()
+    full = {l: oracle.quantize(x, l, oracle.ROUND_SR, g, 448.0, seed=5, want_t=True) for l in (0, 1, 2)}
+    r0, c0, nr, nc = 16, 32, 32, 48
+    win = np.ascontiguousarray(x[r0:r0 + nr, c0:c0 + nc])
+    w = {l: oracle.quantize(win, l, oracle.ROUND_SR, g, 448.0, seed=5, want_t=True, window=(96, r0, c0)) for l in (0, 1, 2)}
+    assert np.array_equal(w[0]["payload"], full[0]["payload"][r0:r0 + nr, c0 // 2:(c0 + nc) // 2])
+    assert np.array_equal(w[0]["scales"], full[0]["scales"][r0:r0 + nr, c0 // 16:(c0 + nc) // 16])
+    assert np.array_equal(w[1]["payload"], full[1]["payload"][c0:c0 + nc, r0 // 2:(r0 + nr) // 2])
+    assert np.array_equal(w[1]["scales"], full[1]["scales"][c0:c0 + nc, r0 // 16:(r0 + nr) // 16])
+    assert np.array_equal(w[2]["payload"], full[2]["payload"][r0:r0 + nr, c0 // 2:(c0 + nc) // 2])
+    assert np.array_equal(w[2]["payload_t"], full[2]["payload_t"][c0:c0 + nc, r0 // 2:(r0 + nr) // 2])
+    # without the window the draws differ
+    plain = oracle.quantize(win, 0, oracle.ROUND_SR, g, 448.0, seed=5)
+    assert not np.array_equal(plain["payload"], w[0]["payload"])
