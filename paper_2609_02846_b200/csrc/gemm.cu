@@ -8,13 +8,20 @@
 // FP32 accumulators in tensor memory.  The factor 2^-32 and the tensor decode factors are applied
 // to the accumulator in the epilogue.
 //
-// One persistent CTA per SM, warp specialised:
+// Persistent, one CTA per SM, CTAs paired into clusters of two that share one 256 x 256 output tile
+// (tcgen05 cta_group::2): each CTA owns 128 rows of A and 128 of the 256 B rows, so it stages and
+// dequantizes 128 + 128 rows per K slice for a 128 x 256 accumulator of its own.  Warp roles per CTA:
 //   warp 0        TMA producer: packed payload tiles (128B-swizzled) and scale tiles, 256 K per stage
-//   warp 1        MMA issuer: 4 x tcgen05.mma (M128 N256 K16) per 64-wide BF16 stage
+//   warp 1        MMA issuer (leader CTA only): 4 x tcgen05.mma (M256 N256 K16) per 64-wide BF16 stage
 //   warp 2        tensor-memory allocation
 //   warps 4-7     epilogue: tcgen05.ld, scale, convert, store (overlaps the next tile's main loop
 //                 through two 256-column accumulators)
-//   warps 8-23    dequantizers: packed smem -> BF16 smem in the 128B-swizzled K-major UMMA layout
+//   warps 8-23    dequantizers: packed smem -> BF16 smem in the 128B-swizzled K-major UMMA layout.  Four
+//                 groups of four warps; group g converts the g-th 64-wide slice of every packed stage into
+//                 BF16 stage g, so four slices are in flight and no group waits for another.
+// The leader learns that both CTAs' BF16 stages are full through one mbarrier that the partner's
+// dequantizers arrive on remotely; stage and accumulator releases come back to both CTAs through
+// tcgen05.commit with a two-CTA multicast mask.  No copy is multicast: every CTA loads its own tiles.
 // Every wait is bounded; a wait that gives up sets the device status word and the CTA drains.
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -28,23 +35,28 @@ __device__ int g_device_status = 0;
 
 namespace {
 
-constexpr int BM = 128, BN = 256;
+constexpr int BM = 128;                     // A rows per CTA (256 per CTA pair)
+constexpr int BN = 256;                     // output columns per tile
+constexpr int BNH = 128;                    // B rows staged by each CTA of the pair
 constexpr int KCHUNK = 256;                 // K per packed stage
 constexpr int KSUB = 64;                    // K per BF16 stage (one 128-byte swizzle row)
-constexpr int PK_STAGES = 2, BF_STAGES = 2;
+constexpr int PK_STAGES = 2;
+constexpr int BF_STAGES = KCHUNK / KSUB;    // 4: one BF16 stage per 64-wide slice of a packed stage
 constexpr int DEQ_WARP0 = 8, DEQ_WARPS = 16, EPI_WARP0 = 4;
+constexpr int DEQ_GROUPS = BF_STAGES;       // dequantizer group g owns slice g of every packed stage and BF16 stage g
+constexpr int GROUP_WARPS = DEQ_WARPS / DEQ_GROUPS;
 constexpr int NUM_THREADS = 32 * (DEQ_WARP0 + DEQ_WARPS);
-constexpr int DEQ_TASKS = 48 / DEQ_WARPS;      // 8-row groups (16 of A, 32 of B) per dequantizer warp and 64-wide slice
+constexpr int DEQ_TASKS = 32 / GROUP_WARPS;    // 8-row groups (16 of A, 16 of B) per warp and slice
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;        // 16384
-constexpr int PK_B_BYTES = BN * KCHUNK / 2;        // 32768
+constexpr int PK_B_BYTES = BNH * KCHUNK / 2;       // 16384
 constexpr int SC_A_BYTES = BM * (KCHUNK / 16);     // 2048
-constexpr int SC_B_BYTES = BN * (KCHUNK / 16);     // 4096
-constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES;   // 55296
+constexpr int SC_B_BYTES = BNH * (KCHUNK / 16);    // 2048
+constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES;   // 36864
 constexpr int BF_A_BYTES = BM * KSUB * 2;          // 16384
-constexpr int BF_B_BYTES = BN * KSUB * 2;          // 32768
-constexpr int BF_STAGE_BYTES = BF_A_BYTES + BF_B_BYTES;                              // 49152
-constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;  // 208896
+constexpr int BF_B_BYTES = BNH * KSUB * 2;         // 16384
+constexpr int BF_STAGE_BYTES = BF_A_BYTES + BF_B_BYTES;                              // 32768
+constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;  // 204800
 constexpr int SMEM_BYTES = SMEM_TILES + 256 + 1024;                                  // barriers + alignment slack
 
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
@@ -56,7 +68,7 @@ struct GemmParams {
     void* out;
     int out_bf16;
     int a_mode, b_mode;           // UE5M3_SCALE_*
-    int tiles_m, tiles_n;
+    int tiles_m, tiles_n;         // 256 x 256 tiles
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -71,11 +83,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster (release at cluster scope).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar), "r"(rank) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
@@ -112,22 +132,39 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Tensor memory of a CTA pair is allocated and freed by the same warp of both CTAs.
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// Arrive (once all MMAs issued so far have retired) on the barrier at this offset in both CTAs of the pair.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+// The same, on this CTA's barrier only.
+__device__ __forceinline__ void umma_commit_local(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t r[32]) {
     asm volatile(
@@ -153,8 +190,8 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
     d |= (uint64_t)2 << 61;                         // 128-byte swizzle
     return d;
 }
-// kind::f16 instruction descriptor: D = F32, A = B = BF16, both K-major, M = 128, N = 256.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// kind::f16 instruction descriptor: D = F32, A = B = BF16, both K-major, M = 256 (two CTAs), N = 256.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 
 __device__ __forceinline__ uint32_t hmul2_bf16(uint32_t a, uint32_t b) {
     uint32_t r;
@@ -191,36 +228,42 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 // ----------------------------------------------------------------------------- kernel
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
             const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
     const uint32_t pk_base = smem_base;
     const uint32_t bf_base = smem_base + PK_STAGES * PK_STAGE_BYTES;
     const uint32_t bar_base = smem_base + SMEM_TILES;
     // barriers (8 bytes each)
-    const uint32_t pk_full = bar_base, pk_empty = bar_base + 16, bf_full = bar_base + 32, bf_empty = bar_base + 48;
-    const uint32_t acc_full = bar_base + 64, acc_empty = bar_base + 80, drain_bar = bar_base + 96;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 128);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 136);
+    const uint32_t pk_full = bar_base, pk_empty = bar_base + 32, bf_full = bar_base + 64, bf_empty = bar_base + 96;
+    const uint32_t acc_full = bar_base + 128, acc_empty = bar_base + 144, drain_bar = bar_base + 160;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 176);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 184);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();                   // 0 = leader of the pair
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int kchunks = (int)(p.Kc / KCHUNK);
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < PK_STAGES; ++s) {
             mbar_init(pk_full + 8 * s, 1);
             mbar_init(pk_empty + 8 * s, DEQ_WARPS);
-            mbar_init(bf_full + 8 * s, DEQ_WARPS);
+        }
+        for (int s = 0; s < BF_STAGES; ++s) {
+            mbar_init(bf_full + 8 * s, 2 * GROUP_WARPS);      // the leader's copy collects both CTAs' groups
             mbar_init(bf_empty + 8 * s, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(acc_full + 8 * s, 1);
-            mbar_init(acc_empty + 8 * s, 4);
+            mbar_init(acc_empty + 8 * s, 8);                  // four epilogue warps in each CTA
         }
         mbar_init(drain_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -229,6 +272,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (warp == 2) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                                       // both CTAs' barriers and tensor memory exist
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -238,48 +282,47 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t it = 0;
             const int a_rows_per_load = (p.a_mode == UE5M3_SCALE_2D) ? 8 : 128;
             const int b_rows_per_load = (p.b_mode == UE5M3_SCALE_2D) ? 8 : 128;
-            const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + 2 * b_rows_per_load * 16;
+            const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + b_rows_per_load * 16;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int mb = tile % p.tiles_m, nb = tile / p.tiles_m;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                const int mb = (tile % p.tiles_m) * 2 + (int)rank;       // 128-row block of A
+                const int nh = (tile / p.tiles_m) * 2 + (int)rank;       // 128-row block of B
                 for (int kc = 0; kc < kchunks; ++kc, ++it) {
-                    const uint32_t s = it & 1, ph = (it >> 1) & 1;
+                    const uint32_t s = it % PK_STAGES, ph = (it / PK_STAGES) & 1;
                     if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t st = pk_base + s * PK_STAGE_BYTES;
                     const uint32_t full = pk_full + 8 * s;
                     mbar_expect_tx(full, tx_bytes);
                     tma_load_2d(st, &map_a, full, kc * (KCHUNK / 2), mb * BM);
-                    tma_load_2d(st + PK_A_BYTES, &map_b, full, kc * (KCHUNK / 2), nb * BN);
-                    // scales: 16 block columns of this K chunk
+                    tma_load_2d(st + PK_A_BYTES, &map_b, full, kc * (KCHUNK / 2), nh * BNH);
+                    // scales: the 16 block columns of this K chunk
                     const uint32_t sa = st + PK_A_BYTES + PK_B_BYTES, sb = sa + SC_A_BYTES;
                     if (p.a_mode == UE5M3_SCALE_1D) tma_load_2d(sa, &map_as, full, kc * 16, mb * BM);
                     else if (p.a_mode == UE5M3_SCALE_2D) tma_load_2d(sa, &map_as, full, kc * 16, mb * (BM / 16));
                     else tma_load_2d(sa, &map_as, full, 0, (mb * kchunks + kc) * 128);
-                    for (int h = 0; h < 2; ++h) {
-                        if (p.b_mode == UE5M3_SCALE_1D) tma_load_2d(sb + h * 2048, &map_bs, full, kc * 16, nb * BN + h * 128);
-                        else if (p.b_mode == UE5M3_SCALE_2D) tma_load_2d(sb + h * 128, &map_bs, full, kc * 16, nb * (BN / 16) + h * 8);
-                        else tma_load_2d(sb + h * 2048, &map_bs, full, 0, ((nb * 2 + h) * kchunks + kc) * 128);
-                    }
+                    if (p.b_mode == UE5M3_SCALE_1D) tma_load_2d(sb, &map_bs, full, kc * 16, nh * BNH);
+                    else if (p.b_mode == UE5M3_SCALE_2D) tma_load_2d(sb, &map_bs, full, kc * 16, nh * (BNH / 16));
+                    else tma_load_2d(sb, &map_bs, full, 0, (nh * kchunks + kc) * 128);
                 }
             }
             // let the copies still in flight land before the CTA's shared memory goes away
-            for (uint32_t back = 0; back < 2 && back < it; ++back) {
+            for (uint32_t back = 0; back < PK_STAGES && back < it; ++back) {
                 const uint32_t j = it - 1 - back;
-                mbar_wait(pk_full + 8 * (j & 1), (j >> 1) & 1, abort_flag);
+                mbar_wait(pk_full + 8 * (j % PK_STAGES), (j / PK_STAGES) & 1, abort_flag);
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA)
+        if (lane == 0 && rank == 0) {
             uint32_t it = 0, tl = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
                 const uint32_t ab = tl & 1, aph = (tl >> 1) & 1;
                 if (!mbar_wait(acc_empty + 8 * ab, aph ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + ab * BN;
-                for (int ks = 0; ks < kchunks * (KCHUNK / KSUB); ++ks, ++it) {
-                    const uint32_t s = it & 1, ph = (it >> 1) & 1;
+                for (int ks = 0; ks < kchunks * BF_STAGES; ++ks, ++it) {
+                    const uint32_t s = it % BF_STAGES, ph = (it / BF_STAGES) & 1;
                     if (!mbar_wait(bf_full + 8 * s, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_s = bf_base + s * BF_STAGE_BYTES, b_s = a_s + BF_A_BYTES;
@@ -287,12 +330,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
                     for (int k = 0; k < KSUB / 16; ++k)
                         umma_bf16(tmem_d, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), kInstrDesc, (ks | k) != 0 ? 1u : 0u);
-                    umma_commit(bf_empty + 8 * s);
+                    umma_commit_pair(bf_empty + 8 * s);        // both CTAs may refill this stage
                 }
-                if (ok) umma_commit(acc_full + 8 * ab);
+                if (ok) umma_commit_pair(acc_full + 8 * ab);   // both CTAs' epilogues may read
             }
             // everything issued must have retired before tensor memory is released
-            umma_commit(drain_bar);
+            umma_commit_local(drain_bar);
             mbar_wait(drain_bar, 0, abort_flag);
         }
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
@@ -301,20 +344,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const float alpha = __fmul_rn(__fmul_rn(__ldg(p.a_decode), 65536.0f), __fmul_rn(__ldg(p.b_decode), 65536.0f));
         uint32_t tl = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
-            const int mb = tile % p.tiles_m, nb = tile / p.tiles_m;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
+            const int mb = (tile % p.tiles_m) * 2 + (int)rank, nb = tile / p.tiles_m;
             const uint32_t ab = tl & 1, aph = (tl >> 1) & 1;
             if (!mbar_wait(acc_full + 8 * ab, aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const int64_t row = (int64_t)mb * BM + q * 32 + lane;
             const int64_t col0 = (int64_t)nb * BN;
+            const bool row_ok = row < p.Mo;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + c * 32, r);
                 tmem_ld_wait();
                 const int64_t col = col0 + c * 32;
-                if (col < p.No) {                      // No is a multiple of 128, so a 32-column group is all in or all out
+                if (row_ok && col < p.No) {            // No is a multiple of 128, so a 32-column group is all in or all out
                     if (p.out_bf16) {
                         uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(p.out) + row * p.ldo + col);
 #pragma unroll
@@ -337,60 +381,62 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty + 8 * ab);
+            if (lane == 0) mbar_arrive_cluster(acc_empty + 8 * ab, 0);     // the leader issues the next tile's MMAs
         }
     } else if (warp >= DEQ_WARP0) {
         // ------------------------------------------------------------------ dequantizers
         const int dw = warp - DEQ_WARP0;
-        const int r7 = lane & 7, j = lane >> 3;       // row inside an 8-row group, 16-value block inside the 64-wide stage
+        const int grp = dw / GROUP_WARPS, gw = dw % GROUP_WARPS;     // slice / BF16 stage of this group, warp inside it
+        const int r7 = lane & 7, j = lane >> 3;       // row inside an 8-row group, 16-value block inside the 64-wide slice
         const int a_shift = (p.a_mode == UE5M3_SCALE_2D) ? 4 : 0, b_shift = (p.b_mode == UE5M3_SCALE_2D) ? 4 : 0;
-        uint32_t it_pk = 0, it_bf = 0;
+        uint8_t* bf = smem_gen + PK_STAGES * PK_STAGE_BYTES + grp * BF_STAGE_BYTES;
+        uint32_t it_pk = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
             for (int kc = 0; kc < kchunks && ok; ++kc, ++it_pk) {
-                const uint32_t ps = it_pk & 1, pph = (it_pk >> 1) & 1;
+                const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
                 if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag)) { ok = false; break; }
                 const uint8_t* st = smem_gen + ps * PK_STAGE_BYTES;
-#pragma unroll 1
-                for (int sub = 0; sub < KCHUNK / KSUB; ++sub, ++it_bf) {
-                    // gather this thread's blocks of the 64-wide slice
-                    uint2 pay[DEQ_TASKS];
-                    uint32_t code[DEQ_TASKS];
+                // gather this thread's blocks of the group's 64-wide slice
+                uint2 pay[DEQ_TASKS];
+                uint32_t code[DEQ_TASKS];
 #pragma unroll
-                    for (int t = 0; t < DEQ_TASKS; ++t) {
-                        const int rg = dw + DEQ_WARPS * t;          // 8-row group: 0..15 are A, 16..47 are B
-                        const bool isA = rg < 16;
-                        const int row = (isA ? rg : rg - 16) * 8 + r7;
-                        const uint8_t* pk = st + (isA ? 0 : PK_A_BYTES) + row * 128 + ((((sub << 1) | (j >> 1)) ^ r7) << 4) + ((j & 1) << 3);
-                        pay[t] = *reinterpret_cast<const uint2*>(pk);
-                        const uint8_t* sc = st + PK_A_BYTES + PK_B_BYTES + (isA ? 0 : SC_A_BYTES);
-                        code[t] = sc[((row >> (isA ? a_shift : b_shift)) << 4) + (sub << 2) + j];
-                    }
-                    const uint32_t bs = it_bf & 1, bph = (it_bf >> 1) & 1;
-                    if (!mbar_wait(bf_empty + 8 * bs, bph ^ 1, abort_flag)) { ok = false; break; }
-                    uint8_t* bf = smem_gen + PK_STAGES * PK_STAGE_BYTES + bs * BF_STAGE_BYTES;
-#pragma unroll
-                    for (int t = 0; t < DEQ_TASKS; ++t) {
-                        const int rg = dw + DEQ_WARPS * t;
-                        const bool isA = rg < 16;
-                        const int row = (isA ? rg : rg - 16) * 8 + r7;
-                        const uint32_t m = scale_pair(code[t]);
-                        uint8_t* dst = bf + (isA ? 0 : BF_A_BYTES) + row * 128;
-                        *reinterpret_cast<uint4*>(dst + (((2 * j) ^ r7) << 4)) = dequant8(pay[t].x, m);
-                        *reinterpret_cast<uint4*>(dst + (((2 * j + 1) ^ r7) << 4)) = dequant8(pay[t].y, m);
-                    }
-                    fence_proxy_async();                 // make the generic-proxy stores visible to the tensor core
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bf_full + 8 * bs);
+                for (int t = 0; t < DEQ_TASKS; ++t) {
+                    const int rg = gw + GROUP_WARPS * t;          // 8-row group: 0..15 are A, 16..31 are B
+                    const bool isA = rg < 16;
+                    const int row = (isA ? rg : rg - 16) * 8 + r7;
+                    const uint8_t* pk = st + (isA ? 0 : PK_A_BYTES) + row * 128 + ((((grp << 1) | (j >> 1)) ^ r7) << 4) + ((j & 1) << 3);
+                    pay[t] = *reinterpret_cast<const uint2*>(pk);
+                    const uint8_t* sc = st + PK_A_BYTES + PK_B_BYTES + (isA ? 0 : SC_A_BYTES);
+                    code[t] = sc[((row >> (isA ? a_shift : b_shift)) << 4) + (grp << 2) + j];
                 }
+                // BF16 stage `grp` is reused once per packed stage
+                if (!mbar_wait(bf_empty + 8 * grp, (it_pk & 1) ^ 1, abort_flag)) { ok = false; break; }
+#pragma unroll
+                for (int t = 0; t < DEQ_TASKS; ++t) {
+                    const int rg = gw + GROUP_WARPS * t;
+                    const bool isA = rg < 16;
+                    const int row = (isA ? rg : rg - 16) * 8 + r7;
+                    const uint32_t m = scale_pair(code[t]);
+                    uint8_t* dst = bf + (isA ? 0 : BF_A_BYTES) + row * 128;
+                    *reinterpret_cast<uint4*>(dst + (((2 * j) ^ r7) << 4)) = dequant8(pay[t].x, m);
+                    *reinterpret_cast<uint4*>(dst + (((2 * j + 1) ^ r7) << 4)) = dequant8(pay[t].y, m);
+                }
+                fence_proxy_async();                 // make the generic-proxy stores visible to the tensor core
                 __syncwarp();
-                if (lane == 0 && ok) mbar_arrive(pk_empty + 8 * ps);
+                if (lane == 0) {
+                    mbar_arrive_cluster(bf_full + 8 * grp, 0);
+                    mbar_arrive(pk_empty + 8 * ps);  // the packed bytes of this stage are in registers or consumed
+                }
             }
         }
     }
 
+    // Neither CTA may leave (or free tensor memory) while its partner can still touch its shared
+    // memory, barriers or accumulators.
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     if (warp == 2) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
@@ -440,18 +486,27 @@ bool make_scale_map(CUtensorMap* m, const uint8_t* scales, int mode, int64_t R, 
 }  // namespace
 
 int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
-    static bool attr_set[64];
+    static int resident_pairs[64];      // CTA pairs that can be resident at once, per device; 0 = not asked yet
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return UE5M3_ERR_CUDA;
-    if (!attr_set[dev]) {
+    if (resident_pairs[dev] == 0) {
         if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return UE5M3_ERR_CUDA;
-        attr_set[dev] = true;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
+        cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel, &cfg) != cudaSuccess || n < 1) {
+            (void)cudaGetLastError();
+            n = num_sms / 2;
+        }
+        resident_pairs[dev] = n < num_sms / 2 ? n : num_sms / 2;
     }
     CUtensorMap ma, mb, mas, mbs;
     const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
     if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
-    if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BN, true)) return UE5M3_ERR_CUDA;
+    if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BNH, true)) return UE5M3_ERR_CUDA;
     if (!make_scale_map(&mas, g.a_scales, g.a_scale_mode, g.Mo, g.Kc)) return UE5M3_ERR_CUDA;
     if (!make_scale_map(&mbs, g.b_scales, g.b_scale_mode, g.No, g.Kc)) return UE5M3_ERR_CUDA;
 
@@ -460,11 +515,12 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     p.a_decode = g.a_decode; p.b_decode = g.b_decode;
     p.out = g.out; p.out_bf16 = g.out_dtype == UE5M3_BF16 ? 1 : 0;
     p.a_mode = g.a_scale_mode; p.b_mode = g.b_scale_mode;
-    p.tiles_m = (int)(g.Mo / BM);
+    p.tiles_m = (int)((g.Mo + 2 * BM - 1) / (2 * BM));
     p.tiles_n = (int)((g.No + BN - 1) / BN);
     const int num_tiles = p.tiles_m * p.tiles_n;
-    const int grid = num_tiles < num_sms ? num_tiles : num_sms;
-    gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, p);
+    const int max_pairs = resident_pairs[dev];
+    const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
+    gemm_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, p);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
