@@ -148,6 +148,24 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def wait_first_sample(self, timeout=20.0):
+        t0 = time.time()
+        while self.proc is not None and time.time() - t0 < timeout:
+            try:
+                if os.path.getsize(self.path) > 0:
+                    return
+            except OSError:
+                return
+            time.sleep(0.05)
+
+    def mark(self):
+        """Samples written before this point (warm-up) are not counted."""
+        try:
+            with open(self.path) as f:
+                self.skip = sum(1 for _ in f)
+        except Exception:
+            self.skip = 0
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
@@ -160,7 +178,9 @@ class ClockSampler:
         sm, mx, pw, reasons = [], [], [], set()
         try:
             with open(self.path) as f:
-                for line in f:
+                for n, line in enumerate(f):
+                    if n < getattr(self, "skip", 0):
+                        continue
                     c = [v.strip() for v in line.split(",")]
                     if len(c) < 7:
                         continue
@@ -253,6 +273,22 @@ KERNEL_BYTES = kernel_bytes()
 GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
 
 
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Step time of the job = the slowest rank's (MAX all-reduce of one number; no data-path collective)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(ms_per_step: float, world: int) -> float:
+    """Whole-job TFLOP/s: every rank runs the same per-rank workload on its own tokens (weak scaling)."""
+    return world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -277,12 +313,14 @@ def run_ours(args):
     step = LinearStep(dev, seed=rank, scale_layout=args.scale_layout)
     K, Wm = args.steps, max(args.warmup, 3)
 
+    sampler = ClockSampler(dev)
+    sampler.start()          # started before the warm-up: its own start-up must not fall into the timed region
+    sampler.wait_first_sample()
     for s in range(Wm):
         step.run(s)
     barrier()
     launches0 = step.launches
-    sampler = ClockSampler(dev)
-    sampler.start()
+    sampler.mark()
     ev = {}
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -296,12 +334,9 @@ def run_ours(args):
     status = lib.last_device_status()
     if status != 0:
         raise SystemExit(f"device status {lib.status_string(status)}")
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / K
-    value = world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e12
+    value = job_value(ms_per_step, world)
     gpu_launches = step.launches - launches0
 
     per_kernel = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in ev.items()}
@@ -337,15 +372,10 @@ def run_ours(args):
             e2e_step(Wm + K + 1 + s)
         b.record()
         barrier()
-        e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e_ms /= n_e2e
+        e_ms = max_over_ranks(a.elapsed_time(b), world, dev) / n_e2e
         h2d = sum(t.numel() * t.element_size() for t in (Xh, Wh, dYh))
         d2h = sum(t.numel() * t.element_size() for t in (Yh, dXh, dWh))
-        e2e = {"value": world * FLOPS_PER_STEP / (e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e_ms, "steps": n_e2e,
+        e2e = {"value": job_value(e_ms, world), "unit": UNIT, "ms_per_step": e_ms, "steps": n_e2e,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank == 0:

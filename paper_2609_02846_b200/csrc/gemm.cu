@@ -71,6 +71,19 @@ struct GemmParams {
     int tiles_m, tiles_n;         // 256 x 256 tiles
 };
 
+// Tile order: groups of kRasterGroup tile rows, and inside a group column by column.  The tiles that are
+// resident at the same time (one per CTA pair) then span about 8 x 9 tiles and share their A and B panels
+// through L2, instead of touching every A panel in each wave.
+constexpr int kRasterGroup = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+    const int per_group = kRasterGroup * tiles_n;
+    const int g = tile / per_group, r = tile - g * per_group;
+    const int first = g * kRasterGroup;
+    const int gsize = min(kRasterGroup, tiles_m - first);
+    tn = r / gsize;
+    tm = first + (r - tn * gsize);
+}
+
 // ----------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -285,8 +298,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + b_rows_per_load * 16;
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-                const int mb = (tile % p.tiles_m) * 2 + (int)rank;       // 128-row block of A
-                const int nh = (tile / p.tiles_m) * 2 + (int)rank;       // 128-row block of B
+                int tm, tn;
+                tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+                const int mb = tm * 2 + (int)rank;                       // 128-row block of A
+                const int nh = tn * 2 + (int)rank;                       // 128-row block of B
                 for (int kc = 0; kc < kchunks; ++kc, ++it) {
                     const uint32_t s = it % PK_STAGES, ph = (it / PK_STAGES) & 1;
                     if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
@@ -345,7 +360,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t tl = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
-            const int mb = (tile % p.tiles_m) * 2 + (int)rank, nb = tile / p.tiles_m;
+            int tm, nb;
+            tile_coords(tile, p.tiles_m, p.tiles_n, tm, nb);
+            const int mb = tm * 2 + (int)rank;
             const uint32_t ab = tl & 1, aph = (tl >> 1) & 1;
             if (!mbar_wait(acc_full + 8 * ab, aph, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -410,6 +427,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint8_t* sc = st + PK_A_BYTES + PK_B_BYTES + (isA ? 0 : SC_A_BYTES);
                     code[t] = sc[((row >> (isA ? a_shift : b_shift)) << 4) + (grp << 2) + j];
                 }
+                // The packed bytes are in registers: hand the stage back to the producer now, so that the next
+                // copy overlaps the arithmetic (the arrive is a release, ordered after this warp's loads).
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pk_empty + 8 * ps);
                 // BF16 stage `grp` is reused once per packed stage
                 if (!mbar_wait(bf_empty + 8 * grp, (it_pk & 1) ^ 1, abort_flag)) { ok = false; break; }
 #pragma unroll
@@ -424,10 +445,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
                 fence_proxy_async();                 // make the generic-proxy stores visible to the tensor core
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive_cluster(bf_full + 8 * grp, 0);
-                    mbar_arrive(pk_empty + 8 * ps);  // the packed bytes of this stage are in registers or consumed
-                }
+                if (lane == 0) mbar_arrive_cluster(bf_full + 8 * grp, 0);
             }
         }
     }
