@@ -271,6 +271,9 @@ def kernel_bytes():
 
 KERNEL_BYTES = kernel_bytes()
 GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the default workload (mean of fprop, dgrad, wgrad;
+# one ncu pass, summary in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt).  Algorithmic bytes: 242 MB per launch.
+GEMM_DRAM_TRAFFIC_BYTES = (140.4e6 + 214.8e6 + 194.1e6 + 47.0e6 + 95.3e6 + 95.4e6) / 3
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -393,7 +396,9 @@ def run_ours(args):
                          "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": gemm_tflops / peaks["bf16_tflops_sustained"],
                          "frac_of_burst_peak": gemm_tflops / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained)",
-                         "avg_launch_ms": gemm_ms, "traffic": None,
+                         "avg_launch_ms": gemm_ms,
+                         "traffic": GEMM_DRAM_TRAFFIC_BYTES if (M_TOK, K_IN, N_OUT) == (8192, 4096, 16384) else None,
+                         "traffic_unit": "bytes of DRAM read+write per launch (ncu, mean of the three GEMMs)",
                          "per_gemm_ms": {k: round(per_kernel[k], 4) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}},
             "quantizer": quant,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches, "clocks": clocks,
