@@ -10,15 +10,18 @@
 //
 // Persistent, one CTA per SM, CTAs paired into clusters of two that share one 256 x 256 output tile
 // (tcgen05 cta_group::2): each CTA owns 128 rows of A and 128 of the 256 B rows, so it stages and
-// dequantizes 128 + 128 rows per K slice for a 128 x 256 accumulator of its own.  Warp roles per CTA:
+// dequantizes 128 + 128 rows per K slice for a 128 x 256 accumulator of its own.  The dequantized A
+// slice goes straight from registers into tensor memory (tcgen05.st; the MMA takes A from TMEM), only
+// the B slice goes through shared memory, which halves the shared-memory traffic of the main loop and
+// leaves room for eight BF16 stages.  Warp roles per CTA:
 //   warp 0        TMA producer: packed payload tiles (128B-swizzled) and scale tiles, 256 K per stage
 //   warp 1        MMA issuer (leader CTA only): 4 x tcgen05.mma (M256 N256 K16) per 64-wide BF16 stage
 //   warp 2        tensor-memory allocation
-//   warps 4-7     epilogue: tcgen05.ld, scale, convert, store (overlaps the next tile's main loop
-//                 through two 256-column accumulators)
-//   warps 8-23    dequantizers: packed smem -> BF16 smem in the 128B-swizzled K-major UMMA layout.  Four
-//                 groups of four warps; group g converts the g-th 64-wide slice of every packed stage into
-//                 BF16 stage g, so four slices are in flight and no group waits for another.
+//   warps 4-7     epilogue: tcgen05.ld, scale, convert, stage in shared memory, TMA store
+//   warps 8-23    dequantizers, four groups of four warps.  Group g converts the g-th 64-wide slice of
+//                 every packed stage; thread t of a group owns row t of the A tile and row t of the B tile.
+//                 Each group ping-pongs between two BF16 stages, so it never waits for its own MMA.
+// Tensor memory: columns 0..255 accumulator, columns 256..511 eight A stages of 32 columns.
 // The leader learns that both CTAs' BF16 stages are full through one mbarrier that the partner's
 // dequantizers arrive on remotely; stage and accumulator releases come back to both CTAs through
 // tcgen05.commit with a two-CTA multicast mask.  No copy is multicast: every CTA loads its own tiles.
@@ -41,23 +44,24 @@ constexpr int BNH = 128;                    // B rows staged by each CTA of the 
 constexpr int KCHUNK = 256;                 // K per packed stage
 constexpr int KSUB = 64;                    // K per BF16 stage (one 128-byte swizzle row)
 constexpr int PK_STAGES = 2;
-constexpr int BF_STAGES = KCHUNK / KSUB;    // 4: one BF16 stage per 64-wide slice of a packed stage
+constexpr int SLICES = KCHUNK / KSUB;       // 4 slices of 64 K per packed stage
+constexpr int BF_STAGES = 2 * SLICES;       // 8: every dequantizer group ping-pongs between two BF16 stages
 constexpr int DEQ_WARP0 = 8, DEQ_WARPS = 16, EPI_WARP0 = 4;
-constexpr int DEQ_GROUPS = BF_STAGES;       // dequantizer group g owns slice g of every packed stage and BF16 stage g
-constexpr int GROUP_WARPS = DEQ_WARPS / DEQ_GROUPS;
+constexpr int DEQ_GROUPS = SLICES;          // dequantizer group g owns slice g of every packed stage
+constexpr int GROUP_WARPS = DEQ_WARPS / DEQ_GROUPS;       // 4 warps = 128 threads = one thread per tile row
 constexpr int NUM_THREADS = 32 * (DEQ_WARP0 + DEQ_WARPS);
-constexpr int DEQ_TASKS = 32 / GROUP_WARPS;    // 8-row groups (16 of A, 16 of B) per warp and slice
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;        // 16384
 constexpr int PK_B_BYTES = BNH * KCHUNK / 2;       // 16384
 constexpr int SC_A_BYTES = BM * (KCHUNK / 16);     // 2048
 constexpr int SC_B_BYTES = BNH * (KCHUNK / 16);    // 2048
 constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES;   // 36864
-constexpr int BF_A_BYTES = BM * KSUB * 2;          // 16384
-constexpr int BF_B_BYTES = BNH * KSUB * 2;         // 16384
-constexpr int BF_STAGE_BYTES = BF_A_BYTES + BF_B_BYTES;                              // 32768
+constexpr int BF_STAGE_BYTES = BNH * KSUB * 2;     // 16384: the B slice; the A slice lives in tensor memory
 constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;  // 204800
-constexpr int SMEM_BYTES = SMEM_TILES + 256 + 1024;                                  // barriers + alignment slack
+constexpr int SMEM_EPI = SMEM_TILES + 1024;        // epilogue staging (1024-aligned for the 128B swizzle) after the barriers
+constexpr int EPI_WARP_BYTES = 4096;               // one 32 x 32 FP32 chunk, or two 32 x 32 BF16 chunks, per epilogue warp
+constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;                     // + alignment slack
+constexpr int TMEM_ACC_COL = 0, TMEM_A_COL = 256, TMEM_A_STAGE_COLS = KSUB / 2;      // 32 columns per A stage
 
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 
@@ -137,6 +141,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+// Bulk tensor store shared -> global of one box; completion is tracked by bulk groups of the issuing thread.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -162,13 +175,28 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// One M256 N256 K16 MMA of the CTA pair: D (tensor memory) (+)= A (tensor memory) * B (shared memory).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t r[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // Arrive (once all MMAs issued so far have retired) on the barrier at this offset in both CTAs of the pair.
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
     const uint16_t mask = 3;
@@ -226,11 +254,15 @@ __device__ __forceinline__ uint32_t scale_pair(uint32_t code) {
 // elements k (low half) and k + 4 (high half); A and B use the same order, which a dot product
 // does not see.
 __device__ __forceinline__ uint4 dequant8(uint32_t w, uint32_t m) {
+    // One code per 16-bit half is isolated, then a multiplication by 2^a + 2^b drops its magnitude bits at
+    // bits 8:6 and its sign at bit 15 in one go (the two shifted copies never overlap, so the sum has no
+    // carries); the multiplications run on the FMA pipe and leave the integer pipe to the masks.
+    const uint32_t w8 = w >> 8;
     uint4 o;
-    o.x = hmul2_bf16(((w << 6) & 0x01C001C0u) | ((w << 12) & 0x80008000u), m);
-    o.y = hmul2_bf16(((w << 2) & 0x01C001C0u) | ((w << 8) & 0x80008000u), m);
-    o.z = hmul2_bf16(((w >> 2) & 0x01C001C0u) | ((w << 4) & 0x80008000u), m);
-    o.w = hmul2_bf16(((w >> 6) & 0x01C001C0u) | (w & 0x80008000u), m);
+    o.x = hmul2_bf16(((w & 0x000F000Fu) * 0x1040u) & 0x81C081C0u, m);     // codes 0 and 4
+    o.y = hmul2_bf16(((w & 0x00F000F0u) * 0x0104u) & 0x81C081C0u, m);     // codes 1 and 5
+    o.z = hmul2_bf16(((w8 & 0x000F000Fu) * 0x1040u) & 0x81C081C0u, m);    // codes 2 and 6
+    o.w = hmul2_bf16(((w8 & 0x00F000F0u) * 0x0104u) & 0x81C081C0u, m);    // codes 3 and 7
     return o;
 }
 
@@ -244,7 +276,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
-            const GemmParams p) {
+            const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -253,10 +285,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const uint32_t bf_base = smem_base + PK_STAGES * PK_STAGE_BYTES;
     const uint32_t bar_base = smem_base + SMEM_TILES;
     // barriers (8 bytes each)
-    const uint32_t pk_full = bar_base, pk_empty = bar_base + 32, bf_full = bar_base + 64, bf_empty = bar_base + 96;
-    const uint32_t acc_full = bar_base + 128, acc_empty = bar_base + 144, drain_bar = bar_base + 160;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 176);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 184);
+    const uint32_t pk_full = bar_base, pk_empty = bar_base + 16, bf_full = bar_base + 32, bf_empty = bar_base + 96;
+    const uint32_t acc_full = bar_base + 160, acc_empty = bar_base + 168, drain_bar = bar_base + 176;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 192);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 200);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();                   // 0 = leader of the pair
@@ -274,13 +306,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             mbar_init(bf_full + 8 * s, 2 * GROUP_WARPS);      // the leader's copy collects both CTAs' groups
             mbar_init(bf_empty + 8 * s, 1);
         }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(acc_full + 8 * s, 1);
-            mbar_init(acc_empty + 8 * s, 8);                  // four epilogue warps in each CTA
-        }
+        mbar_init(acc_full, 1);
+        mbar_init(acc_empty, 8);                              // four epilogue warps in each CTA
         mbar_init(drain_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        prefetch_tmap(&map_a); prefetch_tmap(&map_b); prefetch_tmap(&map_as); prefetch_tmap(&map_bs);
+        prefetch_tmap(&map_a); prefetch_tmap(&map_b); prefetch_tmap(&map_as); prefetch_tmap(&map_bs); prefetch_tmap(&map_out);
     }
     if (warp == 2) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
@@ -332,22 +362,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t it = 0, tl = 0;
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
-                const uint32_t ab = tl & 1, aph = (tl >> 1) & 1;
-                if (!mbar_wait(acc_empty + 8 * ab, aph ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag)) { ok = false; break; }   // epilogues have read tile tl-1
                 tc_fence_after();
-                const uint32_t tmem_d = tmem_base + ab * BN;
-                for (int ks = 0; ks < kchunks * BF_STAGES; ++ks, ++it) {
-                    const uint32_t s = it % BF_STAGES, ph = (it / BF_STAGES) & 1;
+                const uint32_t tmem_d = tmem_base + TMEM_ACC_COL;
+                for (int ks = 0; ks < kchunks * SLICES; ++ks, ++it) {
+                    // slice it: group it % 4, its buffer (it / 4) & 1, used for the (it / 8)-th time
+                    const uint32_t s = (it & 3) + 4 * ((it >> 2) & 1), ph = (it >> 3) & 1;
                     if (!mbar_wait(bf_full + 8 * s, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_s = bf_base + s * BF_STAGE_BYTES, b_s = a_s + BF_A_BYTES;
-                    const uint64_t ad = umma_smem_desc(a_s), bd = umma_smem_desc(b_s);
+                    const uint64_t bd = umma_smem_desc(bf_base + s * BF_STAGE_BYTES);
+                    const uint32_t ta = tmem_base + TMEM_A_COL + s * TMEM_A_STAGE_COLS;
 #pragma unroll
                     for (int k = 0; k < KSUB / 16; ++k)
-                        umma_bf16(tmem_d, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), kInstrDesc, (ks | k) != 0 ? 1u : 0u);
+                        umma_bf16_ts(tmem_d, ta + k * 8, bd + (uint64_t)(k * 2), kInstrDesc, (ks | k) != 0 ? 1u : 0u);
                     umma_commit_pair(bf_empty + 8 * s);        // both CTAs may refill this stage
                 }
-                if (ok) umma_commit_pair(acc_full + 8 * ab);   // both CTAs' epilogues may read
+                if (ok) umma_commit_pair(acc_full);            // both CTAs' epilogues may read
             }
             // everything issued must have retired before tensor memory is released
             umma_commit_local(drain_bar);
@@ -357,56 +387,78 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lane quarter this warp may access
         const float alpha = __fmul_rn(__fmul_rn(__ldg(p.a_decode), 65536.0f), __fmul_rn(__ldg(p.b_decode), 65536.0f));
-        uint32_t tl = 0;
+        // Staging: lane = output row.  The chunk is written in the swizzled layout the output tensor map expects
+        // (conflict-free 16-byte stores) and leaves through the TMA engine, which keeps the row-scattered global
+        // stores off the load/store pipe the dequantizers depend on.  The map clips rows >= Mo and columns >= No.
+        const uint32_t stage = smem_base + SMEM_EPI + q * EPI_WARP_BYTES;
+        uint8_t* stage_gen = smem_gen + SMEM_EPI + q * EPI_WARP_BYTES;
+        uint32_t tl = 0, chunk = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
             int tm, nb;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, nb);
             const int mb = tm * 2 + (int)rank;
-            const uint32_t ab = tl & 1, aph = (tl >> 1) & 1;
-            if (!mbar_wait(acc_full + 8 * ab, aph, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(acc_full, tl & 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const int64_t row = (int64_t)mb * BM + q * 32 + lane;
-            const int64_t col0 = (int64_t)nb * BN;
-            const bool row_ok = row < p.Mo;
+            const int row0 = mb * BM + q * 32, col0 = nb * BN;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < BN / 32; ++c, ++chunk) {
                 uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + c * 32, r);
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_ACC_COL + c * 32, r);
                 tmem_ld_wait();
-                const int64_t col = col0 + c * 32;
-                if (row_ok && col < p.No) {            // No is a multiple of 128, so a 32-column group is all in or all out
-                    if (p.out_bf16) {
-                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(p.out) + row * p.ldo + col);
+                if (c == BN / 32 - 1) {
+                    // the accumulator has been read completely: the leader may start the next tile's MMAs
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
+                }
+                if (p.out_bf16) {
+                    // two 2 KB buffers: the store issued two chunks ago must have read its buffer
+                    if (lane == 0) tma_store_wait_read<1>();
+                    __syncwarp();
+                    const uint32_t boff = (chunk & 1) * 2048;
+                    uint8_t* mine = stage_gen + boff + lane * 64;
+                    const int sw = (lane >> 1) & 3;                   // 64-byte swizzle: 16-byte piece ^= (row / 2) % 4
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * alpha, __uint_as_float(r[8 * v + 1]) * alpha);
-                            o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * alpha, __uint_as_float(r[8 * v + 3]) * alpha);
-                            o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * alpha, __uint_as_float(r[8 * v + 5]) * alpha);
-                            o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * alpha, __uint_as_float(r[8 * v + 7]) * alpha);
-                            dst[v] = o;
-                        }
-                    } else {
-                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + row * p.ldo + col);
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            dst[v] = make_float4(__uint_as_float(r[4 * v + 0]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
-                                                 __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 o;
+                        o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * alpha, __uint_as_float(r[8 * v + 1]) * alpha);
+                        o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * alpha, __uint_as_float(r[8 * v + 3]) * alpha);
+                        o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * alpha, __uint_as_float(r[8 * v + 5]) * alpha);
+                        o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * alpha, __uint_as_float(r[8 * v + 7]) * alpha);
+                        *reinterpret_cast<uint4*>(mine + ((v ^ sw) << 4)) = o;
                     }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) tma_store_2d(&map_out, stage + boff, col0 + c * 32, row0);
+                } else {
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
+                    uint8_t* mine = stage_gen + lane * 128;
+                    const int sw = lane & 7;                          // 128-byte swizzle: 16-byte piece ^= row % 8
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        *reinterpret_cast<float4*>(mine + ((v ^ sw) << 4)) =
+                            make_float4(__uint_as_float(r[4 * v + 0]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
+                                        __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) tma_store_2d(&map_out, stage, col0 + c * 32, row0);
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(acc_empty + 8 * ab, 0);     // the leader issues the next tile's MMAs
         }
+        if (lane == 0) tma_store_wait_all();         // the output is in global memory before the CTA retires
     } else if (warp >= DEQ_WARP0) {
         // ------------------------------------------------------------------ dequantizers
         const int dw = warp - DEQ_WARP0;
-        const int grp = dw / GROUP_WARPS, gw = dw % GROUP_WARPS;     // slice / BF16 stage of this group, warp inside it
-        const int r7 = lane & 7, j = lane >> 3;       // row inside an 8-row group, 16-value block inside the 64-wide slice
-        const int a_shift = (p.a_mode == UE5M3_SCALE_2D) ? 4 : 0, b_shift = (p.b_mode == UE5M3_SCALE_2D) ? 4 : 0;
-        uint8_t* bf = smem_gen + PK_STAGES * PK_STAGE_BYTES + grp * BF_STAGE_BYTES;
+        const int grp = dw / GROUP_WARPS;              // slice of every packed stage this group converts
+        const int q = warp & 3;                        // TMEM lane quarter of this warp (= warp inside the group)
+        const int row = q * 32 + lane;                 // this thread's row of the A tile and of the B tile
+        const int r7 = row & 7;
+        const int a_srow = (p.a_mode == UE5M3_SCALE_2D) ? (row >> 4) : row;
+        const int b_srow = (p.b_mode == UE5M3_SCALE_2D) ? (row >> 4) : row;
+        // the two 16-byte pieces of this row's slice inside the 128B-swizzled packed row
+        const int pk_off0 = row * 128 + (((2 * grp) ^ r7) << 4), pk_off1 = row * 128 + (((2 * grp + 1) ^ r7) << 4);
         uint32_t it_pk = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
@@ -414,38 +466,56 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
                 if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag)) { ok = false; break; }
                 const uint8_t* st = smem_gen + ps * PK_STAGE_BYTES;
-                // gather this thread's blocks of the group's 64-wide slice
-                uint2 pay[DEQ_TASKS];
-                uint32_t code[DEQ_TASKS];
-#pragma unroll
-                for (int t = 0; t < DEQ_TASKS; ++t) {
-                    const int rg = gw + GROUP_WARPS * t;          // 8-row group: 0..15 are A, 16..31 are B
-                    const bool isA = rg < 16;
-                    const int row = (isA ? rg : rg - 16) * 8 + r7;
-                    const uint8_t* pk = st + (isA ? 0 : PK_A_BYTES) + row * 128 + ((((grp << 1) | (j >> 1)) ^ r7) << 4) + ((j & 1) << 3);
-                    pay[t] = *reinterpret_cast<const uint2*>(pk);
-                    const uint8_t* sc = st + PK_A_BYTES + PK_B_BYTES + (isA ? 0 : SC_A_BYTES);
-                    code[t] = sc[((row >> (isA ? a_shift : b_shift)) << 4) + (grp << 2) + j];
-                }
+                const uint4 a0 = *reinterpret_cast<const uint4*>(st + pk_off0);
+                const uint4 a1 = *reinterpret_cast<const uint4*>(st + pk_off1);
+                const uint4 b0 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + pk_off0);
+                const uint4 b1 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + pk_off1);
+                const uint32_t a_codes = *reinterpret_cast<const uint32_t*>(st + PK_A_BYTES + PK_B_BYTES + a_srow * 16 + grp * 4);
+                const uint32_t b_codes = *reinterpret_cast<const uint32_t*>(st + PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + b_srow * 16 + grp * 4);
                 // The packed bytes are in registers: hand the stage back to the producer now, so that the next
                 // copy overlaps the arithmetic (the arrive is a release, ordered after this warp's loads).
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pk_empty + 8 * ps);
-                // BF16 stage `grp` is reused once per packed stage
-                if (!mbar_wait(bf_empty + 8 * grp, (it_pk & 1) ^ 1, abort_flag)) { ok = false; break; }
-#pragma unroll
-                for (int t = 0; t < DEQ_TASKS; ++t) {
-                    const int rg = gw + GROUP_WARPS * t;
-                    const bool isA = rg < 16;
-                    const int row = (isA ? rg : rg - 16) * 8 + r7;
-                    const uint32_t m = scale_pair(code[t]);
-                    uint8_t* dst = bf + (isA ? 0 : BF_A_BYTES) + row * 128;
-                    *reinterpret_cast<uint4*>(dst + (((2 * j) ^ r7) << 4)) = dequant8(pay[t].x, m);
-                    *reinterpret_cast<uint4*>(dst + (((2 * j + 1) ^ r7) << 4)) = dequant8(pay[t].y, m);
+
+                // this group's BF16 stage for this packed stage: two buffers, used alternately
+                const uint32_t bs = grp + 4 * (it_pk & 1);
+                if (!mbar_wait(bf_empty + 8 * bs, ((it_pk >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+
+                // A: 64 values of this row -> 32 tensor-memory columns (column c = K positions 2c, 2c+1)
+                {
+                    const uint32_t m0 = scale_pair(a_codes & 0xFFu), m1 = scale_pair((a_codes >> 8) & 0xFFu);
+                    const uint32_t m2 = scale_pair((a_codes >> 16) & 0xFFu), m3 = scale_pair(a_codes >> 24);
+                    uint32_t r[32];
+                    uint4 v;
+                    v = dequant8(a0.x, m0); r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w;
+                    v = dequant8(a0.y, m0); r[4] = v.x; r[5] = v.y; r[6] = v.z; r[7] = v.w;
+                    v = dequant8(a0.z, m1); r[8] = v.x; r[9] = v.y; r[10] = v.z; r[11] = v.w;
+                    v = dequant8(a0.w, m1); r[12] = v.x; r[13] = v.y; r[14] = v.z; r[15] = v.w;
+                    v = dequant8(a1.x, m2); r[16] = v.x; r[17] = v.y; r[18] = v.z; r[19] = v.w;
+                    v = dequant8(a1.y, m2); r[20] = v.x; r[21] = v.y; r[22] = v.z; r[23] = v.w;
+                    v = dequant8(a1.z, m3); r[24] = v.x; r[25] = v.y; r[26] = v.z; r[27] = v.w;
+                    v = dequant8(a1.w, m3); r[28] = v.x; r[29] = v.y; r[30] = v.z; r[31] = v.w;
+                    tmem_st32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_A_COL + bs * TMEM_A_STAGE_COLS, r);
                 }
-                fence_proxy_async();                 // make the generic-proxy stores visible to the tensor core
+                // B: 64 values of this row -> one 128-byte row of the 128B-swizzled K-major tile
+                {
+                    const uint32_t m0 = scale_pair(b_codes & 0xFFu), m1 = scale_pair((b_codes >> 8) & 0xFFu);
+                    const uint32_t m2 = scale_pair((b_codes >> 16) & 0xFFu), m3 = scale_pair(b_codes >> 24);
+                    uint8_t* dst = smem_gen + PK_STAGES * PK_STAGE_BYTES + bs * BF_STAGE_BYTES + row * 128;
+                    *reinterpret_cast<uint4*>(dst + ((0 ^ r7) << 4)) = dequant8(b0.x, m0);
+                    *reinterpret_cast<uint4*>(dst + ((1 ^ r7) << 4)) = dequant8(b0.y, m0);
+                    *reinterpret_cast<uint4*>(dst + ((2 ^ r7) << 4)) = dequant8(b0.z, m1);
+                    *reinterpret_cast<uint4*>(dst + ((3 ^ r7) << 4)) = dequant8(b0.w, m1);
+                    *reinterpret_cast<uint4*>(dst + ((4 ^ r7) << 4)) = dequant8(b1.x, m2);
+                    *reinterpret_cast<uint4*>(dst + ((5 ^ r7) << 4)) = dequant8(b1.y, m2);
+                    *reinterpret_cast<uint4*>(dst + ((6 ^ r7) << 4)) = dequant8(b1.z, m3);
+                    *reinterpret_cast<uint4*>(dst + ((7 ^ r7) << 4)) = dequant8(b1.w, m3);
+                }
+                tmem_st_wait();                      // the A slice is in tensor memory
+                fence_proxy_async();                 // the B slice is visible to the tensor core
+                tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(bf_full + 8 * grp, 0);
+                if (lane == 0) mbar_arrive_cluster(bf_full + 8 * bs, 0);
             }
         }
     }
@@ -493,6 +563,21 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t row
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output [Mo, No] with leading dimension ldo, stored in boxes of 32 x 32 elements whose shared-memory image is
+// swizzled (64-byte rows for BF16, 128-byte rows for FP32).
+bool make_out_map(CUtensorMap* m, void* out, bool bf16, int64_t Mo, int64_t No, int64_t ldo) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const uint64_t esz = bf16 ? 2 : 4;
+    cuuint64_t dims[2] = {(cuuint64_t)No, (cuuint64_t)Mo};
+    cuuint64_t strides[1] = {(cuuint64_t)ldo * esz};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_scale_map(CUtensorMap* m, const uint8_t* scales, int mode, int64_t R, int64_t Kc) {
     const uint64_t kb = (uint64_t)(Kc / 16);
     if (mode == UE5M3_SCALE_1D) return make_map(m, scales, kb, (uint64_t)R, kb, 16, 128, false);
@@ -527,6 +612,8 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BNH, true)) return UE5M3_ERR_CUDA;
     if (!make_scale_map(&mas, g.a_scales, g.a_scale_mode, g.Mo, g.Kc)) return UE5M3_ERR_CUDA;
     if (!make_scale_map(&mbs, g.b_scales, g.b_scale_mode, g.No, g.Kc)) return UE5M3_ERR_CUDA;
+    CUtensorMap mo;
+    if (!make_out_map(&mo, g.out, g.out_dtype == UE5M3_BF16, g.Mo, g.No, g.ldo)) return UE5M3_ERR_CUDA;
 
     GemmParams p;
     p.Mo = g.Mo; p.No = g.No; p.Kc = g.Kc; p.ldo = g.ldo;
@@ -538,7 +625,7 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int max_pairs = resident_pairs[dev];
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
-    gemm_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, p);
+    gemm_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, mo, p);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
