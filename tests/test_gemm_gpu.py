@@ -110,6 +110,26 @@ def test_linear_forward_backward_small(scale_layout):
     check_gemm_output(dw, yr, sa)
 
 
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_gemm_strided_output_and_ragged_tiles(out_dtype):
+    """Mo and No that are odd multiples of 128 (half-empty 256 x 256 tiles) written into a wider output buffer:
+    nothing outside the [Mo, No] window may be touched."""
+    rng = np.random.default_rng(77)
+    Mo, No, Kc = 384, 128, 512
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x60, 0x90, dec=1.0)
+    qb, bp, bsc = _operand(rng, No, Kc, 2, 0x60, 0x90, dec=0.5)
+    big = torch.full((Mo + 64, No + 192), 7.0, dtype=out_dtype, device=DEV)
+    view = big[:Mo, 64:64 + No]
+    lib.gemm(lib.FPROP, qa, qb, out=view)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    y, sa = oracle.gemm(ap, asc, False, 1.0, bp, bsc, True, 0.5)
+    check_gemm_output(view.contiguous(), y, sa)
+    guard = big.clone()
+    guard[:Mo, 64:64 + No] = 7.0
+    assert torch.all(guard == 7.0)
+
+
 def test_gemm_rejects_bad_shapes():
     rng = np.random.default_rng(1)
     qa, *_ = _operand(rng, 128, 256, 0)
