@@ -273,7 +273,7 @@ KERNEL_BYTES = kernel_bytes()
 GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the default workload (mean of fprop, dgrad, wgrad;
 # one ncu pass, summary in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt).  Algorithmic bytes: 242 MB per launch.
-GEMM_DRAM_TRAFFIC_BYTES = (140.4e6 + 214.8e6 + 194.1e6 + 47.0e6 + 95.3e6 + 95.4e6) / 3
+GEMM_DRAM_TRAFFIC_BYTES = (151.0e6 + 224.2e6 + 202.8e6 + 48.4e6 + 98.2e6 + 101.9e6) / 3
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
