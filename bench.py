@@ -473,6 +473,26 @@ def run_sweep(args):
     return out
 
 
+def run_sweep_oracle(args):
+    """The oracle's quantizer on the host cores, 2^24 elements (rows x 4096), GB/s of the same algorithmic bytes."""
+    import oracle
+    import synth_inputs as si
+    rows = (1 << 24) // 4096
+    x = si.to_numpy_bits(si.row_scaled_tensor(rows, 4096, seed=24))
+    g = oracle.amax(x)
+    row = {"impl": "oracle", "log2_elements": 24, "cores": oracle.num_threads()}
+    for lname, layout in (("1d_row", 0), ("1d_col", 1), ("2d", 2)):
+        for rname, rnd in (("rne", 0), ("sr", 1)):
+            t0 = time.perf_counter()
+            oracle.quantize(x, layout, rnd, g, 448.0, 1)
+            dt = time.perf_counter() - t0
+            row[f"{lname}_{rname}"] = {"ms": round(dt * 1e3, 1), "GB/s": round(_quant_bytes(rows, 4096, layout) / dt / 1e9, 3)}
+    t0 = time.perf_counter()
+    oracle.amax(x)
+    row["amax"] = {"ms": round((time.perf_counter() - t0) * 1e3, 1), "GB/s": round(rows * 4096 * 2 / (time.perf_counter() - t0) / 1e9, 3)}
+    print(json.dumps(row), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -492,6 +512,7 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+        run_sweep_oracle(args)
     else:
         run_ours(args)
 
