@@ -128,10 +128,12 @@ def test_config5_layer_stack(name, K, N):
     _check_linear(16384, K, N, seed=50 + (K + N) // 1024, n_bands=3, T_wgrad_dy=2048.0 if name == "mlp_down" else 448.0)
 
 
-def test_config3_large_quantizer_sizes():
-    """2^28 elements (rows x 4096): row bands against the oracle for every layout/rounding cell, amax exact."""
-    rows = (1 << 28) // 4096
-    x = si.row_scaled_tensor(rows, 4096, seed=28, device=DEV)
+@pytest.mark.parametrize("log2n", [28, 30])
+def test_config3_large_quantizer_sizes(log2n):
+    """2^28 and 2^30 elements (rows x 4096; 2^30 is the largest size of the sweep): row and column bands against
+    the oracle for every layout/rounding cell, amax exact."""
+    rows = (1 << log2n) // 4096
+    x = si.row_scaled_tensor(rows, 4096, seed=log2n, device=DEV)
     g = lib.sample_amax(x)
     rng = np.random.default_rng(3)
     gv = g.item()

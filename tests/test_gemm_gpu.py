@@ -130,6 +130,23 @@ def test_gemm_strided_output_and_ragged_tiles(out_dtype):
     assert torch.all(guard == 7.0)
 
 
+def test_gemm_and_quantizer_are_deterministic():
+    """Same inputs, same bytes: three runs of a linear's forward and backward give identical outputs."""
+    M, K, N = 512, 1024, 768
+    X = si.channel_scaled_activation(M, K, seed=5, device=DEV)
+    W = si.weight(N, K, seed=6, device=DEV)
+    dY = si.heavy_tailed_gradient(M, N, seed=7, device=DEV)
+    ax, aw, ag = lib.sample_amax(X), lib.sample_amax(W), lib.sample_amax(dY)
+    outs = []
+    for _ in range(3):
+        y, qx, qw = lib.linear_forward(X, W, ax, aw)
+        dx, dw = lib.linear_backward(dY, X, qw, ag, ax, seed=3)
+        torch.cuda.synchronize()
+        outs.append((y.clone(), dx.clone(), dw.clone(), qx.payload.clone(), qw.payload_t.clone()))
+    for o in outs[1:]:
+        assert all(torch.equal(a, b) for a, b in zip(outs[0], o))
+
+
 def test_gemm_rejects_bad_shapes():
     rng = np.random.default_rng(1)
     qa, *_ = _operand(rng, 128, 256, 0)

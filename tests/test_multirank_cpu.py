@@ -52,3 +52,24 @@ def test_reference_arm_prints_from_rank0_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "TFLOP/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def _amax_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2609_02846_b200.autograd import reduce_amax_
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    t = torch.tensor([1.5 + 2.0 * rank])                      # each rank sampled its own shard's maximum
+    reduce_amax_(t, dist.group.WORLD)
+    out[rank] = float(t.item())
+    dist.destroy_process_group()
+
+
+def test_refresh_step_amax_is_agreed_across_ranks():
+    """On refresh steps the sampled maxima are MAX-all-reduced (one float per operand): the only exchange of the path."""
+    port = 31500 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_amax_worker, args=(2, port, out), nprocs=2, join=True)
+        res = dict(out)
+    assert res[0] == res[1] == 3.5
