@@ -129,8 +129,8 @@ UE5M3_API int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t col
  * dW = dY^T X; Section 6.1: y = sum_k a_k b_k on the decoded operands, the tensor-scale product
  * applied after accumulation):
  *     C[Mo, No] = (d_A * d_B) * sum_k (s_hat q)_A[m, k] * (s_hat q)_B[n, k]
- * Both operands are K-major.  Every E2M1 x UE5M3 product is exact in BF16; products of two such
- * values are accumulated in FP32 on the tensor cores.  `op` only names the role of the call:
+ * Both operands are K-major.  Every E2M1 x UE5M3 product (times 2^-4) is exact in FP16, subnormals
+ * included; products of two such values are accumulated in FP32 on the tensor cores.  `op` only names the role of the call:
  *     FPROP  A = X  (1D_ROW),        B = W   (2D payload, scales)          Mo = tokens, No = out, Kc = in
  *     DGRAD  A = dY (1D_ROW, SR),    B = W^T (2D payload_t, scales_t)      Mo = tokens, No = in,  Kc = out
  *     WGRAD  A = dY^T (1D_COL, SR),  B = X^T (1D_COL)                      Mo = out,    No = in,  Kc = tokens

@@ -3,26 +3,30 @@
 // C[Mo,No] = (dA dB) * sum_k (s q)_A[m,k] (s q)_B[n,k], both operands K-major.
 //
 // UE5M3 is not a scale type the tensor cores understand, so the kernel turns every
-// (payload, scale) pair into the BF16 number s*q*2^-16 -- exact, because an E2M1 value has
-// at most 2 significant bits and a UE5M3 value at most 4 -- and runs dense BF16 tcgen05 MMAs with
-// FP32 accumulators in tensor memory.  The factor 2^-32 and the tensor decode factors are applied
-// to the accumulator in the epilogue.
+// (payload, scale) pair into the FP16 number s*q*2^-4 and runs dense 16-bit tcgen05 MMAs (kind::f16)
+// with FP32 accumulators in tensor memory.  The conversion is exact: q = n_q/2 with n_q <= 12 and
+// s = n_s * 2^-17 with at most 4 significant bits, so s*q*2^-4 = n_q n_s 2^-22 has at most 6 significant
+// bits, is a multiple of the FP16 subnormal step 2^-24 and is at most 6 * 61440 / 16 = 23040 < 65504.
+// FP16 rather than BF16 because UE5M3 is exactly the top byte of a positive FP16 (same bias, same
+// subnormal step: code << 7 IS the scale) and the hardware converts two E2M1 codes to an FP16 pair in
+// one instruction, which leaves one packed multiplication per two values as the only arithmetic.
+// The factor 2^8 and the tensor decode factors are applied to the accumulator in the epilogue.
 //
 // Persistent, one CTA per SM, CTAs paired into clusters of two that share one 256 x 256 output tile
 // (tcgen05 cta_group::2): each CTA owns 128 rows of A and 128 of the 256 B rows, so it stages and
 // dequantizes 128 + 128 rows per K slice for a 128 x 256 accumulator of its own.  The dequantized A
 // slice goes straight from registers into tensor memory (tcgen05.st; the MMA takes A from TMEM), only
 // the B slice goes through shared memory, which halves the shared-memory traffic of the main loop and
-// leaves room for eight BF16 stages.  Warp roles per CTA:
+// leaves room for eight FP16 stages.  Warp roles per CTA:
 //   warp 0        TMA producer: packed payload tiles (128B-swizzled) and scale tiles, 256 K per stage
-//   warp 1        MMA issuer (leader CTA only): 4 x tcgen05.mma (M256 N256 K16) per 64-wide BF16 stage
+//   warp 1        MMA issuer (leader CTA only): 4 x tcgen05.mma (M256 N256 K16) per 64-wide FP16 stage
 //   warp 2        tensor-memory allocation
 //   warps 4-7     epilogue: tcgen05.ld, scale, convert, stage in shared memory, TMA store
 //   warps 8-23    dequantizers, four groups of four warps.  Group g converts the g-th 64-wide slice of
 //                 every packed stage; thread t of a group owns row t of the A tile and row t of the B tile.
-//                 Each group ping-pongs between two BF16 stages, so it never waits for its own MMA.
+//                 Each group ping-pongs between two FP16 stages, so it never waits for its own MMA.
 // Tensor memory: columns 0..255 accumulator, columns 256..511 eight A stages of 32 columns.
-// The leader learns that both CTAs' BF16 stages are full through one mbarrier that the partner's
+// The leader learns that both CTAs' FP16 stages are full through one mbarrier that the partner's
 // dequantizers arrive on remotely; stage and accumulator releases come back to both CTAs through
 // tcgen05.commit with a two-CTA multicast mask.  No copy is multicast: every CTA loads its own tiles.
 // Every wait is bounded; a wait that gives up sets the device status word and the CTA drains.
@@ -42,10 +46,10 @@ constexpr int BM = 128;                     // A rows per CTA (256 per CTA pair)
 constexpr int BN = 256;                     // output columns per tile
 constexpr int BNH = 128;                    // B rows staged by each CTA of the pair
 constexpr int KCHUNK = 256;                 // K per packed stage
-constexpr int KSUB = 64;                    // K per BF16 stage (one 128-byte swizzle row)
+constexpr int KSUB = 64;                    // K per FP16 stage (one 128-byte swizzle row)
 constexpr int PK_STAGES = 2;
 constexpr int SLICES = KCHUNK / KSUB;       // 4 slices of 64 K per packed stage
-constexpr int BF_STAGES = 2 * SLICES;       // 8: every dequantizer group ping-pongs between two BF16 stages
+constexpr int BF_STAGES = 2 * SLICES;       // 8: every dequantizer group ping-pongs between two FP16 stages
 constexpr int DEQ_WARP0 = 8, DEQ_WARPS = 16, EPI_WARP0 = 4;
 constexpr int DEQ_GROUPS = SLICES;          // dequantizer group g owns slice g of every packed stage
 constexpr int GROUP_WARPS = DEQ_WARPS / DEQ_GROUPS;       // 4 warps = 128 threads = one thread per tile row
@@ -176,7 +180,7 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 // One M256 N256 K16 MMA of the CTA pair: D (tensor memory) (+)= A (tensor memory) * B (shared memory).
-__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
@@ -220,7 +224,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t r[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor of a K-major BF16 tile whose rows are 128 bytes (64 values),
+// Shared-memory matrix descriptor of a K-major 16-bit tile whose rows are 128 bytes (64 values),
 // 128B swizzle: 8-row groups are 1024 bytes apart (stride byte offset), leading byte offset unused (1).
 __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
     uint64_t d = 0;
@@ -231,38 +235,37 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
     d |= (uint64_t)2 << 61;                         // 128-byte swizzle
     return d;
 }
-// kind::f16 instruction descriptor: D = F32, A = B = BF16, both K-major, M = 256 (two CTAs), N = 256.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+// kind::f16 instruction descriptor: D = F32, A = B = F16 (format code 0), both K-major, M = 256 (two CTAs), N = 256.
+constexpr uint32_t kInstrDesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 
-__device__ __forceinline__ uint32_t hmul2_bf16(uint32_t a, uint32_t b) {
+__device__ __forceinline__ uint32_t hmul2_f16(uint32_t a, uint32_t b) {
     uint32_t r;
-    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));     // no .ftz: subnormals are kept
     return r;
 }
 
-// Multiplier s * 2^110 of one block as a BF16 pair.  (code << 4) read as BF16 is s * 2^-112
-// (UE5M3 and BF16 share the subnormal convention), so two exact power-of-two multiplications
-// (2^127, then 2^95) bring it there without leaving the BF16 range.
+// Multiplier s * 2^-4 of one block as an FP16 pair: (code << 7) read as FP16 is s itself, subnormal codes
+// included; the pre-scale keeps s*q inside FP16 and is exact (s * 2^-4 is a multiple of 2^-21).
 __device__ __forceinline__ uint32_t scale_pair(uint32_t code) {
-    const uint32_t raw = (code << 4) * 0x00010001u;
-    return hmul2_bf16(hmul2_bf16(raw, 0x7F007F00u /* 2^127 */), 0x6F006F00u /* 2^95 */);
+    return hmul2_f16((code << 7) * 0x00010001u, 0x2C002C00u /* 2^-4 */);
 }
 
-// Eight packed E2M1 codes -> eight BF16 values s*q*2^-16.  A code's three magnitude bits placed
-// at bits 8:6 of a BF16 read as q * 2^-126 (again the shared subnormal convention), the sign bit
-// goes to bit 15, and one packed multiplication by s * 2^110 finishes the job.  Output word k holds
-// elements k (low half) and k + 4 (high half); A and B use the same order, which a dot product
-// does not see.
+// Eight packed E2M1 codes -> eight FP16 values s*q*2^-4: four hardware conversions (two codes each) and four
+// packed multiplications.  Output word k holds elements 2k and 2k+1 in the order the conversion delivers
+// them; A and B go through the same function, so their K positions match.
 __device__ __forceinline__ uint4 dequant8(uint32_t w, uint32_t m) {
-    // One code per 16-bit half is isolated, then a multiplication by 2^a + 2^b drops its magnitude bits at
-    // bits 8:6 and its sign at bit 15 in one go (the two shifted copies never overlap, so the sum has no
-    // carries); the multiplications run on the FMA pipe and leave the integer pipe to the masks.
-    const uint32_t w8 = w >> 8;
     uint4 o;
-    o.x = hmul2_bf16(((w & 0x000F000Fu) * 0x1040u) & 0x81C081C0u, m);     // codes 0 and 4
-    o.y = hmul2_bf16(((w & 0x00F000F0u) * 0x0104u) & 0x81C081C0u, m);     // codes 1 and 5
-    o.z = hmul2_bf16(((w8 & 0x000F000Fu) * 0x1040u) & 0x81C081C0u, m);    // codes 2 and 6
-    o.w = hmul2_bf16(((w8 & 0x00F000F0u) * 0x0104u) & 0x81C081C0u, m);    // codes 3 and 7
+    asm("{ .reg .b8 b0, b1, b2, b3; .reg .b32 t0, t1, t2, t3;\n\t"
+        "mov.b32 {b0, b1, b2, b3}, %4;\n\t"
+        "cvt.rn.f16x2.e2m1x2 t0, b0;\n\t"
+        "cvt.rn.f16x2.e2m1x2 t1, b1;\n\t"
+        "cvt.rn.f16x2.e2m1x2 t2, b2;\n\t"
+        "cvt.rn.f16x2.e2m1x2 t3, b3;\n\t"
+        "mul.rn.f16x2 %0, t0, %5;\n\t"
+        "mul.rn.f16x2 %1, t1, %5;\n\t"
+        "mul.rn.f16x2 %2, t2, %5;\n\t"
+        "mul.rn.f16x2 %3, t3, %5;\n\t}"
+        : "=r"(o.x), "=r"(o.y), "=r"(o.z), "=r"(o.w) : "r"(w), "r"(m));
     return o;
 }
 
@@ -374,7 +377,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t ta = tmem_base + TMEM_A_COL + s * TMEM_A_STAGE_COLS;
 #pragma unroll
                     for (int k = 0; k < KSUB / 16; ++k)
-                        umma_bf16_ts(tmem_d, ta + k * 8, bd + (uint64_t)(k * 2), kInstrDesc, (ks | k) != 0 ? 1u : 0u);
+                        umma_f16_ts(tmem_d, ta + k * 8, bd + (uint64_t)(k * 2), kInstrDesc, (ks | k) != 0 ? 1u : 0u);
                     umma_commit_pair(bf_empty + 8 * s);        // both CTAs may refill this stage
                 }
                 if (ok) umma_commit_pair(acc_full);            // both CTAs' epilogues may read
@@ -386,7 +389,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lane quarter this warp may access
-        const float alpha = __fmul_rn(__fmul_rn(__ldg(p.a_decode), 65536.0f), __fmul_rn(__ldg(p.b_decode), 65536.0f));
+        const float alpha = __fmul_rn(__fmul_rn(__ldg(p.a_decode), 16.0f), __fmul_rn(__ldg(p.b_decode), 16.0f));
         // Staging: lane = output row.  The chunk is written in the swizzled layout the output tensor map expects
         // (conflict-free 16-byte stores) and leaves through the TMA engine, which keeps the row-scattered global
         // stores off the load/store pipe the dequantizers depend on.  The map clips rows >= Mo and columns >= No.
@@ -477,7 +480,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pk_empty + 8 * ps);
 
-                // this group's BF16 stage for this packed stage: two buffers, used alternately
+                // this group's FP16 stage for this packed stage: two buffers, used alternately
                 const uint32_t bs = grp + 4 * (it_pk & 1);
                 if (!mbar_wait(bf_empty + 8 * bs, ((it_pk >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
 

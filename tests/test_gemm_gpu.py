@@ -65,6 +65,32 @@ def test_gemm_whole_code_range_including_subnormal_and_zero_scales():
     assert np.array_equal(out.cpu().numpy().astype(np.float64), y)       # a single product has no rounding at all
 
 
+def test_every_operand_value_pair_multiplies_exactly():
+    """All 247 nonzero scale codes x 15 nonzero payload codes of A against the same set for B, one product per output:
+    the in-kernel FP16 reconstruction and the tensor-core product are exact for every operand value (subnormal scales
+    included), so the FP32 output equals the rational product bit for bit."""
+    pairs = [(sc, q) for sc in range(1, 0xF8) for q in list(range(1, 8)) + list(range(9, 16))]      # 247 * 14 values
+    R = ((len(pairs) + 127) // 128) * 128
+    Kc = 256
+    payload = np.zeros((R, Kc // 2), np.uint8)
+    scales = np.full((R, Kc // 16), 0x78, np.uint8)
+    for i, (sc, q) in enumerate(pairs):
+        payload[i, 0] = q
+        scales[i, 0] = sc
+    vals = np.zeros(R)
+    vals[:len(pairs)] = [oracle.ue5m3_value(sc) * oracle.e2m1_value(q) for sc, q in pairs]
+    dec = torch.ones(1, device=DEV)
+    qa = lib.QuantizedOperand(torch.from_numpy(payload).to(DEV), torch.from_numpy(scales).to(DEV), dec, lib.SCALE_1D)
+    # B gets the same values scaled down by 2^-20 through its decode factor so that the largest product fits FP32 output
+    qb = lib.QuantizedOperand(qa.payload.clone(), qa.scales.clone(), torch.full((1,), 2.0 ** -20, device=DEV), lib.SCALE_1D)
+    out = lib.gemm(lib.FPROP, qa, qb, torch.float32)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    want = np.outer(vals, vals) * 2.0 ** -20                  # exact in float64: at most 12 significant bits each
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.array_equal(got, want.astype(np.float32).astype(np.float64)) and np.array_equal(want, want.astype(np.float32))
+
+
 def test_small_forward_linear_fp32():
     """M = N = K = 256 forward linear in FP32 with outlier activations and current-amax scales."""
     X = si.outlier_activation(256, 256, seed=0, device=DEV)
