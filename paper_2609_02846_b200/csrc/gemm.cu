@@ -17,15 +17,16 @@
 // dequantizes 128 + 128 rows per K slice for a 128 x 256 accumulator of its own.  The dequantized A
 // slice goes straight from registers into tensor memory (tcgen05.st; the MMA takes A from TMEM), only
 // the B slice goes through shared memory, which halves the shared-memory traffic of the main loop and
-// leaves room for eight FP16 stages.  Warp roles per CTA:
+// leaves room for six FP16 stages next to three packed stages.  Warp roles per CTA:
 //   warp 0        TMA producer: packed payload tiles (128B-swizzled) and scale tiles, 256 K per stage
 //   warp 1        MMA issuer (leader CTA only): 4 x tcgen05.mma (M256 N256 K16) per 64-wide FP16 stage
 //   warp 2        tensor-memory allocation
 //   warps 4-7     epilogue: tcgen05.ld, scale, convert, stage in shared memory, TMA store
 //   warps 8-23    dequantizers, four groups of four warps.  Group g converts the g-th 64-wide slice of
 //                 every packed stage; thread t of a group owns row t of the A tile and row t of the B tile.
-//                 Each group ping-pongs between two FP16 stages, so it never waits for its own MMA.
-// Tensor memory: columns 0..255 accumulator, columns 256..511 eight A stages of 32 columns.
+//                 The six FP16 stages are used round-robin by slice number, so a group refills a stage one and
+//                 a half packed stages after it filled it and never waits for its own latest MMA.
+// Tensor memory: columns 0..255 accumulator, columns 256..447 six A stages of 32 columns.
 // The leader learns that both CTAs' FP16 stages are full through one mbarrier that the partner's
 // dequantizers arrive on remotely; stage and accumulator releases come back to both CTAs through
 // tcgen05.commit with a two-CTA multicast mask.  No copy is multicast: every CTA loads its own tiles.
@@ -47,9 +48,10 @@ constexpr int BN = 256;                     // output columns per tile
 constexpr int BNH = 128;                    // B rows staged by each CTA of the pair
 constexpr int KCHUNK = 256;                 // K per packed stage
 constexpr int KSUB = 64;                    // K per FP16 stage (one 128-byte swizzle row)
-constexpr int PK_STAGES = 2;
+constexpr int PK_STAGES = 3;                // the copy of a packed stage takes about as long as two stages of work
 constexpr int SLICES = KCHUNK / KSUB;       // 4 slices of 64 K per packed stage
-constexpr int BF_STAGES = 2 * SLICES;       // 8: every dequantizer group ping-pongs between two FP16 stages
+constexpr int BF_STAGES = 6;                // FP16 stages, used round-robin by slice number: a group reuses a stage
+                                            // six slices (one and a half packed stages) after it filled it
 constexpr int DEQ_WARP0 = 8, DEQ_WARPS = 16, EPI_WARP0 = 4;
 constexpr int DEQ_GROUPS = SLICES;          // dequantizer group g owns slice g of every packed stage
 constexpr int GROUP_WARPS = DEQ_WARPS / DEQ_GROUPS;       // 4 warps = 128 threads = one thread per tile row
@@ -61,7 +63,7 @@ constexpr int SC_A_BYTES = BM * (KCHUNK / 16);     // 2048
 constexpr int SC_B_BYTES = BNH * (KCHUNK / 16);    // 2048
 constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES;   // 36864
 constexpr int BF_STAGE_BYTES = BNH * KSUB * 2;     // 16384: the B slice; the A slice lives in tensor memory
-constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;  // 204800
+constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;  // 208896
 constexpr int SMEM_EPI = SMEM_TILES + 1024;        // epilogue staging (1024-aligned for the 128B swizzle) after the barriers
 constexpr int EPI_WARP_BYTES = 4096;               // one 32 x 32 FP32 chunk, or two 32 x 32 BF16 chunks, per epilogue warp
 constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;                     // + alignment slack
@@ -288,10 +290,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const uint32_t bf_base = smem_base + PK_STAGES * PK_STAGE_BYTES;
     const uint32_t bar_base = smem_base + SMEM_TILES;
     // barriers (8 bytes each)
-    const uint32_t pk_full = bar_base, pk_empty = bar_base + 16, bf_full = bar_base + 32, bf_empty = bar_base + 96;
-    const uint32_t acc_full = bar_base + 160, acc_empty = bar_base + 168, drain_bar = bar_base + 176;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 192);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 200);
+    const uint32_t pk_full = bar_base, pk_empty = bar_base + 32, bf_full = bar_base + 64, bf_empty = bar_base + 128;
+    const uint32_t acc_full = bar_base + 192, acc_empty = bar_base + 200, drain_bar = bar_base + 208;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 216);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 224);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();                   // 0 = leader of the pair
@@ -369,8 +371,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + TMEM_ACC_COL;
                 for (int ks = 0; ks < kchunks * SLICES; ++ks, ++it) {
-                    // slice it: group it % 4, its buffer (it / 4) & 1, used for the (it / 8)-th time
-                    const uint32_t s = (it & 3) + 4 * ((it >> 2) & 1), ph = (it >> 3) & 1;
+                    // slice number it (converted by group it % 4) lives in stage it % BF_STAGES
+                    const uint32_t s = it % BF_STAGES, ph = (it / BF_STAGES) & 1;
                     if (!mbar_wait(bf_full + 8 * s, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t bd = umma_smem_desc(bf_base + s * BF_STAGE_BYTES);
@@ -480,9 +482,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pk_empty + 8 * ps);
 
-                // this group's FP16 stage for this packed stage: two buffers, used alternately
-                const uint32_t bs = grp + 4 * (it_pk & 1);
-                if (!mbar_wait(bf_empty + 8 * bs, ((it_pk >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                // the FP16 stage of this slice; it is free once the MMAs of slice number - BF_STAGES have retired
+                const uint32_t slice_no = it_pk * SLICES + grp;
+                const uint32_t bs = slice_no % BF_STAGES;
+                if (!mbar_wait(bf_empty + 8 * bs, ((slice_no / BF_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
 
                 // A: 64 values of this row -> 32 tensor-memory columns (column c = K positions 2c, 2c+1)
                 {
