@@ -317,8 +317,9 @@ def run_ours(args):
     K, Wm = args.steps, max(args.warmup, 3)
 
     sampler = ClockSampler(dev)
-    sampler.start()          # started before the warm-up: its own start-up must not fall into the timed region
-    sampler.wait_first_sample()
+    if rank == 0:
+        sampler.start()      # started before the warm-up: its own start-up must not fall into the timed region
+        sampler.wait_first_sample()
     for s in range(Wm):
         step.run(s)
     barrier()

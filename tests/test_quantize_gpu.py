@@ -152,6 +152,47 @@ def test_sample_amax(dtype, shape):
     assert lib.sample_amax(torch.zeros(16, 16, dtype=dtype, device=DEV)).item() == 0.0
 
 
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("scale_layout", [0, 1])
+def test_outputs_stay_inside_their_buffers(layout, scale_layout):
+    """Guard bands around every output buffer: the kernels write exactly the bytes the header promises."""
+    import paper_2609_02846_b200 as lib
+    if layout == oracle.LAYOUT_2D and scale_layout == 1:
+        pytest.skip("tiled scales exist for 1D layouts only")
+    rows, cols = 304, 400                                     # multiples of 16 that are not multiples of any tile size
+    x = si.row_scaled_tensor(rows, cols, seed=12, device=DEV)
+    g = torch.tensor([_amax(x)], device=DEV)
+    R, Kc = (cols, rows) if layout == oracle.LAYOUT_1D_COL else (rows, cols)
+    n_pay = R * Kc // 2
+    n_sc = lib.scales_bytes(rows, cols, layout, scale_layout)
+    GUARD, FILL = 256, 0xA5
+
+    def guarded(n):
+        buf = torch.full((n + 2 * GUARD,), FILL, dtype=torch.uint8, device=DEV)
+        return buf, buf[GUARD:GUARD + n]
+
+    pb, pay = guarded(n_pay); sb, sc = guarded(n_sc)
+    ptb, pay_t = guarded(n_pay); stb, sc_t = guarded(n_sc)
+    dec = torch.full((3,), -7.0, device=DEV)
+    stats = torch.zeros(6, dtype=torch.int64, device=DEV); stats[0] = -1; stats[5] = -1
+    two_d = layout == oracle.LAYOUT_2D
+    out = lib.QuantizedOperand(pay.view(R, Kc // 2), sc if scale_layout else sc.view(-1, Kc // 16), dec[1:2],
+                               lib.SCALE_2D if two_d else lib.SCALE_1D,
+                               pay_t.view(Kc, R // 2) if two_d else None, sc_t.view(Kc // 16, R // 16) if two_d else None)
+    lib.quantize(x, layout, oracle.ROUND_SR, g, 448.0, seed=5, stats=stats[1:5], scale_layout=scale_layout, out=out)
+    torch.cuda.synchronize()
+    for buf in (pb, sb) + ((ptb, stb) if two_d else ()):
+        assert torch.all(buf[:GUARD] == FILL) and torch.all(buf[-GUARD:] == FILL)
+    if not two_d:
+        assert torch.all(ptb == FILL) and torch.all(stb == FILL)
+    assert dec[0].item() == -7.0 and dec[2].item() == -7.0 and dec[1].item() > 0
+    assert stats[0].item() == -1 and stats[5].item() == -1
+    want = oracle_quantize(x, layout, oracle.ROUND_SR, g.item(), 448.0, seed=5, want_t=two_d)
+    assert np.array_equal(pay.view(R, Kc // 2).cpu().numpy(), want["payload"])
+    if two_d:
+        assert np.array_equal(pay_t.view(Kc, R // 2).cpu().numpy(), want["payload_t"])
+
+
 def test_argument_errors_are_reported_not_executed():
     import paper_2609_02846_b200 as lib
     x = torch.zeros(32, 40, dtype=torch.bfloat16, device=DEV)
@@ -168,3 +209,7 @@ def test_argument_errors_are_reported_not_executed():
     assert e.value.status == 3
     with pytest.raises(TypeError):
         lib.quantize(x.half(), lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
+    with pytest.raises(lib.Ue5m3Error):                       # empty input: nothing to quantize is an argument error
+        lib.quantize(x[:0], lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
+    with pytest.raises(lib.Ue5m3Error):
+        lib.sample_amax(x[:0])
