@@ -1,5 +1,7 @@
 """Parity of the CUDA quantizer and tensor maximum with the CPU oracle: every payload byte, scale
 byte, decode factor, stochastic-rounding draw and counter must be identical."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -213,3 +215,32 @@ def test_argument_errors_are_reported_not_executed():
         lib.quantize(x[:0], lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
     with pytest.raises(lib.Ue5m3Error):
         lib.sample_amax(x[:0])
+
+
+def test_philox_matches_curand_device_generator(tmp_path):
+    """The oracle's Philox4x32-10 against cuRAND's device implementation on random counters and keys (the CUDA
+    quantizer's draws are already bit-identical to the oracle's)."""
+    import ctypes
+    import shutil
+    import subprocess
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    if not os.path.exists(nvcc):
+        pytest.skip("nvcc not available to build the cuRAND helper")
+    so = str(tmp_path / "libcurand_philox_check.so")
+    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "curand_philox_check.cu")
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O2", "-shared", "-Xcompiler", "-fPIC", "-o", so, src],
+                   check=True)
+    helper = ctypes.CDLL(so)
+    rng = np.random.default_rng(99)
+    n = 512
+    ctr = rng.integers(0, 2 ** 32, (n, 4), dtype=np.uint32)
+    key = rng.integers(0, 2 ** 32, (n, 2), dtype=np.uint32)
+    ctr[0] = 0; key[0] = 0; ctr[1] = 0xFFFFFFFF; key[1] = 0xFFFFFFFF
+    d_ctr = torch.from_numpy(ctr.view(np.int32)).to(DEV); d_key = torch.from_numpy(key.view(np.int32)).to(DEV)
+    d_out = torch.zeros((n, 4), dtype=torch.int32, device=DEV)
+    rc = helper.curand_philox_blocks(ctypes.c_void_p(d_ctr.data_ptr()), ctypes.c_void_p(d_key.data_ptr()),
+                                     ctypes.c_void_p(d_out.data_ptr()), n)
+    assert rc == 0
+    got = d_out.cpu().numpy().view(np.uint32)
+    for i in range(n):
+        assert list(got[i]) == list(oracle.philox4x32_10(ctr[i], key[i]))
