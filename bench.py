@@ -62,7 +62,7 @@ def measured_peaks():
 # ------------------------------------------------------------------------------------------------
 # CPU oracle arm (the benchmark's cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-SAMPLE_M, SAMPLE_N = 256, 1024
+SAMPLE_M, SAMPLE_N = 512, 1024
 SAMPLE_DESC = (f"same linear cut to M={SAMPLE_M} tokens, K={K_IN}, N={SAMPLE_N}: 5 oracle quantizations + 3 exact "
                "oracle GEMMs, all host threads")
 
