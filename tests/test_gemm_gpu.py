@@ -156,6 +156,25 @@ def test_gemm_strided_output_and_ragged_tiles(out_dtype):
     assert torch.all(guard == 7.0)
 
 
+def test_gemm_random_shapes_and_modes():
+    """A seeded sweep over tile-ragged shapes, scale storage modes, output types and decode factors."""
+    rng = np.random.default_rng(2024)
+    for case in range(16):
+        Mo = int(rng.integers(1, 6)) * 128
+        No = int(rng.integers(1, 6)) * 128
+        Kc = int(rng.integers(1, 5)) * 256
+        ma, mb = int(rng.integers(0, 3)), int(rng.integers(0, 3))
+        out_dtype = torch.float32 if rng.integers(0, 2) else torch.bfloat16
+        da, db = float(np.float32(10.0 ** rng.uniform(-6, 2))), float(np.float32(10.0 ** rng.uniform(-6, 2)))
+        qa, ap, asc = _operand(rng, Mo, Kc, ma, 0x30, 0xA0, dec=da)
+        qb, bp, bsc = _operand(rng, No, Kc, mb, 0x30, 0xA0, dec=db)
+        out = lib.gemm(int(rng.integers(0, 3)), qa, qb, out_dtype)
+        torch.cuda.synchronize()
+        assert lib.last_device_status() == 0
+        y, sa = oracle.gemm(ap, asc, ma == 2, np.float32(da), bp, bsc, mb == 2, np.float32(db))
+        check_gemm_output(out, y, sa)
+
+
 def test_gemm_and_quantizer_are_deterministic():
     """Same inputs, same bytes: three runs of a linear's forward and backward give identical outputs."""
     M, K, N = 512, 1024, 768
