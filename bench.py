@@ -457,14 +457,21 @@ def run_sweep(args):
         for name, (fn, nbytes) in cells.items():
             for _ in range(3):
                 fn()
+            torch.cuda.synchronize()
+            # one launch captured in a CUDA graph: the replay keeps the Python/ctypes call (5-10 us of host time)
+            # out of the device timeline, which matters for the small tensors
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fn()
             ts = []
             for _ in range(args.sweep_iters):
                 if nbytes < (256 << 20):
                     flush.zero_()                      # inputs that fit in L2: flush it between timed launches
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(); fn(); b.record()
+                a.record(); graph.replay(); b.record()
                 torch.cuda.synchronize()
                 ts.append(a.elapsed_time(b))
+            del graph
             ms = statistics.median(ts)
             gbs = nbytes / (ms * 1e-3) / 1e9
             row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3)}
