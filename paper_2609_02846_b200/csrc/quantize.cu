@@ -157,20 +157,28 @@ __device__ __forceinline__ void load_row8(const void* x, int64_t off, float f[8]
     }
 }
 
-// MODE 0: column blocks (output = quantized transpose).  Lane = 2 column groups x 16 row blocks,
-//         so that the 8-byte payload pieces of one output row are contiguous across 16 lanes.
-// MODE 1: 2D tiles.  Lane = 16 column groups x 2 row blocks, so that loads and row-major payload
-//         stores are contiguous across 16 lanes; lanes 2i and 2i+1 hold the halves of one tile.
+// Lane = 16 column groups x 2 row blocks in modes 0 and 1, so that every load instruction of a warp reads 256
+// contiguous bytes of two rows.
+// MODE 0: column blocks (output = quantized transpose): payload and scales go through shared memory and
+//         leave as 16-byte pieces of the transposed rows.  Used for round-to-nearest, which is HBM-bound.
+// MODE 2: column blocks with lane = 2 column groups x 16 row blocks: the 8-byte payload pieces and the scale
+//         bytes of one output row are contiguous across 16 lanes and are stored directly.  Used for stochastic
+//         rounding, which is bound by integer arithmetic and is better off without the staging work.
+// MODE 1: 2D tiles: lanes 2i and 2i+1 hold the halves of one tile; the row-major payload is stored directly
+//         (64 contiguous bytes per row and warp), the optional transposed copy goes through shared memory.
 template <bool IS_BF16, bool SR, bool STATS, int MODE, bool TILED, bool WANT_T>
 __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a) {
-    __shared__ __align__(16) uint8_t s_t[(MODE == 1 && WANT_T) ? kTileCols * (kTileRows / 2) : 16];
+    constexpr bool kColumns = (MODE == 0) || (MODE == 2);
+    constexpr bool kTranspose = (MODE == 0) || WANT_T;
+    __shared__ __align__(16) uint8_t s_t[kTranspose ? kTileCols * (kTileRows / 2) : 16];
+    __shared__ __align__(16) uint8_t s_sc[(MODE == 0) ? (kTileRows / 16) * kTileCols : 16];   // [row block][column]
 
     const TensorConsts tc = cta_tensor_consts(a.amax_held, a.T);
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tc.d;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int cg, rb;   // column group (8 columns) and row block (16 rows) inside the CTA tile
-    if (MODE == 0) { cg = warp * 2 + (lane >> 4); rb = lane & 15; }
+    if (MODE == 2) { cg = warp * 2 + (lane >> 4); rb = lane & 15; }
     else           { cg = lane & 15;              rb = warp * 2 + (lane >> 4); }
     const int64_t c0 = (int64_t)blockIdx.x * kTileCols + cg * 8;
     const int64_t r0 = (int64_t)blockIdx.y * kTileRows + rb * 16;
@@ -214,7 +222,7 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
     float rcol[8];
     uint32_t codes[8];
     uint32_t sat = 0, rep = 0;
-    if (MODE == 0) {
+    if (kColumns) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t fl;
@@ -270,7 +278,7 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
         return wv;
     };
 
-    if (MODE == 0) {
+    if (MODE == 2) {
         if (live) {
             const int64_t kblocks = a.rows >> 4;
             const int64_t rblk = r0 >> 4;
@@ -284,7 +292,8 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
                 a.scales[so] = (uint8_t)codes[j];
             }
         }
-    } else {
+    }
+    if (MODE == 1) {
         if (live) {
 #pragma unroll
             for (int r = 0; r < 16; ++r)
@@ -294,37 +303,64 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
                 if (WANT_T) a.scales_t[(c0 >> 4) * (a.rows >> 4) + (r0 >> 4)] = (uint8_t)codes[0];
             }
         }
-        if (WANT_T) {
-            // shared transpose: s_t[column][row/2], 128 bytes per column, written as 8-byte pieces
-            // whose position is rotated by the column group to spread the banks
+    }
+    if (kTranspose) {
+        // shared transpose: s_t[column][row/2], 128 bytes per column, written as 8-byte pieces
+        // whose position is rotated by the column group to spread the banks
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint2 o;
-                o.x = column_word(j, 0);
-                o.y = column_word(j, 1);
-                const int col = cg * 8 + j;
-                const int piece = (rb + cg) & 15;
-                *reinterpret_cast<uint2*>(s_t + col * (kTileRows / 2) + piece * 8) = o;
+        for (int j = 0; j < 8; ++j) {
+            uint2 o;
+            o.x = column_word(j, 0);
+            o.y = column_word(j, 1);
+            const int col = cg * 8 + j;
+            const int piece = (rb + cg) & 15;
+            *reinterpret_cast<uint2*>(s_t + col * (kTileRows / 2) + piece * 8) = o;
+        }
+        if (MODE == 0) {
+            // scale bytes of this row block for the thread's eight columns (8 contiguous bytes)
+            *reinterpret_cast<uint2*>(s_sc + rb * kTileCols + cg * 8) =
+                make_uint2(codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24),
+                           codes[4] | (codes[5] << 8) | (codes[6] << 16) | (codes[7] << 24));
+        }
+        __syncthreads();
+        uint8_t* const out_t = (MODE == 0) ? a.payload : a.payload_t;
+        // each column of the CTA tile is 128 contiguous output bytes: 8 lanes x 16 bytes
+        const int64_t rbase = (int64_t)blockIdx.y * kTileRows;
+        const bool al16 = ((a.rows >> 1) & 15) == 0;     // output rows start on 16-byte boundaries
+        for (int t = threadIdx.x; t < kTileCols * 8; t += kTileThreads) {
+            const int col = t >> 3, q = t & 7;          // q: 16-byte chunk = row blocks 2q, 2q+1
+            const int64_t c = (int64_t)blockIdx.x * kTileCols + col;
+            const int64_t rr = rbase + q * 32;
+            if (c < a.cols && rr < a.rows) {
+                const int g = col >> 3;
+                const uint2 lo = *reinterpret_cast<const uint2*>(s_t + col * (kTileRows / 2) + (((2 * q) + g) & 15) * 8);
+                const uint2 hi = *reinterpret_cast<const uint2*>(s_t + col * (kTileRows / 2) + (((2 * q + 1) + g) & 15) * 8);
+                uint8_t* dst = out_t + c * (a.rows >> 1) + (rr >> 1);
+                const bool both = rr + 16 < a.rows;
+                if (both && al16) *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                else {
+                    *reinterpret_cast<uint2*>(dst) = lo;
+                    if (both) *reinterpret_cast<uint2*>(dst + 8) = hi;
+                }
             }
-            __syncthreads();
-            // each column of the CTA tile is 128 contiguous output bytes: 8 lanes x 16 bytes
-            const int64_t rbase = (int64_t)blockIdx.y * kTileRows;
-            const bool al16 = ((a.rows >> 1) & 15) == 0;     // output rows start on 16-byte boundaries
-            for (int t = threadIdx.x; t < kTileCols * 8; t += kTileThreads) {
-                const int col = t >> 3, q = t & 7;          // q: 16-byte chunk = row blocks 2q, 2q+1
+        }
+        if (MODE == 0) {
+            // scales of the transposed operand: [column][row block]; the 16 row blocks of this CTA tile are
+            // contiguous for a column, so one thread per column writes them (16 bytes at once when aligned)
+            const int64_t kblocks = a.rows >> 4;
+            const int64_t kb0 = (int64_t)blockIdx.y * (kTileRows / 16);
+            for (int col = threadIdx.x; col < kTileCols; col += kTileThreads) {
                 const int64_t c = (int64_t)blockIdx.x * kTileCols + col;
-                const int64_t rr = rbase + q * 32;
-                if (c < a.cols && rr < a.rows) {
-                    const int g = col >> 3;
-                    const uint2 lo = *reinterpret_cast<const uint2*>(s_t + col * (kTileRows / 2) + (((2 * q) + g) & 15) * 8);
-                    const uint2 hi = *reinterpret_cast<const uint2*>(s_t + col * (kTileRows / 2) + (((2 * q + 1) + g) & 15) * 8);
-                    uint8_t* dst = a.payload_t + c * (a.rows >> 1) + (rr >> 1);
-                    const bool both = rr + 16 < a.rows;
-                    if (both && al16) *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
-                    else {
-                        *reinterpret_cast<uint2*>(dst) = lo;
-                        if (both) *reinterpret_cast<uint2*>(dst + 8) = hi;
-                    }
+                if (c >= a.cols) continue;
+                uint32_t w4[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w4[k >> 2] |= (uint32_t)s_sc[k * kTileCols + col] << (8 * (k & 3));
+                const int nvalid = (int)((kblocks - kb0) < 16 ? (kblocks - kb0) : 16);
+                uint8_t* dst = a.scales + (TILED ? tiled_scale_offset(c, kb0, kblocks) : c * kblocks + kb0);
+                if (nvalid == 16 && (TILED || (kblocks & 15) == 0)) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                } else {
+                    for (int k = 0; k < nvalid; ++k) dst[k] = (uint8_t)(w4[k >> 2] >> (8 * (k & 3)));
                 }
             }
         }
@@ -414,8 +450,9 @@ template <bool IS_BF16, bool SR, bool STATS>
 static cudaError_t launch_tile(const QuantArgs& a, int layout, bool tiled, cudaStream_t st) {
     dim3 grid((unsigned)((a.cols + kTileCols - 1) / kTileCols), (unsigned)((a.rows + kTileRows - 1) / kTileRows));
     if (layout == UE5M3_LAYOUT_1D_COL) {
-        if (tiled) quantize_tile_kernel<IS_BF16, SR, STATS, 0, true, false><<<grid, kTileThreads, 0, st>>>(a);
-        else       quantize_tile_kernel<IS_BF16, SR, STATS, 0, false, false><<<grid, kTileThreads, 0, st>>>(a);
+        constexpr int kMode = SR ? 2 : 0;
+        if (tiled) quantize_tile_kernel<IS_BF16, SR, STATS, kMode, true, false><<<grid, kTileThreads, 0, st>>>(a);
+        else       quantize_tile_kernel<IS_BF16, SR, STATS, kMode, false, false><<<grid, kTileThreads, 0, st>>>(a);
     } else {
         if (a.payload_t) quantize_tile_kernel<IS_BF16, SR, STATS, 1, false, true><<<grid, kTileThreads, 0, st>>>(a);
         else             quantize_tile_kernel<IS_BF16, SR, STATS, 1, false, false><<<grid, kTileThreads, 0, st>>>(a);
