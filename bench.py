@@ -455,7 +455,7 @@ def run_sweep(args):
                                              _quant_bytes(rows, 4096, layout))
         row = {"log2_elements": log2n}
         for name, (fn, nbytes) in cells.items():
-            for _ in range(3):
+            for _ in range(args.sweep_warmup):
                 fn()
             torch.cuda.synchronize()
             # one launch captured in a CUDA graph: the replay keeps the Python/ctypes call (5-10 us of host time)
@@ -474,7 +474,8 @@ def run_sweep(args):
             del graph
             ms = statistics.median(ts)
             gbs = nbytes / (ms * 1e-3) / 1e9
-            row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+            row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3),
+                         "best_GB/s": round(nbytes / (min(ts) * 1e-3) / 1e9, 1)}
         out.append(row)
         print(json.dumps(row), flush=True)
         del x
@@ -482,23 +483,29 @@ def run_sweep(args):
 
 
 def run_sweep_oracle(args):
-    """The oracle's quantizer on the host cores, 2^24 elements (rows x 4096), GB/s of the same algorithmic bytes."""
+    """The oracle's quantizer on the host cores (all cores at 2^24 and 2^26 elements, one core at 2^24), rows x 4096,
+    GB/s of the same algorithmic bytes."""
     import oracle
     import synth_inputs as si
-    rows = (1 << 24) // 4096
-    x = si.to_numpy_bits(si.row_scaled_tensor(rows, 4096, seed=24))
-    g = oracle.amax(x)
-    row = {"impl": "oracle", "log2_elements": 24, "cores": oracle.num_threads()}
-    for lname, layout in (("1d_row", 0), ("1d_col", 1), ("2d", 2)):
-        for rname, rnd in (("rne", 0), ("sr", 1)):
-            t0 = time.perf_counter()
-            oracle.quantize(x, layout, rnd, g, 448.0, 1)
-            dt = time.perf_counter() - t0
-            row[f"{lname}_{rname}"] = {"ms": round(dt * 1e3, 1), "GB/s": round(_quant_bytes(rows, 4096, layout) / dt / 1e9, 3)}
-    t0 = time.perf_counter()
-    oracle.amax(x)
-    row["amax"] = {"ms": round((time.perf_counter() - t0) * 1e3, 1), "GB/s": round(rows * 4096 * 2 / (time.perf_counter() - t0) / 1e9, 3)}
-    print(json.dumps(row), flush=True)
+    all_cores = oracle.num_threads()
+    for log2n, cores in ((24, all_cores), (26, all_cores), (24, 1)):
+        rows = (1 << log2n) // 4096
+        x = si.to_numpy_bits(si.row_scaled_tensor(rows, 4096, seed=log2n))
+        oracle.set_num_threads(cores)
+        g = oracle.amax(x)
+        row = {"impl": "oracle", "log2_elements": log2n, "cores": cores}
+        for lname, layout in (("1d_row", 0), ("1d_col", 1), ("2d", 2)):
+            for rname, rnd in (("rne", 0), ("sr", 1)):
+                t0 = time.perf_counter()
+                oracle.quantize(x, layout, rnd, g, 448.0, 1)
+                dt = time.perf_counter() - t0
+                row[f"{lname}_{rname}"] = {"ms": round(dt * 1e3, 1), "GB/s": round(_quant_bytes(rows, 4096, layout) / dt / 1e9, 3)}
+        t0 = time.perf_counter()
+        oracle.amax(x)
+        dt = time.perf_counter() - t0
+        row["amax"] = {"ms": round(dt * 1e3, 2), "GB/s": round(rows * 4096 * 2 / dt / 1e9, 3)}
+        print(json.dumps(row), flush=True)
+    oracle.set_num_threads(all_cores)
 
 
 def main():
@@ -510,8 +517,9 @@ def main():
     ap.add_argument("--scale-layout", type=int, default=0, choices=[0, 1])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true")
-    ap.add_argument("--sweep-iters", type=int, default=20)
-    ap.add_argument("--sweep-stride", type=int, default=2)
+    ap.add_argument("--sweep-iters", type=int, default=100)
+    ap.add_argument("--sweep-warmup", type=int, default=20)
+    ap.add_argument("--sweep-stride", type=int, default=1)
     ap.add_argument("--shape", default=None, help="M,K,N override for profiling runs (not the benchmark workload)")
     args = ap.parse_args()
     if args.shape:
