@@ -16,6 +16,7 @@ With N > 1 (launched by torchrun) every rank runs the same workload on its own t
 shards over tokens without any exchange, so scaling is "weak" and no collective is on the data path.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 `--sweep` prints the quantizer bandwidth sweep (2^20 .. 2^30 elements) instead of the step benchmark.
+`--stack` times every eligible linear of one 8B-hybrid-shaped layer stack at 16384 tokens.
 """
 from __future__ import annotations
 
@@ -434,6 +435,38 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_stack(args):
+    """One 8B-hybrid-shaped layer stack at 16384 tokens: every eligible linear fwd+bwd, per-linear and aggregate TFLOP/s."""
+    import torch
+    import paper_2609_02846_b200 as lib
+    import synth_inputs as si
+    dev = torch.device("cuda", 0)
+    tokens, out, total_flops, total_ms = 16384, {}, 0.0, 0.0
+    for name, k, n in si.LAYER_STACK:
+        set_shape(tokens, k, n)
+        step = LinearStep(dev, seed=7)
+        for s in range(3):
+            step.run(s)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        iters = max(5, args.steps // 10)
+        a.record()
+        for s in range(iters):
+            step.run(3 + s)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / iters
+        out[name] = {"in": k, "out": n, "ms": round(ms, 4), "TFLOP/s": round(FLOPS_PER_STEP / (ms * 1e-3) / 1e12, 1)}
+        total_flops += FLOPS_PER_STEP
+        total_ms += ms
+        del step
+        torch.cuda.empty_cache()
+    status = lib.last_device_status()
+    print(json.dumps({"workload": "layer stack fwd+bwd, 16384 tokens, six linears", "linears": out, "total_flop": total_flops,
+                      "ms": round(total_ms, 4), "TFLOP/s": round(total_flops / (total_ms * 1e-3) / 1e12, 1),
+                      "device_status": status}), flush=True)
+
+
 def run_sweep(args):
     """Quantizer-only bandwidth sweep: BF16 [rows, 4096], 2^20 .. 2^30 elements, {1D, 2D} x {RNE, SR} + amax."""
     import torch
@@ -517,6 +550,7 @@ def main():
     ap.add_argument("--scale-layout", type=int, default=0, choices=[0, 1])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--stack", action="store_true", help="time the six linears of the 8B-hybrid-shaped layer stack")
     ap.add_argument("--sweep-iters", type=int, default=100)
     ap.add_argument("--sweep-warmup", type=int, default=20)
     ap.add_argument("--sweep-stride", type=int, default=1)
@@ -529,6 +563,8 @@ def main():
     elif args.sweep:
         run_sweep(args)
         run_sweep_oracle(args)
+    elif args.stack:
+        run_stack(args)
     else:
         run_ours(args)
 
