@@ -313,6 +313,12 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     import paper_2609_02846_b200 as lib
+    if not os.path.exists(lib.library_path()):
+        if local == 0:
+            from paper_2609_02846_b200.build import build_library
+            build_library()                     # build product missing (fresh tree): compile it once per node
+        if world > 1:
+            dist.barrier()
     peaks = measured_peaks()
     step = LinearStep(dev, seed=rank, scale_layout=args.scale_layout)
     K, Wm = args.steps, max(args.warmup, 3)

@@ -43,3 +43,17 @@ def read_printed_values():
 @pytest.fixture(scope="session")
 def printed():
     return read_printed_values()
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """On a GPU machine make sure the in-tree CUDA library exists and is current before any GPU test loads it
+    (the library is a build product and is not kept in version control)."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            from paper_2609_02846_b200.build import build_library
+            build_library()
+    except ImportError:
+        pass
+    yield
