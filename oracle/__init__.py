@@ -74,6 +74,15 @@ def lib() -> C.CDLL:
         L.oracle_gemm.argtypes = [i64, i64, i64, vp, vp, C.c_int, f32, vp, vp, C.c_int, f32, vp, vp]
         L.oracle_gemm_cells.restype = None
         L.oracle_gemm_cells.argtypes = [i64, vp, vp, C.c_int, f32, vp, vp, C.c_int, f32, i64, vp, vp, vp, vp]
+        L.oracle_probe_partial.restype = f32
+        L.oracle_probe_partial.argtypes = [i64, vp, vp, C.c_int, vp, vp, C.c_int, i64, i64, i64]
+        L.oracle_probe_combine.restype = f32
+        L.oracle_probe_combine.argtypes = [vp, i64, C.c_int, C.c_int]
+        L.oracle_gemm_probe.restype = None
+        L.oracle_gemm_probe.argtypes = [i64, i64, i64, vp, vp, C.c_int, f32, vp, vp, C.c_int, f32, C.c_int, C.c_int, vp]
+        L.oracle_gemm_probe_cells.restype = None
+        L.oracle_gemm_probe_cells.argtypes = [i64, vp, vp, C.c_int, f32, vp, vp, C.c_int, f32, C.c_int, C.c_int,
+                                              i64, vp, vp, vp]
         L.oracle_bf16_rne.restype = C.c_uint16
         L.oracle_bf16_rne.argtypes = [f64]
         L.oracle_bf16_rne_array.restype = None
@@ -226,6 +235,43 @@ def gemm_cells(ap, asc, a2d, dA, bp, bsc, b2d, dB, ci, cj):
                             _ptr(bp), _ptr(bsc), int(b2d), np.float32(dB),
                             ci.shape[0], _ptr(ci), _ptr(cj), _ptr(y), _ptr(sa))
     return y, sa
+
+
+# ---- GEMM output model of Section 6.2 (64-product RNE partials, RTZ cross-group adds, 1/d grid) ----
+def probe_partial(ap, asc, a2d, bp, bsc, b2d, i, j, group) -> np.float32:
+    """Eq. "issue-partial" for cell (i, j) and 64-product group `group`."""
+    Kc = 2 * ap.shape[1]
+    return np.float32(lib().oracle_probe_partial(Kc, _ptr(ap), _ptr(asc), int(a2d), _ptr(bp), _ptr(bsc), int(b2d),
+                                                 int(i), int(j), int(group)))
+
+
+def probe_combine(partials, cross_rne: bool = False, grid_d: int = 0) -> np.float32:
+    """Eq. "issue-rz" over the given binary32 partials in order, then Q_d (Eq. "grid-denominator")."""
+    p = np.ascontiguousarray(partials, dtype=np.float32)
+    return np.float32(lib().oracle_probe_combine(_ptr(p), p.shape[0], int(cross_rne), int(grid_d)))
+
+
+def gemm_probe(ap, asc, a2d, dA, bp, bsc, b2d, dB, cross_rne: bool = False, grid_d: int = 0) -> np.ndarray:
+    """C = alpha * Q_d(c_J) under the output model; binary32 [Mo, No]."""
+    Mo, Kc = ap.shape[0], 2 * ap.shape[1]
+    No = bp.shape[0]
+    assert bp.shape[1] * 2 == Kc and Kc % 64 == 0
+    y = np.zeros((Mo, No), np.float32)
+    lib().oracle_gemm_probe(Mo, No, Kc, _ptr(ap), _ptr(asc), int(a2d), np.float32(dA),
+                            _ptr(bp), _ptr(bsc), int(b2d), np.float32(dB), int(cross_rne), int(grid_d), _ptr(y))
+    return y
+
+
+def gemm_probe_cells(ap, asc, a2d, dA, bp, bsc, b2d, dB, ci, cj, cross_rne: bool = False, grid_d: int = 0):
+    Kc = 2 * ap.shape[1]
+    assert Kc % 64 == 0
+    ci = np.ascontiguousarray(ci, dtype=np.int64)
+    cj = np.ascontiguousarray(cj, dtype=np.int64)
+    y = np.zeros(ci.shape[0], np.float32)
+    lib().oracle_gemm_probe_cells(Kc, _ptr(ap), _ptr(asc), int(a2d), np.float32(dA),
+                                  _ptr(bp), _ptr(bsc), int(b2d), np.float32(dB), int(cross_rne), int(grid_d),
+                                  ci.shape[0], _ptr(ci), _ptr(cj), _ptr(y))
+    return y
 
 
 def num_threads() -> int:

@@ -28,6 +28,10 @@
  *     in bits 7:4.  The sign of zero is kept.  NaN payload encodes as +6.
  *   - stochastic rounding bits: Philox4x32-10, one call per 8 consecutive
  *     source elements, 16 bits per element (see oracle_sr_bits).
+ *   - GEMM output model (Section 6.2): groups are the 64 consecutive K indices
+ *     64g..64g+63 in ascending order; the partials are of the decoded operands
+ *     s_hat * q; the scale product is alpha = RNE32(dA * dB) and the output is
+ *     RNE32(alpha * Q_d(c)).  The grid step is optional (d = 0 turns it off).
  */
 #include <math.h>
 #include <stdint.h>
@@ -449,6 +453,123 @@ ORACLE_API void oracle_gemm_cells(int64_t Kc,
     #pragma omp parallel for schedule(static)
     for (int64_t t = 0; t < n; ++t)
         exact_cell(Kc, ap, as, a2d, dA, bp, bs, b2d, dB, ci[t], cj[t], &y[t], &sumabs[t]);
+}
+
+/* ------------------------------------------------------------------ */
+/* GEMM output model of Section 6.2 ("probe-matched" accumulation):    */
+/* Eq. "issue-partial", Eq. "issue-rz", Eq. "final-grid"/"grid-        */
+/* denominator".  All values are IEEE-754 binary32.                     */
+/* ------------------------------------------------------------------ */
+
+/* Round-to-nearest-even to binary32 of v * 2^unit_exp for an exact integer v
+ * (|v| < 2^120, results stay inside the normal binary32 range here). */
+static float rne32_of_units(__int128 v, int unit_exp)
+{
+    if (v == 0) return 0.0f;
+    int neg = v < 0;
+    unsigned __int128 a = neg ? (unsigned __int128)(-v) : (unsigned __int128)v;
+    int msb = 127;
+    while (!((a >> msb) & 1)) --msb;                 /* position of the leading one */
+    int shift = msb - 23;                            /* bits dropped to keep 24 */
+    uint32_t q;
+    if (shift <= 0) {
+        q = (uint32_t)a;
+        shift = 0;
+    } else {
+        q = (uint32_t)(a >> shift);
+        unsigned __int128 rem = a & ((((unsigned __int128)1) << shift) - 1);
+        unsigned __int128 half = ((unsigned __int128)1) << (shift - 1);
+        if (rem > half || (rem == half && (q & 1u))) ++q;     /* q may become 2^24: still exact below */
+    }
+    float r = ldexpf((float)q, shift + unit_exp);
+    return neg ? -r : r;
+}
+
+/* Eq. "issue-partial": p_g = RNE32(sum of the 64 products of group g) for cell (i, j); the products
+ * are of the decoded operands s_hat * q without the tensor decode factors. */
+ORACLE_API float oracle_probe_partial(int64_t Kc,
+                                      const uint8_t *ap, const uint8_t *as, int a2d,
+                                      const uint8_t *bp, const uint8_t *bs, int b2d,
+                                      int64_t i, int64_t j, int64_t group)
+{
+    ensure_tables();
+    __int128 acc = 0;
+    for (int64_t k = 64 * group; k < 64 * group + 64; ++k)
+        acc += (__int128)decoded_units(ap, as, Kc, a2d, i, k) * decoded_units(bp, bs, Kc, b2d, j, k);
+    return rne32_of_units(acc, -36);
+}
+
+/* RTZ32(a + b): the binary32 value nearest to the exact sum among those not larger in magnitude. */
+static float rtz32_add(float a, float b)
+{
+    /* binary64 two-sum: s + e == a + b exactly */
+    double x = (double)a, y = (double)b;
+    double s = x + y;
+    double bb = s - x;
+    double e = (x - (s - bb)) + (y - bb);
+    float f = (float)s;                               /* nearest binary32 to s */
+    double over = ((double)f - s) - e;                /* sign of f - (a + b); (double)f - s is exact */
+    if ((f > 0.0f && over > 0.0) || (f < 0.0f && over < 0.0))
+        f = nextafterf(f, 0.0f);                      /* |f| exceeded the exact sum: step toward zero */
+    return f;
+}
+
+/* Eq. "grid-denominator": Q_d(c) = RNE(d c) / d for a power-of-two d; d = 0 disables it.  Ties go to the
+ * even integer index. */
+static float grid_snap(float c, int d)
+{
+    if (d <= 0) return c;
+    float t = c * (float)d;                           /* exact: power-of-two factor */
+    return nearbyintf(t) / (float)d;                  /* default rounding mode: ties to even */
+}
+
+/* Eq. "issue-rz": c_0 = 0, c_{g+1} = R32(c_g + p_g) over n partials in the given order, R = RTZ
+ * (cross_rne = 0) or RNE (cross_rne = 1, the paper's control); then Q_d. */
+ORACLE_API float oracle_probe_combine(const float *p, int64_t n, int cross_rne, int grid_d)
+{
+    float c = 0.0f;
+    for (int64_t g = 0; g < n; ++g)
+        c = cross_rne ? (c + p[g]) : rtz32_add(c, p[g]);
+    return grid_snap(c, grid_d);
+}
+
+static float probe_cell(int64_t Kc,
+                        const uint8_t *ap, const uint8_t *as, int a2d, float dA,
+                        const uint8_t *bp, const uint8_t *bs, int b2d, float dB,
+                        int cross_rne, int grid_d, int64_t i, int64_t j)
+{
+    float c = 0.0f;
+    for (int64_t g = 0; g < Kc / 64; ++g) {
+        float p = oracle_probe_partial(Kc, ap, as, a2d, bp, bs, b2d, i, j, g);
+        c = cross_rne ? (c + p) : rtz32_add(c, p);
+    }
+    float alpha = dA * dB;                            /* the scale product, applied last (Eq. "final-grid") */
+    return alpha * grid_snap(c, grid_d);
+}
+
+/* y[Mo,No] (binary32) under the output model; Kc must be a multiple of 64. */
+ORACLE_API void oracle_gemm_probe(int64_t Mo, int64_t No, int64_t Kc,
+                                  const uint8_t *ap, const uint8_t *as, int a2d, float dA,
+                                  const uint8_t *bp, const uint8_t *bs, int b2d, float dB,
+                                  int cross_rne, int grid_d, float *y)
+{
+    ensure_tables();
+    #pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < Mo; ++i)
+        for (int64_t j = 0; j < No; ++j)
+            y[i * No + j] = probe_cell(Kc, ap, as, a2d, dA, bp, bs, b2d, dB, cross_rne, grid_d, i, j);
+}
+
+ORACLE_API void oracle_gemm_probe_cells(int64_t Kc,
+                                        const uint8_t *ap, const uint8_t *as, int a2d, float dA,
+                                        const uint8_t *bp, const uint8_t *bs, int b2d, float dB,
+                                        int cross_rne, int grid_d,
+                                        int64_t n, const int64_t *ci, const int64_t *cj, float *y)
+{
+    ensure_tables();
+    #pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < n; ++t)
+        y[t] = probe_cell(Kc, ap, as, a2d, dA, bp, bs, b2d, dB, cross_rne, grid_d, ci[t], cj[t]);
 }
 
 /* RNE of a binary64 value to BF16 bits (for the "within 1 ulp" check). */
