@@ -151,6 +151,23 @@ UE5M3_API int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
                void* out, int out_dtype, int64_t ldo, void* stream);
 
 /*
+ * The same product under the GEMM output model of Section 6.2 ("probe-matched" accumulation), bit-exact:
+ *     p_g     = RNE32( sum of the 64 products k = 64g .. 64g+63 of the decoded operands )   Eq. "issue-partial"
+ *     c_0 = 0,  c_{g+1} = RTZ32(c_g + p_g), g ascending                                       Eq. "issue-rz"
+ *     C[m, n] = RNE32( alpha * Q_d(c_G) ),  Q_d(c) = RNE(d c) / d,  alpha = RNE32(d_A * d_B) Eq. "final-grid",
+ *                                                                                             Eq. "grid-denominator"
+ * Arguments, layouts, shape rules, alignment and error behaviour are those of ue5m3_gemm, plus
+ *   cross_rounding      0 = toward zero (the model); 1 = nearest even (the paper's control variant).
+ *   grid_denominator    d: 0 (no grid step) or a power of two up to 65536; the paper's rule is d = 1024.
+ * BF16 output is the FP32 result rounded to nearest even.  The result does not depend on the device's SM count.
+ */
+UE5M3_API int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t Kc,
+               const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
+               const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
+               int cross_rounding, int grid_denominator,
+               void* out, int out_dtype, int64_t ldo, void* stream);
+
+/*
  * Bytes a scale buffer needs.  rows/cols are those of the SOURCE tensor given to ue5m3_quantize.
  * (Section 3.2: one scale per block of B = 16; Section 3.3: one per 16x16 weight tile.)
  * Returns 0 for invalid arguments.

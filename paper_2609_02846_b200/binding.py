@@ -20,7 +20,7 @@ SCALES_ROWMAJOR, SCALES_TILED = 0, 1
 SCALE_1D, SCALE_1D_TILED, SCALE_2D = 0, 1, 2
 FPROP, DGRAD, WGRAD = 0, 1, 2
 
-SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_gemm", "ue5m3_scales_bytes",
+SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_gemm", "ue5m3_gemm_probe_matched", "ue5m3_scales_bytes",
            "ue5m3_unswizzle_scales", "ue5m3_last_device_status", "ue5m3_status_string")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -53,6 +53,8 @@ def _load() -> C.CDLL:
         L.ue5m3_quantize.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, f32, u64, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_gemm.restype = ci
         L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
+        L.ue5m3_gemm_probe_matched.restype = ci
+        L.ue5m3_gemm_probe_matched.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, ci, ci, vp, ci, i64, vp]
         L.ue5m3_scales_bytes.restype = C.c_size_t
         L.ue5m3_scales_bytes.argtypes = [i64, i64, ci, ci]
         L.ue5m3_unswizzle_scales.restype = ci
@@ -202,6 +204,26 @@ def gemm(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dty
                                   _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
                                   _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
                                   _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)), "ue5m3_gemm")
+    return out
+
+
+def gemm_probe_matched(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
+                       out: Optional[torch.Tensor] = None, cross_rounding: int = 0,
+                       grid_denominator: int = 1024) -> torch.Tensor:
+    """The same product under the output model of Section 6.2: 64-product partials rounded to nearest even,
+    cross-group additions toward zero, 1/grid_denominator grid, scale product last (ue5m3_gemm_probe_matched)."""
+    Mo, No, Kc = a.R, b.R, a.Kc
+    if b.Kc != Kc:
+        raise ValueError(f"contraction sizes differ: {Kc} vs {b.Kc}")
+    if out is None:
+        out = torch.empty((Mo, No), dtype=out_dtype, device=a.payload.device)
+    with torch.cuda.device(out.device):
+        _check(_load().ue5m3_gemm_probe_matched(op, Mo, No, Kc,
+                                                _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
+                                                _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
+                                                int(cross_rounding), int(grid_denominator),
+                                                _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)),
+               "ue5m3_gemm_probe_matched")
     return out
 
 

@@ -103,9 +103,9 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
                : UE5M3_ERR_CUDA;
 }
 
-int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
-               int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
-               int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
+static int check_gemm_args(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+                           int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+                           int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo) {
     if (op != UE5M3_FPROP && op != UE5M3_DGRAD && op != UE5M3_WGRAD) return UE5M3_ERR_INVALID_ARG;
     if (!a_payload || !a_scales || !a_decode || !b_payload || !b_scales || !b_decode || !out) return UE5M3_ERR_INVALID_ARG;
     if (Mo <= 0 || No <= 0 || Kc <= 0 || ldo < No) return UE5M3_ERR_INVALID_ARG;
@@ -118,12 +118,39 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
         ((ldo * osz) % 16))
         return UE5M3_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(a_decode) & 3u) || (reinterpret_cast<uintptr_t>(b_decode) & 3u)) return UE5M3_ERR_ALIGN;
+    return UE5M3_OK;
+}
+
+int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+               int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+               int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
+    const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
+                                    b_scale_mode, b_decode, out, out_dtype, ldo);
+    if (bad != UE5M3_OK) return bad;
     const DeviceInfo di = device_info();
     if (!di.ok) return UE5M3_ERR_CUDA;
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
     return launch_gemm(g, di.sms, (cudaStream_t)stream);
+}
+
+int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+                             int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+                             int b_scale_mode, const float* b_decode, int cross_rounding, int grid_denominator,
+                             void* out, int out_dtype, int64_t ldo, void* stream) {
+    const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
+                                    b_scale_mode, b_decode, out, out_dtype, ldo);
+    if (bad != UE5M3_OK) return bad;
+    if (cross_rounding != 0 && cross_rounding != 1) return UE5M3_ERR_INVALID_ARG;
+    if (grid_denominator < 0 || grid_denominator > 65536 || (grid_denominator & (grid_denominator - 1)))
+        return UE5M3_ERR_INVALID_ARG;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
+               out, out_dtype, ldo};
+    return launch_gemm_probe(g, cross_rounding, grid_denominator, di.sms, (cudaStream_t)stream);
 }
 
 int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream) {
@@ -133,6 +160,10 @@ int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t k
     return launch_unswizzle(in, out, R, kblocks, (cudaStream_t)stream) == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
-int ue5m3_last_device_status(void) { return read_and_clear_device_status(); }
+int ue5m3_last_device_status(void) {
+    const int a = read_and_clear_device_status();
+    const int b = read_and_clear_probe_status();
+    return a != UE5M3_OK ? a : b;
+}
 
 }  // extern "C"
