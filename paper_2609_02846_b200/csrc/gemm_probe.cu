@@ -15,17 +15,20 @@
 //   tier 2  the same interval test in FP64; if it closes, one FP64 -> FP32 conversion rounds the exact sum;
 //   tier 3  128-bit integer accumulation of the four significands and a hand-written rounding.
 //
-// Persistent, CTA pairs (tcgen05 cta_group::2) on 256 x 128 output tiles; each CTA holds the running totals
-// c of its 128 x 128 half in registers.  Warp roles per CTA:
+// Persistent, one CTA per SM on 128 x 128 output tiles; the running totals c of a tile live in registers.
+// Nothing here crosses CTAs: the accumulators hand tensor-memory buffers back to the MMA issuer once per
+// group, and that round trip bounds the pipeline, so every barrier is CTA-local (tcgen05 cta_group::1).
+// Warp roles:
 //   warp 0       TMA producer (packed payload and scale tiles, 256 K per stage)
-//   warp 1       tensor-memory allocation; MMA issuer (leader CTA): per 64-wide slice and 64-column half, four
-//                M256 N64 K16 MMAs, each into its own buffer of a ring of six 64-column tensor-memory buffers
-//   warps 2-5    dequantizers: the thread on TMEM lane t converts row t of the A slice (registers -> tensor
-//                memory) and, for t < 64, row t of the B slice (-> 128B-swizzled shared memory)
+//   warp 1       tensor-memory allocation; MMA issuer: per 64-wide slice and 64-column half, four M128 N64 K16
+//                MMAs, each into its own 64-column tensor-memory buffer; two sets of four buffers, so that the
+//                MMAs of one group run while the accumulators work on the previous one
+//   warps 2-5    dequantizers: thread t converts row t of the A slice and row t of the B slice into
+//                128B-swizzled K-major shared-memory tiles
 //   warps 6-21   accumulators: warp w reads TMEM lanes 32 (w % 4) .. +31, columns 16 ((w - 6) / 4) .. +15 of each
 //                buffer, reduces the four block sums of a group and adds the total to c; after the last group
 //                it applies grid and scale product and stores its 16-column runs
-// Tensor memory: columns 0..127 four A stages, columns 128..511 the ring.  Every wait is bounded.
+// Tensor memory: all 512 columns are the two sets.  Every wait is bounded.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdint>
@@ -39,29 +42,28 @@ __device__ int g_probe_status = 0;
 
 namespace {
 
-constexpr int BM = 128;                     // A rows per CTA (256 per CTA pair)
+constexpr int BM = 128;                     // tile rows = A rows staged per CTA
 constexpr int NH = 2;                       // 64-column halves per tile
-constexpr int BN = 64 * NH;                 // output columns per tile
-constexpr int BNH = 32 * NH;                // B rows staged by each CTA of the pair
+constexpr int BN = 64 * NH;                 // tile columns = B rows staged per CTA
 constexpr int KCHUNK = 256;                 // K per packed stage
 constexpr int KSUB = 64;                    // K per FP16 stage = one group of Eq. "issue-partial"
 constexpr int SLICES = KCHUNK / KSUB;
-constexpr int PK_STAGES = 3;
-constexpr int BF_STAGES = 4;                // FP16 stages (A in tensor memory, B in shared memory)
-constexpr int RING = 6;                     // block-sum buffers of 64 columns
+constexpr int PK_STAGES = 2;
+constexpr int BF_STAGES = 4;                // FP16 stages (A and B slices in shared memory)
+constexpr int SETS = 2;                     // sets of four 64-column block-sum buffers
 constexpr int DEQ_WARP0 = 2, DEQ_WARPS = 4, ACC_WARP0 = 6, ACC_WARPS = 16;
 constexpr int NUM_THREADS = 32 * (ACC_WARP0 + ACC_WARPS);
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;        // 16384
-constexpr int PK_B_BYTES = BNH * KCHUNK / 2;       // 8192
+constexpr int PK_B_BYTES = BN * KCHUNK / 2;        // 16384
 constexpr int SC_A_BYTES = BM * (KCHUNK / 16);     // 2048
-constexpr int SC_B_BYTES = BNH * (KCHUNK / 16);    // 1024
-constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES;   // 27648 (a multiple of 1024)
-constexpr int BF_STAGE_BYTES = BNH * KSUB * 2;     // 8192
-constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;
+constexpr int SC_B_BYTES = BN * (KCHUNK / 16);     // 2048
+constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES;   // 36864
+constexpr int BF_A_BYTES = BM * KSUB * 2;          // 16384
+constexpr int BF_STAGE_BYTES = BF_A_BYTES + BN * KSUB * 2;       // 32768
+constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES; // 204800
 constexpr int SMEM_BYTES = SMEM_TILES + 512 + 1024;                                 // barriers, alignment slack
-constexpr int TMEM_A_COL = 0, TMEM_A_STAGE_COLS = KSUB / 2, TMEM_RING_COL = BF_STAGES * TMEM_A_STAGE_COLS;
-static_assert(TMEM_RING_COL + RING * 64 <= 512, "tensor memory budget");
+static_assert(SETS * 4 * 64 <= 512, "tensor memory budget");
 static_assert(PK_STAGE_BYTES % 1024 == 0 && BF_STAGE_BYTES % 1024 == 0, "128B-swizzled tiles start on 1024-byte boundaries");
 
 struct ProbeParams {
@@ -71,7 +73,7 @@ struct ProbeParams {
     void* out;
     int out_bf16;
     int a_mode, b_mode;
-    int tiles_m, tiles_n;         // 256 x BN tiles
+    int tiles_m, tiles_n;         // BM x BN tiles
     int cross_rne;                // 1: the control with nearest-even cross-group additions
     float grid;                   // d of Eq. "grid-denominator" (a power of two) or 0
 };
@@ -90,16 +92,43 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return mbar_wait_status(bar, parity, abort_flag, &g_probe_status);
 }
 
-// kind::f16 instruction descriptor: D = F32, A = B = F16, both K-major, M = 256 (two CTAs), N = 64.
-constexpr uint32_t kInstrDesc = (1u << 4) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+// kind::f16 instruction descriptor: D = F32, A = B = F16, both K-major, M = 128, N = 64.
+constexpr uint32_t kInstrDesc = (1u << 4) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-constexpr int PC = 4;                       // columns per accumulator pass
+// Single-CTA tcgen05 forms.
+__device__ __forceinline__ void tmem_alloc_1(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_1(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D (tensor memory) = A (shared memory) * B (shared memory), M128 N64 K16, accumulator input ignored.
+__device__ __forceinline__ void umma_f16_ss_1(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
+// Arrive on this CTA's barrier once all MMAs issued so far have retired.
+__device__ __forceinline__ void umma_commit_1(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+constexpr int PC = 8;                       // columns per accumulator pass
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float r[PC]) {
     uint32_t u[PC];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]) : "r"(taddr) : "memory");
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7])
+                 : "r"(taddr) : "memory");
 #pragma unroll
     for (int i = 0; i < PC; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ void tmem_ld1(uint32_t taddr, float& r) {
+    uint32_t u;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(u) : "r"(taddr) : "memory");
+    r = __uint_as_float(u);
 }
 
 // Correctly rounded (nearest even) sum of four FP32 numbers whose FP32 interval test failed.
@@ -147,7 +176,7 @@ __device__ __noinline__ float rne_sum4_exact(float t0, float t1, float t2, float
 }
 
 // ----------------------------------------------------------------------------- kernel
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
                   const ProbeParams p) {
@@ -158,13 +187,12 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t bf_base = smem_base + PK_STAGES * PK_STAGE_BYTES;
     const uint32_t bar_base = smem_base + SMEM_TILES;
     const uint32_t pk_full = bar_base, pk_empty = bar_base + 32, bf_full = bar_base + 64, bf_empty = bar_base + 96;
-    const uint32_t ring_full = bar_base + 128, ring_empty = bar_base + 176, drain_bar = bar_base + 224;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 232);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 240);
+    const uint32_t set_full = bar_base + 128, set_empty = bar_base + 160, drain_bar = bar_base + 192;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 200);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 208);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_rank();
-    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int cta = blockIdx.x, num_ctas = gridDim.x;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int kchunks = (int)(p.Kc / KCHUNK);
 
@@ -175,21 +203,20 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             mbar_init(pk_empty + 8 * s, DEQ_WARPS);
         }
         for (int s = 0; s < BF_STAGES; ++s) {
-            mbar_init(bf_full + 8 * s, 2 * DEQ_WARPS);        // the leader's copy collects both CTAs' dequantizers
+            mbar_init(bf_full + 8 * s, DEQ_WARPS);
             mbar_init(bf_empty + 8 * s, 1);
         }
-        for (int s = 0; s < RING; ++s) {
-            mbar_init(ring_full + 8 * s, 1);
-            mbar_init(ring_empty + 8 * s, 2 * ACC_WARPS);     // the leader's copy collects both CTAs' accumulator warps
+        for (int s = 0; s < SETS; ++s) {
+            mbar_init(set_full + 8 * s, 1);
+            mbar_init(set_empty + 8 * s, ACC_WARPS);
         }
         mbar_init(drain_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_a); prefetch_tmap(&map_b); prefetch_tmap(&map_as); prefetch_tmap(&map_bs);
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    if (warp == 1) tmem_alloc_1(smem_u32(tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
-    cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -198,14 +225,13 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         if (lane == 0) {
             uint32_t it = 0;
             const int a_rows_per_load = (p.a_mode == UE5M3_SCALE_2D) ? BM / 16 : BM;
-            const int b_rows_per_load = (p.b_mode == UE5M3_SCALE_2D) ? BNH / 16 : BNH;
+            const int b_rows_per_load = (p.b_mode == UE5M3_SCALE_2D) ? BN / 16 : BN;
             const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + b_rows_per_load * 16;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
                 int tm, tn;
                 tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
-                const int arow0 = (tm * 2 + (int)rank) * BM;             // first A row of this CTA
-                const int brow0 = (tn * 2 + (int)rank) * BNH;            // first B row of this CTA
+                const int arow0 = tm * BM, brow0 = tn * BN;
                 for (int kc = 0; kc < kchunks; ++kc, ++it) {
                     const uint32_t s = it % PK_STAGES, ph = (it / PK_STAGES) & 1;
                     if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
@@ -217,76 +243,71 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     const uint32_t sa = st + PK_A_BYTES + PK_B_BYTES, sb = sa + SC_A_BYTES;
                     if (p.a_mode == UE5M3_SCALE_1D) tma_load_2d(sa, &map_as, full, kc * 16, arow0);
                     else if (p.a_mode == UE5M3_SCALE_2D) tma_load_2d(sa, &map_as, full, kc * 16, arow0 / 16);
-                    else tma_load_2d(sa, &map_as, full, 0, ((arow0 >> 7) * kchunks + kc) * 128);
+                    else tma_load_2d(sa, &map_as, full, 0, (tm * kchunks + kc) * 128);
                     if (p.b_mode == UE5M3_SCALE_1D) tma_load_2d(sb, &map_bs, full, kc * 16, brow0);
                     else if (p.b_mode == UE5M3_SCALE_2D) tma_load_2d(sb, &map_bs, full, kc * 16, brow0 / 16);
-                    else tma_load_2d(sb, &map_bs, full, 0, ((brow0 >> 7) * kchunks + kc) * 128 + (brow0 & 127));
+                    else tma_load_2d(sb, &map_bs, full, 0, (tn * kchunks + kc) * 128);
                 }
             }
+            // let the copies still in flight land before the CTA's shared memory goes away
             for (uint32_t back = 0; back < PK_STAGES && back < it; ++back) {
                 const uint32_t j = it - 1 - back;
                 mbar_wait(pk_full + 8 * (j % PK_STAGES), (j / PK_STAGES) & 1, abort_flag);
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (leader CTA)
-        if (lane == 0 && rank == 0) {
-            uint32_t it = 0, rj = 0;
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, gh = 0;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
                 for (int ks = 0; ks < kchunks * SLICES && ok; ++ks, ++it) {
                     const uint32_t s = it % BF_STAGES, ph = (it / BF_STAGES) & 1;
                     if (!mbar_wait(bf_full + 8 * s, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t bd = umma_smem_desc(bf_base + s * BF_STAGE_BYTES);
-                    const uint32_t ta = tmem_base + TMEM_A_COL + s * TMEM_A_STAGE_COLS;
+                    const uint64_t ad = umma_smem_desc(bf_base + s * BF_STAGE_BYTES);
+                    const uint64_t bd = umma_smem_desc(bf_base + s * BF_STAGE_BYTES + BF_A_BYTES);
 #pragma unroll 1
-                    for (int h = 0; h < NH && ok; ++h) {
-#pragma unroll 1
-                        for (int b = 0; b < KSUB / 16; ++b, ++rj) {
-                            const uint32_t buf = rj % RING;
-                            if (!mbar_wait(ring_empty + 8 * buf, ((rj / RING) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                            tc_fence_after();
-                            // block b of the slice, B rows 32 h .. 32 h + 31 of each CTA, into a zeroed buffer
-                            umma_f16_ts(tmem_base + TMEM_RING_COL + buf * 64, ta + b * 8,
-                                        bd + (uint64_t)(h * (32 * 128 / 16) + b * 2), kInstrDesc, 0u);
-                            umma_commit_pair(ring_full + 8 * buf);
-                        }
+                    for (int h = 0; h < NH; ++h, ++gh) {
+                        // the four blocks of this group and half go to the four buffers of set gh % SETS
+                        const uint32_t set = gh % SETS;
+                        if (!mbar_wait(set_empty + 8 * set, ((gh / SETS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int b = 0; b < KSUB / 16; ++b)
+                            umma_f16_ss_1(tmem_base + (set * 4 + b) * 64, ad + (uint64_t)(b * 2),
+                                          bd + (uint64_t)(h * (64 * 128 / 16) + b * 2), kInstrDesc);
+                        umma_commit_1(set_full + 8 * set);
                     }
-                    if (ok) umma_commit_pair(bf_empty + 8 * s);
+                    if (ok) umma_commit_1(bf_empty + 8 * s);
                 }
             }
-            umma_commit_local(drain_bar);
+            // everything issued must have retired before tensor memory is released
+            umma_commit_1(drain_bar);
             mbar_wait(drain_bar, 0, abort_flag);
         }
     } else if (warp >= DEQ_WARP0 && warp < DEQ_WARP0 + DEQ_WARPS) {
         // ------------------------------------------------------------------ dequantizers
-        const int q = warp & 3;
-        const int row = q * 32 + lane;
+        const int row = (warp - DEQ_WARP0) * 32 + lane;       // this thread's row of the A tile and of the B tile
         const int r7 = row & 7;
-        const bool has_b = row < BNH;                  // warp-uniform
         const int a_srow = (p.a_mode == UE5M3_SCALE_2D) ? (row >> 4) : row;
         const int b_srow = (p.b_mode == UE5M3_SCALE_2D) ? (row >> 4) : row;
         uint32_t it_pk = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
             for (int kc = 0; kc < kchunks && ok; ++kc, ++it_pk) {
                 const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
                 if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag)) { ok = false; break; }
                 const uint8_t* st = smem_gen + ps * PK_STAGE_BYTES;
                 const uint4 a_codes4 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + PK_B_BYTES + a_srow * 16);
-                uint4 b_codes4 = make_uint4(0, 0, 0, 0);
-                if (has_b) b_codes4 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + b_srow * 16);
+                const uint4 b_codes4 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + b_srow * 16);
 #pragma unroll 1
                 for (int sl = 0; sl < SLICES; ++sl) {
                     const int off0 = row * 128 + (((2 * sl) ^ r7) << 4), off1 = row * 128 + (((2 * sl + 1) ^ r7) << 4);
                     const uint4 a0 = *reinterpret_cast<const uint4*>(st + off0);
                     const uint4 a1 = *reinterpret_cast<const uint4*>(st + off1);
-                    uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
-                    if (has_b) {
-                        b0 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + off0);
-                        b1 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + off1);
-                    }
+                    const uint4 b0 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + off0);
+                    const uint4 b1 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + off1);
                     const uint32_t a_codes = sl == 0 ? a_codes4.x : sl == 1 ? a_codes4.y : sl == 2 ? a_codes4.z : a_codes4.w;
                     const uint32_t b_codes = sl == 0 ? b_codes4.x : sl == 1 ? b_codes4.y : sl == 2 ? b_codes4.z : b_codes4.w;
                     if (sl == SLICES - 1) {
@@ -297,26 +318,24 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     const uint32_t slice_no = it_pk * SLICES + sl;
                     const uint32_t bs = slice_no % BF_STAGES;
                     if (!mbar_wait(bf_empty + 8 * bs, ((slice_no / BF_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
+                    uint8_t* stage_gen = smem_gen + PK_STAGES * PK_STAGE_BYTES + bs * BF_STAGE_BYTES;
                     {
                         const uint32_t m0 = scale_pair(a_codes & 0xFFu), m1 = scale_pair((a_codes >> 8) & 0xFFu);
                         const uint32_t m2 = scale_pair((a_codes >> 16) & 0xFFu), m3 = scale_pair(a_codes >> 24);
-                        uint32_t r[32];
-                        uint4 v;
-                        v = dequant8(a0.x, m0); r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w;
-                        v = dequant8(a0.y, m0); r[4] = v.x; r[5] = v.y; r[6] = v.z; r[7] = v.w;
-                        v = dequant8(a0.z, m1); r[8] = v.x; r[9] = v.y; r[10] = v.z; r[11] = v.w;
-                        v = dequant8(a0.w, m1); r[12] = v.x; r[13] = v.y; r[14] = v.z; r[15] = v.w;
-                        v = dequant8(a1.x, m2); r[16] = v.x; r[17] = v.y; r[18] = v.z; r[19] = v.w;
-                        v = dequant8(a1.y, m2); r[20] = v.x; r[21] = v.y; r[22] = v.z; r[23] = v.w;
-                        v = dequant8(a1.z, m3); r[24] = v.x; r[25] = v.y; r[26] = v.z; r[27] = v.w;
-                        v = dequant8(a1.w, m3); r[28] = v.x; r[29] = v.y; r[30] = v.z; r[31] = v.w;
-                        tmem_st32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_A_COL + bs * TMEM_A_STAGE_COLS, r);
+                        uint8_t* dst = stage_gen + row * 128;
+                        *reinterpret_cast<uint4*>(dst + ((0 ^ r7) << 4)) = dequant8(a0.x, m0);
+                        *reinterpret_cast<uint4*>(dst + ((1 ^ r7) << 4)) = dequant8(a0.y, m0);
+                        *reinterpret_cast<uint4*>(dst + ((2 ^ r7) << 4)) = dequant8(a0.z, m1);
+                        *reinterpret_cast<uint4*>(dst + ((3 ^ r7) << 4)) = dequant8(a0.w, m1);
+                        *reinterpret_cast<uint4*>(dst + ((4 ^ r7) << 4)) = dequant8(a1.x, m2);
+                        *reinterpret_cast<uint4*>(dst + ((5 ^ r7) << 4)) = dequant8(a1.y, m2);
+                        *reinterpret_cast<uint4*>(dst + ((6 ^ r7) << 4)) = dequant8(a1.z, m3);
+                        *reinterpret_cast<uint4*>(dst + ((7 ^ r7) << 4)) = dequant8(a1.w, m3);
                     }
-                    if (has_b) {
+                    {
                         const uint32_t m0 = scale_pair(b_codes & 0xFFu), m1 = scale_pair((b_codes >> 8) & 0xFFu);
                         const uint32_t m2 = scale_pair((b_codes >> 16) & 0xFFu), m3 = scale_pair(b_codes >> 24);
-                        uint8_t* dst = smem_gen + PK_STAGES * PK_STAGE_BYTES + bs * BF_STAGE_BYTES + row * 128;
+                        uint8_t* dst = stage_gen + BF_A_BYTES + row * 128;
                         *reinterpret_cast<uint4*>(dst + ((0 ^ r7) << 4)) = dequant8(b0.x, m0);
                         *reinterpret_cast<uint4*>(dst + ((1 ^ r7) << 4)) = dequant8(b0.y, m0);
                         *reinterpret_cast<uint4*>(dst + ((2 ^ r7) << 4)) = dequant8(b0.z, m1);
@@ -326,11 +345,9 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         *reinterpret_cast<uint4*>(dst + ((6 ^ r7) << 4)) = dequant8(b1.z, m3);
                         *reinterpret_cast<uint4*>(dst + ((7 ^ r7) << 4)) = dequant8(b1.w, m3);
                     }
-                    tmem_st_wait();
-                    fence_proxy_async();
-                    tc_fence_before();
+                    fence_proxy_async();                 // the slices are visible to the tensor core
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(bf_full + 8 * bs, 0);
+                    if (lane == 0) mbar_arrive(bf_full + 8 * bs);
                 }
             }
         }
@@ -338,11 +355,11 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // ------------------------------------------------------------------ accumulators
         const int q = warp & 3;                        // TMEM lane quarter
         const int cg = (warp - ACC_WARP0) >> 2;        // 16-column group of every 64-column buffer
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_RING_COL + cg * 16;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + cg * 16;
         const float alpha = __fmul_rn(__ldg(p.a_decode), __ldg(p.b_decode));
-        uint32_t rj = 0;
+        uint32_t gh = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
             int tm, tn;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
             float c[NH][16];
@@ -353,70 +370,61 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll 1
             for (int ks = 0; ks < kchunks * SLICES && ok; ++ks) {
 #pragma unroll
-                for (int h = 0; h < NH; ++h) {
-                    uint32_t col[4];
-#pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        const uint32_t j = rj + b, buf = j % RING;
-                        col[b] = buf * 64;
-                        if (ok && !mbar_wait(ring_full + 8 * buf, (j / RING) & 1, abort_flag)) ok = false;
-                    }
-                    if (!ok) break;
+                for (int h = 0; h < NH; ++h, ++gh) {
+                    const uint32_t set = gh % SETS;
+                    if (!mbar_wait(set_full + 8 * set, (gh / SETS) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
+                    const uint32_t base = lane_addr + set * 256;
 #pragma unroll
                     for (int pass = 0; pass < 16 / PC; ++pass) {
                         float t[4][PC];
 #pragma unroll
-                        for (int b = 0; b < 4; ++b) tmem_ld_cols(lane_addr + col[b] + pass * PC, t[b]);
+                        for (int b = 0; b < 4; ++b) tmem_ld_cols(base + b * 64 + pass * PC, t[b]);
                         tmem_ld_wait();
-                        if (pass == 16 / PC - 1) {
-                            // all four buffers have been read by this warp
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) {
-#pragma unroll
-                                for (int b = 0; b < 4; ++b) mbar_arrive_cluster(ring_empty + 8 * ((rj + b) % RING), 0);
-                            }
-                        }
-                        float pg[PC];
                         bool inexact = false;
 #pragma unroll
                         for (int e = 0; e < PC; ++e) {
                             float lo = __fadd_rd(t[0][e], t[1][e]), hi = __fadd_ru(t[0][e], t[1][e]);
                             lo = __fadd_rd(lo, t[2][e]); hi = __fadd_ru(hi, t[2][e]);
                             lo = __fadd_rd(lo, t[3][e]); hi = __fadd_ru(hi, t[3][e]);
-                            pg[e] = lo;
+                            t[0][e] = lo;                                  // the group total when lo == hi
                             inexact |= (lo != hi);
                         }
                         if (__any_sync(0xFFFFFFFFu, inexact)) {
+                            // Rare: some addition rounded.  The block sums are still in tensor memory; take them
+                            // again one column at a time and sum exactly.
 #pragma unroll 1
                             for (int e = 0; e < PC; ++e) {
-                                // element e of the register arrays, selected without dynamic indexing
-                                float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f, pe = 0.0f;
-#pragma unroll
-                                for (int k = 0; k < PC; ++k)
-                                    if (k == e) { s0 = t[0][k]; s1 = t[1][k]; s2 = t[2][k]; s3 = t[3][k]; pe = pg[k]; }
+                                float s0, s1, s2, s3;
+                                tmem_ld1(base + 0 * 64 + pass * PC + e, s0);
+                                tmem_ld1(base + 1 * 64 + pass * PC + e, s1);
+                                tmem_ld1(base + 2 * 64 + pass * PC + e, s2);
+                                tmem_ld1(base + 3 * 64 + pass * PC + e, s3);
+                                tmem_ld_wait();
                                 const float lo = __fadd_rd(__fadd_rd(__fadd_rd(s0, s1), s2), s3);
                                 const float hi = __fadd_ru(__fadd_ru(__fadd_ru(s0, s1), s2), s3);
-                                if (lo != hi) pe = rne_sum4_exact(s0, s1, s2, s3);
+                                const float pe = (lo != hi) ? rne_sum4_exact(s0, s1, s2, s3) : lo;
 #pragma unroll
                                 for (int k = 0; k < PC; ++k)
-                                    if (k == e) pg[k] = pe;
+                                    if (k == e) t[0][k] = pe;
                             }
                         }
 #pragma unroll
                         for (int e = 0; e < PC; ++e)
-                            c[h][pass * PC + e] = p.cross_rne ? __fadd_rn(c[h][pass * PC + e], pg[e]) : __fadd_rz(c[h][pass * PC + e], pg[e]);
+                            c[h][pass * PC + e] = p.cross_rne ? __fadd_rn(c[h][pass * PC + e], t[0][e]) : __fadd_rz(c[h][pass * PC + e], t[0][e]);
                     }
-                    rj += 4;
+                    // this warp is done with the set
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(set_empty + 8 * set);
                 }
             }
             if (!ok) break;
             // ---- grid, scale product, store: lane = output row, 16 consecutive columns per half
-            const int64_t grow = (int64_t)(tm * 2 + (int)rank) * BM + q * 32 + lane;
+            const int64_t grow = (int64_t)tm * BM + q * 32 + lane;
 #pragma unroll
             for (int h = 0; h < NH; ++h) {
-                const int64_t gcol = (int64_t)tn * BN + (cg >> 1) * BNH + h * 32 + (cg & 1) * 16;
+                const int64_t gcol = (int64_t)tn * BN + h * 64 + cg * 16;
                 float y[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
@@ -439,12 +447,12 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
     }
 
+    // tensor memory is freed only when no role can touch it any more
     tc_fence_before();
     __syncthreads();
-    cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc_1(tmem_base, 512);
     }
 }
 
@@ -459,43 +467,33 @@ bool make_scale_map_rows(CUtensorMap* m, const uint8_t* scales, int mode, int64_
 }  // namespace
 
 int launch_gemm_probe(const GemmArgs& g, int cross_rne, int grid_denominator, int num_sms, cudaStream_t st) {
-    static int resident_pairs[64];
+    static bool configured[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return UE5M3_ERR_CUDA;
-    if (resident_pairs[dev] == 0) {
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(gemm_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return UE5M3_ERR_CUDA;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
-        cfg.blockDim = dim3(NUM_THREADS, 1, 1);
-        cfg.dynamicSmemBytes = SMEM_BYTES;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_probe_kernel, &cfg) != cudaSuccess || n < 1) {
-            (void)cudaGetLastError();
-            n = num_sms / 2;
-        }
-        resident_pairs[dev] = n < num_sms / 2 ? n : num_sms / 2;
+        configured[dev] = true;
     }
     CUtensorMap ma, mb, mas, mbs;
     const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
     if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
-    if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BNH, true)) return UE5M3_ERR_CUDA;
+    if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BN, true)) return UE5M3_ERR_CUDA;
     if (!make_scale_map_rows(&mas, g.a_scales, g.a_scale_mode, g.Mo, g.Kc, BM)) return UE5M3_ERR_CUDA;
-    if (!make_scale_map_rows(&mbs, g.b_scales, g.b_scale_mode, g.No, g.Kc, BNH)) return UE5M3_ERR_CUDA;
+    if (!make_scale_map_rows(&mbs, g.b_scales, g.b_scale_mode, g.No, g.Kc, BN)) return UE5M3_ERR_CUDA;
 
     ProbeParams p;
     p.Mo = g.Mo; p.No = g.No; p.Kc = g.Kc; p.ldo = g.ldo;
     p.a_decode = g.a_decode; p.b_decode = g.b_decode;
     p.out = g.out; p.out_bf16 = g.out_dtype == UE5M3_BF16 ? 1 : 0;
     p.a_mode = g.a_scale_mode; p.b_mode = g.b_scale_mode;
-    p.tiles_m = (int)((g.Mo + 2 * BM - 1) / (2 * BM));
+    p.tiles_m = (int)((g.Mo + BM - 1) / BM);
     p.tiles_n = (int)((g.No + BN - 1) / BN);
     p.cross_rne = cross_rne;
     p.grid = (float)grid_denominator;
     const int num_tiles = p.tiles_m * p.tiles_n;
-    const int max_pairs = resident_pairs[dev];
-    const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
-    gemm_probe_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, p);
+    const int ctas = num_tiles < num_sms ? num_tiles : num_sms;       // one CTA per SM: the kernel holds all tensor memory
+    gemm_probe_kernel<<<ctas, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, p);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
