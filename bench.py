@@ -473,6 +473,75 @@ def run_stack(args):
                       "device_status": status}), flush=True)
 
 
+# FP32 lanes per SM per clock and directed-rounding additions per output cell and 64-product group
+# (6 for the exactness interval of the four block sums, 1 toward zero into the running total).
+PROBE_FP32_LANES_PER_SM, PROBE_ADDS_PER_GROUP = 128, 7
+
+
+def run_probe(args):
+    """The three GEMMs of the benchmark linear under the output model of Section 6.2 (ue5m3_gemm_probe_matched),
+    each timed alone on the quantized operands of one step; the oracle's model GEMM timed beside it on a sample."""
+    import torch
+    import paper_2609_02846_b200 as lib
+    dev = torch.device("cuda", 0)
+    step = LinearStep(dev, seed=7)
+    step.run(0)
+    q = step.q
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler(dev)
+    sampler.start()
+    sampler.wait_first_sample()
+    jobs = (("fprop", lib.FPROP, q["x"], q["w"], step.Y), ("dgrad", lib.DGRAD, q["g"], q["w"].transposed(), step.dX),
+            ("wgrad", lib.WGRAD, q["gt"], q["xt"], step.dW))
+    iters = max(3, args.steps // 20)
+    per_op, total_ms = {}, 0.0
+    for name, op, a, b, out in jobs:
+        for _ in range(max(3, args.warmup)):
+            lib.gemm_probe_matched(op, a, b, out=out)
+        torch.cuda.synchronize()
+        if name == "fprop":
+            sampler.mark()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            lib.gemm_probe_matched(op, a, b, out=out)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        per_op[name] = {"ms": round(ms, 4), "TFLOP/s": round(2.0 * M_TOK * K_IN * N_OUT / (ms * 1e-3) / 1e12, 1)}
+        total_ms += ms
+    clocks = sampler.stop()
+    status = lib.last_device_status()
+    tflops = 3 * 2.0 * M_TOK * K_IN * N_OUT / (total_ms * 1e-3) / 1e12
+    sm_hz = (clocks.get("sm_max_mhz") or 1965.0) * 1e6
+    peak = props.multi_processor_count * PROBE_FP32_LANES_PER_SM * sm_hz / PROBE_ADDS_PER_GROUP * 128 / 1e12
+    line = {"metric": "probe_matched_gemm_tflops", "value": round(tflops, 1), "unit": "TFLOP/s", "n_gpus": 1,
+            "dtype": "e2m1 x ue5m3 operands, exact 64-product partials, f32 toward-zero accumulation",
+            "config": {"workload": f"fprop, dgrad, wgrad of linear M={M_TOK} K={K_IN} N={N_OUT} under the Section 6.2 output model, "
+                                   "grid 1/1024, operands from one quantized step", "launches_timed_per_gemm": iters},
+            "per_gemm": per_op,
+            "roofline": {"bound": "alu", "achieved": round(tflops, 1), "peak": round(peak, 1), "unit": "TFLOP/s",
+                         "frac": round(tflops / peak, 3), "traffic": None,
+                         "peak_derivation": f"{props.multi_processor_count} SMs x {PROBE_FP32_LANES_PER_SM} FP32 lanes x max SM clock / "
+                                            f"{PROBE_ADDS_PER_GROUP} directed-rounding adds per cell and 64-group x 128 flop per cell and group"},
+            "device_status": status, "clocks": clocks}
+    if not args.no_cpu_baseline:
+        import oracle
+        qa, qb = q["x"], q["w"]
+        rows, cols = 64, 64
+        ap, asc = qa.payload[:rows].cpu().numpy(), qa.scales[:rows].cpu().numpy()
+        bp, bsc = qb.payload[:cols].cpu().numpy(), qb.scales[:cols // 16].cpu().numpy()
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 10.0:
+            oracle.gemm_probe(ap, asc, False, float(qa.decode.item()), bp, bsc, True, float(qb.decode.item()), grid_d=1024)
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        line["cpu_baseline"] = {"value": round(2.0 * rows * cols * K_IN / dt / 1e12, 6), "unit": "TFLOP/s", "cores": oracle.num_threads(),
+                                "kind": "oracle", "sample": f"fprop cut to {rows} x {cols} outputs, K={K_IN}, about 10 s"}
+    print(json.dumps(line), flush=True)
+
+
 def run_sweep(args):
     """Quantizer-only bandwidth sweep: BF16 [rows, 4096], 2^20 .. 2^30 elements, {1D, 2D} x {RNE, SR} + amax."""
     import torch
@@ -557,6 +626,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--stack", action="store_true", help="time the six linears of the 8B-hybrid-shaped layer stack")
+    ap.add_argument("--probe", action="store_true", help="time the GEMMs under the Section 6.2 output model")
     ap.add_argument("--sweep-iters", type=int, default=100)
     ap.add_argument("--sweep-warmup", type=int, default=20)
     ap.add_argument("--sweep-stride", type=int, default=1)
@@ -571,6 +641,8 @@ def main():
         run_sweep_oracle(args)
     elif args.stack:
         run_stack(args)
+    elif args.probe:
+        run_probe(args)
     else:
         run_ours(args)
 

@@ -125,6 +125,19 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float r[PC]) {
 #pragma unroll
     for (int i = 0; i < PC; ++i) r[i] = __uint_as_float(u[i]);
 }
+// Packed pairs of FP32 (one instruction adds two lanes' worth of values with the stated rounding).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2_rd(uint64_t a, uint64_t b) { uint64_t r; asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t add2_ru(uint64_t a, uint64_t b) { uint64_t r; asm("add.rp.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t add2_rz(uint64_t a, uint64_t b) { uint64_t r; asm("add.rz.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t add2_rn(uint64_t a, uint64_t b) { uint64_t r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 __device__ __forceinline__ void tmem_ld1(uint32_t taddr, float& r) {
     uint32_t u;
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(u) : "r"(taddr) : "memory");
@@ -362,11 +375,11 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
             int tm, tn;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
-            float c[NH][16];
+            uint64_t c[NH][8];                             // running totals, two columns per word
 #pragma unroll
             for (int h = 0; h < NH; ++h)
 #pragma unroll
-                for (int e = 0; e < 16; ++e) c[h][e] = 0.0f;
+                for (int e = 0; e < 8; ++e) c[h][e] = 0ull;
 #pragma unroll 1
             for (int ks = 0; ks < kchunks * SLICES && ok; ++ks) {
 #pragma unroll
@@ -381,14 +394,18 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                         for (int b = 0; b < 4; ++b) tmem_ld_cols(base + b * 64 + pass * PC, t[b]);
                         tmem_ld_wait();
+                        uint64_t tot[PC / 2];
                         bool inexact = false;
 #pragma unroll
-                        for (int e = 0; e < PC; ++e) {
-                            float lo = __fadd_rd(t[0][e], t[1][e]), hi = __fadd_ru(t[0][e], t[1][e]);
-                            lo = __fadd_rd(lo, t[2][e]); hi = __fadd_ru(hi, t[2][e]);
-                            lo = __fadd_rd(lo, t[3][e]); hi = __fadd_ru(hi, t[3][e]);
-                            t[0][e] = lo;                                  // the group total when lo == hi
-                            inexact |= (lo != hi);
+                        for (int e = 0; e < PC / 2; ++e) {
+                            const uint64_t t0 = pack2(t[0][2 * e], t[0][2 * e + 1]), t1 = pack2(t[1][2 * e], t[1][2 * e + 1]);
+                            const uint64_t t2 = pack2(t[2][2 * e], t[2][2 * e + 1]), t3 = pack2(t[3][2 * e], t[3][2 * e + 1]);
+                            const uint64_t lo = add2_rd(add2_rd(add2_rd(t0, t1), t2), t3);
+                            const uint64_t hi = add2_ru(add2_ru(add2_ru(t0, t1), t2), t3);
+                            float l0, l1, h0, h1;
+                            unpack2(lo, l0, l1); unpack2(hi, h0, h1);
+                            tot[e] = lo;                                   // the group totals when lo == hi
+                            inexact |= (l0 != h0) | (l1 != h1);
                         }
                         if (__any_sync(0xFFFFFFFFu, inexact)) {
                             // Rare: some addition rounded.  The block sums are still in tensor memory; take them
@@ -405,13 +422,22 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                                 const float hi = __fadd_ru(__fadd_ru(__fadd_ru(s0, s1), s2), s3);
                                 const float pe = (lo != hi) ? rne_sum4_exact(s0, s1, s2, s3) : lo;
 #pragma unroll
-                                for (int k = 0; k < PC; ++k)
-                                    if (k == e) t[0][k] = pe;
+                                for (int k = 0; k < PC / 2; ++k) {
+                                    float v0, v1;
+                                    unpack2(tot[k], v0, v1);
+                                    if (2 * k == e) v0 = pe;
+                                    if (2 * k + 1 == e) v1 = pe;
+                                    tot[k] = pack2(v0, v1);
+                                }
                             }
                         }
+                        if (p.cross_rne) {
 #pragma unroll
-                        for (int e = 0; e < PC; ++e)
-                            c[h][pass * PC + e] = p.cross_rne ? __fadd_rn(c[h][pass * PC + e], t[0][e]) : __fadd_rz(c[h][pass * PC + e], t[0][e]);
+                            for (int e = 0; e < PC / 2; ++e) c[h][pass * (PC / 2) + e] = add2_rn(c[h][pass * (PC / 2) + e], tot[e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < PC / 2; ++e) c[h][pass * (PC / 2) + e] = add2_rz(c[h][pass * (PC / 2) + e], tot[e]);
+                        }
                     }
                     // this warp is done with the set
                     tc_fence_before();
@@ -427,8 +453,10 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 const int64_t gcol = (int64_t)tn * BN + h * 64 + cg * 16;
                 float y[16];
 #pragma unroll
+                for (int e = 0; e < 8; ++e) unpack2(c[h][e], y[2 * e], y[2 * e + 1]);
+#pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    float v = __fmul_rn(c[h][e], 256.0f);                 // undo the operands' 2^-4 pre-scales (exact)
+                    float v = __fmul_rn(y[e], 256.0f);                    // undo the operands' 2^-4 pre-scales (exact)
                     if (p.grid > 0.0f) v = __fdiv_rn(rintf(__fmul_rn(v, p.grid)), p.grid);
                     y[e] = __fmul_rn(alpha, v);
                 }

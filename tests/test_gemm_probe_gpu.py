@@ -149,3 +149,33 @@ def test_probe_matched_rejects_bad_arguments():
         lib.gemm_probe_matched(lib.FPROP, qa, qb, grid_denominator=1000)      # not a power of two
     with pytest.raises(lib.Ue5m3Error):
         lib.gemm_probe_matched(lib.FPROP, qa, qb, cross_rounding=2)
+
+
+def test_probe_matched_full_size_linear_sampled_cells():
+    """The benchmark linear (M = 8192, K = 4096, N = 16384) in the launch configuration the benchmark times: all three
+    GEMMs on operands of one quantized step, 4096 sampled cells each (tile corners and interiors included), FP32
+    bit for bit and BF16 as the rounded FP32."""
+    M, K, N = 8192, 4096, 16384
+    x = si.channel_scaled_activation(M, K, seed=22, device=DEV)
+    w = si.weight(N, K, seed=23, device=DEV)
+    dy = si.heavy_tailed_gradient(M, N, seed=24, device=DEV)
+    gx, gw, gg = lib.sample_amax(x), lib.sample_amax(w), lib.sample_amax(dy)
+    qx = lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, gx)
+    qw = lib.quantize(w, lib.LAYOUT_2D, lib.ROUND_RNE, gw, want_transpose=True)
+    qg = lib.quantize(dy, lib.LAYOUT_1D_ROW, lib.ROUND_SR, gg, seed=44)
+    qgt = lib.quantize(dy, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, seed=45)
+    qxt = lib.quantize(x, lib.LAYOUT_1D_COL, lib.ROUND_RNE, gx)
+    rng = np.random.default_rng(77)
+    for op, a, b in ((lib.FPROP, qx, qw), (lib.DGRAD, qg, qw.transposed()), (lib.WGRAD, qgt, qxt)):
+        Mo, No = a.R, b.R
+        ci = np.concatenate([rng.integers(0, Mo, 4000), [0, 127, 128, Mo - 1] * 24])
+        cj = np.concatenate([rng.integers(0, No, 4000), np.repeat([0, 63, 64, 127, 128, No - 1], 16)])
+        want = oracle.gemm_probe_cells(a.payload.cpu().numpy(), a.scales.cpu().numpy(), a.scale_mode == lib.SCALE_2D,
+                                       float(a.decode.item()), b.payload.cpu().numpy(), b.scales.cpu().numpy(),
+                                       b.scale_mode == lib.SCALE_2D, float(b.decode.item()), ci, cj, grid_d=1024)
+        out32 = _run(a, b, torch.float32, grid_denominator=1024)
+        got = out32[torch.from_numpy(ci).to(DEV), torch.from_numpy(cj).to(DEV)].cpu().numpy()
+        assert np.array_equal(_bits(got), _bits(want)), op
+        out16 = _run(a, b, torch.bfloat16, grid_denominator=1024)
+        assert torch.equal(out16, out32.to(torch.bfloat16)), op
+        del out32, out16
