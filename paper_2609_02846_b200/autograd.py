@@ -51,7 +51,7 @@ class _Ue5m3LinearFn(torch.autograd.Function):
         _check_dims(M, K, N)
         ax = layer.scale_x.get(x, step)
         aw = layer.scale_w.get(w, step)
-        y, _, qw = B.linear_forward(x, w, ax, aw, layer.target_T, x.dtype)
+        y, _, qw = B.linear_forward(x, w, ax, aw, layer.target_T, x.dtype, grid_denominator=layer.grid_denominator)
         ctx.save_for_backward(x)
         ctx.qw, ctx.ax, ctx.layer, ctx.step = qw, ax, layer, step
         return y
@@ -63,21 +63,27 @@ class _Ue5m3LinearFn(torch.autograd.Function):
         dy = dy.contiguous()
         ag = layer.scale_dy.get(dy, step)
         dx, dw = B.linear_backward(dy, x, ctx.qw, ag, ctx.ax, seed=layer.seed * 1000003 + step, target_T=layer.target_T,
-                                   target_T_wgrad_dy=layer.target_T_wgrad_dy, out_dtype=dy.dtype)
+                                   target_T_wgrad_dy=layer.target_T_wgrad_dy, out_dtype=dy.dtype,
+                                   grid_denominator=layer.grid_denominator, grad_rounding=layer.grad_rounding)
         return dx, dw, None, None
 
 
 class Ue5m3Linear(torch.nn.Module):
     """y = x W^T with UE5M3-FP4 operands in all three GEMMs.  `x` is [tokens, in_features] (bfloat16 or float32);
-    call `advance()` once per optimizer step so that the held references refresh every `interval` steps."""
+    call `advance()` once per optimizer step so that the held references refresh every `interval` steps.
+    `grid_denominator` not None runs the three products under the Section 6.2 output model (0: without its grid
+    step); `grad_rounding` is the rounding of the upstream gradient (stochastic by default)."""
 
     def __init__(self, in_features: int, out_features: int, device="cuda", dtype=torch.bfloat16, interval: int = 50,
-                 target_T: float = 448.0, target_T_wgrad_dy: Optional[float] = None, seed: int = 0, group=None):
+                 target_T: float = 448.0, target_T_wgrad_dy: Optional[float] = None, seed: int = 0, group=None,
+                 grid_denominator: Optional[int] = None, grad_rounding: int = B.ROUND_SR):
         super().__init__()
         self.weight = torch.nn.Parameter(torch.empty(out_features, in_features, device=device, dtype=dtype).normal_(0, 0.02))
         self.target_T = float(target_T)
         self.target_T_wgrad_dy = float(target_T if target_T_wgrad_dy is None else target_T_wgrad_dy)
         self.seed = int(seed)
+        self.grid_denominator = grid_denominator
+        self.grad_rounding = int(grad_rounding)
         self.step = 0
         self.scale_x, self.scale_w, self.scale_dy = (OperandScale(interval, group) for _ in range(3))
 

@@ -252,24 +252,34 @@ class AmaxCache:
         return self.held
 
 
+def _multiply(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype, grid_denominator: Optional[int]):
+    """`gemm`, or `gemm_probe_matched` with the given grid when `grid_denominator` is not None."""
+    if grid_denominator is None:
+        return gemm(op, a, b, out_dtype)
+    return gemm_probe_matched(op, a, b, out_dtype, grid_denominator=grid_denominator)
+
+
 def linear_forward(x: torch.Tensor, w: torch.Tensor, amax_x: torch.Tensor, amax_w: torch.Tensor,
                    target_T: float = 448.0, out_dtype: torch.dtype = torch.bfloat16,
-                   scale_layout: int = SCALES_ROWMAJOR):
+                   scale_layout: int = SCALES_ROWMAJOR, grid_denominator: Optional[int] = None):
     """Y = X W^T: quantize X (1D along K, RNE) and W (2D tiles, RNE, with transposed copy), multiply.
-    Returns (Y, qx, qw); qw carries the transposed view the backward pass needs."""
+    Returns (Y, qx, qw); qw carries the transposed view the backward pass needs.  `grid_denominator` not None
+    selects the Section 6.2 output model for the product (0 = that model without its grid step)."""
     qx = quantize(x, LAYOUT_1D_ROW, ROUND_RNE, amax_x, target_T, scale_layout=scale_layout)
     qw = quantize(w, LAYOUT_2D, ROUND_RNE, amax_w, target_T, want_transpose=True)
-    return gemm(FPROP, qx, qw, out_dtype), qx, qw
+    return _multiply(FPROP, qx, qw, out_dtype, grid_denominator), qx, qw
 
 
 def linear_backward(dy: torch.Tensor, x: torch.Tensor, qw: QuantizedOperand, amax_dy: torch.Tensor,
                     amax_x: torch.Tensor, seed: int, target_T: float = 448.0, target_T_wgrad_dy: float = 448.0,
-                    out_dtype: torch.dtype = torch.bfloat16, scale_layout: int = SCALES_ROWMAJOR):
-    """dX = dY W and dW = dY^T X.  dY is rounded stochastically, once per GEMM with seeds 4*seed and
-    4*seed + 1; the saved activation X is re-quantized along the token dimension with RNE."""
-    qdy = quantize(dy, LAYOUT_1D_ROW, ROUND_SR, amax_dy, target_T, seed=4 * seed, scale_layout=scale_layout)
-    dx = gemm(DGRAD, qdy, qw.transposed(), out_dtype)
-    qdy_t = quantize(dy, LAYOUT_1D_COL, ROUND_SR, amax_dy, target_T_wgrad_dy, seed=4 * seed + 1, scale_layout=scale_layout)
+                    out_dtype: torch.dtype = torch.bfloat16, scale_layout: int = SCALES_ROWMAJOR,
+                    grid_denominator: Optional[int] = None, grad_rounding: int = ROUND_SR):
+    """dX = dY W and dW = dY^T X.  dY is rounded stochastically by default, once per GEMM with seeds 4*seed and
+    4*seed + 1 (`grad_rounding = ROUND_RNE` gives the nearest-even control); the saved activation X is
+    re-quantized along the token dimension with RNE."""
+    qdy = quantize(dy, LAYOUT_1D_ROW, grad_rounding, amax_dy, target_T, seed=4 * seed, scale_layout=scale_layout)
+    dx = _multiply(DGRAD, qdy, qw.transposed(), out_dtype, grid_denominator)
+    qdy_t = quantize(dy, LAYOUT_1D_COL, grad_rounding, amax_dy, target_T_wgrad_dy, seed=4 * seed + 1, scale_layout=scale_layout)
     qx_t = quantize(x, LAYOUT_1D_COL, ROUND_RNE, amax_x, target_T, scale_layout=scale_layout)
-    dw = gemm(WGRAD, qdy_t, qx_t, out_dtype)
+    dw = _multiply(WGRAD, qdy_t, qx_t, out_dtype, grid_denominator)
     return dx, dw

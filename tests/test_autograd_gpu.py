@@ -42,6 +42,38 @@ def test_linear_function_matches_oracle():
     assert rel < 0.2
 
 
+@pytest.mark.parametrize("grad_rounding", [lib.ROUND_SR, lib.ROUND_RNE])
+def test_linear_function_under_the_output_model_is_bit_exact(grad_rounding):
+    """The layer with the Section 6.2 output model: forward output and both gradients equal the oracle's pipeline
+    (quantize, model GEMM, BF16 rounding) bit for bit."""
+    M, K, N = 256, 512, 256
+    layer = Ue5m3Linear(K, N, device=DEV, seed=3, grid_denominator=1024, grad_rounding=grad_rounding)
+    with torch.no_grad():
+        layer.weight.copy_(si.weight(N, K, seed=2, device=DEV))
+    x = si.channel_scaled_activation(M, K, seed=1, device=DEV).requires_grad_(True)
+    dy = si.heavy_tailed_gradient(M, N, seed=4, device=DEV)
+    y = layer(x)
+    y.backward(dy)
+    torch.cuda.synchronize()
+    Xn, Wn, Gn = si.to_numpy_bits(x.detach()), si.to_numpy_bits(layer.weight.detach()), si.to_numpy_bits(dy)
+    gx, gw, gg = oracle.amax(Xn), oracle.amax(Wn), oracle.amax(Gn)
+    seed = 3 * 1000003 + 0
+    ox = oracle.quantize(Xn, 0, 0, gx); ow = oracle.quantize(Wn, 2, 0, gw, want_t=True)
+    og = oracle.quantize(Gn, 0, grad_rounding, gg, seed=4 * seed); ogt = oracle.quantize(Gn, 1, grad_rounding, gg, seed=4 * seed + 1)
+    oxt = oracle.quantize(Xn, 1, 0, gx)
+
+    def same(out, a, a_t, b, b_t, b2d):
+        want = oracle.gemm_probe(a["payload_t" if a_t else "payload"], a["scales_t" if a_t else "scales"], False, a["decode"],
+                                 b["payload_t" if b_t else "payload"], b["scales_t" if b_t else "scales"], b2d, b["decode"],
+                                 grid_d=1024)
+        want_bits = torch.from_numpy(want).to(torch.bfloat16).view(torch.uint16)
+        assert torch.equal(out.detach().cpu().view(torch.uint16), want_bits)
+
+    same(y, ox, False, ow, False, True)
+    same(x.grad, og, False, ow, True, True)
+    same(layer.weight.grad, ogt, False, oxt, False, False)
+
+
 def test_hold_policy_inside_the_layer():
     layer = Ue5m3Linear(256, 256, device=DEV, interval=50)
     x = si.channel_scaled_activation(256, 256, seed=1, device=DEV)
