@@ -244,3 +244,48 @@ def test_philox_matches_curand_device_generator(tmp_path):
     got = d_out.cpu().numpy().view(np.uint32)
     for i in range(n):
         assert list(got[i]) == list(oracle.philox4x32_10(ctr[i], key[i]))
+
+
+@pytest.mark.parametrize("T", [64.0, 448.0, 1024.0, 2048.0, 8192.0, 32768.0])
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_scale_target_sweep(T, layout):
+    """The scale target is a free parameter of the call (Section 5.2: 448 by default, 2048 for selected operands):
+    byte and counter parity at every target, and the stale-growth headroom U_max / T of Proposition 1 — a tensor that
+    has grown by rho since its reference was sampled saturates a block scale exactly when T rho exceeds 61440."""
+    x = si.heavy_tailed_gradient(256, 512, seed=5, device=DEV)
+    g = _amax(x)
+    for rounding in ROUNDINGS:
+        _, got = lib_quantize(x, layout, rounding, g, T, seed=3)
+        want = oracle_quantize(x, layout, rounding, g, T, seed=3)
+        assert_same_quantization(got, want)
+        assert want["stats"]["scale_saturated"] == 0
+        assert int(want["scales"].max()) == oracle.ue5m3_encode(np.float32(T))   # the block holding the maximum gets code(T)
+    headroom = 61440.0 / T
+    for rho, expect_saturation in ((0.98 * headroom, False), (1.07 * headroom, True)):
+        stale = np.float32(g / rho)                        # the held reference is rho times too small
+        _, got = lib_quantize(x, layout, oracle.ROUND_RNE, float(stale), T)
+        want = oracle_quantize(x, layout, oracle.ROUND_RNE, float(stale), T)
+        assert_same_quantization(got, want)
+        assert (want["stats"]["scale_saturated"] > 0) == expect_saturation
+        assert int(want["scales"].max()) <= 0xF7
+
+
+def test_raised_target_moves_small_block_scales_away_from_zero():
+    """Section 5.2: T = 2048 maps small block scales about 4.6x farther from zero than T = 448 — fewer blocks of a
+    heavy-tailed gradient land on subnormal or repaired zero scale codes, at every block's code the ratio is 2048/448
+    up to the code grid."""
+    x = si.heavy_tailed_gradient(512, 1024, seed=6, device=DEV) * 1e-3
+    x[:, ::7] *= 1e-4                                      # columns of very small gradient components
+    g = _amax(x)
+    _, lo = lib_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, 448.0)
+    _, hi = lib_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, 2048.0)
+    for got, T in ((lo, 448.0), (hi, 2048.0)):
+        assert_same_quantization(got, oracle_quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, T))
+    v_lo = np.array([oracle.ue5m3_value(int(c)) for c in lo["scales"].ravel()])
+    v_hi = np.array([oracle.ue5m3_value(int(c)) for c in hi["scales"].ravel()])
+    normal = (lo["scales"].ravel() >= 0x10) & (hi["scales"].ravel() < 0xF0)
+    ratio = v_hi[normal] / v_lo[normal]
+    assert np.all(np.abs(ratio / (2048.0 / 448.0) - 1) < 0.14)           # one code step is at most 1/8
+    assert abs(np.median(ratio) - 4.571) < 0.2
+    assert (hi["scales"] < 8).sum() <= (lo["scales"] < 8).sum()
+    assert hi["stats"]["zero_repaired"] <= lo["stats"]["zero_repaired"]
