@@ -125,6 +125,28 @@ UE5M3_API int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t col
                    int scale_layout, void* stream);
 
 /*
+ * Both 1D quantizations of one tensor from a single read (Section 5.3: the backward pass needs dY along its
+ * columns for dX = dY W and along its rows for dW = dY^T X; likewise X along K for Y and along the tokens for dW).
+ * The row outputs are exactly what ue5m3_quantize(..., UE5M3_LAYOUT_1D_ROW, rounding, ..., target_T_row, seed_row)
+ * writes and the column outputs exactly what UE5M3_LAYOUT_1D_COL with (target_T_col, seed_col) writes; the call
+ * moves 2 + 2 * 0.5625 bytes per BF16 element instead of 2 * (2 + 0.5625).
+ *   x, dtype, rows, cols, ld, rounding, amax_held, scale_layout, stream     as in ue5m3_quantize.
+ *   payload_row [rows, cols/2], scales_row (rows x cols/16 blocks)           device, 16-byte aligned.
+ *   payload_col [cols, rows/2], scales_col (cols x rows/16 blocks)           device, 16-byte aligned.
+ *   decode_row, decode_col   device, 1 float each, optional (NULL to skip).
+ *   stats_row, stats_col     device, 4 x uint64 each, both or neither; counters as in ue5m3_quantize.
+ * Errors as in ue5m3_quantize.
+ */
+UE5M3_API int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
+                   const float* amax_held, float target_T_row, float target_T_col,
+                   uint64_t seed_row, uint64_t seed_col,
+                   uint8_t* payload_row, uint8_t* scales_row,
+                   uint8_t* payload_col, uint8_t* scales_col,
+                   float* decode_row, float* decode_col,
+                   uint64_t* stats_row, uint64_t* stats_col,
+                   int scale_layout, void* stream);
+
+/*
  * Block-scaled GEMM on quantized operands (paper, Section 5.3: Y = X W^T, dX = dY W,
  * dW = dY^T X; Section 6.1: y = sum_k a_k b_k on the decoded operands, the tensor-scale product
  * applied after accumulation):

@@ -20,7 +20,7 @@ SCALES_ROWMAJOR, SCALES_TILED = 0, 1
 SCALE_1D, SCALE_1D_TILED, SCALE_2D = 0, 1, 2
 FPROP, DGRAD, WGRAD = 0, 1, 2
 
-SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_gemm", "ue5m3_gemm_probe_matched", "ue5m3_scales_bytes",
+SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_quantize_dual", "ue5m3_gemm", "ue5m3_gemm_probe_matched", "ue5m3_scales_bytes",
            "ue5m3_unswizzle_scales", "ue5m3_last_device_status", "ue5m3_status_string")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -51,6 +51,8 @@ def _load() -> C.CDLL:
         L.ue5m3_sample_amax.argtypes = [vp, ci, i64, i64, i64, vp, vp]
         L.ue5m3_quantize.restype = ci
         L.ue5m3_quantize.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, f32, u64, vp, vp, vp, vp, vp, vp, ci, vp]
+        L.ue5m3_quantize_dual.restype = ci
+        L.ue5m3_quantize_dual.argtypes = [vp, ci, i64, i64, i64, ci, vp, f32, f32, u64, u64, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_gemm.restype = ci
         L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_probe_matched.restype = ci
@@ -180,6 +182,41 @@ def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tenso
             C.c_float(target_T), C.c_uint64(int(seed) & (2 ** 64 - 1)),
             _dev_ptr(out.payload), _dev_ptr(out.scales), _dev_ptr(out.payload_t), _dev_ptr(out.scales_t),
             _dev_ptr(out.decode), _dev_ptr(stats), scale_layout, _stream(x)), "ue5m3_quantize")
+    return out
+
+
+def quantize_dual(x: torch.Tensor, rounding: int, amax_held: torch.Tensor, target_T_row: float = 448.0,
+                  target_T_col: float = 448.0, seed_row: int = 0, seed_col: int = 0,
+                  stats_row: Optional[torch.Tensor] = None, stats_col: Optional[torch.Tensor] = None,
+                  scale_layout: int = SCALES_ROWMAJOR,
+                  out: Optional[tuple] = None) -> tuple:
+    """ue5m3_quantize_dual: the 1D_ROW and the 1D_COL quantization of `x` from one read.  Returns (row, col)
+    operands, each identical to what `quantize` produces for that layout, target and seed."""
+    rows, cols, ld = _matrix(x)
+    dev = x.device
+    u8 = dict(dtype=torch.uint8, device=dev)
+    if out is None:
+        ops = []
+        for layout, (R, K) in ((LAYOUT_1D_ROW, (rows, cols)), (LAYOUT_1D_COL, (cols, rows))):
+            nbytes = scales_bytes(rows, cols, layout, scale_layout)
+            if nbytes == 0:
+                _check(2, "ue5m3_quantize_dual (rows and cols must be positive multiples of 16)")
+            scales = torch.zeros(nbytes, **u8) if scale_layout == SCALES_TILED else torch.empty((R, K // 16), **u8)
+            ops.append(QuantizedOperand(torch.empty((R, K // 2), **u8), scales, torch.empty(1, dtype=torch.float32, device=dev),
+                                        SCALE_1D_TILED if scale_layout == SCALES_TILED else SCALE_1D))
+        out = tuple(ops)
+    row, col = out
+    for st in (stats_row, stats_col):
+        if st is not None and (st.dtype != torch.int64 or st.numel() != 4):
+            raise ValueError("stats must be int64 tensors with 4 elements")
+    with torch.cuda.device(dev):
+        _check(_load().ue5m3_quantize_dual(
+            _dev_ptr(x), _dtype_code(x), rows, cols, ld, rounding, _dev_ptr(amax_held),
+            C.c_float(target_T_row), C.c_float(target_T_col),
+            C.c_uint64(int(seed_row) & (2 ** 64 - 1)), C.c_uint64(int(seed_col) & (2 ** 64 - 1)),
+            _dev_ptr(row.payload), _dev_ptr(row.scales), _dev_ptr(col.payload), _dev_ptr(col.scales),
+            _dev_ptr(row.decode), _dev_ptr(col.decode), _dev_ptr(stats_row), _dev_ptr(stats_col),
+            scale_layout, _stream(x)), "ue5m3_quantize_dual")
     return out
 
 

@@ -103,6 +103,40 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
                : UE5M3_ERR_CUDA;
 }
 
+int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,
+                        const float* amax_held, float target_T_row, float target_T_col, uint64_t seed_row, uint64_t seed_col,
+                        uint8_t* payload_row, uint8_t* scales_row, uint8_t* payload_col, uint8_t* scales_col,
+                        float* decode_row, float* decode_col, uint64_t* stats_row, uint64_t* stats_col, int scale_layout,
+                        void* stream) {
+    if (!x || !amax_held || !payload_row || !scales_row || !payload_col || !scales_col || rows <= 0 || cols <= 0 || ld < cols)
+        return UE5M3_ERR_INVALID_ARG;
+    if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
+    if (rounding != UE5M3_ROUND_RNE && rounding != UE5M3_ROUND_SR) return UE5M3_ERR_INVALID_ARG;
+    if (scale_layout != UE5M3_SCALES_ROWMAJOR && scale_layout != UE5M3_SCALES_TILED) return UE5M3_ERR_INVALID_ARG;
+    for (float T : {target_T_row, target_T_col})
+        if (!(T > 0.0f) || T > 61440.0f || T != (float)(int)T) return UE5M3_ERR_INVALID_ARG;
+    if ((stats_row == nullptr) != (stats_col == nullptr)) return UE5M3_ERR_INVALID_ARG;
+    if ((rows % 16) || (cols % 16)) return UE5M3_ERR_SHAPE;
+    const int64_t esz = dtype == UE5M3_F32 ? 4 : 2;
+    if (!aligned16(x) || ((ld * esz) % 16) || !aligned16(payload_row) || !aligned16(scales_row) || !aligned16(payload_col) ||
+        !aligned16(scales_col))
+        return UE5M3_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(amax_held) & 3u) || (reinterpret_cast<uintptr_t>(decode_row) & 3u) ||
+        (reinterpret_cast<uintptr_t>(decode_col) & 3u) || (reinterpret_cast<uintptr_t>(stats_row) & 7u) ||
+        (reinterpret_cast<uintptr_t>(stats_col) & 7u))
+        return UE5M3_ERR_ALIGN;
+    if (rows * (cols / 16) >= ((int64_t)1 << 32) - 256) return UE5M3_ERR_UNSUPPORTED;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    QuantArgs a{x, rows, cols, ld, amax_held, target_T_col, seed_col, payload_col, scales_col, nullptr, nullptr, decode_col,
+                reinterpret_cast<unsigned long long*>(stats_col),
+                payload_row, scales_row, target_T_row, seed_row, decode_row, reinterpret_cast<unsigned long long*>(stats_row)};
+    return launch_quantize_dual(a, dtype, rounding, scale_layout == UE5M3_SCALES_TILED, (cudaStream_t)stream) == cudaSuccess
+               ? UE5M3_OK
+               : UE5M3_ERR_CUDA;
+}
+
 static int check_gemm_args(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
                            int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
                            int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo) {

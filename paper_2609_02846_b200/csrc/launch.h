@@ -17,6 +17,14 @@ struct QuantArgs {
     uint8_t* scales_t;
     float* decode_out;
     unsigned long long* stats;
+    // Second output set of the dual-layout call (ue5m3_quantize_dual): the 1D_ROW quantization of the same
+    // tensor, produced from the same read.  The fields above then describe the 1D_COL quantization.
+    uint8_t* row_payload;
+    uint8_t* row_scales;
+    float row_T;
+    uint64_t row_seed;
+    float* row_decode;
+    unsigned long long* row_stats;
 };
 
 struct GemmArgs {
@@ -27,6 +35,7 @@ struct GemmArgs {
 };
 
 cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, cudaStream_t st);
+cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bool tiled, cudaStream_t st);
 cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* out, int num_sms,
                         cudaStream_t st);
 cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, cudaStream_t st);

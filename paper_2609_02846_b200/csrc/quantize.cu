@@ -66,6 +66,15 @@ __device__ __forceinline__ TensorConsts cta_tensor_consts(const float* amax_held
     return s_tc;
 }
 
+// The same for two targets at once (dual-layout call: columns with T, rows with T_row).
+__device__ __forceinline__ void cta_tensor_consts2(const float* amax_held, float T, float T_row, TensorConsts& tc, TensorConsts& tcr) {
+    __shared__ TensorConsts s_tc2[2];
+    if (threadIdx.x == 0) { const float g = __ldg(amax_held); s_tc2[0] = tensor_consts(g, T); s_tc2[1] = tensor_consts(g, T_row); }
+    __syncthreads();
+    tc = s_tc2[0];
+    tcr = s_tc2[1];
+}
+
 template <bool IS_BF16, bool SR, bool STATS, bool TILED>
 __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a, int kb_shift) {
     const TensorConsts tc = cta_tensor_consts(a.amax_held, a.T);
@@ -166,15 +175,24 @@ __device__ __forceinline__ void load_row8(const void* x, int64_t off, float f[8]
 //         rounding, which is bound by integer arithmetic and is better off without the staging work.
 // MODE 1: 2D tiles: lanes 2i and 2i+1 hold the halves of one tile; the row-major payload is stored directly
 //         (64 contiguous bytes per row and warp), the optional transposed copy goes through shared memory.
+// MODE 3: dual layout: MODE 0 plus the 1D_ROW quantization of the same register tile (a row block of 16 is this
+//         lane's 8 columns and lane ^ 1's): the tensor is read once for both operands of a backward pass.
 template <bool IS_BF16, bool SR, bool STATS, int MODE, bool TILED, bool WANT_T>
 __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a) {
-    constexpr bool kColumns = (MODE == 0) || (MODE == 2);
-    constexpr bool kTranspose = (MODE == 0) || WANT_T;
+    constexpr bool kDual = MODE == 3;
+    constexpr bool kStaged = (MODE == 0) || kDual;       // column output through shared memory
+    constexpr bool kColumns = kStaged || (MODE == 2);
+    constexpr bool kTranspose = kStaged || WANT_T;
     __shared__ __align__(16) uint8_t s_t[kTranspose ? kTileCols * (kTileRows / 2) : 16];
-    __shared__ __align__(16) uint8_t s_sc[(MODE == 0) ? (kTileRows / 16) * kTileCols : 16];   // [row block][column]
+    __shared__ __align__(16) uint8_t s_sc[kStaged ? (kTileRows / 16) * kTileCols : 16];   // [row block][column]
 
-    const TensorConsts tc = cta_tensor_consts(a.amax_held, a.T);
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tc.d;
+    TensorConsts tc, tcr;
+    if (kDual) cta_tensor_consts2(a.amax_held, a.T, a.row_T, tc, tcr);
+    else { tc = cta_tensor_consts(a.amax_held, a.T); tcr = tc; }
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        if (a.decode_out) *a.decode_out = tc.d;
+        if (kDual && a.row_decode) *a.row_decode = tcr.d;
+    }
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int cg, rb;   // column group (8 columns) and row block (16 rows) inside the CTA tile
@@ -245,6 +263,7 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
     // ---- pass 2: encode.  nib[r] = the 8 codes of row r (column j in bits 4j+3:4j) ----
     uint32_t nib[16];
     uint32_t clip = 0;
+    uint32_t sat_r = 0, rep_r = 0, clip_r = 0;
 #pragma unroll
     for (int r = 0; r < 16; ++r) {
         float f[8];
@@ -252,6 +271,41 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
         else { uint4 v; load_row8<false>(a.x, base + r * a.ld, f, v); }
         uint32_t w[4] = {0, 0, 0, 0};
         if (SR) sr_bits8(a.seed, ((uint64_t)(r0 + r) * (uint64_t)a.cols + (uint64_t)c0) >> 3, w);
+        if (kDual) {
+            // ---- the row operand: block = 16 consecutive columns of row r0 + r, held by lanes 2i and 2i + 1 ----
+            float m = 0.0f;
+            if (IS_BF16) {
+                uint32_t pm = bf16x2_absmax(bf16x2_absmax(0u, raw[r].x), raw[r].y);
+                pm = bf16x2_absmax(bf16x2_absmax(pm, raw[r].z), raw[r].w);
+                m = fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xFFFF0000u));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(f[j]));
+            }
+            m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+            float rrow;
+            uint32_t fl;
+            const uint32_t code_r = block_scale(m, tcr, rrow, fl);
+            if ((lane & 1) == 0) { sat_r += fl & 1u; rep_r += (fl >> 1) & 1u; }
+            uint32_t wr[4] = {0, 0, 0, 0};
+            if (SR) sr_bits8(a.row_seed, ((uint64_t)(r0 + r) * (uint64_t)a.cols + (uint64_t)c0) >> 3, wr);
+            const uint32_t orow = encode8<SR>(f, rrow, wr, clip_r);
+            const int64_t kbpr = a.cols >> 4;
+            // four lanes (even column groups) -> four consecutive scale bytes
+            uint32_t s4 = code_r | (__shfl_down_sync(0xFFFFFFFFu, code_r, 2) << 8);
+            s4 |= __shfl_down_sync(0xFFFFFFFFu, s4, 4) << 16;
+            if (live) {
+                *reinterpret_cast<uint32_t*>(a.row_payload + (r0 + r) * (a.cols >> 1) + (c0 >> 1)) = orow;
+                const int64_t kb = c0 >> 4;
+                if (TILED) {
+                    if ((cg & 1) == 0) a.row_scales[tiled_scale_offset(r0 + r, kb, kbpr)] = (uint8_t)code_r;
+                } else if ((kbpr & 3) == 0) {
+                    if ((cg & 7) == 0) *reinterpret_cast<uint32_t*>(a.row_scales + (r0 + r) * kbpr + kb) = s4;   // cols % 64 == 0
+                } else if ((cg & 1) == 0) {
+                    a.row_scales[(r0 + r) * kbpr + kb] = (uint8_t)code_r;
+                }
+            }
+        }
         float z[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) z[j] = __fmul_rn(f[j], rcol[j]);
@@ -316,14 +370,14 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
             const int piece = (rb + cg) & 15;
             *reinterpret_cast<uint2*>(s_t + col * (kTileRows / 2) + piece * 8) = o;
         }
-        if (MODE == 0) {
+        if (kStaged) {
             // scale bytes of this row block for the thread's eight columns (8 contiguous bytes)
             *reinterpret_cast<uint2*>(s_sc + rb * kTileCols + cg * 8) =
                 make_uint2(codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24),
                            codes[4] | (codes[5] << 8) | (codes[6] << 16) | (codes[7] << 24));
         }
         __syncthreads();
-        uint8_t* const out_t = (MODE == 0) ? a.payload : a.payload_t;
+        uint8_t* const out_t = kStaged ? a.payload : a.payload_t;
         // each column of the CTA tile is 128 contiguous output bytes: 8 lanes x 16 bytes
         const int64_t rbase = (int64_t)blockIdx.y * kTileRows;
         const bool al16 = ((a.rows >> 1) & 15) == 0;     // output rows start on 16-byte boundaries
@@ -344,7 +398,7 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
                 }
             }
         }
-        if (MODE == 0) {
+        if (kStaged) {
             // scales of the transposed operand: [column][row block]; the 16 row blocks of this CTA tile are
             // contiguous for a column, so one thread per column writes them (16 bytes at once when aligned)
             const int64_t kblocks = a.rows >> 4;
@@ -369,6 +423,7 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
     if (STATS) {
         const uint32_t lv = live ? 1u : 0u;
         warp_add_stats(a.stats, lv * sat, lv * rep, lv * clip, lv * nonf);
+        if (kDual) warp_add_stats(a.row_stats, lv * sat_r, lv * rep_r, lv * clip_r, lv * nonf);
     }
 }
 
@@ -469,6 +524,25 @@ static cudaError_t launch_any(const QuantArgs& a, int layout, bool tiled, cudaSt
 cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, cudaStream_t st) {
     const bool bf = dtype == UE5M3_BF16, sr = rounding == UE5M3_ROUND_SR, stt = a.stats != nullptr;
 #define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_any<B, S, T>(a, layout, tiled, st);
+    UE5M3_DISPATCH(true, false, false) UE5M3_DISPATCH(true, true, false)
+    UE5M3_DISPATCH(true, false, true)  UE5M3_DISPATCH(true, true, true)
+    UE5M3_DISPATCH(false, false, false) UE5M3_DISPATCH(false, true, false)
+    UE5M3_DISPATCH(false, false, true)  UE5M3_DISPATCH(false, true, true)
+#undef UE5M3_DISPATCH
+    return cudaErrorInvalidValue;
+}
+
+template <bool IS_BF16, bool SR, bool STATS>
+static cudaError_t launch_dual(const QuantArgs& a, bool tiled, cudaStream_t st) {
+    dim3 grid((unsigned)((a.cols + kTileCols - 1) / kTileCols), (unsigned)((a.rows + kTileRows - 1) / kTileRows));
+    if (tiled) quantize_tile_kernel<IS_BF16, SR, STATS, 3, true, false><<<grid, kTileThreads, 0, st>>>(a);
+    else       quantize_tile_kernel<IS_BF16, SR, STATS, 3, false, false><<<grid, kTileThreads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bool tiled, cudaStream_t st) {
+    const bool bf = dtype == UE5M3_BF16, sr = rounding == UE5M3_ROUND_SR, stt = a.stats != nullptr;
+#define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_dual<B, S, T>(a, tiled, st);
     UE5M3_DISPATCH(true, false, false) UE5M3_DISPATCH(true, true, false)
     UE5M3_DISPATCH(true, false, true)  UE5M3_DISPATCH(true, true, true)
     UE5M3_DISPATCH(false, false, false) UE5M3_DISPATCH(false, true, false)

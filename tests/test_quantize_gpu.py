@@ -289,3 +289,43 @@ def test_raised_target_moves_small_block_scales_away_from_zero():
     assert abs(np.median(ratio) - 4.571) < 0.2
     assert (hi["scales"] < 8).sum() <= (lo["scales"] < 8).sum()
     assert hi["stats"]["zero_repaired"] <= lo["stats"]["zero_repaired"]
+
+
+@pytest.mark.parametrize("rounding", ROUNDINGS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("shape", [(16, 16), (256, 256), (272, 4112), (1040, 208), (512, 1024)])
+@pytest.mark.parametrize("scale_layout", [0, 1])
+def test_dual_layout_call_equals_the_two_single_calls(rounding, dtype, shape, scale_layout):
+    """One read, both 1D operands: every byte, decode factor and counter equals the oracle's row and column
+    quantizations with their own targets and seeds."""
+    import paper_2609_02846_b200 as lib
+    rows, cols = shape
+    x = si.heavy_tailed_gradient(rows, cols, seed=rows + cols, device=DEV, dtype=dtype)
+    x[3, 5] = 0.0
+    g = torch.tensor([_amax(x) * 0.5], dtype=torch.float32, device=DEV)      # stale reference: some clipping and saturation
+    st_r = torch.zeros(4, dtype=torch.int64, device=DEV)
+    st_c = torch.zeros(4, dtype=torch.int64, device=DEV)
+    row, col = lib.quantize_dual(x, rounding, g, 448.0, 2048.0, seed_row=40, seed_col=41, stats_row=st_r, stats_col=st_c,
+                                 scale_layout=scale_layout)
+    torch.cuda.synchronize()
+    for op, st, layout, T, seed, (R, K) in ((row, st_r, oracle.LAYOUT_1D_ROW, 448.0, 40, (rows, cols)),
+                                            (col, st_c, oracle.LAYOUT_1D_COL, 2048.0, 41, (cols, rows))):
+        want = oracle_quantize(x, layout, rounding, float(g.item()), T, seed=seed)
+        scales = lib.unswizzle_scales(op.scales, R, K // 16) if scale_layout == 1 else op.scales
+        got = dict(payload=op.payload.cpu().numpy(), scales=scales.cpu().numpy(), payload_t=None, scales_t=None,
+                   decode=np.float32(op.decode.item()), stats=dict(zip(oracle.STAT_NAMES, st.cpu().tolist())))
+        assert_same_quantization(got, want)
+
+
+def test_dual_layout_call_without_counters_and_into_given_buffers():
+    import paper_2609_02846_b200 as lib
+    x = si.channel_scaled_activation(512, 768, seed=4, device=DEV)
+    g = lib.sample_amax(x)
+    first = lib.quantize_dual(x, oracle.ROUND_RNE, g)
+    again = lib.quantize_dual(x * 2, oracle.ROUND_RNE, g, out=first)
+    assert again is first
+    single_r = lib.quantize(x * 2, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
+    single_c = lib.quantize(x * 2, lib.LAYOUT_1D_COL, lib.ROUND_RNE, g)
+    assert torch.equal(first[0].payload, single_r.payload) and torch.equal(first[0].scales, single_r.scales)
+    assert torch.equal(first[1].payload, single_c.payload) and torch.equal(first[1].scales, single_c.scales)
+    assert torch.equal(first[0].decode, single_r.decode) and torch.equal(first[1].decode, single_c.decode)
