@@ -74,7 +74,7 @@ __device__ __forceinline__ uint32_t e2m1x2_rne(float lo, float hi) {
 __device__ __forceinline__ void sr_accumulate(float z, uint32_t word, int j, uint32_t& mags, uint32_t& signs) {
     const float t = fminf(z, 6.0f);                       // NaN -> +6, sign of everything else kept
     const float a = fminf(fabsf(t), 6.0f);
-    const float b = (a < 1.0f) ? __fmaf_rn(a, 0.5f, 0.5f) : a;
+    const float b = fmaxf(a, __fmaf_rn(a, 0.5f, 0.5f));     // a/2 + 1/2 exceeds a exactly when a < 1: no compare, no select
     const uint32_t r = (j & 1) ? (word >> 10) : (word << 6);           // draw * 2^6 ...
     const uint32_t Bp = __float_as_uint(b) + ((r & 0x3FFFC0u) | 32u);  // ... + 2^5, added below the kept bit
     // bits 24:22 of Bp are the magnitude code plus 4 (mod 8); bit 31 of t is the sign
