@@ -68,6 +68,9 @@ def lib() -> C.CDLL:
         L.oracle_quantize_window.restype = C.c_int
         L.oracle_quantize_window.argtypes = [vp, C.c_int, i64, i64, i64, C.c_int, C.c_int, f32, f32, u64, i64, i64, i64,
                                              vp, vp, vp, vp, C.POINTER(f32), vp]
+        L.oracle_quantize_window_block.restype = C.c_int
+        L.oracle_quantize_window_block.argtypes = [vp, C.c_int, i64, i64, i64, C.c_int, C.c_int, f32, f32, u64, i64, i64, i64,
+                                                   C.c_int, vp, vp, vp, vp, C.POINTER(f32), vp]
         L.oracle_dequantize.restype = None
         L.oracle_dequantize.argtypes = [vp, vp, i64, i64, C.c_int, f32, vp]
         L.oracle_gemm.restype = None
@@ -171,9 +174,11 @@ def tensor_constants(g, T):
 
 # ---- quantizer -----------------------------------------------------------------------------
 def quantize(x: np.ndarray, layout: int, rounding: int, g, T=448.0, seed: int = 0, want_t: bool = False,
-             window=None):
+             window=None, block: int = 16):
     """Returns dict(payload, scales, payload_t, scales_t, decode, stats) in canonical layout.
-    window = (full_cols, row0, col0): x is that window of a larger tensor (matters for SR draws only)."""
+    window = (full_cols, row0, col0): x is that window of a larger tensor (matters for SR draws only).
+    block = 32 is the block-size control: one scale per 32 elements (32 x 32 in 2D), written to every
+    16-element slot it covers."""
     assert x.ndim == 2 and x.strides[1] == x.itemsize
     rows, cols = x.shape
     full_cols, row0, col0 = window if window is not None else (cols, 0, 0)
@@ -193,13 +198,13 @@ def quantize(x: np.ndarray, layout: int, rounding: int, g, T=448.0, seed: int = 
         scales_t = np.zeros((cols // 16, rows // 16), np.uint8)
     dec = C.c_float()
     stats = np.zeros(4, np.uint64)
-    rc = lib().oracle_quantize_window(_ptr(x), _dtype_code(x), rows, cols, ld, layout, rounding,
-                                      np.float32(g), np.float32(T), int(seed) & (2**64 - 1),
-                                      full_cols, row0, col0,
-                                      _ptr(payload), _ptr(scales), _ptr(payload_t), _ptr(scales_t),
-                                      C.byref(dec), _ptr(stats))
+    rc = lib().oracle_quantize_window_block(_ptr(x), _dtype_code(x), rows, cols, ld, layout, rounding,
+                                            np.float32(g), np.float32(T), int(seed) & (2**64 - 1),
+                                            full_cols, row0, col0, int(block),
+                                            _ptr(payload), _ptr(scales), _ptr(payload_t), _ptr(scales_t),
+                                            C.byref(dec), _ptr(stats))
     if rc != 0:
-        raise ValueError("oracle_quantize: sizes and window offsets must be multiples of 16")
+        raise ValueError("oracle_quantize: sizes and window offsets must be multiples of 16 (of the block size along a blocked dimension)")
     return dict(payload=payload, scales=scales, payload_t=payload_t, scales_t=scales_t,
                 decode=np.float32(dec.value), stats=dict(zip(STAT_NAMES, (int(v) for v in stats))))
 

@@ -305,15 +305,21 @@ static void quantize_block(const void *x, int dtype, window_t win, int64_t ld,
  *                payload_t [cols, rows/2], scales_t [cols/16, rows/16].
  * Returns 0, or -1 for shapes that are not multiples of 16.
  */
-ORACLE_API int oracle_quantize_window(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
-                                      int layout, int rounding, float g, float T, uint64_t seed,
-                                      int64_t full_cols, int64_t row0, int64_t col0,
-                                      uint8_t *payload, uint8_t *scales,
-                                      uint8_t *payload_t, uint8_t *scales_t,
-                                      float *decode_out, uint64_t *stats_out)
+ORACLE_API int oracle_quantize_window_block(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                                            int layout, int rounding, float g, float T, uint64_t seed,
+                                            int64_t full_cols, int64_t row0, int64_t col0, int block,
+                                            uint8_t *payload, uint8_t *scales,
+                                            uint8_t *payload_t, uint8_t *scales_t,
+                                            float *decode_out, uint64_t *stats_out)
 {
+    /* block = B of Eq. "microscaling": 16 (the recipe) or 32 (the block-size control of Section 5.5).  The scale
+     * arrays keep one byte per 16 elements; a block of 32 writes its byte to both (in 2D: all four) slots. */
+    if (block != 16 && block != 32) return -1;
+    const int B = block, rep = block / 16;
     if (rows <= 0 || cols <= 0 || (rows % 16) || (cols % 16)) return -1;
-    if ((row0 % 16) || (col0 % 16) || row0 < 0 || col0 < 0 || col0 + cols > full_cols) return -1;
+    if (layout != LAYOUT_1D_COL && (cols % B)) return -1;
+    if (layout != LAYOUT_1D_ROW && (rows % B)) return -1;
+    if ((row0 % B) || (col0 % B) || row0 < 0 || col0 < 0 || col0 + cols > full_cols) return -1;
     window_t win = { full_cols, row0, col0 };
     float g_eff, S, G, d;
     oracle_tensor_constants(g, T, &g_eff, &S, &G, &d);
@@ -325,40 +331,43 @@ ORACLE_API int oracle_quantize_window(const void *x, int dtype, int64_t rows, in
     if (layout == LAYOUT_1D_ROW) {
         #pragma omp parallel for reduction(+ : s0, s1, s2, s3) schedule(static)
         for (int64_t r = 0; r < rows; ++r)
-            for (int64_t kb = 0; kb < cols / 16; ++kb) {
-                pos_t mem[16]; int codes[16]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
-                for (int j = 0; j < 16; ++j) { mem[j].r = r; mem[j].c = 16 * kb + j; }
-                quantize_block(x, dtype, win, ld, mem, 16, S, G, rounding, seed, codes, &sc, stats);
+            for (int64_t kb = 0; kb < cols / B; ++kb) {
+                pos_t mem[32]; int codes[32]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
+                for (int j = 0; j < B; ++j) { mem[j].r = r; mem[j].c = B * kb + j; }
+                quantize_block(x, dtype, win, ld, mem, B, S, G, rounding, seed, codes, &sc, stats);
                 s0 += stats[0]; s1 += stats[1]; s2 += stats[2]; s3 += stats[3];
-                scales[r * (cols / 16) + kb] = (uint8_t)sc;
-                for (int j = 0; j < 16; ++j) put_nibble(payload, cols / 2, r, 16 * kb + j, codes[j]);
+                for (int q = 0; q < rep; ++q) scales[r * (cols / 16) + rep * kb + q] = (uint8_t)sc;
+                for (int j = 0; j < B; ++j) put_nibble(payload, cols / 2, r, B * kb + j, codes[j]);
             }
     } else if (layout == LAYOUT_1D_COL) {
         #pragma omp parallel for reduction(+ : s0, s1, s2, s3) schedule(static)
         for (int64_t c = 0; c < cols; ++c)
-            for (int64_t rb = 0; rb < rows / 16; ++rb) {
-                pos_t mem[16]; int codes[16]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
-                for (int j = 0; j < 16; ++j) { mem[j].r = 16 * rb + j; mem[j].c = c; }
-                quantize_block(x, dtype, win, ld, mem, 16, S, G, rounding, seed, codes, &sc, stats);
+            for (int64_t rb = 0; rb < rows / B; ++rb) {
+                pos_t mem[32]; int codes[32]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
+                for (int j = 0; j < B; ++j) { mem[j].r = B * rb + j; mem[j].c = c; }
+                quantize_block(x, dtype, win, ld, mem, B, S, G, rounding, seed, codes, &sc, stats);
                 s0 += stats[0]; s1 += stats[1]; s2 += stats[2]; s3 += stats[3];
-                scales[c * (rows / 16) + rb] = (uint8_t)sc;
-                for (int j = 0; j < 16; ++j) put_nibble(payload, rows / 2, c, 16 * rb + j, codes[j]);
+                for (int q = 0; q < rep; ++q) scales[c * (rows / 16) + rep * rb + q] = (uint8_t)sc;
+                for (int j = 0; j < B; ++j) put_nibble(payload, rows / 2, c, B * rb + j, codes[j]);
             }
     } else if (layout == LAYOUT_2D) {
         #pragma omp parallel for reduction(+ : s0, s1, s2, s3) schedule(static)
-        for (int64_t rb = 0; rb < rows / 16; ++rb)
-            for (int64_t cb = 0; cb < cols / 16; ++cb) {
-                pos_t mem[256]; int codes[256]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
-                for (int i = 0; i < 16; ++i)
-                    for (int j = 0; j < 16; ++j) { mem[16 * i + j].r = 16 * rb + i; mem[16 * i + j].c = 16 * cb + j; }
-                quantize_block(x, dtype, win, ld, mem, 256, S, G, rounding, seed, codes, &sc, stats);
+        for (int64_t rb = 0; rb < rows / B; ++rb)
+            for (int64_t cb = 0; cb < cols / B; ++cb) {
+                pos_t mem[1024]; int codes[1024]; int sc; uint64_t stats[4] = {0, 0, 0, 0};
+                for (int i = 0; i < B; ++i)
+                    for (int j = 0; j < B; ++j) { mem[B * i + j].r = B * rb + i; mem[B * i + j].c = B * cb + j; }
+                quantize_block(x, dtype, win, ld, mem, B * B, S, G, rounding, seed, codes, &sc, stats);
                 s0 += stats[0]; s1 += stats[1]; s2 += stats[2]; s3 += stats[3];
-                scales[rb * (cols / 16) + cb] = (uint8_t)sc;
-                if (scales_t) scales_t[cb * (rows / 16) + rb] = (uint8_t)sc;
-                for (int i = 0; i < 16; ++i)
-                    for (int j = 0; j < 16; ++j) {
-                        put_nibble(payload, cols / 2, 16 * rb + i, 16 * cb + j, codes[16 * i + j]);
-                        if (payload_t) put_nibble(payload_t, rows / 2, 16 * cb + j, 16 * rb + i, codes[16 * i + j]);
+                for (int qi = 0; qi < rep; ++qi)
+                    for (int qj = 0; qj < rep; ++qj) {
+                        scales[(rep * rb + qi) * (cols / 16) + rep * cb + qj] = (uint8_t)sc;
+                        if (scales_t) scales_t[(rep * cb + qj) * (rows / 16) + rep * rb + qi] = (uint8_t)sc;
+                    }
+                for (int i = 0; i < B; ++i)
+                    for (int j = 0; j < B; ++j) {
+                        put_nibble(payload, cols / 2, B * rb + i, B * cb + j, codes[B * i + j]);
+                        if (payload_t) put_nibble(payload_t, rows / 2, B * cb + j, B * rb + i, codes[B * i + j]);
                     }
             }
     } else {
@@ -366,6 +375,18 @@ ORACLE_API int oracle_quantize_window(const void *x, int dtype, int64_t rows, in
     }
     if (stats_out) { stats_out[0] = s0; stats_out[1] = s1; stats_out[2] = s2; stats_out[3] = s3; }
     return 0;
+}
+
+/* The recipe's block size, B = 16 (Table 1). */
+ORACLE_API int oracle_quantize_window(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                                      int layout, int rounding, float g, float T, uint64_t seed,
+                                      int64_t full_cols, int64_t row0, int64_t col0,
+                                      uint8_t *payload, uint8_t *scales,
+                                      uint8_t *payload_t, uint8_t *scales_t,
+                                      float *decode_out, uint64_t *stats_out)
+{
+    return oracle_quantize_window_block(x, dtype, rows, cols, ld, layout, rounding, g, T, seed, full_cols, row0, col0, 16,
+                                        payload, scales, payload_t, scales_t, decode_out, stats_out);
 }
 
 /* The whole tensor is the window at (0, 0). */

@@ -265,21 +265,23 @@ def test_amax_and_hold_schedule(printed):
 # ------------------------------------------------------------------------------------------
 # Whole quantizer against the textbook statement in exact rationals (Eq. "microscaling")
 # ------------------------------------------------------------------------------------------
-def _blocks(rows, cols, layout):
-    """Block membership written independently of the oracle: lists of (r, c) plus where the codes go."""
-    out = []
+def _blocks(rows, cols, layout, B=16):
+    """Block membership written independently of the oracle: lists of (r, c) plus the scale slots (one per 16
+    elements, so a block of 32 owns two, in 2D four) that must hold the block's code."""
+    out, rep = [], B // 16
     if layout == oracle.LAYOUT_1D_ROW:
         for r in range(rows):
-            for kb in range(cols // 16):
-                out.append(([(r, 16 * kb + j) for j in range(16)], (r, kb)))
+            for kb in range(cols // B):
+                out.append(([(r, B * kb + j) for j in range(B)], [(r, rep * kb + q) for q in range(rep)]))
     elif layout == oracle.LAYOUT_1D_COL:
         for c in range(cols):
-            for rb in range(rows // 16):
-                out.append(([(16 * rb + j, c) for j in range(16)], (c, rb)))
+            for rb in range(rows // B):
+                out.append(([(B * rb + j, c) for j in range(B)], [(c, rep * rb + q) for q in range(rep)]))
     else:
-        for rb in range(rows // 16):
-            for cb in range(cols // 16):
-                out.append(([(16 * rb + i, 16 * cb + j) for i in range(16) for j in range(16)], (rb, cb)))
+        for rb in range(rows // B):
+            for cb in range(cols // B):
+                out.append(([(B * rb + i, B * cb + j) for i in range(B) for j in range(B)],
+                            [(rep * rb + qi, rep * cb + qj) for qi in range(rep) for qj in range(rep)]))
     return out
 
 
@@ -291,28 +293,30 @@ def _nearest_ue5m3(u):
 
 @pytest.mark.parametrize("layout", [oracle.LAYOUT_1D_ROW, oracle.LAYOUT_1D_COL, oracle.LAYOUT_2D])
 @pytest.mark.parametrize("as_bf16", [False, True])
-def test_quantizer_equals_rational_microscaling(layout, as_bf16):
+@pytest.mark.parametrize("B", [16, 32])
+def test_quantizer_equals_rational_microscaling(layout, as_bf16, B):
     """With g = T 2^k the tensor multiplier is exact, so q_i must be the E2M1 value nearest to the
-    exact rational x_i T F / (g s_hat), s_hat the UE5M3 value nearest to a_B T / g."""
+    exact rational x_i T F / (g s_hat), s_hat the UE5M3 value nearest to a_B T / g; B = 16 is the recipe's
+    block size (Table 1), B = 32 the block-size control (Section 5.5)."""
     rng = np.random.default_rng(11 + layout)
-    rows, cols = 32, 48
+    rows, cols = (32, 48) if B == 16 else (64, 96)
     xf = (rng.normal(0, 1, (rows, cols)) * 10.0 ** rng.uniform(-2, 2, (rows, 1))).astype(np.float32)
     xf[4, 9] = 0.0
-    xf[:16, :16] *= 1e-9                                   # a tile that needs the zero-scale rule
+    xf[:B, :B] *= 1e-9                                     # a tile that needs the zero-scale rule
     xf = torch.from_numpy(xf).to(torch.bfloat16).float().numpy()
     x = bf16_bits(xf) if as_bf16 else xf
     T = 448.0
     g = T * 2.0 ** -1                                      # 224: stale reference, several blocks clip
-    q = oracle.quantize(x, layout, oracle.ROUND_RNE, g, T, want_t=True)
+    q = oracle.quantize(x, layout, oracle.ROUND_RNE, g, T, want_t=True, block=B)
     assert q["decode"] == f32(g) / f32(6 * T)
     n_checked = n_skipped = clip = repaired = 0
-    for members, (orow, ocol) in _blocks(rows, cols, layout):
+    for members, slots in _blocks(rows, cols, layout, B):
         aB = max(abs(Fr(float(xf[r, c]))) for r, c in members)
         code = _nearest_ue5m3(aB * Fr(T) / Fr(g))
         if code == 0:
             code = 0x78
             repaired += 1
-        assert q["scales"][orow, ocol] == code
+        assert all(q["scales"][orow, ocol] == code for orow, ocol in slots)
         s_hat = Fr(oracle.ue5m3_value(code))
         for r, c in members:
             z = Fr(float(xf[r, c])) * 6 * Fr(T) / (Fr(g) * s_hat)
