@@ -57,6 +57,11 @@ enum {
 
 enum { UE5M3_F32 = 0, UE5M3_BF16 = 1 };                                   /* element types */
 enum { UE5M3_LAYOUT_1D_ROW = 0, UE5M3_LAYOUT_1D_COL = 1, UE5M3_LAYOUT_2D = 2 };
+/* OR into the layout argument of ue5m3_quantize for the block-size control of Section 5.5 (B = 32 instead of 16):
+ * one scale per 32 elements along the blocked dimension (32 x 32 tiles in 2D), written to every 16-element slot
+ * it covers, so that buffers, scale layouts and the GEMM calls are unchanged.  The blocked dimensions must be
+ * multiples of 32. */
+enum { UE5M3_BLOCK_32 = 0x100 };
 enum { UE5M3_ROUND_RNE = 0, UE5M3_ROUND_SR = 1 };
 enum { UE5M3_SCALES_ROWMAJOR = 0, UE5M3_SCALES_TILED = 1 };
 enum { UE5M3_SCALE_1D = 0, UE5M3_SCALE_1D_TILED = 1, UE5M3_SCALE_2D = 2 };  /* how a GEMM operand's scales are stored */

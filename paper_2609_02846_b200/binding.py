@@ -15,6 +15,7 @@ import torch
 
 F32, BF16 = 0, 1
 LAYOUT_1D_ROW, LAYOUT_1D_COL, LAYOUT_2D = 0, 1, 2
+BLOCK_32 = 0x100            # OR into a layout: the block-size control (one scale per 32 elements)
 ROUND_RNE, ROUND_SR = 0, 1
 SCALES_ROWMAJOR, SCALES_TILED = 0, 1
 SCALE_1D, SCALE_1D_TILED, SCALE_2D = 0, 1, 2
@@ -146,8 +147,12 @@ class QuantizedOperand:
 
 def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tensor, target_T: float = 448.0,
              seed: int = 0, want_transpose: bool = False, stats: Optional[torch.Tensor] = None,
-             scale_layout: int = SCALES_ROWMAJOR, out: Optional[QuantizedOperand] = None) -> QuantizedOperand:
-    """ue5m3_quantize.  `stats` (int64[4], device) is accumulated into when given."""
+             scale_layout: int = SCALES_ROWMAJOR, out: Optional[QuantizedOperand] = None,
+             block: int = 16) -> QuantizedOperand:
+    """ue5m3_quantize.  `stats` (int64[4], device) is accumulated into when given.  `block = 32` selects the
+    block-size control (one scale per 32 elements, stored in every 16-element slot it covers)."""
+    if block not in (16, 32):
+        raise ValueError("block must be 16 or 32")
     rows, cols, ld = _matrix(x)
     dev = x.device
     u8 = dict(dtype=torch.uint8, device=dev)
@@ -178,8 +183,8 @@ def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tenso
         raise ValueError("stats must be an int64 tensor with 4 elements")
     with torch.cuda.device(dev):
         _check(_load().ue5m3_quantize(
-            _dev_ptr(x), _dtype_code(x), rows, cols, ld, layout, rounding, _dev_ptr(amax_held),
-            C.c_float(target_T), C.c_uint64(int(seed) & (2 ** 64 - 1)),
+            _dev_ptr(x), _dtype_code(x), rows, cols, ld, layout | (BLOCK_32 if block == 32 else 0), rounding,
+            _dev_ptr(amax_held), C.c_float(target_T), C.c_uint64(int(seed) & (2 ** 64 - 1)),
             _dev_ptr(out.payload), _dev_ptr(out.scales), _dev_ptr(out.payload_t), _dev_ptr(out.scales_t),
             _dev_ptr(out.decode), _dev_ptr(stats), scale_layout, _stream(x)), "ue5m3_quantize")
     return out

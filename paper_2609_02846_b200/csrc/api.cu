@@ -76,6 +76,8 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
                    const float* amax_held, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
                    uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
                    void* stream) {
+    const int block32 = (layout & UE5M3_BLOCK_32) ? 1 : 0;
+    layout &= ~UE5M3_BLOCK_32;
     if (!x || !amax_held || !payload || !scales || rows <= 0 || cols <= 0 || ld < cols) return UE5M3_ERR_INVALID_ARG;
     if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
     if (layout != UE5M3_LAYOUT_1D_ROW && layout != UE5M3_LAYOUT_1D_COL && layout != UE5M3_LAYOUT_2D) return UE5M3_ERR_INVALID_ARG;
@@ -86,6 +88,7 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
     if (layout != UE5M3_LAYOUT_2D && payload_t) return UE5M3_ERR_INVALID_ARG;
     if (layout == UE5M3_LAYOUT_2D && scale_layout != UE5M3_SCALES_ROWMAJOR) return UE5M3_ERR_INVALID_ARG;
     if ((rows % 16) || (cols % 16)) return UE5M3_ERR_SHAPE;
+    if (block32 && ((layout != UE5M3_LAYOUT_1D_COL && (cols % 32)) || (layout != UE5M3_LAYOUT_1D_ROW && (rows % 32)))) return UE5M3_ERR_SHAPE;
     const int64_t esz = dtype == UE5M3_F32 ? 4 : 2;
     if (!aligned16(x) || ((ld * esz) % 16) || !aligned16(payload) || !aligned16(scales)) return UE5M3_ERR_ALIGN;
     if (payload_t && (!aligned16(payload_t) || !aligned16(scales_t))) return UE5M3_ERR_ALIGN;
@@ -98,6 +101,7 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
     QuantArgs a{x, rows, cols, ld, amax_held, target_T, seed, payload, scales, payload_t, scales_t, decode_out,
                 reinterpret_cast<unsigned long long*>(stats)};
+    a.block32 = block32;
     return launch_quantize(a, dtype, layout, rounding, scale_layout == UE5M3_SCALES_TILED, (cudaStream_t)stream) == cudaSuccess
                ? UE5M3_OK
                : UE5M3_ERR_CUDA;
@@ -131,7 +135,8 @@ int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, in
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
     QuantArgs a{x, rows, cols, ld, amax_held, target_T_col, seed_col, payload_col, scales_col, nullptr, nullptr, decode_col,
                 reinterpret_cast<unsigned long long*>(stats_col),
-                payload_row, scales_row, target_T_row, seed_row, decode_row, reinterpret_cast<unsigned long long*>(stats_row)};
+                payload_row, scales_row, target_T_row, seed_row, decode_row, reinterpret_cast<unsigned long long*>(stats_row),
+                0};
     return launch_quantize_dual(a, dtype, rounding, scale_layout == UE5M3_SCALES_TILED, (cudaStream_t)stream) == cudaSuccess
                ? UE5M3_OK
                : UE5M3_ERR_CUDA;

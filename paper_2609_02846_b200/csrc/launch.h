@@ -25,6 +25,7 @@ struct QuantArgs {
     uint64_t row_seed;
     float* row_decode;
     unsigned long long* row_stats;
+    int block32;            // 1: one scale per 32 elements (32 x 32 in 2D), written to every 16-element slot it covers
 };
 
 struct GemmArgs {

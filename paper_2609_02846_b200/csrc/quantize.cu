@@ -111,9 +111,12 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a, 
         for (int j = 0; j < 16; ++j) aB = fmaxf(aB, fabsf(f[j]));
     }
 
+    // block of 32: the neighbouring thread holds the other half (blocks per row are even, so pairs never straddle rows)
+    if (a.block32) aB = fmaxf(aB, __shfl_xor_sync(0xFFFFFFFFu, aB, 1));
     float rB;
     uint32_t flags;
     const uint32_t code = block_scale(aB, tc, rB, flags);
+    if (a.block32 && (threadIdx.x & 1)) flags = 0;             // one count per block
 
     uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};
     if (SR) {
@@ -237,25 +240,37 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
     }
 
     // ---- block scales ----
+    // Blocks of 32: the thread holding the adjacent 16 rows is lane ^ 16 (lane ^ 1 in mode 2), the one holding the
+    // adjacent 16 columns of a 2D tile lane ^ 2; CTA tiles start on multiples of 32, so partners share a block.
+    constexpr int kRowPartner = (MODE == 2) ? 1 : 16;
     float rcol[8];
     uint32_t codes[8];
     uint32_t sat = 0, rep = 0;
     if (kColumns) {
+        if (a.block32) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) colmax[j] = fmaxf(colmax[j], __shfl_xor_sync(0xFFFFFFFFu, colmax[j], kRowPartner));
+        }
+        const bool counts = !a.block32 || (lane & kRowPartner) == 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t fl;
             codes[j] = block_scale(colmax[j], tc, rcol[j], fl);
-            sat += fl & 1u; rep += (fl >> 1) & 1u;
+            if (counts) { sat += fl & 1u; rep += (fl >> 1) & 1u; }
         }
     } else {
         float m = colmax[0];
 #pragma unroll
         for (int j = 1; j < 8; ++j) m = fmaxf(m, colmax[j]);
         m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+        if (a.block32) {
+            m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+            m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 16));
+        }
         uint32_t fl;
         float r;
         const uint32_t code = block_scale(m, tc, r, fl);
-        if ((lane & 1) == 0) { sat += fl & 1u; rep += (fl >> 1) & 1u; }
+        if ((lane & (a.block32 ? 19 : 1)) == 0) { sat += fl & 1u; rep += (fl >> 1) & 1u; }
 #pragma unroll
         for (int j = 0; j < 8; ++j) { rcol[j] = r; codes[j] = code; }
     }
@@ -283,10 +298,11 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
                 for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(f[j]));
             }
             m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+            if (a.block32) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
             float rrow;
             uint32_t fl;
             const uint32_t code_r = block_scale(m, tcr, rrow, fl);
-            if ((lane & 1) == 0) { sat_r += fl & 1u; rep_r += (fl >> 1) & 1u; }
+            if ((lane & (a.block32 ? 3 : 1)) == 0) { sat_r += fl & 1u; rep_r += (fl >> 1) & 1u; }
             uint32_t wr[4] = {0, 0, 0, 0};
             if (SR) sr_bits8(a.row_seed, ((uint64_t)(r0 + r) * (uint64_t)a.cols + (uint64_t)c0) >> 3, wr);
             const uint32_t orow = encode8<SR>(f, rrow, wr, clip_r);

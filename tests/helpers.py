@@ -7,16 +7,16 @@ import paper_2609_02846_b200 as lib
 from synth_inputs import to_numpy_bits
 
 
-def oracle_quantize(x: torch.Tensor, layout, rounding, g, T=448.0, seed=0, want_t=False):
-    return oracle.quantize(to_numpy_bits(x), layout, rounding, g, T, seed, want_t)
+def oracle_quantize(x: torch.Tensor, layout, rounding, g, T=448.0, seed=0, want_t=False, block=16):
+    return oracle.quantize(to_numpy_bits(x), layout, rounding, g, T, seed, want_t, block=block)
 
 
-def lib_quantize(x, layout, rounding, g, T=448.0, seed=0, want_t=False, with_stats=True, scale_layout=0):
+def lib_quantize(x, layout, rounding, g, T=448.0, seed=0, want_t=False, with_stats=True, scale_layout=0, block=16):
     """Returns (QuantizedOperand, canonical numpy dict like the oracle's)."""
     dev = x.device
     g_dev = g if isinstance(g, torch.Tensor) else torch.tensor([g], dtype=torch.float32, device=dev)
     stats = torch.zeros(4, dtype=torch.int64, device=dev) if with_stats else None
-    q = lib.quantize(x, layout, rounding, g_dev, T, seed, want_t, stats, scale_layout)
+    q = lib.quantize(x, layout, rounding, g_dev, T, seed, want_t, stats, scale_layout, block=block)
     scales = q.scales
     if scale_layout == lib.SCALES_TILED:
         R = q.payload.shape[0]

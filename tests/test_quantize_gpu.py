@@ -329,3 +329,62 @@ def test_dual_layout_call_without_counters_and_into_given_buffers():
     assert torch.equal(first[0].payload, single_r.payload) and torch.equal(first[0].scales, single_r.scales)
     assert torch.equal(first[1].payload, single_c.payload) and torch.equal(first[1].scales, single_c.scales)
     assert torch.equal(first[0].decode, single_r.decode) and torch.equal(first[1].decode, single_c.decode)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("rounding", ROUNDINGS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("shape", [(32, 32), (256, 256), (288, 4128), (1056, 224)])
+def test_block_32_control_matches_oracle(layout, rounding, dtype, shape):
+    """The block-size control (Section 5.5: the same recipe with B = 32): bytes, counters and the replicated scale
+    slots equal the oracle's; a block-32 scale code is the larger of the two (2D: four) block-16 codes."""
+    rows, cols = shape
+    x = si.heavy_tailed_gradient(rows, cols, seed=rows ^ cols, device=DEV, dtype=dtype)
+    g = _amax(x) * 0.25                                    # stale reference: clipping, no saturation yet
+    x[:32, :32] *= 1e-12                                   # a whole block that needs the zero-scale rule
+    for scale_layout in (0, 1) if layout != oracle.LAYOUT_2D else (0,):
+        _, got = lib_quantize(x, layout, rounding, g, seed=7, want_t=layout == oracle.LAYOUT_2D, scale_layout=scale_layout,
+                              block=32)
+        want = oracle_quantize(x, layout, rounding, g, seed=7, want_t=layout == oracle.LAYOUT_2D, block=32)
+        assert_same_quantization(got, want)
+    assert want["stats"]["zero_repaired"] >= 1
+    fine = oracle_quantize(x, layout, rounding, g, seed=7)
+    s16, s32 = fine["scales"].astype(np.int32), want["scales"].astype(np.int32)
+    s16 = np.where(s16 == 0x78, np.where(s32 == 0x78, 0x78, 0), s16)      # repaired zero codes carry no order
+    pair = np.maximum(s16[:, 0::2], s16[:, 1::2])
+    if layout == oracle.LAYOUT_2D:
+        pair = np.maximum(pair[0::2], pair[1::2])
+        assert np.array_equal(np.repeat(np.repeat(pair, 2, axis=0), 2, axis=1)[s32 != 0x78], s32[s32 != 0x78])
+    else:
+        assert np.array_equal(np.repeat(pair, 2, axis=1)[s32 != 0x78], s32[s32 != 0x78])
+
+
+def test_block_32_operands_run_through_the_unchanged_gemm():
+    import paper_2609_02846_b200 as lib
+    from helpers import check_gemm_output
+    M, K, N = 256, 512, 256
+    x = si.channel_scaled_activation(M, K, seed=1, device=DEV)
+    w = si.weight(N, K, seed=2, device=DEV)
+    qx, ox = lib_quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, _amax(x), block=32)
+    qw, ow = lib_quantize(w, lib.LAYOUT_2D, lib.ROUND_RNE, _amax(w), block=32)
+    y = lib.gemm(lib.FPROP, qx, qw, torch.float32)
+    yr, sa = oracle.gemm(ox["payload"], ox["scales"], False, ox["decode"], ow["payload"], ow["scales"], True, ow["decode"])
+    check_gemm_output(y, yr, sa)
+    # the coarser blocks cost accuracy against the unquantized product, as the control is meant to show
+    exact = x.double() @ w.double().T
+    qx16, _ = lib_quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, _amax(x))
+    qw16, _ = lib_quantize(w, lib.LAYOUT_2D, lib.ROUND_RNE, _amax(w))
+    y16 = lib.gemm(lib.FPROP, qx16, qw16, torch.float32)
+    err32 = (y.double() - exact).norm() / exact.norm()
+    err16 = (y16.double() - exact).norm() / exact.norm()
+    assert err16 < err32 < 3 * err16
+
+
+def test_block_32_rejects_dimensions_that_are_not_multiples_of_32():
+    import paper_2609_02846_b200 as lib
+    x = si.weight(48, 64, seed=1, device=DEV)
+    g = lib.sample_amax(x)
+    lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g, block=32)            # columns are the blocked dimension
+    for layout in (lib.LAYOUT_1D_COL, lib.LAYOUT_2D):
+        with pytest.raises(lib.Ue5m3Error):
+            lib.quantize(x, layout, lib.ROUND_RNE, g, block=32)
