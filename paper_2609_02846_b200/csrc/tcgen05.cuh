@@ -21,12 +21,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster (release at cluster scope).
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.  The arrive carries the default
+// release at CTA scope: what it publishes (this CTA's shared and tensor memory, already fenced for the async proxy) is
+// read by this CTA's own tensor core, never by threads of the other CTA, and a cluster-scope release was measured to
+// stall the arriving warp for about a thousand cycles.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar, uint32_t rank) {
     asm volatile(
         "{\n\t.reg .b32 ra;\n\t"
         "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
         ::"r"(bar), "r"(rank) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
