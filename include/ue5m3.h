@@ -110,6 +110,9 @@ UE5M3_API int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t 
  *                                   scales [rows/16, cols/16]; if payload_t and scales_t are both
  *                                   non-null they receive the same codes for x^T:
  *                                   payload_t [cols, rows/2], scales_t [cols/16, rows/16].
+ *              Any of the three may be OR-ed with UE5M3_BLOCK_32 (blocks of 32, or 32x32 tiles; the
+ *              blocked dimensions must then be multiples of 32; scale shapes stay as above, each
+ *              scale repeated in the slots it covers; counters [0] and [1] count blocks of 32).
  *   amax_held  device, 1 float (g).        target_T  integer-valued, 0 < T <= 61440 (448 or 2048).
  *   seed       used only for UE5M3_ROUND_SR.
  *   payload, scales       device outputs, both 16-byte aligned.
