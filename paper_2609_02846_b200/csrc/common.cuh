@@ -74,13 +74,16 @@ __device__ __forceinline__ uint32_t e2m1x2_rne(float lo, float hi) {
 __device__ __forceinline__ void sr_accumulate(float z, uint32_t word, int j, uint32_t& mags, uint32_t& signs) {
     const float t = fminf(z, 6.0f);                       // NaN -> +6, sign of everything else kept
     const float a = fminf(fabsf(t), 6.0f);
-    const float b = fmaxf(a, __fmaf_rn(a, 0.5f, 0.5f));     // a/2 + 1/2 exceeds a exactly when a < 1: no compare, no select
-    const uint32_t r = (j & 1) ? (word >> 10) : (word << 6);           // draw * 2^6 ...
-    const uint32_t Bp = __float_as_uint(b) + ((r & 0x3FFFC0u) | 32u);  // ... + 2^5, added below the kept bit
+    const float b = fmaxf(a, __fmaf_rn(a, 0.5f, 0.5f));   // a/2 + 1/2 exceeds a exactly when a < 1: no compare, no select
+    // The kernel is bound by the integer/logic pipe, the multiply-add pipe has room: the draw is placed below
+    // the kept bit and the sign into its nibble by integer multiply-adds instead of shift-and-mask pairs.
+    const uint32_t draw = (j & 1) ? (word >> 16) : (word & 0xFFFFu);
+    uint32_t Bp;
+    asm("mad.lo.u32 %0, %1, 64, %2;" : "=r"(Bp) : "r"(draw), "r"(__float_as_uint(b) + 32u));    // draw * 2^6 + 2^5 + bits(b)
     // bits 24:22 of Bp are the magnitude code plus 4 (mod 8); bit 31 of t is the sign
     const uint32_t m = (22 - 4 * j >= 0) ? (Bp >> (22 - 4 * j)) : (Bp << (4 * j - 22));
     mags |= m & (7u << (4 * j));
-    signs |= (__float_as_uint(t) >> (28 - 4 * j)) & (8u << (4 * j));
+    asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(signs) : "r"(__float_as_uint(t) >> 31), "r"(8u << (4 * j)));
 }
 __device__ __forceinline__ uint32_t sr_finish(uint32_t mags, uint32_t signs) { return (mags ^ 0x44444444u) | signs; }
 
