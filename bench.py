@@ -374,7 +374,7 @@ def run_ours(args):
         bufs = [tuple(getattr(step, n) for n in names), tuple(torch.empty_like(getattr(step, n)) for n in names)]
         s_in, s_out, main = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev), torch.cuda.current_stream()
         in_done, comp_done, out_done = [None, None], [None, None], [None, None]
-        n_e2e = max(2, min(K, 10))
+        n_e2e = max(2, min(K, 50))        # long enough that filling and draining the three-stage pipeline is amortised
 
         def e2e_step(s):
             b_ = s & 1
