@@ -66,7 +66,7 @@ constexpr int PK_STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + SC_B_BYTES
 constexpr int BF_STAGE_BYTES = BNH * KSUB * 2;     // 16384: the B slice; the A slice lives in tensor memory
 constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES;  // 208896
 constexpr int SMEM_EPI = SMEM_TILES + 1024;        // epilogue staging (1024-aligned for the 128B swizzle) after the barriers
-constexpr int EPI_WARP_BYTES = 4096;               // one 32 x 32 FP32 chunk, or two 32 x 32 BF16 chunks, per epilogue warp
+constexpr int EPI_WARP_BYTES = 4096;               // one box of 32 rows x 128 bytes per epilogue warp
 constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;                     // + alignment slack
 constexpr int TMEM_ACC_COL = 0, TMEM_A_COL = 256, TMEM_A_STAGE_COLS = KSUB / 2;      // 32 columns per A stage
 
@@ -220,7 +220,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // stores off the load/store pipe the dequantizers depend on.  The map clips rows >= Mo and columns >= No.
         const uint32_t stage = smem_base + SMEM_EPI + q * EPI_WARP_BYTES;
         uint8_t* stage_gen = smem_gen + SMEM_EPI + q * EPI_WARP_BYTES;
-        uint32_t tl = 0, chunk = 0;
+        uint32_t tl = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
             int tm, nb;
@@ -229,37 +229,53 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (!mbar_wait(acc_full, tl & 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const int row0 = mb * BM + q * 32, col0 = nb * BN;
+            if (p.out_bf16) {
+                // 64-column chunks: two tensor-memory loads fill one 4 KB box (32 rows of 128 bytes, 128B swizzle), then
+                // one proxy fence and one TMA store — half as many fences and stores as 32-column boxes would need.
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c, ++chunk) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_ACC_COL + c * 32, r);
-                tmem_ld_wait();
-                if (c == BN / 32 - 1) {
-                    // the accumulator has been read completely: the leader may start the next tile's MMAs
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
-                }
-                if (p.out_bf16) {
-                    // two 2 KB buffers: the store issued two chunks ago must have read its buffer
-                    if (lane == 0) tma_store_wait_read<1>();
-                    __syncwarp();
-                    const uint32_t boff = (chunk & 1) * 2048;
-                    uint8_t* mine = stage_gen + boff + lane * 64;
-                    const int sw = (lane >> 1) & 3;                   // 64-byte swizzle: 16-byte piece ^= (row / 2) % 4
+                for (int c = 0; c < BN / 64; ++c) {
+                    uint8_t* mine = stage_gen + lane * 128;
+                    const int sw = lane & 7;                              // 16-byte piece ^= row % 8
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 o;
-                        o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * alpha, __uint_as_float(r[8 * v + 1]) * alpha);
-                        o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * alpha, __uint_as_float(r[8 * v + 3]) * alpha);
-                        o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * alpha, __uint_as_float(r[8 * v + 5]) * alpha);
-                        o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * alpha, __uint_as_float(r[8 * v + 7]) * alpha);
-                        *reinterpret_cast<uint4*>(mine + ((v ^ sw) << 4)) = o;
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_ACC_COL + c * 64 + half * 32, r);
+                        tmem_ld_wait();
+                        if (c == BN / 64 - 1 && half == 1) {
+                            // the accumulator has been read completely: the leader may start the next tile's MMAs
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
+                        }
+                        if (half == 0) {
+                            if (lane == 0) tma_store_wait_read<0>();      // the previous store has read the box
+                            __syncwarp();
+                        }
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * alpha, __uint_as_float(r[8 * v + 1]) * alpha);
+                            o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * alpha, __uint_as_float(r[8 * v + 3]) * alpha);
+                            o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * alpha, __uint_as_float(r[8 * v + 5]) * alpha);
+                            o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * alpha, __uint_as_float(r[8 * v + 7]) * alpha);
+                            *reinterpret_cast<uint4*>(mine + (((half * 4 + v) ^ sw) << 4)) = o;
+                        }
                     }
                     fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) tma_store_2d(&map_out, stage + boff, col0 + c * 32, row0);
-                } else {
+                    if (lane == 0) tma_store_2d(&map_out, stage, col0 + c * 64, row0);
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_ACC_COL + c * 32, r);
+                    tmem_ld_wait();
+                    if (c == BN / 32 - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
+                    }
                     if (lane == 0) tma_store_wait_read<0>();
                     __syncwarp();
                     uint8_t* mine = stage_gen + lane * 128;
@@ -361,18 +377,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 }
 
 // ----------------------------------------------------------------------------- host side
-// Output [Mo, No] with leading dimension ldo, stored in boxes of 32 x 32 elements whose shared-memory image is
-// swizzled (64-byte rows for BF16, 128-byte rows for FP32).
+// Output [Mo, No] with leading dimension ldo, stored in boxes of 32 rows x 128 bytes (64 BF16 or 32 FP32 columns) whose
+// shared-memory image is 128B-swizzled.
 bool make_out_map(CUtensorMap* m, void* out, bool bf16, int64_t Mo, int64_t No, int64_t ldo) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const uint64_t esz = bf16 ? 2 : 4;
     cuuint64_t dims[2] = {(cuuint64_t)No, (cuuint64_t)Mo};
     cuuint64_t strides[1] = {(cuuint64_t)ldo * esz};
-    cuuint32_t box[2] = {32, 32};
+    cuuint32_t box[2] = {bf16 ? 64u : 32u, 32};
     cuuint32_t estr[2] = {1, 1};
     return fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
