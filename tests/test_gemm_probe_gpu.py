@@ -179,3 +179,15 @@ def test_probe_matched_full_size_linear_sampled_cells():
         out16 = _run(a, b, torch.bfloat16, grid_denominator=1024)
         assert torch.equal(out16, out32.to(torch.bfloat16)), op
         del out32, out16
+
+
+def test_probe_matched_deep_contraction():
+    """Kc = 16384 (the weight-gradient depth of a 16384-token batch): 256 toward-zero additions per cell."""
+    rng = np.random.default_rng(31)
+    Mo, No, Kc = 128, 256, 16384
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x68, 0x88, dec=0.01)
+    qb, bp, bsc = _operand(rng, No, Kc, 0, 0x68, 0x88, dec=0.02)
+    for cross in (0, 1):
+        out = _run(qa, qb, cross_rounding=cross, grid_denominator=1024)
+        want = oracle.gemm_probe(ap, asc, False, 0.01, bp, bsc, False, np.float32(0.02), cross_rne=bool(cross), grid_d=1024)
+        _assert_bit_equal(out, want)
