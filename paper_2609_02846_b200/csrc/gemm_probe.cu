@@ -63,7 +63,7 @@ constexpr int BF_A_BYTES = BM * KSUB * 2;          // 16384
 constexpr int BF_STAGE_BYTES = BF_A_BYTES + BN * KSUB * 2;       // 32768
 constexpr int SMEM_TILES = PK_STAGES * PK_STAGE_BYTES + BF_STAGES * BF_STAGE_BYTES; // 204800
 constexpr int SMEM_BYTES = SMEM_TILES + 512 + 1024;                                 // barriers, alignment slack
-static_assert(SETS * 4 * 64 <= 512, "tensor memory budget");
+static_assert(SETS * 4 * 64 <= 512, "the two sets must fit the 512 tensor-memory columns");
 static_assert(PK_STAGE_BYTES % 1024 == 0 && BF_STAGE_BYTES % 1024 == 0, "128B-swizzled tiles start on 1024-byte boundaries");
 
 struct ProbeParams {
