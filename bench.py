@@ -542,6 +542,37 @@ def run_probe(args):
     print(json.dumps(line), flush=True)
 
 
+def run_current(args):
+    """The per-batch (D = 1) reference policy: tensor maximum + quantization of X- and dY-sized tensors, as two calls and
+    as the one ue5m3_quantize_current call (the second pass directly behind the first on the same stream)."""
+    import torch
+    import paper_2609_02846_b200 as lib
+    import synth_inputs as si
+    dev = torch.device("cuda", 0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = {}
+    for name, rows, cols in (("X", M_TOK, K_IN), ("dY", M_TOK, N_OUT)):
+        x = si.channel_scaled_activation(rows, cols, seed=3, device=dev)
+        g = lib.sample_amax(x)
+        q = lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g)
+        res = {}
+        for label, fn in (("amax", lambda: lib.sample_amax(x, g)),
+                          ("quantize", lambda: lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, g, out=q)),
+                          ("quantize_current", lambda: lib.quantize_current(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, amax_out=g, out=q))):
+            ts = []
+            for _ in range(max(5, args.steps // 10)):
+                flush.fill_(1)                                   # start every measurement with x out of L2
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3)
+            res[label] = round(statistics.median(ts), 1)
+        res["MiB"] = rows * cols * 2 >> 20
+        out[name] = res
+    print(json.dumps({"workload": "per-batch reference policy, BF16, 1D rows, RNE; microseconds, L2 flushed before each measurement",
+                      "tensors": out}), flush=True)
+
+
 def run_sweep(args):
     """Quantizer-only bandwidth sweep: BF16 [rows, 4096], 2^20 .. 2^30 elements, {1D, 2D} x {RNE, SR} + amax."""
     import torch
@@ -626,6 +657,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--stack", action="store_true", help="time the six linears of the 8B-hybrid-shaped layer stack")
+    ap.add_argument("--current", action="store_true", help="time the per-batch (D = 1) reference policy")
     ap.add_argument("--probe", action="store_true", help="time the GEMMs under the Section 6.2 output model")
     ap.add_argument("--sweep-iters", type=int, default=100)
     ap.add_argument("--sweep-warmup", type=int, default=20)
@@ -643,6 +675,8 @@ def main():
         run_stack(args)
     elif args.probe:
         run_probe(args)
+    elif args.current:
+        run_current(args)
     else:
         run_ours(args)
 

@@ -133,6 +133,21 @@ UE5M3_API int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t col
                    int scale_layout, void* stream);
 
 /*
+ * Current scaling (the D = 1 policy of Table "delayed-scaling policies": the reference is recomputed for every
+ * batch): the tensor maximum of x is written to *amax_out and x is quantized against it, both on `stream`, the
+ * second pass directly behind the first.  The maximum must be complete before any element is scaled, so the tensor is
+ * read twice; the second read comes from the L2 cache only for tensors well below its size (a 64 MiB stream is not
+ * retained on B200).  The result equals ue5m3_sample_amax followed by ue5m3_quantize with amax_held = amax_out.
+ * Arguments, layouts and errors are those of the two calls (cols a multiple of 16 here).
+ */
+UE5M3_API int ue5m3_quantize_current(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                   int layout, int rounding, float* amax_out, float target_T, uint64_t seed,
+                   uint8_t* payload, uint8_t* scales,
+                   uint8_t* payload_t, uint8_t* scales_t,
+                   float* decode_out, uint64_t* stats,
+                   int scale_layout, void* stream);
+
+/*
  * Both 1D quantizations of one tensor from a single read (Section 5.3: the backward pass needs dY along its
  * columns for dX = dY W and along its rows for dW = dY^T X; likewise X along K for Y and along the tokens for dW).
  * The row outputs are exactly what ue5m3_quantize(..., UE5M3_LAYOUT_1D_ROW, rounding, ..., target_T_row, seed_row)

@@ -21,7 +21,7 @@ SCALES_ROWMAJOR, SCALES_TILED = 0, 1
 SCALE_1D, SCALE_1D_TILED, SCALE_2D = 0, 1, 2
 FPROP, DGRAD, WGRAD = 0, 1, 2
 
-SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_quantize_dual", "ue5m3_gemm", "ue5m3_gemm_probe_matched", "ue5m3_scales_bytes",
+SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_quantize_dual", "ue5m3_quantize_current", "ue5m3_gemm", "ue5m3_gemm_probe_matched", "ue5m3_scales_bytes",
            "ue5m3_unswizzle_scales", "ue5m3_last_device_status", "ue5m3_status_string")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -52,6 +52,8 @@ def _load() -> C.CDLL:
         L.ue5m3_sample_amax.argtypes = [vp, ci, i64, i64, i64, vp, vp]
         L.ue5m3_quantize.restype = ci
         L.ue5m3_quantize.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, f32, u64, vp, vp, vp, vp, vp, vp, ci, vp]
+        L.ue5m3_quantize_current.restype = ci
+        L.ue5m3_quantize_current.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, f32, u64, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_quantize_dual.restype = ci
         L.ue5m3_quantize_dual.argtypes = [vp, ci, i64, i64, i64, ci, vp, f32, f32, u64, u64, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_gemm.restype = ci
@@ -145,6 +147,32 @@ class QuantizedOperand:
         return QuantizedOperand(self.payload_t, self.scales_t, self.decode, SCALE_2D, self.payload, self.scales)
 
 
+def _alloc_operand(x: torch.Tensor, layout: int, want_transpose: bool, scale_layout: int) -> QuantizedOperand:
+    """Output buffers of one quantization of `x`."""
+    rows, cols, _ = _matrix(x)
+    dev = x.device
+    u8 = dict(dtype=torch.uint8, device=dev)
+    nbytes = scales_bytes(rows, cols, layout, scale_layout)
+    if nbytes == 0:
+        _check(2, "ue5m3_quantize (rows and cols must be positive multiples of 16)")
+    if layout == LAYOUT_1D_ROW:
+        payload = torch.empty((rows, cols // 2), **u8)
+        sshape = (rows, cols // 16)
+    elif layout == LAYOUT_1D_COL:
+        payload = torch.empty((cols, rows // 2), **u8)
+        sshape = (cols, rows // 16)
+    else:
+        payload = torch.empty((rows, cols // 2), **u8)
+        sshape = (rows // 16, cols // 16)
+    scales = torch.zeros(nbytes, **u8) if scale_layout == SCALES_TILED else torch.empty(sshape, **u8)
+    payload_t = scales_t = None
+    if layout == LAYOUT_2D and want_transpose:
+        payload_t = torch.empty((cols, rows // 2), **u8)
+        scales_t = torch.empty((cols // 16, rows // 16), **u8)
+    mode = SCALE_2D if layout == LAYOUT_2D else (SCALE_1D_TILED if scale_layout == SCALES_TILED else SCALE_1D)
+    return QuantizedOperand(payload, scales, torch.empty(1, dtype=torch.float32, device=dev), mode, payload_t, scales_t)
+
+
 def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tensor, target_T: float = 448.0,
              seed: int = 0, want_transpose: bool = False, stats: Optional[torch.Tensor] = None,
              scale_layout: int = SCALES_ROWMAJOR, out: Optional[QuantizedOperand] = None,
@@ -155,30 +183,8 @@ def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tenso
         raise ValueError("block must be 16 or 32")
     rows, cols, ld = _matrix(x)
     dev = x.device
-    u8 = dict(dtype=torch.uint8, device=dev)
     if out is None:
-        nbytes = scales_bytes(rows, cols, layout, scale_layout)
-        if nbytes == 0:
-            _check(2, "ue5m3_quantize (rows and cols must be positive multiples of 16)")
-        if layout == LAYOUT_1D_ROW:
-            payload = torch.empty((rows, cols // 2), **u8)
-            sshape = (rows, cols // 16)
-        elif layout == LAYOUT_1D_COL:
-            payload = torch.empty((cols, rows // 2), **u8)
-            sshape = (cols, rows // 16)
-        else:
-            payload = torch.empty((rows, cols // 2), **u8)
-            sshape = (rows // 16, cols // 16)
-        if scale_layout == SCALES_TILED:
-            scales = torch.zeros(nbytes, **u8)
-        else:
-            scales = torch.empty(sshape, **u8)
-        payload_t = scales_t = None
-        if layout == LAYOUT_2D and want_transpose:
-            payload_t = torch.empty((cols, rows // 2), **u8)
-            scales_t = torch.empty((cols // 16, rows // 16), **u8)
-        mode = SCALE_2D if layout == LAYOUT_2D else (SCALE_1D_TILED if scale_layout == SCALES_TILED else SCALE_1D)
-        out = QuantizedOperand(payload, scales, torch.empty(1, dtype=torch.float32, device=dev), mode, payload_t, scales_t)
+        out = _alloc_operand(x, layout, want_transpose, scale_layout)
     if stats is not None and (stats.dtype != torch.int64 or stats.numel() != 4):
         raise ValueError("stats must be an int64 tensor with 4 elements")
     with torch.cuda.device(dev):
@@ -188,6 +194,26 @@ def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tenso
             _dev_ptr(out.payload), _dev_ptr(out.scales), _dev_ptr(out.payload_t), _dev_ptr(out.scales_t),
             _dev_ptr(out.decode), _dev_ptr(stats), scale_layout, _stream(x)), "ue5m3_quantize")
     return out
+
+
+def quantize_current(x: torch.Tensor, layout: int, rounding: int, target_T: float = 448.0, seed: int = 0,
+                     want_transpose: bool = False, stats: Optional[torch.Tensor] = None,
+                     scale_layout: int = SCALES_ROWMAJOR, amax_out: Optional[torch.Tensor] = None,
+                     out: Optional[QuantizedOperand] = None):
+    """ue5m3_quantize_current: the per-batch (D = 1) reference policy.  Returns (operand, amax) where amax is the
+    tensor maximum the operand was scaled by (device float32[1])."""
+    if amax_out is None:
+        amax_out = torch.empty(1, dtype=torch.float32, device=x.device)
+    if out is None:
+        out = _alloc_operand(x, layout, want_transpose, scale_layout)
+    rows, cols, ld = _matrix(x)
+    with torch.cuda.device(x.device):
+        _check(_load().ue5m3_quantize_current(
+            _dev_ptr(x), _dtype_code(x), rows, cols, ld, layout, rounding, _dev_ptr(amax_out),
+            C.c_float(target_T), C.c_uint64(int(seed) & (2 ** 64 - 1)),
+            _dev_ptr(out.payload), _dev_ptr(out.scales), _dev_ptr(out.payload_t), _dev_ptr(out.scales_t),
+            _dev_ptr(out.decode), _dev_ptr(stats), scale_layout, _stream(x)), "ue5m3_quantize_current")
+    return out, amax_out
 
 
 def quantize_dual(x: torch.Tensor, rounding: int, amax_held: torch.Tensor, target_T_row: float = 448.0,

@@ -72,12 +72,11 @@ int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int6
                                                                                                         : UE5M3_ERR_CUDA;
 }
 
-int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int layout, int rounding,
-                   const float* amax_held, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
-                   uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
-                   void* stream) {
-    const int block32 = (layout & UE5M3_BLOCK_32) ? 1 : 0;
-    layout &= ~UE5M3_BLOCK_32;
+// Argument checks of ue5m3_quantize (layout without the block-size flag).
+static int check_quantize_args(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int layout, int block32,
+                               int rounding, const float* amax_held, float target_T, const uint8_t* payload,
+                               const uint8_t* scales, const uint8_t* payload_t, const uint8_t* scales_t,
+                               const float* decode_out, const uint64_t* stats, int scale_layout) {
     if (!x || !amax_held || !payload || !scales || rows <= 0 || cols <= 0 || ld < cols) return UE5M3_ERR_INVALID_ARG;
     if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
     if (layout != UE5M3_LAYOUT_1D_ROW && layout != UE5M3_LAYOUT_1D_COL && layout != UE5M3_LAYOUT_2D) return UE5M3_ERR_INVALID_ARG;
@@ -96,6 +95,18 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
         (reinterpret_cast<uintptr_t>(stats) & 7u))
         return UE5M3_ERR_ALIGN;
     if (rows * (cols / 16) >= ((int64_t)1 << 32) - 256) return UE5M3_ERR_UNSUPPORTED;   // 32-bit block index
+    return UE5M3_OK;
+}
+
+int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int layout, int rounding,
+                   const float* amax_held, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
+                   uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
+                   void* stream) {
+    const int block32 = (layout & UE5M3_BLOCK_32) ? 1 : 0;
+    layout &= ~UE5M3_BLOCK_32;
+    const int bad = check_quantize_args(x, dtype, rows, cols, ld, layout, block32, rounding, amax_held, target_T, payload, scales,
+                                        payload_t, scales_t, decode_out, stats, scale_layout);
+    if (bad != UE5M3_OK) return bad;
     const DeviceInfo di = device_info();
     if (!di.ok) return UE5M3_ERR_CUDA;
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
@@ -105,6 +116,21 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
     return launch_quantize(a, dtype, layout, rounding, scale_layout == UE5M3_SCALES_TILED, (cudaStream_t)stream) == cudaSuccess
                ? UE5M3_OK
                : UE5M3_ERR_CUDA;
+}
+
+int ue5m3_quantize_current(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int layout, int rounding,
+                           float* amax_out, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
+                           uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
+                           void* stream) {
+    // both calls' arguments are checked before anything is launched
+    const int bad = check_quantize_args(x, dtype, rows, cols, ld, layout & ~UE5M3_BLOCK_32, (layout & UE5M3_BLOCK_32) ? 1 : 0,
+                                        rounding, amax_out, target_T, payload, scales, payload_t, scales_t, decode_out, stats,
+                                        scale_layout);
+    if (bad != UE5M3_OK) return bad;
+    const int rc = ue5m3_sample_amax(x, dtype, rows, cols, ld, amax_out, stream);
+    if (rc != UE5M3_OK) return rc;
+    return ue5m3_quantize(x, dtype, rows, cols, ld, layout, rounding, amax_out, target_T, seed, payload, scales, payload_t,
+                          scales_t, decode_out, stats, scale_layout, stream);
 }
 
 int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int rounding,

@@ -388,3 +388,26 @@ def test_block_32_rejects_dimensions_that_are_not_multiples_of_32():
     for layout in (lib.LAYOUT_1D_COL, lib.LAYOUT_2D):
         with pytest.raises(lib.Ue5m3Error):
             lib.quantize(x, layout, lib.ROUND_RNE, g, block=32)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("rounding", ROUNDINGS)
+def test_current_scaling_call_equals_amax_then_quantize(layout, rounding):
+    """The per-batch (D = 1) reference policy in one call: the maximum it reports and every output byte equal the
+    oracle's amax followed by its quantizer."""
+    import paper_2609_02846_b200 as lib
+    x = si.heavy_tailed_gradient(272, 528, seed=17, device=DEV)
+    stats = torch.zeros(4, dtype=torch.int64, device=DEV)
+    q, amax = lib.quantize_current(x, layout, rounding, 448.0, seed=5, want_transpose=layout == oracle.LAYOUT_2D, stats=stats)
+    torch.cuda.synchronize()
+    g = oracle.amax(si.to_numpy_bits(x))
+    assert amax.item() == g
+    want = oracle_quantize(x, layout, rounding, g, 448.0, seed=5, want_t=layout == oracle.LAYOUT_2D)
+    got = dict(payload=q.payload.cpu().numpy(), scales=q.scales.cpu().numpy(),
+               payload_t=None if q.payload_t is None else q.payload_t.cpu().numpy(),
+               scales_t=None if q.scales_t is None else q.scales_t.cpu().numpy(),
+               decode=np.float32(q.decode.item()), stats=dict(zip(oracle.STAT_NAMES, stats.cpu().tolist())))
+    assert_same_quantization(got, want)
+    assert want["stats"]["scale_saturated"] == 0 and int(want["scales"].max()) == oracle.ue5m3_encode(np.float32(448.0))
+    with pytest.raises(lib.Ue5m3Error):
+        lib.quantize_current(x[:, :520], layout, rounding)          # 520 columns: not a multiple of 16, nothing is launched
