@@ -213,6 +213,23 @@ UE5M3_API int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t K
                void* out, int out_dtype, int64_t ldo, void* stream);
 
 /*
+ * Failure-detection self-test of the two GEMM kernels (the paper has no counterpart: its Section 7.1 only notes one
+ * restart of a run).  Every device-side wait of ue5m3_gemm and ue5m3_gemm_probe_matched is bounded; this call shows
+ * what happens when one runs out, without faulting or hanging the GPU: the kernel is launched on the given operands
+ * with its copy producer switched off and the bound of every wait set to wait_limit_cycles SM clocks, so each
+ * consumer's first wait expires, all roles drain, tensor memory is released and the kernel returns.  `out` is not
+ * written.  Afterwards ue5m3_last_device_status() returns UE5M3_ERR_TIMEOUT once and UE5M3_OK from then on, and the
+ * context stays usable.
+ *   which               0 = the kernel of ue5m3_gemm, 1 = the kernel of ue5m3_gemm_probe_matched.
+ *   wait_limit_cycles   1000 .. 4e9 (about 2e6 is one millisecond).
+ * All other arguments, and their checks and errors, are those of ue5m3_gemm.
+ */
+UE5M3_API int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc,
+               const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
+               const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
+               void* out, int out_dtype, int64_t ldo, int64_t wait_limit_cycles, void* stream);
+
+/*
  * Bytes a scale buffer needs.  rows/cols are those of the SOURCE tensor given to ue5m3_quantize.
  * (Section 3.2: one scale per block of B = 16; Section 3.3: one per 16x16 weight tile.)
  * Returns 0 for invalid arguments.

@@ -279,7 +279,7 @@ static void quantize_block(const void *x, int dtype, window_t win, int64_t ld,
     int code = oracle_ue5m3_encode(u);
     if (code == 0) { code = 0x78; stats[STAT_ZERO_REPAIRED]++; }   /* zero-scale rule: value 1 */
     float s_hat = (float)UE_TAB[code];                  /* exact */
-    float inv = 1.0f / s_hat;                           /* "before reciprocal computation" */
+    float inv = 1.0f / s_hat;                           /* Section 5.4, zero-scale rule: the reciprocal is taken of the stored value */
     float rB = G * inv;
     for (int i = 0; i < n; ++i) {
         float v = load_elem(x, dtype, mem[i].r * ld + mem[i].c);

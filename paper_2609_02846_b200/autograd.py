@@ -37,6 +37,24 @@ class OperandScale:
         return held
 
 
+_layer_counter = 0            # layers built so far in this process: the default stream id of a new layer
+
+
+def sr_stream_seed(layer_seed: int, rank: int, step: int) -> int:
+    """Base seed of one backward pass.  Eq. "sr" wants independent draws: two layers of the same shape, two
+    data-parallel ranks and two steps must not share a draw stream (the draw depends only on the seed and the element
+    index), otherwise their rounding errors are correlated and do not average out in the gradient all-reduce.
+    The three fields sit in disjoint bit ranges (step: 24 bits, rank: 14 bits, layer: 24 bits) of a 62-bit value,
+    since `linear_backward` uses 4 * seed and 4 * seed + 1 for its two quantizations."""
+    return ((int(layer_seed) & 0xFFFFFF) << 38) | ((int(rank) & 0x3FFF) << 24) | (int(step) & 0xFFFFFF)
+
+
+def _group_rank(group) -> int:
+    if group is not None and torch.distributed.is_initialized():
+        return torch.distributed.get_rank(group)
+    return 0
+
+
 def _check_dims(M: int, K: int, N: int) -> None:
     for name, v in (("tokens", M), ("in_features", K), ("out_features", N)):
         if v % 256:
@@ -62,7 +80,7 @@ class _Ue5m3LinearFn(torch.autograd.Function):
         layer, step = ctx.layer, ctx.step
         dy = dy.contiguous()
         ag = layer.scale_dy.get(dy, step)
-        dx, dw = B.linear_backward(dy, x, ctx.qw, ag, ctx.ax, seed=layer.seed * 1000003 + step, target_T=layer.target_T,
+        dx, dw = B.linear_backward(dy, x, ctx.qw, ag, ctx.ax, seed=sr_stream_seed(layer.seed, layer.rank, step), target_T=layer.target_T,
                                    target_T_wgrad_dy=layer.target_T_wgrad_dy, out_dtype=dy.dtype,
                                    grid_denominator=layer.grid_denominator, grad_rounding=layer.grad_rounding)
         return dx, dw, None, None
@@ -72,16 +90,21 @@ class Ue5m3Linear(torch.nn.Module):
     """y = x W^T with UE5M3-FP4 operands in all three GEMMs.  `x` is [tokens, in_features] (bfloat16 or float32);
     call `advance()` once per optimizer step so that the held references refresh every `interval` steps.
     `grid_denominator` not None runs the three products under the Section 6.2 output model (0: without its grid
-    step); `grad_rounding` is the rounding of the upstream gradient (stochastic by default)."""
+    step); `grad_rounding` is the rounding of the upstream gradient (stochastic by default).  `seed` names the layer's
+    stochastic-rounding stream (default: the count of layers built before it); the rank inside `group` and the step are
+    mixed in, so layers, ranks and steps draw independently."""
 
     def __init__(self, in_features: int, out_features: int, device="cuda", dtype=torch.bfloat16, interval: int = 50,
-                 target_T: float = 448.0, target_T_wgrad_dy: Optional[float] = None, seed: int = 0, group=None,
+                 target_T: float = 448.0, target_T_wgrad_dy: Optional[float] = None, seed: Optional[int] = None, group=None,
                  grid_denominator: Optional[int] = None, grad_rounding: int = B.ROUND_SR):
         super().__init__()
         self.weight = torch.nn.Parameter(torch.empty(out_features, in_features, device=device, dtype=dtype).normal_(0, 0.02))
         self.target_T = float(target_T)
         self.target_T_wgrad_dy = float(target_T if target_T_wgrad_dy is None else target_T_wgrad_dy)
-        self.seed = int(seed)
+        global _layer_counter
+        self.seed = _layer_counter if seed is None else int(seed)     # default: a stream of its own per layer
+        _layer_counter += 1
+        self.rank = _group_rank(group)          # mixed into the draws only; the tensor references stay rank-independent
         self.grid_denominator = grid_denominator
         self.grad_rounding = int(grad_rounding)
         self.step = 0

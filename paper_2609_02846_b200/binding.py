@@ -21,8 +21,9 @@ SCALES_ROWMAJOR, SCALES_TILED = 0, 1
 SCALE_1D, SCALE_1D_TILED, SCALE_2D = 0, 1, 2
 FPROP, DGRAD, WGRAD = 0, 1, 2
 
-SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_quantize_dual", "ue5m3_quantize_current", "ue5m3_gemm", "ue5m3_gemm_probe_matched", "ue5m3_scales_bytes",
-           "ue5m3_unswizzle_scales", "ue5m3_last_device_status", "ue5m3_status_string")
+SYMBOLS = ("ue5m3_sample_amax", "ue5m3_quantize", "ue5m3_quantize_dual", "ue5m3_quantize_current", "ue5m3_gemm",
+           "ue5m3_gemm_probe_matched", "ue5m3_gemm_stall_selftest", "ue5m3_scales_bytes", "ue5m3_unswizzle_scales",
+           "ue5m3_last_device_status", "ue5m3_status_string")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libue5m3.so")
@@ -60,6 +61,8 @@ def _load() -> C.CDLL:
         L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_probe_matched.restype = ci
         L.ue5m3_gemm_probe_matched.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, ci, ci, vp, ci, i64, vp]
+        L.ue5m3_gemm_stall_selftest.restype = ci
+        L.ue5m3_gemm_stall_selftest.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, i64, vp]
         L.ue5m3_scales_bytes.restype = C.c_size_t
         L.ue5m3_scales_bytes.argtypes = [i64, i64, ci, ci]
         L.ue5m3_unswizzle_scales.restype = ci
@@ -199,9 +202,14 @@ def quantize(x: torch.Tensor, layout: int, rounding: int, amax_held: torch.Tenso
 def quantize_current(x: torch.Tensor, layout: int, rounding: int, target_T: float = 448.0, seed: int = 0,
                      want_transpose: bool = False, stats: Optional[torch.Tensor] = None,
                      scale_layout: int = SCALES_ROWMAJOR, amax_out: Optional[torch.Tensor] = None,
-                     out: Optional[QuantizedOperand] = None):
+                     out: Optional[QuantizedOperand] = None, block: int = 16):
     """ue5m3_quantize_current: the per-batch (D = 1) reference policy.  Returns (operand, amax) where amax is the
-    tensor maximum the operand was scaled by (device float32[1])."""
+    tensor maximum the operand was scaled by (device float32[1]).  `layout` is one of the three LAYOUT_* values;
+    `block = 32` selects the block-size control as in `quantize`."""
+    if block not in (16, 32):
+        raise ValueError("block must be 16 or 32")
+    if layout not in (LAYOUT_1D_ROW, LAYOUT_1D_COL, LAYOUT_2D):
+        raise ValueError("layout must be LAYOUT_1D_ROW, LAYOUT_1D_COL or LAYOUT_2D (pass block=32 for the block-size control)")
     if amax_out is None:
         amax_out = torch.empty(1, dtype=torch.float32, device=x.device)
     if out is None:
@@ -209,7 +217,7 @@ def quantize_current(x: torch.Tensor, layout: int, rounding: int, target_T: floa
     rows, cols, ld = _matrix(x)
     with torch.cuda.device(x.device):
         _check(_load().ue5m3_quantize_current(
-            _dev_ptr(x), _dtype_code(x), rows, cols, ld, layout, rounding, _dev_ptr(amax_out),
+            _dev_ptr(x), _dtype_code(x), rows, cols, ld, layout | (BLOCK_32 if block == 32 else 0), rounding, _dev_ptr(amax_out),
             C.c_float(target_T), C.c_uint64(int(seed) & (2 ** 64 - 1)),
             _dev_ptr(out.payload), _dev_ptr(out.scales), _dev_ptr(out.payload_t), _dev_ptr(out.scales_t),
             _dev_ptr(out.decode), _dev_ptr(stats), scale_layout, _stream(x)), "ue5m3_quantize_current")
@@ -293,6 +301,19 @@ def gemm_probe_matched(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dt
                                                 _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)),
                "ue5m3_gemm_probe_matched")
     return out
+
+
+def gemm_stall_selftest(which: int, a: QuantizedOperand, b: QuantizedOperand, out: torch.Tensor,
+                        wait_limit_cycles: int = 2_000_000) -> None:
+    """ue5m3_gemm_stall_selftest: launches the chosen GEMM kernel (0: ue5m3_gemm, 1: ue5m3_gemm_probe_matched) with its
+    copy producer switched off and every wait bounded by `wait_limit_cycles`; `out` is left untouched and
+    `last_device_status()` then reports the timeout once."""
+    with torch.cuda.device(out.device):
+        _check(_load().ue5m3_gemm_stall_selftest(int(which), a.R, b.R, a.Kc,
+                                                 _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
+                                                 _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
+                                                 _dev_ptr(out), _dtype_code(out), out.stride(0), int(wait_limit_cycles),
+                                                 _stream(out)), "ue5m3_gemm_stall_selftest")
 
 
 def last_device_status() -> int:

@@ -1,6 +1,8 @@
 // C ABI of the UE5M3-FP4 library: argument checks on the host, then kernel launches.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <cstdint>
+#include <mutex>
 #include "../../include/ue5m3.h"
 #include "launch.h"
 
@@ -9,19 +11,26 @@ namespace ue5m3 {
 struct DeviceInfo { int ok; int sms; int major; };
 
 static DeviceInfo device_info() {
-    // one entry per device ordinal; filled on first use with that device current
+    // one entry per device ordinal; filled once, on first use with that device current (concurrent first calls
+    // are serialised by the once-flag; a failed query leaves ok = 0 for good)
     static DeviceInfo cache[64];
-    static bool known[64];
+    static std::once_flag asked[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DeviceInfo{0, 0, 0};
-    if (!known[dev]) {
-        cudaDeviceProp p;
-        if (cudaGetDeviceProperties(&p, dev) != cudaSuccess) return DeviceInfo{0, 0, 0};
-        cache[dev] = DeviceInfo{1, p.multiProcessorCount, p.major};
-        known[dev] = true;
-    }
+    std::call_once(asked[dev], [&]() {
+        int sms = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess)
+            cache[dev] = DeviceInfo{1, sms, major};
+    });
     return cache[dev];
 }
+
+// One NVTX range per C-ABI call (visible in a timeline profiler; a no-op when no tool is attached).
+struct ApiRange {
+    explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+    ~ApiRange() { nvtxRangePop(); }
+};
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -60,6 +69,7 @@ size_t ue5m3_scales_bytes(int64_t rows, int64_t cols, int layout, int scale_layo
 }
 
 int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* amax_out, void* stream) {
+    const ApiRange range_("ue5m3_sample_amax");
     if (!x || !amax_out || rows <= 0 || cols <= 0 || ld < cols) return UE5M3_ERR_INVALID_ARG;
     if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
     if (cols % 8) return UE5M3_ERR_SHAPE;
@@ -102,6 +112,7 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
                    const float* amax_held, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
                    uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
                    void* stream) {
+    const ApiRange range_("ue5m3_quantize");
     const int block32 = (layout & UE5M3_BLOCK_32) ? 1 : 0;
     layout &= ~UE5M3_BLOCK_32;
     const int bad = check_quantize_args(x, dtype, rows, cols, ld, layout, block32, rounding, amax_held, target_T, payload, scales,
@@ -122,6 +133,7 @@ int ue5m3_quantize_current(const void* x, int dtype, int64_t rows, int64_t cols,
                            float* amax_out, float target_T, uint64_t seed, uint8_t* payload, uint8_t* scales,
                            uint8_t* payload_t, uint8_t* scales_t, float* decode_out, uint64_t* stats, int scale_layout,
                            void* stream) {
+    const ApiRange range_("ue5m3_quantize_current");
     // both calls' arguments are checked before anything is launched
     const int bad = check_quantize_args(x, dtype, rows, cols, ld, layout & ~UE5M3_BLOCK_32, (layout & UE5M3_BLOCK_32) ? 1 : 0,
                                         rounding, amax_out, target_T, payload, scales, payload_t, scales_t, decode_out, stats,
@@ -138,6 +150,7 @@ int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, in
                         uint8_t* payload_row, uint8_t* scales_row, uint8_t* payload_col, uint8_t* scales_col,
                         float* decode_row, float* decode_col, uint64_t* stats_row, uint64_t* stats_col, int scale_layout,
                         void* stream) {
+    const ApiRange range_("ue5m3_quantize_dual");
     if (!x || !amax_held || !payload_row || !scales_row || !payload_col || !scales_col || rows <= 0 || cols <= 0 || ld < cols)
         return UE5M3_ERR_INVALID_ARG;
     if (dtype != UE5M3_F32 && dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
@@ -189,6 +202,7 @@ static int check_gemm_args(int op, int64_t Mo, int64_t No, int64_t Kc, const uin
 int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
                int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
                int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
+    const ApiRange range_("ue5m3_gemm");
     const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
                                     b_scale_mode, b_decode, out, out_dtype, ldo);
     if (bad != UE5M3_OK) return bad;
@@ -204,6 +218,7 @@ int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t Kc, const u
                              int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
                              int b_scale_mode, const float* b_decode, int cross_rounding, int grid_denominator,
                              void* out, int out_dtype, int64_t ldo, void* stream) {
+    const ApiRange range_("ue5m3_gemm_probe_matched");
     const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
                                     b_scale_mode, b_decode, out, out_dtype, ldo);
     if (bad != UE5M3_OK) return bad;
@@ -218,7 +233,28 @@ int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t Kc, const u
     return launch_gemm_probe(g, cross_rounding, grid_denominator, di.sms, (cudaStream_t)stream);
 }
 
+int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+                               int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+                               int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo,
+                               int64_t wait_limit_cycles, void* stream) {
+    const ApiRange range_("ue5m3_gemm_stall_selftest");
+    if (which != 0 && which != 1) return UE5M3_ERR_INVALID_ARG;
+    if (wait_limit_cycles < 1000 || wait_limit_cycles > 4000000000LL) return UE5M3_ERR_INVALID_ARG;
+    const int bad = check_gemm_args(UE5M3_FPROP, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
+                                    b_scale_mode, b_decode, out, out_dtype, ldo);
+    if (bad != UE5M3_OK) return bad;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
+               out, out_dtype, ldo};
+    g.wait_limit_cycles = wait_limit_cycles;
+    g.stall_producer = 1;
+    return which == 0 ? launch_gemm(g, di.sms, (cudaStream_t)stream) : launch_gemm_probe(g, 0, 0, di.sms, (cudaStream_t)stream);
+}
+
 int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream) {
+    const ApiRange range_("ue5m3_unswizzle_scales");
     if (!in || !out || R <= 0 || kblocks <= 0) return UE5M3_ERR_INVALID_ARG;
     const DeviceInfo di = device_info();
     if (!di.ok) return UE5M3_ERR_CUDA;

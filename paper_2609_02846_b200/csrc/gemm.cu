@@ -34,6 +34,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdint>
+#include <mutex>
 #include "../../include/ue5m3.h"
 #include "launch.h"
 #include "tcgen05.cuh"
@@ -78,6 +79,8 @@ struct GemmParams {
     int out_bf16;
     int a_mode, b_mode;           // UE5M3_SCALE_*
     int tiles_m, tiles_n;         // 256 x 256 tiles
+    long long wait_limit;         // bound of every device-side wait, SM clocks
+    int stall_producer;           // self-test: the copy producer issues nothing, so every consumer wait runs out
 };
 
 // Tile order: groups of kRasterGroup tile rows, and inside a group column by column.  The tiles that are
@@ -93,8 +96,8 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
     tm = first + (r - tn * gsize);
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    return mbar_wait_status(bar, parity, abort_flag, &g_device_status);
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
+    return mbar_wait_status(bar, parity, abort_flag, &g_device_status, limit);
 }
 
 // kind::f16 instruction descriptor: D = F32, A = B = F16 (format code 0), both K-major, M = 256 (two CTAs), N = 256.
@@ -155,14 +158,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int b_rows_per_load = (p.b_mode == UE5M3_SCALE_2D) ? 8 : 128;
             const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + b_rows_per_load * 16;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            for (int tile = pair; tile < num_tiles && ok && !p.stall_producer; tile += num_pairs) {
                 int tm, tn;
                 tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
                 const int mb = tm * 2 + (int)rank;                       // 128-row block of A
                 const int nh = tn * 2 + (int)rank;                       // 128-row block of B
                 for (int kc = 0; kc < kchunks; ++kc, ++it) {
                     const uint32_t s = it % PK_STAGES, ph = (it / PK_STAGES) & 1;
-                    if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                     const uint32_t st = pk_base + s * PK_STAGE_BYTES;
                     const uint32_t full = pk_full + 8 * s;
                     mbar_expect_tx(full, tx_bytes);
@@ -178,10 +181,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     else tma_load_2d(sb, &map_bs, full, 0, (nh * kchunks + kc) * 128);
                 }
             }
-            // let the copies still in flight land before the CTA's shared memory goes away
+            // let the copies still in flight land before the CTA's shared memory goes away (every one of them was
+            // issued, so it completes: this wait ignores the abort flag)
             for (uint32_t back = 0; back < PK_STAGES && back < it; ++back) {
                 const uint32_t j = it - 1 - back;
-                mbar_wait(pk_full + 8 * (j % PK_STAGES), (j / PK_STAGES) & 1, abort_flag);
+                mbar_wait_drain(pk_full + 8 * (j % PK_STAGES), (j / PK_STAGES) & 1, &g_device_status, p.wait_limit);
             }
         }
     } else if (warp == 1) {
@@ -190,13 +194,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t it = 0, tl = 0;
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
-                if (!mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag)) { ok = false; break; }   // epilogues have read tile tl-1
+                if (!mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }   // epilogues have read tile tl-1
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + TMEM_ACC_COL;
                 for (int ks = 0; ks < kchunks * SLICES; ++ks, ++it) {
                     // slice number it (converted by group it % 4) lives in stage it % BF_STAGES
                     const uint32_t s = it % BF_STAGES, ph = (it / BF_STAGES) & 1;
-                    if (!mbar_wait(bf_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bf_full + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t bd = umma_smem_desc(bf_base + s * BF_STAGE_BYTES);
                     const uint32_t ta = tmem_base + TMEM_A_COL + s * TMEM_A_STAGE_COLS;
@@ -209,7 +213,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
             // everything issued must have retired before tensor memory is released
             umma_commit_local(drain_bar);
-            mbar_wait(drain_bar, 0, abort_flag);
+            mbar_wait_drain(drain_bar, 0, &g_device_status, p.wait_limit);
         }
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------------------------ epilogue
@@ -226,7 +230,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             int tm, nb;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, nb);
             const int mb = tm * 2 + (int)rank;
-            if (!mbar_wait(acc_full, tl & 1, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(acc_full, tl & 1, abort_flag, p.wait_limit)) { ok = false; break; }
             tc_fence_after();
             const int row0 = mb * BM + q * 32, col0 = nb * BN;
             if (p.out_bf16) {
@@ -308,7 +312,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
             for (int kc = 0; kc < kchunks && ok; ++kc, ++it_pk) {
                 const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
-                if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag, p.wait_limit)) { ok = false; break; }
                 const uint8_t* st = smem_gen + ps * PK_STAGE_BYTES;
                 const uint4 a0 = *reinterpret_cast<const uint4*>(st + pk_off0);
                 const uint4 a1 = *reinterpret_cast<const uint4*>(st + pk_off1);
@@ -324,7 +328,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 // the FP16 stage of this slice; it is free once the MMAs of slice number - BF_STAGES have retired
                 const uint32_t slice_no = it_pk * SLICES + grp;
                 const uint32_t bs = slice_no % BF_STAGES;
-                if (!mbar_wait(bf_empty + 8 * bs, ((slice_no / BF_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bf_empty + 8 * bs, ((slice_no / BF_STAGES) & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
 
                 // A: 64 values of this row -> 32 tensor-memory columns (column c = K positions 2c, 2c+1)
                 {
@@ -403,12 +407,13 @@ bool make_scale_map(CUtensorMap* m, const uint8_t* scales, int mode, int64_t R, 
 }  // namespace
 
 int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
-    static int resident_pairs[64];      // CTA pairs that can be resident at once, per device; 0 = not asked yet
+    // CTA pairs that can be resident at once, per device; asked once per device, concurrent first calls serialised
+    static int resident_pairs[64];
+    static std::once_flag asked[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return UE5M3_ERR_CUDA;
-    if (resident_pairs[dev] == 0) {
-        if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-            return UE5M3_ERR_CUDA;
+    std::call_once(asked[dev], [&]() {
+        if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
         cfg.blockDim = dim3(NUM_THREADS, 1, 1);
@@ -419,7 +424,8 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
             n = num_sms / 2;
         }
         resident_pairs[dev] = n < num_sms / 2 ? n : num_sms / 2;
-    }
+    });
+    if (resident_pairs[dev] < 1) return UE5M3_ERR_CUDA;
     CUtensorMap ma, mb, mas, mbs;
     const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
     if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
@@ -436,6 +442,8 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     p.a_mode = g.a_scale_mode; p.b_mode = g.b_scale_mode;
     p.tiles_m = (int)((g.Mo + 2 * BM - 1) / (2 * BM));
     p.tiles_n = (int)((g.No + BN - 1) / BN);
+    p.wait_limit = g.wait_limit_cycles > 0 ? g.wait_limit_cycles : WAIT_LIMIT_CYCLES;
+    p.stall_producer = g.stall_producer;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int max_pairs = resident_pairs[dev];
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;

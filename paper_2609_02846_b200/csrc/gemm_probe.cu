@@ -32,6 +32,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdint>
+#include <mutex>
 #include "../../include/ue5m3.h"
 #include "launch.h"
 #include "tcgen05.cuh"
@@ -76,6 +77,8 @@ struct ProbeParams {
     int tiles_m, tiles_n;         // BM x BN tiles
     int cross_rne;                // 1: the control with nearest-even cross-group additions
     float grid;                   // d of Eq. "grid-denominator" (a power of two) or 0
+    long long wait_limit;         // bound of every device-side wait, SM clocks
+    int stall_producer;           // self-test: the copy producer issues nothing, so every consumer wait runs out
 };
 
 constexpr int kRasterGroup = 8;
@@ -88,8 +91,8 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
     tm = first + (r - tn * gsize);
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    return mbar_wait_status(bar, parity, abort_flag, &g_probe_status);
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
+    return mbar_wait_status(bar, parity, abort_flag, &g_probe_status, limit);
 }
 
 // kind::f16 instruction descriptor: D = F32, A = B = F16, both K-major, M = 128, N = 64.
@@ -241,13 +244,13 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const int b_rows_per_load = (p.b_mode == UE5M3_SCALE_2D) ? BN / 16 : BN;
             const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + b_rows_per_load * 16;
             bool ok = true;
-            for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
+            for (int tile = cta; tile < num_tiles && ok && !p.stall_producer; tile += num_ctas) {
                 int tm, tn;
                 tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
                 const int arow0 = tm * BM, brow0 = tn * BN;
                 for (int kc = 0; kc < kchunks; ++kc, ++it) {
                     const uint32_t s = it % PK_STAGES, ph = (it / PK_STAGES) & 1;
-                    if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                     const uint32_t st = smem_base + s * PK_STAGE_BYTES;
                     const uint32_t full = pk_full + 8 * s;
                     mbar_expect_tx(full, tx_bytes);
@@ -265,7 +268,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             // let the copies still in flight land before the CTA's shared memory goes away
             for (uint32_t back = 0; back < PK_STAGES && back < it; ++back) {
                 const uint32_t j = it - 1 - back;
-                mbar_wait(pk_full + 8 * (j % PK_STAGES), (j / PK_STAGES) & 1, abort_flag);
+                mbar_wait_drain(pk_full + 8 * (j % PK_STAGES), (j / PK_STAGES) & 1, &g_probe_status, p.wait_limit);
             }
         }
     } else if (warp == 1) {
@@ -276,7 +279,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
                 for (int ks = 0; ks < kchunks * SLICES && ok; ++ks, ++it) {
                     const uint32_t s = it % BF_STAGES, ph = (it / BF_STAGES) & 1;
-                    if (!mbar_wait(bf_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bf_full + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t ad = umma_smem_desc(bf_base + s * BF_STAGE_BYTES);
                     const uint64_t bd = umma_smem_desc(bf_base + s * BF_STAGE_BYTES + BF_A_BYTES);
@@ -284,7 +287,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     for (int h = 0; h < NH; ++h, ++gh) {
                         // the four blocks of this group and half go to the four buffers of set gh % SETS
                         const uint32_t set = gh % SETS;
-                        if (!mbar_wait(set_empty + 8 * set, ((gh / SETS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(set_empty + 8 * set, ((gh / SETS) & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                         tc_fence_after();
 #pragma unroll
                         for (int b = 0; b < KSUB / 16; ++b)
@@ -297,7 +300,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
             // everything issued must have retired before tensor memory is released
             umma_commit_1(drain_bar);
-            mbar_wait(drain_bar, 0, abort_flag);
+            mbar_wait_drain(drain_bar, 0, &g_probe_status, p.wait_limit);
         }
     } else if (warp >= DEQ_WARP0 && warp < DEQ_WARP0 + DEQ_WARPS) {
         // ------------------------------------------------------------------ dequantizers
@@ -310,7 +313,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         for (int tile = cta; tile < num_tiles && ok; tile += num_ctas) {
             for (int kc = 0; kc < kchunks && ok; ++kc, ++it_pk) {
                 const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
-                if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag, p.wait_limit)) { ok = false; break; }
                 const uint8_t* st = smem_gen + ps * PK_STAGE_BYTES;
                 const uint4 a_codes4 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + PK_B_BYTES + a_srow * 16);
                 const uint4 b_codes4 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + b_srow * 16);
@@ -330,7 +333,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     }
                     const uint32_t slice_no = it_pk * SLICES + sl;
                     const uint32_t bs = slice_no % BF_STAGES;
-                    if (!mbar_wait(bf_empty + 8 * bs, ((slice_no / BF_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bf_empty + 8 * bs, ((slice_no / BF_STAGES) & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                     uint8_t* stage_gen = smem_gen + PK_STAGES * PK_STAGE_BYTES + bs * BF_STAGE_BYTES;
                     {
                         const uint32_t m0 = scale_pair(a_codes & 0xFFu), m1 = scale_pair((a_codes >> 8) & 0xFFu);
@@ -385,7 +388,7 @@ gemm_probe_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                 for (int h = 0; h < NH; ++h, ++gh) {
                     const uint32_t set = gh % SETS;
-                    if (!mbar_wait(set_full + 8 * set, (gh / SETS) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(set_full + 8 * set, (gh / SETS) & 1, abort_flag, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t base = lane_addr + set * 256;
 #pragma unroll
@@ -496,13 +499,14 @@ bool make_scale_map_rows(CUtensorMap* m, const uint8_t* scales, int mode, int64_
 
 int launch_gemm_probe(const GemmArgs& g, int cross_rne, int grid_denominator, int num_sms, cudaStream_t st) {
     static bool configured[64];
+    static std::once_flag asked[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return UE5M3_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-            return UE5M3_ERR_CUDA;
-        configured[dev] = true;
-    }
+    std::call_once(asked[dev], [&]() {
+        configured[dev] =
+            cudaFuncSetAttribute(gemm_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    });
+    if (!configured[dev]) return UE5M3_ERR_CUDA;
     CUtensorMap ma, mb, mas, mbs;
     const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
     if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
@@ -519,6 +523,8 @@ int launch_gemm_probe(const GemmArgs& g, int cross_rne, int grid_denominator, in
     p.tiles_n = (int)((g.No + BN - 1) / BN);
     p.cross_rne = cross_rne;
     p.grid = (float)grid_denominator;
+    p.wait_limit = g.wait_limit_cycles > 0 ? g.wait_limit_cycles : WAIT_LIMIT_CYCLES;
+    p.stall_producer = g.stall_producer;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int ctas = num_tiles < num_sms ? num_tiles : num_sms;       // one CTA per SM: the kernel holds all tensor memory
     gemm_probe_kernel<<<ctas, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, p);

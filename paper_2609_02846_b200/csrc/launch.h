@@ -33,6 +33,10 @@ struct GemmArgs {
     const uint8_t* a_payload; const uint8_t* a_scales; int a_scale_mode; const float* a_decode;
     const uint8_t* b_payload; const uint8_t* b_scales; int b_scale_mode; const float* b_decode;
     void* out; int out_dtype; int64_t ldo;
+    // Failure-detection self-test only (ue5m3_gemm_stall_selftest): bound of every device-side wait in SM clocks
+    // (0 = the default, about two seconds) and 1 to launch with the copy producer switched off.
+    long long wait_limit_cycles = 0;
+    int stall_producer = 0;
 };
 
 cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, cudaStream_t st);

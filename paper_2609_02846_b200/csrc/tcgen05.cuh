@@ -7,7 +7,7 @@
 
 namespace ue5m3 {
 
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // default bound of a device-side wait: about two seconds
 
 // ----------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -41,24 +41,41 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after WAIT_LIMIT_CYCLES or as soon as another role has given up.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status_word) {
+// Bounded wait: gives up after `limit` SM clocks or as soon as another role of the CTA has given up.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status_word,
+                                                   long long limit) {
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             atomicExch(status_word, (int)UE5M3_ERR_TIMEOUT);
             return false;
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait_status(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status_word) {
+__device__ __forceinline__ bool mbar_wait_status(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status_word,
+                                                 long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status_word);
+    return mbar_wait_slow(bar, parity, abort_flag, status_word, limit);
+}
+// Drain wait: for something this thread really issued (a copy, a commit), which therefore completes.  It does not
+// look at the abort flag -- after another role gave up the issued work is still in flight and the CTA's shared and
+// tensor memory must outlive it -- and stops only on the clock, as a last resort.
+static __device__ __noinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, int* status_word, long long limit) {
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > limit) {
+            atomicExch(status_word, (int)UE5M3_ERR_TIMEOUT);
+            return false;
+        }
+    }
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -206,15 +223,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 inline EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    // resolved once per process; concurrent first calls are serialised by the function-local static
+    static const EncodeTiledFn fn = []() -> EncodeTiledFn {
         void* ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &ptr, 12000, cudaEnableDefault, &qres) != cudaSuccess ||
             qres != cudaDriverEntryPointSuccess)
             return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
+        return reinterpret_cast<EncodeTiledFn>(ptr);
+    }();
     return fn;
 }
 

@@ -175,6 +175,25 @@ def test_gemm_random_shapes_and_modes():
         check_gemm_output(out, y, sa)
 
 
+@pytest.mark.parametrize("shape", [(2432, 384, 256), (4352, 128, 512), (2304, 640, 256)])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_gemm_grouped_tile_order_with_ragged_last_group(shape, out_dtype):
+    """More than eight 256-row tile rows, and a count that is not a multiple of eight: the persistent scheduler visits
+    tiles in groups of eight tile rows, column by column inside a group, and the last group is short (2432 rows = 9.5
+    tile rows, 4352 = 17, 2304 = 9).  The whole output is compared with the exact oracle, so a tile visited twice,
+    skipped or written to the wrong place cannot pass."""
+    Mo, No, Kc = shape
+    rng = np.random.default_rng(Mo * 7 + No)
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x50, 0xA0, dec=0.25)
+    qb, bp, bsc = _operand(rng, No, Kc, 2, 0x50, 0xA0, dec=1.0 / 512.0)
+    out = torch.full((Mo, No), float("nan"), dtype=out_dtype, device=DEV)
+    lib.gemm(lib.WGRAD, qa, qb, out=out)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    y, sa = oracle.gemm(ap, asc, False, 0.25, bp, bsc, True, np.float32(1.0 / 512.0))
+    check_gemm_output(out, y, sa)
+
+
 def test_gemm_and_quantizer_are_deterministic():
     """Same inputs, same bytes: three runs of a linear's forward and backward give identical outputs."""
     M, K, N = 512, 1024, 768

@@ -73,3 +73,40 @@ def test_refresh_step_amax_is_agreed_across_ranks():
         mp.spawn(_amax_worker, args=(2, port, out), nprocs=2, join=True)
         res = dict(out)
     assert res[0] == res[1] == 3.5
+
+
+def test_layers_ranks_and_steps_draw_from_different_streams():
+    """Eq. "sr" assumes independent draws: the base seed of a backward pass differs between two layers built with the
+    default seed, between two data-parallel ranks and between two steps, and so do the 16-bit draws the oracle's
+    generator gives for the same element index; both quantizations of dY inside one pass (4s and 4s + 1) differ too."""
+    import oracle
+    from paper_2609_02846_b200 import autograd
+    a = autograd.Ue5m3Linear(256, 256, device="cpu")
+    b = autograd.Ue5m3Linear(256, 256, device="cpu")
+    assert a.seed != b.seed and a.rank == b.rank == 0
+    seeds = {autograd.sr_stream_seed(layer, rank, step) for layer in (a.seed, b.seed) for rank in (0, 1, 7) for step in (0, 1, 50)}
+    assert len(seeds) == 18 and max(seeds) < 2 ** 62
+    streams = set()
+    for s in seeds:
+        for role in (0, 1):
+            streams.add(tuple(oracle.sr_bits(4 * s + role, i) for i in range(16)))
+    assert len(streams) == 36
+
+
+def _rank_seed_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2609_02846_b200 import autograd
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    layer = autograd.Ue5m3Linear(256, 256, device="cpu", seed=5, group=dist.group.WORLD)
+    out[rank] = (layer.rank, autograd.sr_stream_seed(layer.seed, layer.rank, 3))
+    dist.destroy_process_group()
+
+
+def test_rank_is_mixed_into_the_gradient_draws():
+    port = 33500 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_rank_seed_worker, args=(2, port, out), nprocs=2, join=True)
+        res = dict(out)
+    assert res[0][0] == 0 and res[1][0] == 1 and res[0][1] != res[1][1]

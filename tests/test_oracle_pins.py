@@ -489,6 +489,149 @@ def test_sr_col_layout_uses_source_indices():
 
 
 # ------------------------------------------------------------------------------------------
+# The quantizer for a general reference g: exact rationals with only the named binary32 roundings
+# ------------------------------------------------------------------------------------------
+def rn32(q):
+    """Round an exact rational to binary32 (nearest, ties to even significand, subnormals below 2^-126); exact result
+    as a Fraction.  Written from the IEEE-754 definition: quantum 2^(e-23) for 2^e <= |q| < 2^(e+1), e >= -126."""
+    q = Fr(q)
+    if q == 0:
+        return Fr(0)
+    a = abs(q)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fr(2) ** e > a:
+        e -= 1
+    assert Fr(2) ** e <= a < Fr(2) ** (e + 1)
+    quantum = Fr(2) ** (max(e, -126) - 23)
+    n, rem = divmod(a, quantum)
+    if rem * 2 > quantum or (rem * 2 == quantum and n % 2 == 1):
+        n += 1
+    r = n * quantum
+    assert r < Fr(2) ** 128
+    return r if q > 0 else -r
+
+
+def _philox4x32(ctr, key, rounds=10):
+    """Philox4x32 from its definition (Salmon et al. 2011, Section 3.3 and Table 2 constants), Python integers."""
+    c = list(ctr)
+    k = list(key)
+    for _ in range(rounds):
+        p0, p1 = 0xD2511F53 * c[0], 0xCD9E8D57 * c[2]
+        c = [(p1 >> 32) ^ c[1] ^ k[0], p1 & 0xFFFFFFFF, (p0 >> 32) ^ c[3] ^ k[1], p0 & 0xFFFFFFFF]
+        k = [(k[0] + 0x9E3779B9) & 0xFFFFFFFF, (k[1] + 0xBB67AE85) & 0xFFFFFFFF]
+    return c
+
+
+def _draw16(seed, i):
+    w = _philox4x32([(i >> 3) & 0xFFFFFFFF, (i >> 3) >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32])
+    return (w[(i & 7) >> 1] >> (16 * (i & 1))) & 0xFFFF
+
+
+def _e2m1_nearest_even(a):
+    """Index of the E2M1 magnitude nearest to 0 <= a <= 6, ties to the even index (fraction bit 0)."""
+    return min(range(8), key=lambda c: (abs(E2M1_MAGS[c] - a), c % 2))
+
+
+def _e2m1_stochastic(a, r16):
+    """Eq. "sr" resolved to 16 bits: a (already a binary32 value in [0, 6]) lies in [q-, q+); below 1 it is first rounded
+    to the binary32 grid of [1, 2) (a multiple of 2^-23).  With L = 2^22 (a - q-)/(q+ - q-) (an integer: every E2M1 gap is
+    2^22 binary32 steps of its binade) it goes up iff L + 64 r16 + 32 >= 2^22."""
+    if a < 1:
+        a = rn32(a + 1) - 1
+    lo = max(c for c in range(8) if E2M1_MAGS[c] <= a)
+    if lo == 7:
+        return 7
+    L = (a - E2M1_MAGS[lo]) / (E2M1_MAGS[lo + 1] - E2M1_MAGS[lo]) * 2 ** 22
+    assert L.denominator == 1
+    return lo + 1 if L + 64 * r16 + 32 >= 2 ** 22 else lo
+
+
+@pytest.mark.parametrize("layout", [oracle.LAYOUT_1D_ROW, oracle.LAYOUT_1D_COL, oracle.LAYOUT_2D])
+@pytest.mark.parametrize("rounding", [oracle.ROUND_RNE, oracle.ROUND_SR])
+@pytest.mark.parametrize("T", [448.0, 2048.0])
+@pytest.mark.parametrize("g_kind", ["hundred", "fraction_of_max", "current_max", "stale"])
+def test_quantizer_equals_stepwise_rational_restatement_for_general_g(layout, rounding, T, g_kind):
+    """Non-dyadic references: S = RN32(T/g), G = RN32(6T/g), d = RN32(g/(6T)), u_B = RN32(a_B S), 1/s = RN32(1/s_hat),
+    r_B = RN32(G RN32(1/s_hat)), z = RN32(x r_B) -- exactly these seven roundings, everything else in exact rationals
+    (Eq. "scale-target" right-hand form, Eq. "microscaling", zero-scale rule, Eq. "sr").  Every scale byte, payload nibble,
+    the decode factor and the clip / repair / saturation counters must agree; no element is skipped."""
+    rng = np.random.default_rng(101 + layout + 3 * rounding + int(T))
+    rows, cols = (16, 32) if layout == oracle.LAYOUT_1D_ROW else (16, 16)
+    x = (rng.normal(0, 1, (rows, cols)) * 10.0 ** rng.uniform(-1.5, 1.5, (rows, cols))).astype(np.float32)
+    x[0, 3] = -0.0
+    x[rows - 1, cols - 1] = np.float32(1e-12)
+    if layout == oracle.LAYOUT_1D_ROW:
+        x[1, 16:] *= np.float32(1e-9)                       # one block that needs the zero-scale rule
+    amax = float(np.abs(x).max())
+    g = {"hundred": 100.0, "fraction_of_max": float(np.float32(0.37 * amax)), "current_max": amax,
+         "stale": float(np.float32(amax / 201.0))}[g_kind]    # T rho = 201 T > 61440: Proposition 1 says saturation
+    seed = 0x9E3779B97F4A7C15
+    q = oracle.quantize(x, layout, rounding, g, T, seed=seed, want_t=True)
+
+    gF, TF = Fr(float(np.float32(g))), Fr(T)
+    S, G, d = rn32(TF / gF), rn32(6 * TF / gF), rn32(gF / (6 * TF))
+    assert Fr(float(q["decode"])) == d
+    clip = repaired = saturated = 0
+    for members, slots in _blocks(rows, cols, layout):
+        aB = max(abs(Fr(float(x[r, c]))) for r, c in members)
+        u = rn32(aB * S)
+        saturated += u > 61440
+        code = _nearest_ue5m3(u)
+        if code == 0:
+            code, repaired = 0x78, repaired + 1
+        assert all(q["scales"][orow, ocol] == code for orow, ocol in slots)
+        rB = rn32(G * rn32(1 / Fr(oracle.ue5m3_value(code))))
+        for r, c in members:
+            z = rn32(Fr(float(x[r, c])) * rB)
+            clip += abs(z) > 6
+            a = min(abs(z), Fr(6))
+            mag = _e2m1_nearest_even(a) if rounding == oracle.ROUND_RNE else _e2m1_stochastic(a, _draw16(seed, r * cols + c))
+            want = (8 if np.signbit(x[r, c]) else 0) | mag
+            if layout == oracle.LAYOUT_1D_COL:
+                got = (q["payload"][c, r // 2] >> (4 * (r % 2))) & 0xF
+            else:
+                got = (q["payload"][r, c // 2] >> (4 * (c % 2))) & 0xF
+            assert got == want, (r, c, float(z), got, want)
+            if layout == oracle.LAYOUT_2D:
+                assert (q["payload_t"][c, r // 2] >> (4 * (r % 2))) & 0xF == want
+    assert q["stats"] == dict(scale_saturated=saturated, zero_repaired=repaired, payload_clipped=clip, nonfinite=0)
+    if g_kind == "current_max":
+        assert saturated == 0 and (q["scales"] == oracle.ue5m3_encode(T)).any()      # a_B = g  =>  u_B = T
+    if g_kind == "stale":
+        assert saturated > 0 and clip > 0
+
+
+def test_operation_order_of_the_scale_is_pinned():
+    """The right-hand form of Eq. "scale-target", u_B = a_B (T/g) with the quotient rounded first, differs from
+    RN32(RN32(a_B T)/g) in the last bit for some inputs.  Block maxima placed within a few binary32 steps of a UE5M3
+    midpoint separate the two orders (different scale bytes); the oracle must follow the first."""
+    T = 448.0
+    found = 0
+    rng = np.random.default_rng(5)
+    mids = [Fr(17, 16), Fr(19, 16), Fr(21, 8), Fr(27, 2), Fr(25, 64)]      # midpoints between adjacent UE5M3 values
+    for _ in range(400):
+        g = float(np.float32(rng.uniform(1.0, 200.0)))
+        S = rn32(Fr(T) / Fr(g))
+        for mid in mids:
+            a0 = np.float32(float(mid / S))
+            for step in range(-3, 4):
+                aB = a0
+                for _s in range(abs(step)):
+                    aB = np.nextafter(aB, np.float32(np.inf if step > 0 else 0), dtype=np.float32)
+                u1 = rn32(Fr(float(aB)) * S)
+                u2 = rn32(rn32(Fr(float(aB)) * Fr(T)) / Fr(g))
+                c1, c2 = _nearest_ue5m3(u1), _nearest_ue5m3(u2)
+                if c1 != c2:
+                    x = np.zeros((16, 16), np.float32)
+                    x[3, 5] = -aB
+                    assert oracle.quantize(x, oracle.LAYOUT_1D_ROW, oracle.ROUND_RNE, g, T)["scales"][3, 0] == c1
+                    found += 1
+        if found >= 8:
+            break
+    assert found >= 8
+
+
+# ------------------------------------------------------------------------------------------
 # GEMM (Section 5.3 / 6.1: plain sums over the decoded operands)
 # ------------------------------------------------------------------------------------------
 def _rand_operand(rng, R, Kc, scale2d):
