@@ -124,7 +124,7 @@ int ue5m3_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t
     QuantArgs a{x, rows, cols, ld, amax_held, target_T, seed, payload, scales, payload_t, scales_t, decode_out,
                 reinterpret_cast<unsigned long long*>(stats)};
     a.block32 = block32;
-    return launch_quantize(a, dtype, layout, rounding, scale_layout == UE5M3_SCALES_TILED, (cudaStream_t)stream) == cudaSuccess
+    return launch_quantize(a, dtype, layout, rounding, scale_layout == UE5M3_SCALES_TILED, di.sms, (cudaStream_t)stream) == cudaSuccess
                ? UE5M3_OK
                : UE5M3_ERR_CUDA;
 }

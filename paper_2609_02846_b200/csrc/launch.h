@@ -5,6 +5,13 @@
 
 namespace ue5m3 {
 
+// The ten round-key pairs of Philox4x32-10 for one seed (k[2r], k[2r + 1] = key of round r).  They depend only on
+// the seed, so the launcher computes them on the host and they travel with the launch parameters.
+struct PhiloxKeys {
+    uint32_t k[20];
+    uint32_t m0k0_hi, m0k0_lo;      // 0xD2511F53 * k[0]: the second round's first product when the counter is below 2^32
+};
+
 struct QuantArgs {
     const void* x;
     int64_t rows, cols, ld;
@@ -26,6 +33,9 @@ struct QuantArgs {
     float* row_decode;
     unsigned long long* row_stats;
     int block32;            // 1: one scale per 32 elements (32 x 32 in 2D), written to every 16-element slot it covers
+    PhiloxKeys keys;        // round keys of `seed`, filled in by the launcher (stochastic rounding only)
+    PhiloxKeys row_keys;    // round keys of `row_seed` (dual-layout call)
+    int small_counter;      // 1: fewer than 2^35 elements, so every Philox counter fits in 32 bits
 };
 
 struct GemmArgs {
@@ -39,7 +49,7 @@ struct GemmArgs {
     int stall_producer = 0;
 };
 
-cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, cudaStream_t st);
+cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, int num_sms, cudaStream_t st);
 cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bool tiled, cudaStream_t st);
 cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* out, int num_sms,
                         cudaStream_t st);

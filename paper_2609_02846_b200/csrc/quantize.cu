@@ -34,119 +34,255 @@ __device__ __forceinline__ void warp_add_stats(unsigned long long* stats, uint32
 
 __device__ __forceinline__ bool nonfinite(float v) { return !(fabsf(v) < __int_as_float(0x7f800000)); }
 
-// Eight consecutive elements -> four payload bytes (one 32-bit word), RNE or SR.
-template <bool SR>
-__device__ __forceinline__ uint32_t encode8(const float f[8], float rB, const uint32_t w[4], uint32_t& clip) {
+// Eight consecutive elements -> the eight values the saturating hardware conversion will encode: the products
+// z = f * r themselves for round-to-nearest (the conversion rounds), or their stochastic roundings, which already lie
+// on the E2M1 grid.  `r` holds the per-element multipliers.  SANITIZE: NaN products are replaced by +Inf before the
+// stochastic rounding (callers that already removed NaNs from their inputs pass false).
+template <bool SR, bool SANITIZE>
+__device__ __forceinline__ void round_values8(const float f[8], const float r[8], const uint32_t w[4], float v[8], uint32_t& clip) {
     float z[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) z[j] = __fmul_rn(f[j], rB);
+    for (int j = 0; j < 8; ++j) z[j] = __fmul_rn(f[j], r[j]);
 #pragma unroll
     for (int j = 0; j < 8; ++j) clip += (fabsf(z[j]) > 6.0f) ? 1u : 0u;
-    uint32_t out = 0;
     if (SR) {
-        uint32_t mags = 0, signs = 0;
+        if (SANITIZE) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) sr_accumulate(z[j], w[j >> 1], j, mags, signs);
-        out = sr_finish(mags, signs);
+            for (int j = 0; j < 8; ++j) z[j] = fminf(z[j], __int_as_float(0x7f800000));   // NaN -> +Inf -> +6
+        }
+        sr_values8(z, w, v);
     } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) out |= e2m1x2_rne(z[2 * j], z[2 * j + 1]) << (8 * j);
+        for (int j = 0; j < 8; ++j) v[j] = z[j];
     }
+}
+// Eight values -> four payload bytes (element j in bits 4j+3:4j).
+__device__ __forceinline__ uint32_t pack8(const float v[8]) {
+    uint32_t out = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) out |= e2m1x2_rne(v[2 * j], v[2 * j + 1]) << (8 * j);
     return out;
+}
+template <bool SR, bool SANITIZE>
+__device__ __forceinline__ uint32_t encode8(const float f[8], float rB, const uint32_t w[4], uint32_t& clip) {
+    const float r[8] = {rB, rB, rB, rB, rB, rB, rB, rB};
+    float v[8];
+    round_values8<SR, SANITIZE>(f, r, w, v, clip);
+    return pack8(v);
+}
+
+// ---------------------------------------------------------------------------------------
+// Per-CTA set-up: tensor constants (three IEEE divisions by thread 0) and the table code -> r_B
+// ---------------------------------------------------------------------------------------
+struct CtaTables {
+    TensorConsts tc[2];        // [0]: target T, [1]: the row target of the dual-layout call
+    float lut[2][256];         // scale_multiplier(code, G) for the two targets
+};
+
+// Fills the tables; every thread of a 256-thread CTA owns one code.  Two barriers.
+template <bool DUAL>
+__device__ __forceinline__ void cta_setup(CtaTables& t, const float* amax_held, float T, float T_row) {
+    if (threadIdx.x == 0) {
+        const float g = __ldg(amax_held);
+        t.tc[0] = tensor_consts(g, T);
+        if (DUAL) t.tc[1] = tensor_consts(g, T_row);
+    }
+    __syncthreads();
+    t.lut[0][threadIdx.x] = scale_multiplier(threadIdx.x, t.tc[0].G);
+    if (DUAL) t.lut[1][threadIdx.x] = scale_multiplier(threadIdx.x, t.tc[1].G);
+    __syncthreads();
 }
 
 // ---------------------------------------------------------------------------------------
 // 1D blocks along the contiguous dimension
 // ---------------------------------------------------------------------------------------
-// Tensor constants are computed once per CTA (three IEEE divisions) and broadcast through shared memory.
-__device__ __forceinline__ TensorConsts cta_tensor_consts(const float* amax_held, float T) {
-    __shared__ TensorConsts s_tc;
-    if (threadIdx.x == 0) s_tc = tensor_consts(__ldg(amax_held), T);
-    __syncthreads();
-    return s_tc;
-}
-
-// The same for two targets at once (dual-layout call: columns with T, rows with T_row).
-__device__ __forceinline__ void cta_tensor_consts2(const float* amax_held, float T, float T_row, TensorConsts& tc, TensorConsts& tcr) {
-    __shared__ TensorConsts s_tc2[2];
-    if (threadIdx.x == 0) { const float g = __ldg(amax_held); s_tc2[0] = tensor_consts(g, T); s_tc2[1] = tensor_consts(g, T_row); }
-    __syncthreads();
-    tc = s_tc2[0];
-    tcr = s_tc2[1];
-}
-
+// Persistent: the grid is sized to the device (resident CTAs x SMs) and every thread walks over blocks with the
+// grid stride, so the set-up above is paid once per CTA and there is no partial last wave.
 template <bool IS_BF16, bool SR, bool STATS, bool TILED>
-__global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(QuantArgs a, int kb_shift) {
-    const TensorConsts tc = cta_tensor_consts(a.amax_held, a.T);
-    const uint32_t kbpr = (uint32_t)(a.cols >> 4);
-    const uint32_t nblocks = (uint32_t)a.rows * kbpr;          // the launcher guarantees < 2^32 blocks
-    const uint32_t idx = blockIdx.x * kRowThreads + threadIdx.x;
-    if (idx == 0 && a.decode_out) *a.decode_out = tc.d;
-    const bool live = idx < nblocks;
-    const uint32_t idc = live ? idx : 0;
-    // blocks per row is a power of two for the usual widths: shift instead of divide
-    const uint32_t row = (kb_shift >= 0) ? (idc >> kb_shift) : (idc / kbpr);
-    const uint32_t kb = idc - row * kbpr;
+__global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(const __grid_constant__ QuantArgs a, int kb_shift) {
+    static_assert(kRowThreads == 256, "one table entry per thread");
+    __shared__ CtaTables tab;
+    cta_setup<false>(tab, a.amax_held, a.T, a.T);
+    const float S = tab.tc[0].S;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tab.tc[0].d;
+    // NaN inputs under stochastic rounding: BF16 words are cleaned once per block when a NaN-propagating maximum
+    // says so (free otherwise); with counters, or FP32 inputs, every product is cleaned instead.
+    constexpr bool kRawSanitize = SR && IS_BF16 && !STATS;
+    constexpr bool kSanitizeZ = SR && !kRawSanitize;
 
-    float f[16];
-    float aB = 0.0f;
-    if (IS_BF16) {
-        const uint16_t* p = reinterpret_cast<const uint16_t*>(a.x) + (int64_t)row * a.ld + kb * 16;
-        const uint4 v0 = ldg_nc_v4(p), v1 = ldg_nc_v4(p + 8);
-        uint32_t m = bf16x2_absmax(0u, v0.x);
-        m = bf16x2_absmax(m, v0.y); m = bf16x2_absmax(m, v0.z); m = bf16x2_absmax(m, v0.w);
-        m = bf16x2_absmax(m, v1.x); m = bf16x2_absmax(m, v1.y); m = bf16x2_absmax(m, v1.z); m = bf16x2_absmax(m, v1.w);
-        aB = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
-        unpack_bf16x8(v0, f);
-        unpack_bf16x8(v1, f + 8);
-    } else {
-        const float* p = reinterpret_cast<const float*>(a.x) + (int64_t)row * a.ld + kb * 16;
+    const uint32_t kbpr = (uint32_t)(a.cols >> 4);
+    const uint32_t nblocks = (uint32_t)a.rows * kbpr;          // the launcher guarantees < 2^32 - 2^16 blocks
+    uint32_t sat = 0, rep = 0, clip = 0, nonf = 0;
+    // all lanes of a warp make the same number of trips (the scale bytes travel through shuffles)
+    for (uint32_t base = blockIdx.x * kRowThreads; base < nblocks; base += gridDim.x * kRowThreads) {
+        const uint32_t idx = base + threadIdx.x;
+        const bool live = idx < nblocks;
+        const uint32_t idc = live ? idx : 0;
+        // blocks per row is a power of two for the usual widths: shift instead of divide
+        const uint32_t row = (kb_shift >= 0) ? (idc >> kb_shift) : (idc / kbpr);
+        const uint32_t kb = idc - row * kbpr;
+
+        float f[16];
+        float aB = 0.0f;
+        if (IS_BF16) {
+            const uint16_t* p = reinterpret_cast<const uint16_t*>(a.x) + (int64_t)row * a.ld + kb * 16;
+            const uint4 v0 = ldg_nc_v4(p), v1 = ldg_nc_v4(p + 8);
+            uint32_t raw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+            uint32_t m = 0;
+            if (kRawSanitize) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint4 v = ldg_nc_v4(p + 4 * q);
-            f[4 * q + 0] = __uint_as_float(v.x); f[4 * q + 1] = __uint_as_float(v.y);
-            f[4 * q + 2] = __uint_as_float(v.z); f[4 * q + 3] = __uint_as_float(v.w);
+                for (int q = 0; q < 8; ++q) m = bf16x2_absmax_nan(m, raw[q]);
+                if (bf16x2_any_nan(m)) {             // rare: the block holds a NaN
+                    m = 0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { m = bf16x2_absmax(m, raw[q]); raw[q] = bf16x2_nan_to_inf(raw[q]); }
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) m = bf16x2_absmax(m, raw[q]);
+            }
+            m = bf16x2_magnitudes(m);
+            aB = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+#pragma unroll
+            for (int q = 0; q < 8; ++q) unpack_bf16x2(raw[q], f[2 * q], f[2 * q + 1]);
+        } else {
+            const float* p = reinterpret_cast<const float*>(a.x) + (int64_t)row * a.ld + kb * 16;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 v = ldg_nc_v4(p + 4 * q);
+                f[4 * q + 0] = __uint_as_float(v.x); f[4 * q + 1] = __uint_as_float(v.y);
+                f[4 * q + 2] = __uint_as_float(v.z); f[4 * q + 3] = __uint_as_float(v.w);
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) aB = fmaxf(aB, fabsf(f[j]));
+        }
+
+        // block of 32: the neighbouring thread holds the other half (blocks per row are even, so pairs never straddle rows)
+        if (a.block32) aB = fmaxf(aB, __shfl_xor_sync(0xFFFFFFFFu, aB, 1));
+        float rB;
+        uint32_t flags;
+        const uint32_t code = block_scale(aB, S, tab.lut[0], rB, flags);
+        if (a.block32 && (threadIdx.x & 1)) flags = 0;             // one count per block
+
+        uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};
+        if (SR) {
+            // element index of the block = 16 * idx (rows are whole numbers of blocks): groups 2 idx and 2 idx + 1
+            const uint64_t g0 = (uint64_t)idc * 2;
+            sr_bits8(a.keys, g0, a.small_counter != 0, w0);
+            sr_bits8(a.keys, g0 + 1, a.small_counter != 0, w1);
+        }
+        uint32_t bclip = 0;
+        uint2 out;
+        out.x = encode8<SR, kSanitizeZ>(f, rB, w0, bclip);
+        out.y = encode8<SR, kSanitizeZ>(f + 8, rB, w1, bclip);
+
+        if (live) *reinterpret_cast<uint2*>(a.payload + (uint64_t)idx * 8) = out;
+
+        if (TILED) {
+            if (live) a.scales[tiled_scale_offset((int64_t)row, kb, kbpr)] = (uint8_t)code;
+        } else {
+            // row-major scales are indexed by the flat block index: four lanes share one 32-bit store
+            uint32_t sc = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
+            sc |= __shfl_down_sync(0xFFFFFFFFu, sc, 2) << 16;
+            if (live && (threadIdx.x & 3) == 0) *reinterpret_cast<uint32_t*>(a.scales + idx) = sc;
+        }
+
+        if (STATS) {
+            uint32_t bnonf = 0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) bnonf += nonfinite(f[j]) ? 1u : 0u;
+            const uint32_t lv = live ? 1u : 0u;
+            sat += lv * (flags & 1u); rep += lv * ((flags >> 1) & 1u); clip += lv * bclip; nonf += lv * bnonf;
+        }
+    }
+    if (STATS) warp_add_stats(a.stats, sat, rep, clip, nonf);
+}
+
+// The common case -- rows stored back to back (ld == cols), row-major scales, 32-byte aligned BF16 source: the tensor is
+// one flat run of blocks.  A thread takes two blocks per trip, 256 blocks apart, each with ONE 256-bit load (a warp
+// instruction reads 1 KB of contiguous memory), needs no row/column arithmetic, and the Philox groups of block i are
+// 2i and 2i + 1.
+__device__ __forceinline__ void ldg_nc_v8(const void* p, uint32_t r[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]) : "l"(p));
+}
+
+constexpr int kFlatBlocksPerTrip = 2;
+
+template <bool SR, bool STATS>
+__global__ void __launch_bounds__(kRowThreads) quantize_row_flat_kernel(const __grid_constant__ QuantArgs a, uint32_t nblocks) {
+    static_assert(kRowThreads == 256, "one table entry per thread");
+    __shared__ CtaTables tab;
+    cta_setup<false>(tab, a.amax_held, a.T, a.T);
+    const float S = tab.tc[0].S;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tab.tc[0].d;
+    constexpr bool kRawSanitize = SR && !STATS;
+    constexpr bool kSanitizeZ = SR && !kRawSanitize;
+    const bool small = a.small_counter != 0;
+    constexpr uint32_t kTrip = kRowThreads * kFlatBlocksPerTrip;
+
+    uint32_t sat = 0, rep = 0, clip = 0, nonf = 0;
+    for (uint32_t base = blockIdx.x * kTrip; base < nblocks; base += gridDim.x * kTrip) {
+        uint32_t raw[kFlatBlocksPerTrip][8];
+        uint32_t idx[kFlatBlocksPerTrip];
+        bool live[kFlatBlocksPerTrip];
+#pragma unroll
+        for (int b = 0; b < kFlatBlocksPerTrip; ++b) {
+            idx[b] = base + b * kRowThreads + threadIdx.x;
+            live[b] = idx[b] < nblocks;
+            ldg_nc_v8(reinterpret_cast<const uint8_t*>(a.x) + (uint64_t)(live[b] ? idx[b] : 0) * 32, raw[b]);
         }
 #pragma unroll
-        for (int j = 0; j < 16; ++j) aB = fmaxf(aB, fabsf(f[j]));
-    }
-
-    // block of 32: the neighbouring thread holds the other half (blocks per row are even, so pairs never straddle rows)
-    if (a.block32) aB = fmaxf(aB, __shfl_xor_sync(0xFFFFFFFFu, aB, 1));
-    float rB;
-    uint32_t flags;
-    const uint32_t code = block_scale(aB, tc, rB, flags);
-    if (a.block32 && (threadIdx.x & 1)) flags = 0;             // one count per block
-
-    uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};
-    if (SR) {
-        const uint64_t g0 = ((uint64_t)row * (uint64_t)a.cols + (uint64_t)kb * 16) >> 3;
-        sr_bits8(a.seed, g0, w0);
-        sr_bits8(a.seed, g0 + 1, w1);
-    }
-    uint32_t clip = 0;
-    uint2 out;
-    out.x = encode8<SR>(f, rB, w0, clip);
-    out.y = encode8<SR>(f + 8, rB, w1, clip);
-
-    if (live) *reinterpret_cast<uint2*>(a.payload + (uint64_t)idx * 8) = out;
-
-    if (TILED) {
-        if (live) a.scales[tiled_scale_offset((int64_t)row, kb, kbpr)] = (uint8_t)code;
-    } else {
-        // row-major scales are indexed by the flat block index: four lanes share one 32-bit store
-        uint32_t s = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
-        s |= __shfl_down_sync(0xFFFFFFFFu, s, 2) << 16;
-        if (live && (threadIdx.x & 3) == 0) *reinterpret_cast<uint32_t*>(a.scales + idx) = s;
-    }
-
-    if (STATS) {
-        uint32_t nonf = 0;
+        for (int b = 0; b < kFlatBlocksPerTrip; ++b) {
+            uint32_t m = 0;
+            if (kRawSanitize) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) nonf += nonfinite(f[j]) ? 1u : 0u;
-        const uint32_t lv = live ? 1u : 0u;
-        warp_add_stats(a.stats, lv * (flags & 1u), lv * ((flags >> 1) & 1u), lv * clip, lv * nonf);
+                for (int q = 0; q < 8; ++q) m = bf16x2_absmax_nan(m, raw[b][q]);
+                if (bf16x2_any_nan(m)) {             // rare: the block holds a NaN
+                    m = 0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { m = bf16x2_absmax(m, raw[b][q]); raw[b][q] = bf16x2_nan_to_inf(raw[b][q]); }
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) m = bf16x2_absmax(m, raw[b][q]);
+            }
+            m = bf16x2_magnitudes(m);
+            float aB = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+            // block of 32: the neighbouring thread holds the other half (an even number of blocks per row)
+            if (a.block32) aB = fmaxf(aB, __shfl_xor_sync(0xFFFFFFFFu, aB, 1));
+            float rB;
+            uint32_t flags;
+            const uint32_t code = block_scale(aB, S, tab.lut[0], rB, flags);
+            if (a.block32 && (threadIdx.x & 1)) flags = 0;
+            float f[16];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) unpack_bf16x2(raw[b][q], f[2 * q], f[2 * q + 1]);
+            uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};
+            if (SR) {
+                const uint64_t g0 = (uint64_t)(live[b] ? idx[b] : 0) * 2;
+                sr_bits8(a.keys, g0, small, w0);
+                sr_bits8(a.keys, g0 + 1, small, w1);
+            }
+            uint32_t bclip = 0;
+            uint2 out;
+            out.x = encode8<SR, kSanitizeZ>(f, rB, w0, bclip);
+            out.y = encode8<SR, kSanitizeZ>(f + 8, rB, w1, bclip);
+            if (live[b]) *reinterpret_cast<uint2*>(a.payload + (uint64_t)idx[b] * 8) = out;
+            // four lanes share one 32-bit store of scale bytes (nblocks is a multiple of 4 here)
+            uint32_t sc = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
+            sc |= __shfl_down_sync(0xFFFFFFFFu, sc, 2) << 16;
+            if (live[b] && (threadIdx.x & 3) == 0) *reinterpret_cast<uint32_t*>(a.scales + idx[b]) = sc;
+            if (STATS) {
+                uint32_t bnonf = 0;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) bnonf += nonfinite(f[j]) ? 1u : 0u;
+                const uint32_t lv = live[b] ? 1u : 0u;
+                sat += lv * (flags & 1u); rep += lv * ((flags >> 1) & 1u); clip += lv * bclip; nonf += lv * bnonf;
+            }
+        }
     }
+    if (STATS) warp_add_stats(a.stats, sat, rep, clip, nonf);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -181,21 +317,18 @@ __device__ __forceinline__ void load_row8(const void* x, int64_t off, float f[8]
 // MODE 3: dual layout: MODE 0 plus the 1D_ROW quantization of the same register tile (a row block of 16 is this
 //         lane's 8 columns and lane ^ 1's): the tensor is read once for both operands of a backward pass.
 template <bool IS_BF16, bool SR, bool STATS, int MODE, bool TILED, bool WANT_T>
-__global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a) {
+__global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile_kernel(const __grid_constant__ QuantArgs a) {
+    static_assert(kTileThreads == 256, "one table entry per thread");
     constexpr bool kDual = MODE == 3;
     constexpr bool kStaged = (MODE == 0) || kDual;       // column output through shared memory
     constexpr bool kColumns = kStaged || (MODE == 2);
     constexpr bool kTranspose = kStaged || WANT_T;
+    // NaN inputs under stochastic rounding (see quantize_row_kernel)
+    constexpr bool kRawSanitize = SR && IS_BF16 && !STATS;
+    constexpr bool kSanitizeZ = SR && !kRawSanitize;
     __shared__ __align__(16) uint8_t s_t[kTranspose ? kTileCols * (kTileRows / 2) : 16];
     __shared__ __align__(16) uint8_t s_sc[kStaged ? (kTileRows / 16) * kTileCols : 16];   // [row block][column]
-
-    TensorConsts tc, tcr;
-    if (kDual) cta_tensor_consts2(a.amax_held, a.T, a.row_T, tc, tcr);
-    else { tc = cta_tensor_consts(a.amax_held, a.T); tcr = tc; }
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
-        if (a.decode_out) *a.decode_out = tc.d;
-        if (kDual && a.row_decode) *a.row_decode = tcr.d;
-    }
+    __shared__ CtaTables tab;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int cg, rb;   // column group (8 columns) and row block (16 rows) inside the CTA tile
@@ -206,36 +339,70 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
     const bool live = (c0 < a.cols) && (r0 < a.rows);
     const int64_t base = live ? (r0 * a.ld + c0) : 0;
 
-    // ---- pass 1: load the 16 x 8 register tile, column maxima ----
+    // ---- pass 1: load the 16 x 8 register tile (the loads are in flight while the CTA's tables are built) ----
     uint4 raw[IS_BF16 ? 16 : 1];
+    if (IS_BF16) {
+#pragma unroll
+        for (int r = 0; r < 16; ++r) raw[r] = ldg_nc_v4(reinterpret_cast<const uint16_t*>(a.x) + base + r * a.ld);
+    }
+
+    cta_setup<kDual>(tab, a.amax_held, a.T, a.row_T);
+    const float S = tab.tc[0].S, S_row = tab.tc[kDual ? 1 : 0].S;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        if (a.decode_out) *a.decode_out = tab.tc[0].d;
+        if (kDual && a.row_decode) *a.row_decode = tab.tc[1].d;
+    }
+
+    // ---- column maxima ----
     float colmax[8];
     uint32_t cm[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int j = 0; j < 8; ++j) colmax[j] = 0.0f;
     uint32_t nonf = 0;
+    bool has_nan = false;
+    if (IS_BF16) {
+        if (kRawSanitize) {
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        float f[8];
-        uint4 v;
-        load_row8<IS_BF16>(a.x, base + r * a.ld, f, v);
-        if (IS_BF16) {
-            raw[r] = v;
-            cm[0] = bf16x2_absmax(cm[0], v.x); cm[1] = bf16x2_absmax(cm[1], v.y);
-            cm[2] = bf16x2_absmax(cm[2], v.z); cm[3] = bf16x2_absmax(cm[3], v.w);
-        } else {
+            for (int r = 0; r < 16; ++r) {
+                cm[0] = bf16x2_absmax_nan(cm[0], raw[r].x); cm[1] = bf16x2_absmax_nan(cm[1], raw[r].y);
+                cm[2] = bf16x2_absmax_nan(cm[2], raw[r].z); cm[3] = bf16x2_absmax_nan(cm[3], raw[r].w);
+            }
+            has_nan = bf16x2_any_nan(cm[0]) || bf16x2_any_nan(cm[1]) || bf16x2_any_nan(cm[2]) || bf16x2_any_nan(cm[3]);
+        }
+        if (!kRawSanitize || has_nan) {              // the maxima that ignore NaNs (second case: rare)
+            cm[0] = cm[1] = cm[2] = cm[3] = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) colmax[j] = fmaxf(colmax[j], fabsf(f[j]));
+            for (int r = 0; r < 16; ++r) {
+                cm[0] = bf16x2_absmax(cm[0], raw[r].x); cm[1] = bf16x2_absmax(cm[1], raw[r].y);
+                cm[2] = bf16x2_absmax(cm[2], raw[r].z); cm[3] = bf16x2_absmax(cm[3], raw[r].w);
+            }
         }
         if (STATS) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) nonf += nonfinite(f[j]) ? 1u : 0u;
+            for (int r = 0; r < 16; ++r) {
+                float f[8];
+                unpack_bf16x8(raw[r], f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) nonf += nonfinite(f[j]) ? 1u : 0u;
+            }
         }
-    }
-    if (IS_BF16) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            colmax[2 * q] = __uint_as_float(cm[q] << 16);
-            colmax[2 * q + 1] = __uint_as_float(cm[q] & 0xFFFF0000u);
+            colmax[2 * q] = __uint_as_float((cm[q] << 16) & 0x7FFF0000u);
+            colmax[2 * q + 1] = __uint_as_float(cm[q] & 0x7FFF0000u);
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+            float f[8];
+            uint4 v;
+            load_row8<false>(a.x, base + r * a.ld, f, v);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) colmax[j] = fmaxf(colmax[j], fabsf(f[j]));
+            if (STATS) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) nonf += nonfinite(f[j]) ? 1u : 0u;
+            }
         }
     }
 
@@ -255,7 +422,7 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t fl;
-            codes[j] = block_scale(colmax[j], tc, rcol[j], fl);
+            codes[j] = block_scale(colmax[j], S, tab.lut[0], rcol[j], fl);
             if (counts) { sat += fl & 1u; rep += (fl >> 1) & 1u; }
         }
     } else {
@@ -269,84 +436,92 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
         }
         uint32_t fl;
         float r;
-        const uint32_t code = block_scale(m, tc, r, fl);
+        const uint32_t code = block_scale(m, S, tab.lut[0], r, fl);
         if ((lane & (a.block32 ? 19 : 1)) == 0) { sat += fl & 1u; rep += (fl >> 1) & 1u; }
 #pragma unroll
         for (int j = 0; j < 8; ++j) { rcol[j] = r; codes[j] = code; }
     }
 
-    // ---- pass 2: encode.  nib[r] = the 8 codes of row r (column j in bits 4j+3:4j) ----
-    uint32_t nib[16];
+    // ---- pass 2: encode, two rows at a time.  Outputs stored along the rows of the source (2D payload, the row operand
+    // of the dual call) pair horizontal neighbours in one conversion; outputs stored along its columns pair the two
+    // rows, which is the byte the transposed payload holds -- so nothing has to be transposed nibble by nibble.
+    // tcol[j][h]: the 8 codes of column j for rows 8h .. 8h+7 (row r in bits 4(r%8)+3 : 4(r%8)).
+    uint32_t tcol[kColumns || WANT_T ? 8 : 1][2];
+    if (kColumns || WANT_T) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) tcol[j][0] = tcol[j][1] = 0;
+    }
     uint32_t clip = 0;
     uint32_t sat_r = 0, rep_r = 0, clip_r = 0;
+    // group of Philox draws of the 8 elements of row r0 + r: ((r0 + r) * cols + c0) / 8
+    const uint64_t group0 = ((uint64_t)r0 * (uint64_t)a.cols + (uint64_t)c0) >> 3;
+    const uint64_t group_step = (uint64_t)a.cols >> 3;
+    const bool small = a.small_counter != 0;
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        float f[8];
-        if (IS_BF16) { unpack_bf16x8(raw[r], f); }
-        else { uint4 v; load_row8<false>(a.x, base + r * a.ld, f, v); }
-        uint32_t w[4] = {0, 0, 0, 0};
-        if (SR) sr_bits8(a.seed, ((uint64_t)(r0 + r) * (uint64_t)a.cols + (uint64_t)c0) >> 3, w);
-        if (kDual) {
-            // ---- the row operand: block = 16 consecutive columns of row r0 + r, held by lanes 2i and 2i + 1 ----
-            float m = 0.0f;
+    for (int rp = 0; rp < 8; ++rp) {
+        float v[2][8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int r = 2 * rp + h;
+            float f[8];
             if (IS_BF16) {
-                uint32_t pm = bf16x2_absmax(bf16x2_absmax(0u, raw[r].x), raw[r].y);
-                pm = bf16x2_absmax(bf16x2_absmax(pm, raw[r].z), raw[r].w);
-                m = fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xFFFF0000u));
-            } else {
+                uint4 x = raw[r];
+                if (kRawSanitize && has_nan) {
+                    x.x = bf16x2_nan_to_inf(x.x); x.y = bf16x2_nan_to_inf(x.y);
+                    x.z = bf16x2_nan_to_inf(x.z); x.w = bf16x2_nan_to_inf(x.w);
+                }
+                unpack_bf16x8(x, f);
+            } else { uint4 x; load_row8<false>(a.x, base + r * a.ld, f, x); }
+            uint32_t w[4] = {0, 0, 0, 0};
+            if (SR) sr_bits8(a.keys, group0 + (uint64_t)r * group_step, small, w);
+            if (kDual) {
+                // ---- the row operand: block = 16 consecutive columns of row r0 + r, held by lanes 2i and 2i + 1 ----
+                float m = 0.0f;
+                if (IS_BF16) {
+                    uint32_t pm = bf16x2_absmax(bf16x2_absmax(0u, raw[r].x), raw[r].y);
+                    pm = bf16x2_magnitudes(bf16x2_absmax(bf16x2_absmax(pm, raw[r].z), raw[r].w));
+                    m = fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xFFFF0000u));
+                } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(f[j]));
-            }
-            m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-            if (a.block32) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-            float rrow;
-            uint32_t fl;
-            const uint32_t code_r = block_scale(m, tcr, rrow, fl);
-            if ((lane & (a.block32 ? 3 : 1)) == 0) { sat_r += fl & 1u; rep_r += (fl >> 1) & 1u; }
-            uint32_t wr[4] = {0, 0, 0, 0};
-            if (SR) sr_bits8(a.row_seed, ((uint64_t)(r0 + r) * (uint64_t)a.cols + (uint64_t)c0) >> 3, wr);
-            const uint32_t orow = encode8<SR>(f, rrow, wr, clip_r);
-            const int64_t kbpr = a.cols >> 4;
-            // four lanes (even column groups) -> four consecutive scale bytes
-            uint32_t s4 = code_r | (__shfl_down_sync(0xFFFFFFFFu, code_r, 2) << 8);
-            s4 |= __shfl_down_sync(0xFFFFFFFFu, s4, 4) << 16;
-            if (live) {
-                *reinterpret_cast<uint32_t*>(a.row_payload + (r0 + r) * (a.cols >> 1) + (c0 >> 1)) = orow;
-                const int64_t kb = c0 >> 4;
-                if (TILED) {
-                    if ((cg & 1) == 0) a.row_scales[tiled_scale_offset(r0 + r, kb, kbpr)] = (uint8_t)code_r;
-                } else if ((kbpr & 3) == 0) {
-                    if ((cg & 7) == 0) *reinterpret_cast<uint32_t*>(a.row_scales + (r0 + r) * kbpr + kb) = s4;   // cols % 64 == 0
-                } else if ((cg & 1) == 0) {
-                    a.row_scales[(r0 + r) * kbpr + kb] = (uint8_t)code_r;
+                    for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(f[j]));
+                }
+                m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+                if (a.block32) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+                float rrow;
+                uint32_t fl;
+                const uint32_t code_r = block_scale(m, S_row, tab.lut[kDual ? 1 : 0], rrow, fl);
+                if ((lane & (a.block32 ? 3 : 1)) == 0) { sat_r += fl & 1u; rep_r += (fl >> 1) & 1u; }
+                uint32_t wr[4] = {0, 0, 0, 0};
+                if (SR) sr_bits8(a.row_keys, group0 + (uint64_t)r * group_step, small, wr);
+                const uint32_t orow = encode8<SR, kSanitizeZ>(f, rrow, wr, clip_r);
+                const int64_t kbpr = a.cols >> 4;
+                // four lanes (even column groups) -> four consecutive scale bytes
+                uint32_t s4 = code_r | (__shfl_down_sync(0xFFFFFFFFu, code_r, 2) << 8);
+                s4 |= __shfl_down_sync(0xFFFFFFFFu, s4, 4) << 16;
+                if (live) {
+                    *reinterpret_cast<uint32_t*>(a.row_payload + (r0 + r) * (a.cols >> 1) + (c0 >> 1)) = orow;
+                    const int64_t kb = c0 >> 4;
+                    if (TILED) {
+                        if ((cg & 1) == 0) a.row_scales[tiled_scale_offset(r0 + r, kb, kbpr)] = (uint8_t)code_r;
+                    } else if ((kbpr & 3) == 0) {
+                        if ((cg & 7) == 0) *reinterpret_cast<uint32_t*>(a.row_scales + (r0 + r) * kbpr + kb) = s4;   // cols % 64 == 0
+                    } else if ((cg & 1) == 0) {
+                        a.row_scales[(r0 + r) * kbpr + kb] = (uint8_t)code_r;
+                    }
                 }
             }
+            round_values8<SR, kSanitizeZ>(f, rcol, w, v[h], clip);
+            if (MODE == 1) {
+                // 2D: the row-major payload of this row (64 contiguous bytes per row and warp)
+                const uint32_t o = pack8(v[h]);
+                if (live) *reinterpret_cast<uint32_t*>(a.payload + (r0 + r) * (a.cols >> 1) + (c0 >> 1)) = o;
+            }
         }
-        float z[8];
+        if (kColumns || WANT_T) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) z[j] = __fmul_rn(f[j], rcol[j]);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) clip += (fabsf(z[j]) > 6.0f) ? 1u : 0u;
-        uint32_t o = 0;
-        if (SR) {
-            uint32_t mags = 0, signs = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) sr_accumulate(z[j], w[j >> 1], j, mags, signs);
-            o = sr_finish(mags, signs);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) o |= e2m1x2_rne(z[2 * j], z[2 * j + 1]) << (8 * j);
+            for (int j = 0; j < 8; ++j) tcol[j][rp >> 2] |= e2m1x2_rne(v[0][j], v[1][j]) << (8 * (rp & 3));
         }
-        nib[r] = o;
     }
-
-    // transposed pieces: for column j the 16 codes down the rows, row r in bits 4r+3:4r
-    auto column_word = [&](int j, int half) -> uint32_t {
-        uint32_t wv = 0;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) wv |= ((nib[8 * half + r] >> (4 * j)) & 0xFu) << (4 * r);
-        return wv;
-    };
 
     if (MODE == 2) {
         if (live) {
@@ -355,8 +530,8 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 uint2 o;
-                o.x = column_word(j, 0);
-                o.y = column_word(j, 1);
+                o.x = tcol[j][0];
+                o.y = tcol[j][1];
                 *reinterpret_cast<uint2*>(a.payload + (c0 + j) * (a.rows >> 1) + (r0 >> 1)) = o;
                 const int64_t so = TILED ? tiled_scale_offset(c0 + j, rblk, kblocks) : (c0 + j) * kblocks + rblk;
                 a.scales[so] = (uint8_t)codes[j];
@@ -365,9 +540,6 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
     }
     if (MODE == 1) {
         if (live) {
-#pragma unroll
-            for (int r = 0; r < 16; ++r)
-                *reinterpret_cast<uint32_t*>(a.payload + (r0 + r) * (a.cols >> 1) + (c0 >> 1)) = nib[r];
             if ((lane & 1) == 0) {
                 a.scales[(r0 >> 4) * (a.cols >> 4) + (c0 >> 4)] = (uint8_t)codes[0];
                 if (WANT_T) a.scales_t[(c0 >> 4) * (a.rows >> 4) + (r0 >> 4)] = (uint8_t)codes[0];
@@ -380,8 +552,8 @@ __global__ void __launch_bounds__(kTileThreads) quantize_tile_kernel(QuantArgs a
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint2 o;
-            o.x = column_word(j, 0);
-            o.y = column_word(j, 1);
+            o.x = tcol[j][0];
+            o.y = tcol[j][1];
             const int col = cg * 8 + j;
             const int piece = (rb + cg) & 15;
             *reinterpret_cast<uint2*>(s_t + col * (kTileRows / 2) + piece * 8) = o;
@@ -477,7 +649,8 @@ __global__ void __launch_bounds__(kAmaxThreads) amax_kernel(const void* x, int64
         }
     }
     if (IS_BF16) {
-        const uint32_t p = bf16x2_max(bf16x2_max(pm0, pm1), bf16x2_max(pm2, pm3));
+        const uint32_t p = bf16x2_max(bf16x2_max(bf16x2_magnitudes(pm0), bf16x2_magnitudes(pm1)),
+                                      bf16x2_max(bf16x2_magnitudes(pm2), bf16x2_magnitudes(pm3)));
         m = fmaxf(__uint_as_float(p << 16), __uint_as_float(p & 0xFFFF0000u));
     }
 #pragma unroll
@@ -505,16 +678,50 @@ __global__ void unswizzle_scales_kernel(const uint8_t* in, uint8_t* out, int64_t
 // ---------------------------------------------------------------------------------------
 // Host-side launchers (called from the C ABI)
 // ---------------------------------------------------------------------------------------
-template <bool IS_BF16, bool SR, bool STATS>
-static cudaError_t launch_row(const QuantArgs& a, bool tiled, cudaStream_t st) {
+// CTAs of `kernel` that fit on one SM, asked once per kernel instance (thread-safe static initialisation).
+template <typename K>
+static int resident_ctas_per_sm(K kernel, int threads) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        n = 1;
+    }
+    return n;
+}
+
+template <bool IS_BF16, bool SR, bool STATS, bool TILED>
+static cudaError_t launch_row_t(const QuantArgs& a, int num_sms, cudaStream_t st) {
+    static const int per_sm = resident_ctas_per_sm(quantize_row_kernel<IS_BF16, SR, STATS, TILED>, kRowThreads);
     const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
-    const unsigned grid = (unsigned)((nblocks + kRowThreads - 1) / kRowThreads);
+    uint64_t grid = (nblocks + kRowThreads - 1) / kRowThreads;
+    const uint64_t resident = (uint64_t)per_sm * (uint64_t)num_sms;
+    if (grid > resident) grid = resident;          // persistent: one wave, every thread strides over the blocks
     const uint64_t kbpr = (uint64_t)(a.cols >> 4);
     int kb_shift = -1;
     if ((kbpr & (kbpr - 1)) == 0) { kb_shift = 0; while ((1ull << kb_shift) < kbpr) ++kb_shift; }
-    if (tiled) quantize_row_kernel<IS_BF16, SR, STATS, true><<<grid, kRowThreads, 0, st>>>(a, kb_shift);
-    else       quantize_row_kernel<IS_BF16, SR, STATS, false><<<grid, kRowThreads, 0, st>>>(a, kb_shift);
+    quantize_row_kernel<IS_BF16, SR, STATS, TILED><<<(unsigned)grid, kRowThreads, 0, st>>>(a, kb_shift);
     return cudaGetLastError();
+}
+
+template <bool SR, bool STATS>
+static cudaError_t launch_row_flat(const QuantArgs& a, int num_sms, cudaStream_t st) {
+    static const int per_sm = resident_ctas_per_sm(quantize_row_flat_kernel<SR, STATS>, kRowThreads);
+    const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
+    const uint64_t per_cta = (uint64_t)kRowThreads * kFlatBlocksPerTrip;
+    uint64_t grid = (nblocks + per_cta - 1) / per_cta;
+    const uint64_t resident = (uint64_t)per_sm * (uint64_t)num_sms;
+    if (grid > resident) grid = resident;
+    quantize_row_flat_kernel<SR, STATS><<<(unsigned)grid, kRowThreads, 0, st>>>(a, (uint32_t)nblocks);
+    return cudaGetLastError();
+}
+
+template <bool IS_BF16, bool SR, bool STATS>
+static cudaError_t launch_row(const QuantArgs& a, bool tiled, int num_sms, cudaStream_t st) {
+    const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
+    // BF16 rows back to back on a 32-byte boundary, row-major scales, a multiple of four blocks
+    if (IS_BF16 && !tiled && a.ld == a.cols && (nblocks & 3) == 0 && (reinterpret_cast<uintptr_t>(a.x) & 31u) == 0)
+        return launch_row_flat<SR, STATS>(a, num_sms, st);
+    return tiled ? launch_row_t<IS_BF16, SR, STATS, true>(a, num_sms, st) : launch_row_t<IS_BF16, SR, STATS, false>(a, num_sms, st);
 }
 
 template <bool IS_BF16, bool SR, bool STATS>
@@ -532,14 +739,17 @@ static cudaError_t launch_tile(const QuantArgs& a, int layout, bool tiled, cudaS
 }
 
 template <bool IS_BF16, bool SR, bool STATS>
-static cudaError_t launch_any(const QuantArgs& a, int layout, bool tiled, cudaStream_t st) {
-    if (layout == UE5M3_LAYOUT_1D_ROW) return launch_row<IS_BF16, SR, STATS>(a, tiled, st);
+static cudaError_t launch_any(const QuantArgs& a, int layout, bool tiled, int num_sms, cudaStream_t st) {
+    if (layout == UE5M3_LAYOUT_1D_ROW) return launch_row<IS_BF16, SR, STATS>(a, tiled, num_sms, st);
     return launch_tile<IS_BF16, SR, STATS>(a, layout, tiled, st);
 }
 
-cudaError_t launch_quantize(const QuantArgs& a, int dtype, int layout, int rounding, bool tiled, cudaStream_t st) {
+cudaError_t launch_quantize(const QuantArgs& args, int dtype, int layout, int rounding, bool tiled, int num_sms, cudaStream_t st) {
+    QuantArgs a = args;
     const bool bf = dtype == UE5M3_BF16, sr = rounding == UE5M3_ROUND_SR, stt = a.stats != nullptr;
-#define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_any<B, S, T>(a, layout, tiled, st);
+    if (sr) a.keys = philox_round_keys(a.seed);
+    a.small_counter = (uint64_t)a.rows * (uint64_t)a.cols < (1ull << 35) ? 1 : 0;
+#define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_any<B, S, T>(a, layout, tiled, num_sms, st);
     UE5M3_DISPATCH(true, false, false) UE5M3_DISPATCH(true, true, false)
     UE5M3_DISPATCH(true, false, true)  UE5M3_DISPATCH(true, true, true)
     UE5M3_DISPATCH(false, false, false) UE5M3_DISPATCH(false, true, false)
@@ -556,8 +766,11 @@ static cudaError_t launch_dual(const QuantArgs& a, bool tiled, cudaStream_t st) 
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bool tiled, cudaStream_t st) {
+cudaError_t launch_quantize_dual(const QuantArgs& args, int dtype, int rounding, bool tiled, cudaStream_t st) {
+    QuantArgs a = args;
     const bool bf = dtype == UE5M3_BF16, sr = rounding == UE5M3_ROUND_SR, stt = a.stats != nullptr;
+    if (sr) { a.keys = philox_round_keys(a.seed); a.row_keys = philox_round_keys(a.row_seed); }
+    a.small_counter = (uint64_t)a.rows * (uint64_t)a.cols < (1ull << 35) ? 1 : 0;
 #define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_dual<B, S, T>(a, tiled, st);
     UE5M3_DISPATCH(true, false, false) UE5M3_DISPATCH(true, true, false)
     UE5M3_DISPATCH(true, false, true)  UE5M3_DISPATCH(true, true, true)
