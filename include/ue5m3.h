@@ -95,7 +95,7 @@ UE5M3_API int ue5m3_sample_amax(const void* x, int dtype, int64_t rows, int64_t 
  *
  * Stochastic rounding rounds |z| up to the next E2M1 magnitude with probability equal to its
  * relative position between the two neighbours, resolved to 16 bits: the 16 random bits of source
- * element i = row * cols + col are taken from Philox4x32-10 with key = (seed low, seed high) and
+ * element i = row * cols + col are taken from Philox4x32 with 7 rounds, key = (seed low, seed high) and
  * counter = (low32(i>>3), high32(i>>3), 0, 0): element lane j = i & 7 uses half (j & 1) of output
  * word j >> 1.  Block scales are never rounded stochastically.
  *

@@ -54,6 +54,8 @@ def lib() -> C.CDLL:
         L.oracle_e2m1_encode_sr.argtypes = [f32, u32]
         L.oracle_philox4x32_10.restype = None
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        L.oracle_philox4x32.restype = None
+        L.oracle_philox4x32.argtypes = [vp, vp, C.c_int, vp]
         L.oracle_sr_bits.restype = u32
         L.oracle_sr_bits.argtypes = [u64, u64]
         L.oracle_amax.restype = f32
@@ -135,6 +137,18 @@ def philox4x32_10(ctr, key):
     out = np.zeros(4, dtype=np.uint32)
     lib().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
     return out
+
+
+def philox4x32(ctr, key, rounds: int):
+    """Philox4x32 with the given number of rounds (10: the generator's default; 7: what the draws use)."""
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().oracle_philox4x32(_ptr(c), _ptr(k), int(rounds), _ptr(out))
+    return out
+
+
+SR_PHILOX_ROUNDS = 7
 
 
 def sr_bits(seed: int, index: int) -> int:

@@ -26,8 +26,8 @@
  *     else 1.0.
  *   - payload nibble order: element 2p in bits 3:0 of byte p, element 2p+1
  *     in bits 7:4.  The sign of zero is kept.  NaN payload encodes as +6.
- *   - stochastic rounding bits: Philox4x32-10, one call per 8 consecutive
- *     source elements, 16 bits per element (see oracle_sr_bits).
+ *   - stochastic rounding bits: Philox4x32 with 7 rounds, one call per 8
+ *     consecutive source elements, 16 bits per element (see oracle_sr_bits).
  *   - GEMM output model (Section 6.2): groups are the 64 consecutive K indices
  *     64g..64g+63 in ascending order; the partials are of the decoded operands
  *     s_hat * q; the scale product is alpha = RNE32(dA * dB) and the output is
@@ -158,12 +158,15 @@ ORACLE_API int oracle_e2m1_encode_sr(float z, uint32_t r16)
     return sign | mag;
 }
 
-/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw 2011). */
-ORACLE_API void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+/* Philox4x32-R (Salmon, Moraes, Dror, Shaw 2011): R rounds of the bijection, the key bumped by the Weyl
+ * constants after every round.  R = 10 is the generator's default and the one the published known-answer
+ * vectors and cuRAND cover; R = 7 is the smallest round count its authors report as passing the full
+ * statistical batteries, and the one the stochastic-rounding draws use (see oracle_sr_bits). */
+ORACLE_API void oracle_philox4x32(const uint32_t ctr[4], const uint32_t key[2], int rounds, uint32_t out[4])
 {
     uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
     uint32_t k0 = key[0], k1 = key[1];
-    for (int round = 0; round < 10; ++round) {
+    for (int round = 0; round < rounds; ++round) {
         uint64_t p0 = (uint64_t)0xD2511F53u * c0;
         uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
         uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
@@ -177,17 +180,27 @@ ORACLE_API void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+ORACLE_API void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    oracle_philox4x32(ctr, key, 10, out);
+}
+
+#define SR_PHILOX_ROUNDS 7
+
 /* The 16 random bits of source element i (logical row-major index
  * row * cols + col of the SOURCE tensor, independent of ld and of layout):
- * key = (seed low, seed high), counter = (low32(i>>3), high32(i>>3), 0, 0),
- * lane j = i & 7 takes half (j & 1) of word j >> 1. */
+ * Philox4x32-7 with key = (seed low, seed high), counter = (low32(i>>3),
+ * high32(i>>3), 0, 0); lane j = i & 7 takes half (j & 1) of word j >> 1.
+ * The paper fixes neither generator nor bits per draw (Section 5.3 only asks
+ * for an unbiased Q_SR); seven rounds instead of the default ten is a reading
+ * taken for the cost of the draw on the GPU, within the generator family. */
 ORACLE_API uint32_t oracle_sr_bits(uint64_t seed, uint64_t i)
 {
     uint64_t blk = i >> 3;
     uint32_t ctr[4] = { (uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u };
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
     uint32_t w[4];
-    oracle_philox4x32_10(ctr, key, w);
+    oracle_philox4x32(ctr, key, SR_PHILOX_ROUNDS, w);
     int j = (int)(i & 7);
     return (w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
 }

@@ -101,13 +101,13 @@ __device__ __forceinline__ void sr_values8(const float z[8], const uint32_t w[4]
     }
 }
 
-// Philox4x32-10 (Salmon et al. 2011).  The ten round keys depend only on the seed: the host computes them once
-// per call and they reach the kernel as launch parameters, so a round is two 32 x 32 -> 64 bit products and two
-// three-input exclusive-ors.
+// Philox4x32 (Salmon et al. 2011) with kPhiloxRounds = 7 rounds.  The round keys depend only on the seed: the host
+// computes them once per call and they reach the kernel as launch parameters, so a round is two 32 x 32 -> 64 bit
+// products and two three-input exclusive-ors.
 __host__ __device__ inline PhiloxKeys philox_round_keys(uint64_t seed) {
     PhiloxKeys K;
     uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
-    for (int r = 0; r < 10; ++r) {
+    for (int r = 0; r < kPhiloxRounds; ++r) {
         K.k[2 * r] = k0;
         K.k[2 * r + 1] = k1;
         k0 += 0x9E3779B9u;
@@ -119,10 +119,10 @@ __host__ __device__ inline PhiloxKeys philox_round_keys(uint64_t seed) {
     return K;
 }
 
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              const PhiloxKeys& K, uint32_t out[4]) {
+__device__ __forceinline__ void philox4x32(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                           const PhiloxKeys& K, uint32_t out[4]) {
 #pragma unroll
-    for (int r = 0; r < 10; ++r) {
+    for (int r = 0; r < kPhiloxRounds; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
         const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
         c0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k[2 * r];
@@ -134,8 +134,8 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 }
 
 // The same generator for a counter (c0, 0, 0, 0): the first round has one product (the other factor is zero) and
-// leaves c0' = k[0], so the second round's first product is the launch constant m0k0; 17 products instead of 20.
-__device__ __forceinline__ void philox4x32_10_c0(uint32_t c0, const PhiloxKeys& K, uint32_t out[4]) {
+// leaves c0' = k[0], so the second round's first product is the launch constant m0k0: three products fewer.
+__device__ __forceinline__ void philox4x32_c0(uint32_t c0, const PhiloxKeys& K, uint32_t out[4]) {
     const uint64_t q = (uint64_t)0xD2511F53u * c0;
     // after round 0: (k[0], 0, hi(q) ^ k[1], lo(q));  round 1:
     const uint64_t p1 = (uint64_t)0xCD9E8D57u * ((uint32_t)(q >> 32) ^ K.k[1]);
@@ -144,7 +144,7 @@ __device__ __forceinline__ void philox4x32_10_c0(uint32_t c0, const PhiloxKeys& 
     uint32_t a2 = K.m0k0_hi ^ (uint32_t)q ^ K.k[3];
     uint32_t a3 = K.m0k0_lo;
 #pragma unroll
-    for (int r = 2; r < 10; ++r) {
+    for (int r = 2; r < kPhiloxRounds; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * a0;
         const uint64_t pp = (uint64_t)0xCD9E8D57u * a2;
         a0 = (uint32_t)(pp >> 32) ^ a1 ^ K.k[2 * r];
@@ -155,11 +155,12 @@ __device__ __forceinline__ void philox4x32_10_c0(uint32_t c0, const PhiloxKeys& 
     out[0] = a0; out[1] = a1; out[2] = a2; out[3] = a3;
 }
 
-// Random bits of the 8 source elements whose logical index i has i >> 3 == group.  `small` (uniform over the
-// launch): every group number is below 2^32.
-__device__ __forceinline__ void sr_bits8(const PhiloxKeys& K, uint64_t group, bool small, uint32_t w[4]) {
-    if (small) philox4x32_10_c0((uint32_t)group, K, w);
-    else philox4x32_10((uint32_t)group, (uint32_t)(group >> 32), 0u, 0u, K, w);
+// Random bits of the 8 source elements whose logical index i has i >> 3 == group.  SMALL: the tensor has fewer
+// than 2^35 elements, so every group number is below 2^32 (chosen per launch by the host).
+template <bool SMALL>
+__device__ __forceinline__ void sr_bits8(const PhiloxKeys& K, uint64_t group, uint32_t w[4]) {
+    if (SMALL) philox4x32_c0((uint32_t)group, K, w);
+    else philox4x32((uint32_t)group, (uint32_t)(group >> 32), 0u, 0u, K, w);
 }
 
 // ---------------------------------------------------------------------------------------

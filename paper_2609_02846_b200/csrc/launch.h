@@ -5,10 +5,11 @@
 
 namespace ue5m3 {
 
-// The ten round-key pairs of Philox4x32-10 for one seed (k[2r], k[2r + 1] = key of round r).  They depend only on
+// The round-key pairs of Philox4x32-7 for one seed (k[2r], k[2r + 1] = key of round r).  They depend only on
 // the seed, so the launcher computes them on the host and they travel with the launch parameters.
+constexpr int kPhiloxRounds = 7;
 struct PhiloxKeys {
-    uint32_t k[20];
+    uint32_t k[2 * kPhiloxRounds];
     uint32_t m0k0_hi, m0k0_lo;      // 0xD2511F53 * k[0]: the second round's first product when the counter is below 2^32
 };
 

@@ -1,14 +1,16 @@
 // Fused UE5M3-FP4 quantizer kernels and the tensor-maximum reduction (sm_100a).
 //
-// Three streaming kernels, all HBM-bound by design:
-//   quantize_row_kernel  one thread per 16-element block along the contiguous dimension:
-//                        one 256-bit (BF16) or two 256-bit (FP32) loads, 8 payload bytes and one
-//                        scale byte out.
-//   quantize_tile_kernel each thread owns a 16-row x 8-column register tile.  MODE_COL forms
-//                        blocks down the rows and writes the quantized transpose; MODE_2D forms
-//                        16x16 tiles from two neighbouring lanes and writes the row-major payload
-//                        plus (optionally) the transposed copy through a shared-memory transpose.
-//   amax_kernel          max |x| with packed BF16 compares and one integer atomicMax per CTA.
+// Streaming kernels, bound by HBM (round to nearest) or by integer arithmetic (stochastic rounding):
+//   quantize_row_kernel       1D blocks along the contiguous dimension, one thread per 16-element block, persistent
+//                             grid; quantize_row_flat_kernel is its round-to-nearest fast path for contiguous BF16
+//                             tensors (one 256-bit load per block).
+//   quantize_tile_kernel      each thread owns a 16-row x 8-column register tile.  MODE 0 forms blocks down the rows
+//                             and writes the quantized transpose, MODE 1 forms 16x16 tiles from two neighbouring
+//                             lanes and writes the row-major payload plus (optionally) the transposed copy, MODE 3
+//                             writes the row and the column operand of the same tensor.  Column outputs are
+//                             converted two rows at a time, which yields the transposed bytes directly.
+//   amax_kernel               max |x| with packed BF16 compares and one integer atomicMax per CTA.
+// Every CTA first tabulates the per-element multiplier of each of the 256 scale codes in shared memory.
 #include "common.cuh"
 #include "launch.h"
 
@@ -98,8 +100,10 @@ __device__ __forceinline__ void cta_setup(CtaTables& t, const float* amax_held, 
 // ---------------------------------------------------------------------------------------
 // Persistent: the grid is sized to the device (resident CTAs x SMs) and every thread walks over blocks with the
 // grid stride, so the set-up above is paid once per CTA and there is no partial last wave.
-template <bool IS_BF16, bool SR, bool STATS, bool TILED>
+// RND: 0 = round to nearest even, 1 = stochastic rounding with 32-bit Philox counters, 2 = with 64-bit counters.
+template <bool IS_BF16, int RND, bool STATS, bool TILED>
 __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(const __grid_constant__ QuantArgs a, int kb_shift) {
+    constexpr bool SR = RND != 0, SMALL = RND == 1;
     static_assert(kRowThreads == 256, "one table entry per thread");
     __shared__ CtaTables tab;
     cta_setup<false>(tab, a.amax_held, a.T, a.T);
@@ -168,8 +172,8 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(const __grid_
         if (SR) {
             // element index of the block = 16 * idx (rows are whole numbers of blocks): groups 2 idx and 2 idx + 1
             const uint64_t g0 = (uint64_t)idc * 2;
-            sr_bits8(a.keys, g0, a.small_counter != 0, w0);
-            sr_bits8(a.keys, g0 + 1, a.small_counter != 0, w1);
+            sr_bits8<SMALL>(a.keys, g0, w0);
+            sr_bits8<SMALL>(a.keys, g0 + 1, w1);
         }
         uint32_t bclip = 0;
         uint2 out;
@@ -198,88 +202,58 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(const __grid_
     if (STATS) warp_add_stats(a.stats, sat, rep, clip, nonf);
 }
 
-// The common case -- rows stored back to back (ld == cols), row-major scales, 32-byte aligned BF16 source: the tensor is
-// one flat run of blocks.  A thread takes two blocks per trip, 256 blocks apart, each with ONE 256-bit load (a warp
-// instruction reads 1 KB of contiguous memory), needs no row/column arithmetic, and the Philox groups of block i are
-// 2i and 2i + 1.
+// Round to nearest, the common case -- BF16 rows stored back to back (ld == cols) on a 32-byte boundary, row-major
+// scales: the tensor is one flat run of blocks, each fetched with ONE 256-bit load (a warp instruction reads 1 KB of
+// contiguous memory) and no row/column arithmetic.  Measured against the general kernel: +7 % at 2^29 elements.
 __device__ __forceinline__ void ldg_nc_v8(const void* p, uint32_t r[8]) {
     asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]) : "l"(p));
 }
 
-constexpr int kFlatBlocksPerTrip = 2;
-
-template <bool SR, bool STATS>
+template <bool STATS>
 __global__ void __launch_bounds__(kRowThreads) quantize_row_flat_kernel(const __grid_constant__ QuantArgs a, uint32_t nblocks) {
     static_assert(kRowThreads == 256, "one table entry per thread");
     __shared__ CtaTables tab;
     cta_setup<false>(tab, a.amax_held, a.T, a.T);
     const float S = tab.tc[0].S;
     if (blockIdx.x == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tab.tc[0].d;
-    constexpr bool kRawSanitize = SR && !STATS;
-    constexpr bool kSanitizeZ = SR && !kRawSanitize;
-    const bool small = a.small_counter != 0;
-    constexpr uint32_t kTrip = kRowThreads * kFlatBlocksPerTrip;
 
     uint32_t sat = 0, rep = 0, clip = 0, nonf = 0;
-    for (uint32_t base = blockIdx.x * kTrip; base < nblocks; base += gridDim.x * kTrip) {
-        uint32_t raw[kFlatBlocksPerTrip][8];
-        uint32_t idx[kFlatBlocksPerTrip];
-        bool live[kFlatBlocksPerTrip];
+    for (uint32_t base = blockIdx.x * kRowThreads; base < nblocks; base += gridDim.x * kRowThreads) {
+        const uint32_t idx = base + threadIdx.x;
+        const bool live = idx < nblocks;
+        uint32_t raw[8];
+        ldg_nc_v8(reinterpret_cast<const uint8_t*>(a.x) + (uint64_t)(live ? idx : 0) * 32, raw);
+        uint32_t m = 0;
 #pragma unroll
-        for (int b = 0; b < kFlatBlocksPerTrip; ++b) {
-            idx[b] = base + b * kRowThreads + threadIdx.x;
-            live[b] = idx[b] < nblocks;
-            ldg_nc_v8(reinterpret_cast<const uint8_t*>(a.x) + (uint64_t)(live[b] ? idx[b] : 0) * 32, raw[b]);
-        }
+        for (int q = 0; q < 8; ++q) m = bf16x2_absmax(m, raw[q]);
+        m = bf16x2_magnitudes(m);
+        float aB = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+        // block of 32: the neighbouring thread holds the other half (an even number of blocks per row)
+        if (a.block32) aB = fmaxf(aB, __shfl_xor_sync(0xFFFFFFFFu, aB, 1));
+        float rB;
+        uint32_t flags;
+        const uint32_t code = block_scale(aB, S, tab.lut[0], rB, flags);
+        if (a.block32 && (threadIdx.x & 1)) flags = 0;
+        float f[16];
 #pragma unroll
-        for (int b = 0; b < kFlatBlocksPerTrip; ++b) {
-            uint32_t m = 0;
-            if (kRawSanitize) {
+        for (int q = 0; q < 8; ++q) unpack_bf16x2(raw[q], f[2 * q], f[2 * q + 1]);
+        const uint32_t none[4] = {0, 0, 0, 0};
+        uint32_t bclip = 0;
+        uint2 out;
+        out.x = encode8<false, false>(f, rB, none, bclip);
+        out.y = encode8<false, false>(f + 8, rB, none, bclip);
+        if (live) *reinterpret_cast<uint2*>(a.payload + (uint64_t)idx * 8) = out;
+        // four lanes share one 32-bit store of scale bytes (the block count is a multiple of 4 here)
+        uint32_t sc = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
+        sc |= __shfl_down_sync(0xFFFFFFFFu, sc, 2) << 16;
+        if (live && (threadIdx.x & 3) == 0) *reinterpret_cast<uint32_t*>(a.scales + idx) = sc;
+        if (STATS) {
+            uint32_t bnonf = 0;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) m = bf16x2_absmax_nan(m, raw[b][q]);
-                if (bf16x2_any_nan(m)) {             // rare: the block holds a NaN
-                    m = 0;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) { m = bf16x2_absmax(m, raw[b][q]); raw[b][q] = bf16x2_nan_to_inf(raw[b][q]); }
-                }
-            } else {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) m = bf16x2_absmax(m, raw[b][q]);
-            }
-            m = bf16x2_magnitudes(m);
-            float aB = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
-            // block of 32: the neighbouring thread holds the other half (an even number of blocks per row)
-            if (a.block32) aB = fmaxf(aB, __shfl_xor_sync(0xFFFFFFFFu, aB, 1));
-            float rB;
-            uint32_t flags;
-            const uint32_t code = block_scale(aB, S, tab.lut[0], rB, flags);
-            if (a.block32 && (threadIdx.x & 1)) flags = 0;
-            float f[16];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) unpack_bf16x2(raw[b][q], f[2 * q], f[2 * q + 1]);
-            uint32_t w0[4] = {0, 0, 0, 0}, w1[4] = {0, 0, 0, 0};
-            if (SR) {
-                const uint64_t g0 = (uint64_t)(live[b] ? idx[b] : 0) * 2;
-                sr_bits8(a.keys, g0, small, w0);
-                sr_bits8(a.keys, g0 + 1, small, w1);
-            }
-            uint32_t bclip = 0;
-            uint2 out;
-            out.x = encode8<SR, kSanitizeZ>(f, rB, w0, bclip);
-            out.y = encode8<SR, kSanitizeZ>(f + 8, rB, w1, bclip);
-            if (live[b]) *reinterpret_cast<uint2*>(a.payload + (uint64_t)idx[b] * 8) = out;
-            // four lanes share one 32-bit store of scale bytes (nblocks is a multiple of 4 here)
-            uint32_t sc = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
-            sc |= __shfl_down_sync(0xFFFFFFFFu, sc, 2) << 16;
-            if (live[b] && (threadIdx.x & 3) == 0) *reinterpret_cast<uint32_t*>(a.scales + idx[b]) = sc;
-            if (STATS) {
-                uint32_t bnonf = 0;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) bnonf += nonfinite(f[j]) ? 1u : 0u;
-                const uint32_t lv = live[b] ? 1u : 0u;
-                sat += lv * (flags & 1u); rep += lv * ((flags >> 1) & 1u); clip += lv * bclip; nonf += lv * bnonf;
-            }
+            for (int j = 0; j < 16; ++j) bnonf += nonfinite(f[j]) ? 1u : 0u;
+            const uint32_t lv = live ? 1u : 0u;
+            sat += lv * (flags & 1u); rep += lv * ((flags >> 1) & 1u); clip += lv * bclip; nonf += lv * bnonf;
         }
     }
     if (STATS) warp_add_stats(a.stats, sat, rep, clip, nonf);
@@ -305,23 +279,21 @@ __device__ __forceinline__ void load_row8(const void* x, int64_t off, float f[8]
     }
 }
 
-// Lane = 16 column groups x 2 row blocks in modes 0 and 1, so that every load instruction of a warp reads 256
-// contiguous bytes of two rows.
+// Lane = 16 column groups x 2 row blocks, so that every load instruction of a warp reads 256 contiguous bytes of
+// two rows.
 // MODE 0: column blocks (output = quantized transpose): payload and scales go through shared memory and
-//         leave as 16-byte pieces of the transposed rows.  Used for round-to-nearest, which is HBM-bound.
-// MODE 2: column blocks with lane = 2 column groups x 16 row blocks: the 8-byte payload pieces and the scale
-//         bytes of one output row are contiguous across 16 lanes and are stored directly.  Used for stochastic
-//         rounding, which is bound by integer arithmetic and is better off without the staging work.
+//         leave as 16-byte pieces of the transposed rows.
 // MODE 1: 2D tiles: lanes 2i and 2i+1 hold the halves of one tile; the row-major payload is stored directly
 //         (64 contiguous bytes per row and warp), the optional transposed copy goes through shared memory.
 // MODE 3: dual layout: MODE 0 plus the 1D_ROW quantization of the same register tile (a row block of 16 is this
 //         lane's 8 columns and lane ^ 1's): the tensor is read once for both operands of a backward pass.
-template <bool IS_BF16, bool SR, bool STATS, int MODE, bool TILED, bool WANT_T>
+template <bool IS_BF16, int RND, bool STATS, int MODE, bool TILED, bool WANT_T>
 __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile_kernel(const __grid_constant__ QuantArgs a) {
+    constexpr bool SR = RND != 0, SMALL = RND == 1;
     static_assert(kTileThreads == 256, "one table entry per thread");
     constexpr bool kDual = MODE == 3;
     constexpr bool kStaged = (MODE == 0) || kDual;       // column output through shared memory
-    constexpr bool kColumns = kStaged || (MODE == 2);
+    constexpr bool kColumns = kStaged;
     constexpr bool kTranspose = kStaged || WANT_T;
     // NaN inputs under stochastic rounding (see quantize_row_kernel)
     constexpr bool kRawSanitize = SR && IS_BF16 && !STATS;
@@ -332,8 +304,8 @@ __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int cg, rb;   // column group (8 columns) and row block (16 rows) inside the CTA tile
-    if (MODE == 2) { cg = warp * 2 + (lane >> 4); rb = lane & 15; }
-    else           { cg = lane & 15;              rb = warp * 2 + (lane >> 4); }
+    cg = lane & 15;
+    rb = warp * 2 + (lane >> 4);
     const int64_t c0 = (int64_t)blockIdx.x * kTileCols + cg * 8;
     const int64_t r0 = (int64_t)blockIdx.y * kTileRows + rb * 16;
     const bool live = (c0 < a.cols) && (r0 < a.rows);
@@ -407,9 +379,9 @@ __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile
     }
 
     // ---- block scales ----
-    // Blocks of 32: the thread holding the adjacent 16 rows is lane ^ 16 (lane ^ 1 in mode 2), the one holding the
+    // Blocks of 32: the thread holding the adjacent 16 rows is lane ^ 16, the one holding the
     // adjacent 16 columns of a 2D tile lane ^ 2; CTA tiles start on multiples of 32, so partners share a block.
-    constexpr int kRowPartner = (MODE == 2) ? 1 : 16;
+    constexpr int kRowPartner = 16;
     float rcol[8];
     uint32_t codes[8];
     uint32_t sat = 0, rep = 0;
@@ -456,7 +428,6 @@ __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile
     // group of Philox draws of the 8 elements of row r0 + r: ((r0 + r) * cols + c0) / 8
     const uint64_t group0 = ((uint64_t)r0 * (uint64_t)a.cols + (uint64_t)c0) >> 3;
     const uint64_t group_step = (uint64_t)a.cols >> 3;
-    const bool small = a.small_counter != 0;
 #pragma unroll
     for (int rp = 0; rp < 8; ++rp) {
         float v[2][8];
@@ -473,7 +444,7 @@ __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile
                 unpack_bf16x8(x, f);
             } else { uint4 x; load_row8<false>(a.x, base + r * a.ld, f, x); }
             uint32_t w[4] = {0, 0, 0, 0};
-            if (SR) sr_bits8(a.keys, group0 + (uint64_t)r * group_step, small, w);
+            if (SR) sr_bits8<SMALL>(a.keys, group0 + (uint64_t)r * group_step, w);
             if (kDual) {
                 // ---- the row operand: block = 16 consecutive columns of row r0 + r, held by lanes 2i and 2i + 1 ----
                 float m = 0.0f;
@@ -492,7 +463,7 @@ __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile
                 const uint32_t code_r = block_scale(m, S_row, tab.lut[kDual ? 1 : 0], rrow, fl);
                 if ((lane & (a.block32 ? 3 : 1)) == 0) { sat_r += fl & 1u; rep_r += (fl >> 1) & 1u; }
                 uint32_t wr[4] = {0, 0, 0, 0};
-                if (SR) sr_bits8(a.row_keys, group0 + (uint64_t)r * group_step, small, wr);
+                if (SR) sr_bits8<SMALL>(a.row_keys, group0 + (uint64_t)r * group_step, wr);
                 const uint32_t orow = encode8<SR, kSanitizeZ>(f, rrow, wr, clip_r);
                 const int64_t kbpr = a.cols >> 4;
                 // four lanes (even column groups) -> four consecutive scale bytes
@@ -523,21 +494,6 @@ __global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile
         }
     }
 
-    if (MODE == 2) {
-        if (live) {
-            const int64_t kblocks = a.rows >> 4;
-            const int64_t rblk = r0 >> 4;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint2 o;
-                o.x = tcol[j][0];
-                o.y = tcol[j][1];
-                *reinterpret_cast<uint2*>(a.payload + (c0 + j) * (a.rows >> 1) + (r0 >> 1)) = o;
-                const int64_t so = TILED ? tiled_scale_offset(c0 + j, rblk, kblocks) : (c0 + j) * kblocks + rblk;
-                a.scales[so] = (uint8_t)codes[j];
-            }
-        }
-    }
     if (MODE == 1) {
         if (live) {
             if ((lane & 1) == 0) {
@@ -689,9 +645,9 @@ static int resident_ctas_per_sm(K kernel, int threads) {
     return n;
 }
 
-template <bool IS_BF16, bool SR, bool STATS, bool TILED>
+template <bool IS_BF16, int RND, bool STATS, bool TILED>
 static cudaError_t launch_row_t(const QuantArgs& a, int num_sms, cudaStream_t st) {
-    static const int per_sm = resident_ctas_per_sm(quantize_row_kernel<IS_BF16, SR, STATS, TILED>, kRowThreads);
+    static const int per_sm = resident_ctas_per_sm(quantize_row_kernel<IS_BF16, RND, STATS, TILED>, kRowThreads);
     const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
     uint64_t grid = (nblocks + kRowThreads - 1) / kRowThreads;
     const uint64_t resident = (uint64_t)per_sm * (uint64_t)num_sms;
@@ -699,83 +655,85 @@ static cudaError_t launch_row_t(const QuantArgs& a, int num_sms, cudaStream_t st
     const uint64_t kbpr = (uint64_t)(a.cols >> 4);
     int kb_shift = -1;
     if ((kbpr & (kbpr - 1)) == 0) { kb_shift = 0; while ((1ull << kb_shift) < kbpr) ++kb_shift; }
-    quantize_row_kernel<IS_BF16, SR, STATS, TILED><<<(unsigned)grid, kRowThreads, 0, st>>>(a, kb_shift);
+    quantize_row_kernel<IS_BF16, RND, STATS, TILED><<<(unsigned)grid, kRowThreads, 0, st>>>(a, kb_shift);
     return cudaGetLastError();
 }
 
-template <bool SR, bool STATS>
+template <bool STATS>
 static cudaError_t launch_row_flat(const QuantArgs& a, int num_sms, cudaStream_t st) {
-    static const int per_sm = resident_ctas_per_sm(quantize_row_flat_kernel<SR, STATS>, kRowThreads);
+    static const int per_sm = resident_ctas_per_sm(quantize_row_flat_kernel<STATS>, kRowThreads);
     const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
-    const uint64_t per_cta = (uint64_t)kRowThreads * kFlatBlocksPerTrip;
-    uint64_t grid = (nblocks + per_cta - 1) / per_cta;
+    uint64_t grid = (nblocks + kRowThreads - 1) / kRowThreads;
     const uint64_t resident = (uint64_t)per_sm * (uint64_t)num_sms;
     if (grid > resident) grid = resident;
-    quantize_row_flat_kernel<SR, STATS><<<(unsigned)grid, kRowThreads, 0, st>>>(a, (uint32_t)nblocks);
+    quantize_row_flat_kernel<STATS><<<(unsigned)grid, kRowThreads, 0, st>>>(a, (uint32_t)nblocks);
     return cudaGetLastError();
 }
 
-template <bool IS_BF16, bool SR, bool STATS>
+template <bool IS_BF16, int RND, bool STATS>
 static cudaError_t launch_row(const QuantArgs& a, bool tiled, int num_sms, cudaStream_t st) {
     const uint64_t nblocks = (uint64_t)a.rows * (uint64_t)(a.cols >> 4);
-    // BF16 rows back to back on a 32-byte boundary, row-major scales, a multiple of four blocks
-    if (IS_BF16 && !tiled && a.ld == a.cols && (nblocks & 3) == 0 && (reinterpret_cast<uintptr_t>(a.x) & 31u) == 0)
-        return launch_row_flat<SR, STATS>(a, num_sms, st);
-    return tiled ? launch_row_t<IS_BF16, SR, STATS, true>(a, num_sms, st) : launch_row_t<IS_BF16, SR, STATS, false>(a, num_sms, st);
+    // BF16 rows back to back on a 32-byte boundary, row-major scales, a multiple of four blocks: round-to-nearest
+    // takes the flat kernel (measured: 256-bit loads are worth 7 % at 2^29 elements); stochastic rounding is bound
+    // by arithmetic and measured no faster there, so it stays on the general kernel
+    if (IS_BF16 && RND == 0 && !tiled && a.ld == a.cols && (nblocks & 3) == 0 && (reinterpret_cast<uintptr_t>(a.x) & 31u) == 0)
+        return launch_row_flat<STATS>(a, num_sms, st);
+    return tiled ? launch_row_t<IS_BF16, RND, STATS, true>(a, num_sms, st) : launch_row_t<IS_BF16, RND, STATS, false>(a, num_sms, st);
 }
 
-template <bool IS_BF16, bool SR, bool STATS>
+template <bool IS_BF16, int RND, bool STATS>
 static cudaError_t launch_tile(const QuantArgs& a, int layout, bool tiled, cudaStream_t st) {
     dim3 grid((unsigned)((a.cols + kTileCols - 1) / kTileCols), (unsigned)((a.rows + kTileRows - 1) / kTileRows));
     if (layout == UE5M3_LAYOUT_1D_COL) {
-        constexpr int kMode = SR ? 2 : 0;
-        if (tiled) quantize_tile_kernel<IS_BF16, SR, STATS, kMode, true, false><<<grid, kTileThreads, 0, st>>>(a);
-        else       quantize_tile_kernel<IS_BF16, SR, STATS, kMode, false, false><<<grid, kTileThreads, 0, st>>>(a);
+        if (tiled) quantize_tile_kernel<IS_BF16, RND, STATS, 0, true, false><<<grid, kTileThreads, 0, st>>>(a);
+        else       quantize_tile_kernel<IS_BF16, RND, STATS, 0, false, false><<<grid, kTileThreads, 0, st>>>(a);
     } else {
-        if (a.payload_t) quantize_tile_kernel<IS_BF16, SR, STATS, 1, false, true><<<grid, kTileThreads, 0, st>>>(a);
-        else             quantize_tile_kernel<IS_BF16, SR, STATS, 1, false, false><<<grid, kTileThreads, 0, st>>>(a);
+        if (a.payload_t) quantize_tile_kernel<IS_BF16, RND, STATS, 1, false, true><<<grid, kTileThreads, 0, st>>>(a);
+        else             quantize_tile_kernel<IS_BF16, RND, STATS, 1, false, false><<<grid, kTileThreads, 0, st>>>(a);
     }
     return cudaGetLastError();
 }
 
-template <bool IS_BF16, bool SR, bool STATS>
+template <bool IS_BF16, int RND, bool STATS>
 static cudaError_t launch_any(const QuantArgs& a, int layout, bool tiled, int num_sms, cudaStream_t st) {
-    if (layout == UE5M3_LAYOUT_1D_ROW) return launch_row<IS_BF16, SR, STATS>(a, tiled, num_sms, st);
-    return launch_tile<IS_BF16, SR, STATS>(a, layout, tiled, st);
+    if (layout == UE5M3_LAYOUT_1D_ROW) return launch_row<IS_BF16, RND, STATS>(a, tiled, num_sms, st);
+    return launch_tile<IS_BF16, RND, STATS>(a, layout, tiled, st);
 }
 
 cudaError_t launch_quantize(const QuantArgs& args, int dtype, int layout, int rounding, bool tiled, int num_sms, cudaStream_t st) {
     QuantArgs a = args;
-    const bool bf = dtype == UE5M3_BF16, sr = rounding == UE5M3_ROUND_SR, stt = a.stats != nullptr;
-    if (sr) a.keys = philox_round_keys(a.seed);
+    const bool bf = dtype == UE5M3_BF16, stt = a.stats != nullptr;
     a.small_counter = (uint64_t)a.rows * (uint64_t)a.cols < (1ull << 35) ? 1 : 0;
-#define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_any<B, S, T>(a, layout, tiled, num_sms, st);
-    UE5M3_DISPATCH(true, false, false) UE5M3_DISPATCH(true, true, false)
-    UE5M3_DISPATCH(true, false, true)  UE5M3_DISPATCH(true, true, true)
-    UE5M3_DISPATCH(false, false, false) UE5M3_DISPATCH(false, true, false)
-    UE5M3_DISPATCH(false, false, true)  UE5M3_DISPATCH(false, true, true)
+    const int rnd = rounding != UE5M3_ROUND_SR ? 0 : (a.small_counter ? 1 : 2);
+    if (rnd) a.keys = philox_round_keys(a.seed);
+#define UE5M3_DISPATCH(B, R, T) if (bf == B && rnd == R && stt == T) return launch_any<B, R, T>(a, layout, tiled, num_sms, st);
+    UE5M3_DISPATCH(true, 0, false) UE5M3_DISPATCH(true, 1, false) UE5M3_DISPATCH(true, 2, false)
+    UE5M3_DISPATCH(true, 0, true)  UE5M3_DISPATCH(true, 1, true)  UE5M3_DISPATCH(true, 2, true)
+    UE5M3_DISPATCH(false, 0, false) UE5M3_DISPATCH(false, 1, false) UE5M3_DISPATCH(false, 2, false)
+    UE5M3_DISPATCH(false, 0, true)  UE5M3_DISPATCH(false, 1, true)  UE5M3_DISPATCH(false, 2, true)
 #undef UE5M3_DISPATCH
     return cudaErrorInvalidValue;
 }
 
-template <bool IS_BF16, bool SR, bool STATS>
+template <bool IS_BF16, int RND, bool STATS>
 static cudaError_t launch_dual(const QuantArgs& a, bool tiled, cudaStream_t st) {
     dim3 grid((unsigned)((a.cols + kTileCols - 1) / kTileCols), (unsigned)((a.rows + kTileRows - 1) / kTileRows));
-    if (tiled) quantize_tile_kernel<IS_BF16, SR, STATS, 3, true, false><<<grid, kTileThreads, 0, st>>>(a);
-    else       quantize_tile_kernel<IS_BF16, SR, STATS, 3, false, false><<<grid, kTileThreads, 0, st>>>(a);
+    if (tiled) quantize_tile_kernel<IS_BF16, RND, STATS, 3, true, false><<<grid, kTileThreads, 0, st>>>(a);
+    else       quantize_tile_kernel<IS_BF16, RND, STATS, 3, false, false><<<grid, kTileThreads, 0, st>>>(a);
     return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_dual(const QuantArgs& args, int dtype, int rounding, bool tiled, cudaStream_t st) {
     QuantArgs a = args;
-    const bool bf = dtype == UE5M3_BF16, sr = rounding == UE5M3_ROUND_SR, stt = a.stats != nullptr;
-    if (sr) { a.keys = philox_round_keys(a.seed); a.row_keys = philox_round_keys(a.row_seed); }
+    const bool bf = dtype == UE5M3_BF16, stt = a.stats != nullptr;
     a.small_counter = (uint64_t)a.rows * (uint64_t)a.cols < (1ull << 35) ? 1 : 0;
-#define UE5M3_DISPATCH(B, S, T) if (bf == B && sr == S && stt == T) return launch_dual<B, S, T>(a, tiled, st);
-    UE5M3_DISPATCH(true, false, false) UE5M3_DISPATCH(true, true, false)
-    UE5M3_DISPATCH(true, false, true)  UE5M3_DISPATCH(true, true, true)
-    UE5M3_DISPATCH(false, false, false) UE5M3_DISPATCH(false, true, false)
-    UE5M3_DISPATCH(false, false, true)  UE5M3_DISPATCH(false, true, true)
+    const int rnd = rounding != UE5M3_ROUND_SR ? 0 : (a.small_counter ? 1 : 2);
+    if (rnd) { a.keys = philox_round_keys(a.seed); a.row_keys = philox_round_keys(a.row_seed); }
+#define UE5M3_DISPATCH(B, R, T) if (bf == B && rnd == R && stt == T) return launch_dual<B, R, T>(a, tiled, st);
+    UE5M3_DISPATCH(true, 0, false) UE5M3_DISPATCH(true, 1, false) UE5M3_DISPATCH(true, 2, false)
+    UE5M3_DISPATCH(true, 0, true)  UE5M3_DISPATCH(true, 1, true)  UE5M3_DISPATCH(true, 2, true)
+    UE5M3_DISPATCH(false, 0, false) UE5M3_DISPATCH(false, 1, false) UE5M3_DISPATCH(false, 2, false)
+    UE5M3_DISPATCH(false, 0, true)  UE5M3_DISPATCH(false, 1, true)  UE5M3_DISPATCH(false, 2, true)
 #undef UE5M3_DISPATCH
     return cudaErrorInvalidValue;
 }

@@ -406,10 +406,46 @@ def test_philox_known_answers():
         assert list(oracle.philox4x32_10(w[0:4], w[4:6])) == w[6:10]
 
 
+def test_philox_round_function_from_the_definition():
+    """The generator as Python integers, written from its definition, reproduces the published 10-round vectors; the
+    oracle's generic routine must then agree with it for every round count, in particular the 7 rounds the draws use
+    (the published vectors cover only the default of 10)."""
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        rows = [[int(v, 16) for v in l.split()] for l in f if l.strip() and not l.startswith("#")]
+    for w in rows:
+        assert _philox4x32(w[0:4], w[4:6], 10) == w[6:10]
+    rng = np.random.default_rng(8)
+    for rounds in (1, 2, 7, 10):
+        for w in rows + [[int(v) for v in rng.integers(0, 2 ** 32, 6)] for _ in range(8)] + [[5, 0, 0, 0, 9, 1]]:
+            assert [int(v) for v in oracle.philox4x32(w[0:4], w[4:6], rounds)] == _philox4x32(w[0:4], w[4:6], rounds)
+    assert oracle.SR_PHILOX_ROUNDS == 7
+
+
+def test_seven_round_draws_are_uniform_and_decorrelated():
+    """Sanity of the 7-round draws on the counters the quantizer uses (consecutive small integers, two nearby keys):
+    16-bit draws uniform per bit, per byte bucket and pairwise uncorrelated between neighbouring elements, between
+    the two keys of a backward pass, and between a counter and its successor."""
+    n = 1 << 15
+    a = np.array([_draw16(40, i) for i in range(n)], dtype=np.float64)
+    b = np.array([_draw16(41, i) for i in range(n)], dtype=np.float64)
+    for d in (a, b):
+        assert abs(d.mean() / 65535.0 - 0.5) < 4 * (1 / np.sqrt(12 * n))
+        hist = np.bincount((d.astype(np.int64) >> 8), minlength=256)
+        chi2 = ((hist - n / 256) ** 2 / (n / 256)).sum()
+        assert chi2 < 255 + 5 * np.sqrt(2 * 255)                       # chi-square with 255 degrees of freedom
+        bits = ((d.astype(np.int64)[:, None] >> np.arange(16)) & 1).mean(axis=0)
+        assert np.all(np.abs(bits - 0.5) < 5 * 0.5 / np.sqrt(n))
+    def corr(x, y):
+        return abs(np.corrcoef(x, y)[0, 1])
+    lim = 5 / np.sqrt(n)
+    assert corr(a, b) < lim and corr(a[:-1], a[1:]) < lim and corr(a[:-8], a[8:]) < lim and corr(a[::8][:-1], a[::8][1:]) < lim * 3
+
+
 def test_sr_bits_indexing():
     seed = 0x0123456789ABCDEF
     for i in (0, 5, 8, 1023, 2 ** 35 + 3):
-        w = oracle.philox4x32_10([(i >> 3) & 0xFFFFFFFF, (i >> 3) >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32])
+        assert oracle.sr_bits(seed, i) == _draw16(seed, i)
+        w = oracle.philox4x32([(i >> 3) & 0xFFFFFFFF, (i >> 3) >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32], 7)
         j = i & 7
         assert oracle.sr_bits(seed, i) == (int(w[j >> 1]) >> (16 * (j & 1))) & 0xFFFF
     draws = np.array([oracle.sr_bits(3, i) for i in range(1 << 14)])
@@ -523,7 +559,7 @@ def _philox4x32(ctr, key, rounds=10):
 
 
 def _draw16(seed, i):
-    w = _philox4x32([(i >> 3) & 0xFFFFFFFF, (i >> 3) >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32])
+    w = _philox4x32([(i >> 3) & 0xFFFFFFFF, (i >> 3) >> 32, 0, 0], [seed & 0xFFFFFFFF, seed >> 32], rounds=7)
     return (w[(i & 7) >> 1] >> (16 * (i & 1))) & 0xFFFF
 
 
