@@ -142,7 +142,7 @@ class ClockSampler:
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
-            cmd = ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"]
+            cmd = ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "25"]
             if self.gpu_id:
                 cmd += ["-i", self.gpu_id]
             self.proc = subprocess.Popen(cmd, stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
@@ -176,25 +176,33 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, pw, reasons = [], [], [], set()
+        rows = []
         try:
             with open(self.path) as f:
-                for n, line in enumerate(f):
-                    if n < getattr(self, "skip", 0):
-                        continue
+                for line in f:
                     c = [v.strip() for v in line.split(",")]
                     if len(c) < 7:
                         continue
                     try:
-                        sm.append(float(c[0])); mx.append(float(c[1])); pw.append(float(c[2]))
+                        rows.append((float(c[0]), float(c[1]), float(c[2]), c[3:7]))
                     except ValueError:
                         continue
-                    for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[3:7]):
-                        if v.lower().startswith("active"):
-                            reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
+        skip = getattr(self, "skip", 0)
+        # a timed region shorter than the sampling interval may hold no sample: then the last samples of the warm-up
+        # (the same launch sequence, directly before the region) stand in, and the record says so
+        picked = rows[skip:]
+        if not picked and rows:
+            picked = rows[-3:]
+            out["note"] = "no sample fell inside the timed region; these are the last samples of the warm-up before it"
+        sm, mx, pw, reasons = [], [], [], set()
+        for a, b, c_, flags in picked:
+            sm.append(a); mx.append(b); pw.append(c_)
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), flags):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(pw), samples=len(sm))
         out["reasons"] = sorted(reasons)
@@ -231,27 +239,46 @@ class LinearStep:
         ev.setdefault(name, []).append((a, b))
         return r
 
-    def run(self, step, ev=None):
+    def run(self, step, ev=None, per_kernel=False):
+        """One step.  With `ev`, CUDA events bracket every GEMM launch and every GROUP of consecutive quantizer
+        launches (names in QUANT_GROUPS), so that the quantizer time of a step has no event gaps inside a group;
+        `per_kernel=True` brackets every quantizer launch separately instead (breakdown pass, not the timed region)."""
         lib = self.lib
         refresh = self.cx.refreshes_at(step)
         gx, gw, gg = self.cx.get(self.X, step), self.cw.get(self.W, step), self.cg.get(self.dY, step)
         self.launches += 3 if refresh else 0
         sl = self.scale_layout
         q = self.q
-        q["x"] = self._timed("q_x_row", lambda: lib.quantize(self.X, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, gx, 448.0,
-                                                             scale_layout=sl, out=q.get("x")), ev)
-        q["w"] = self._timed("q_w_2d", lambda: lib.quantize(self.W, lib.LAYOUT_2D, lib.ROUND_RNE, gw, 448.0,
-                                                            want_transpose=True, out=q.get("w")), ev)
+        evk = ev if per_kernel else None
+        evg = None if per_kernel else ev
+
+        def fwd_quant():
+            q["x"] = self._timed("q_x_row", lambda: lib.quantize(self.X, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, gx, 448.0,
+                                                                 scale_layout=sl, out=q.get("x")), evk)
+            q["w"] = self._timed("q_w_2d", lambda: lib.quantize(self.W, lib.LAYOUT_2D, lib.ROUND_RNE, gw, 448.0,
+                                                                want_transpose=True, out=q.get("w")), evk)
+
+        def dgrad_quant():
+            q["g"] = self._timed("q_dy_row_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_ROW, lib.ROUND_SR, gg, 448.0,
+                                                                     seed=4 * step, scale_layout=sl, out=q.get("g")), evk)
+
+        def wgrad_quant():
+            q["gt"] = self._timed("q_dy_col_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, 448.0,
+                                                                      seed=4 * step + 1, scale_layout=sl, out=q.get("gt")), evk)
+            q["xt"] = self._timed("q_x_col", lambda: lib.quantize(self.X, lib.LAYOUT_1D_COL, lib.ROUND_RNE, gx, 448.0,
+                                                                  scale_layout=sl, out=q.get("xt")), evk)
+
+        self._timed("quant_fwd", fwd_quant, evg)
         self._timed("gemm_fprop", lambda: lib.gemm(lib.FPROP, q["x"], q["w"], out=self.Y), ev)
-        q["g"] = self._timed("q_dy_row_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_ROW, lib.ROUND_SR, gg, 448.0,
-                                                                 seed=4 * step, scale_layout=sl, out=q.get("g")), ev)
+        self._timed("quant_dgrad", dgrad_quant, evg)
         self._timed("gemm_dgrad", lambda: lib.gemm(lib.DGRAD, q["g"], q["w"].transposed(), out=self.dX), ev)
-        q["gt"] = self._timed("q_dy_col_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, 448.0,
-                                                                  seed=4 * step + 1, scale_layout=sl, out=q.get("gt")), ev)
-        q["xt"] = self._timed("q_x_col", lambda: lib.quantize(self.X, lib.LAYOUT_1D_COL, lib.ROUND_RNE, gx, 448.0,
-                                                              scale_layout=sl, out=q.get("xt")), ev)
+        self._timed("quant_wgrad", wgrad_quant, evg)
         self._timed("gemm_wgrad", lambda: lib.gemm(lib.WGRAD, q["gt"], q["xt"], out=self.dW), ev)
         self.launches += 8
+
+
+QUANT_GROUPS = {"quant_fwd": ("q_x_row", "q_w_2d"), "quant_dgrad": ("q_dy_row_sr",), "quant_wgrad": ("q_dy_col_sr", "q_x_col")}
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 
 
 # algorithmic bytes of each streaming kernel per launch (BF16 in, payload + scales out)
@@ -353,15 +380,63 @@ def run_ours(args):
     per_kernel = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in ev.items()}
     gemm_ms = statistics.mean(per_kernel[k] for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad"))
     gemm_tflops = GEMM_FLOPS / (gemm_ms * 1e-3) / 1e12
-    quant = {}
-    qbytes = qms = 0.0
+    # quantizers inside the timed region: one event pair per group of consecutive quantizer launches
+    qbytes = float(sum(KERNEL_BYTES.values()))
+    qms = sum(per_kernel[g] for g in QUANT_GROUPS)
+    quant = {"timing": "inside the timed region: one CUDA-event pair around each group of consecutive quantizer launches "
+                       "(no event between the launches of a group)",
+             "groups": {g: {"kernels": list(ks), "ms": round(per_kernel[g], 4),
+                            "GB/s": round(sum(KERNEL_BYTES[k] for k in ks) / (per_kernel[g] * 1e-3) / 1e9, 1)}
+                        for g, ks in QUANT_GROUPS.items()},
+             "all": {"ms": round(qms, 4), "GB/s": round(qbytes / (qms * 1e-3) / 1e9, 1),
+                     "frac_of_measured_hbm": round(qbytes / (qms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),
+                     "frac_of_nominal_8TBs": round(qbytes / (qms * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 3),
+                     "share_of_step": round(qms / ms_per_step, 3)}}
+
+    # ---- breakdown pass (outside the timed region): every quantizer launch with its own event pair ----
+    evb = {}
+    for s_ in range(min(K, 20)):
+        step.run(Wm + K + s_, evb, per_kernel=True)
+    torch.cuda.synchronize()
+    pk = {}
     for k, nbytes in KERNEL_BYTES.items():
-        gbs = nbytes / (per_kernel[k] * 1e-3) / 1e9
-        quant[k] = {"ms": round(per_kernel[k], 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3)}
-        qbytes += nbytes
-        qms += per_kernel[k]
-    quant["all"] = {"ms": round(qms, 4), "GB/s": round(qbytes / (qms * 1e-3) / 1e9, 1),
-                    "frac_of_measured_hbm": round(qbytes / (qms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
+        ms = statistics.mean(a.elapsed_time(b) for a, b in evb[k])
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        pk[k] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+    quant["per_kernel"] = pk
+    quant["per_kernel_timing"] = ("separate pass after the timed region, one event pair per launch: each figure includes the "
+                                  "launch gap of a single short kernel (a few microseconds)")
+
+    # ---- sustained leg: at least two seconds of back-to-back steps under the power cap ----
+    sustained = None
+    if rank == 0 and world == 1 and not args.no_sustained:
+        sampler2 = ClockSampler(dev)
+        sampler2.start()
+        sampler2.wait_first_sample()
+        n_sus = max(50, int(2200.0 / ms_per_step))
+        for s_ in range(20):
+            step.run(Wm + K + 20 + s_)
+        torch.cuda.synchronize()
+        sampler2.mark()
+        evs = {}
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for s_ in range(n_sus):
+            step.run(Wm + K + 40 + s_, evs)
+        s1.record()
+        torch.cuda.synchronize()
+        clk2 = sampler2.stop()
+        sus_ms = s0.elapsed_time(s1) / n_sus
+        sus_gemm_ms = statistics.mean(a.elapsed_time(b) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad") for a, b in evs[k])
+        sus_gemm = GEMM_FLOPS / (sus_gemm_ms * 1e-3) / 1e12
+        sustained = {"seconds": round(sus_ms * n_sus * 1e-3, 2), "steps": n_sus, "ms_per_step": round(sus_ms, 4),
+                     "tflops_per_step": round(FLOPS_PER_STEP / (sus_ms * 1e-3) / 1e12, 1),
+                     "gemm_tflops_per_launch": round(sus_gemm, 1), "gemm_avg_launch_ms": round(sus_gemm_ms, 4),
+                     "gemm_frac_of_sustained_peak": round(sus_gemm / peaks["bf16_tflops_sustained"], 3),
+                     "gemm_frac_of_burst_peak": round(sus_gemm / peaks["bf16_tflops"], 3),
+                     "gemm_frac_of_nominal_2250": round(sus_gemm / NOMINAL_BF16_TFLOPS, 3),
+                     "clocks": clk2,
+                     "gemm_launch_ms_x_sm_mhz": None if not clk2.get("sm_mhz") else round(sus_gemm_ms * clk2["sm_mhz"], 1)}
 
     # ---- end to end: host buffers in, results back to the host, every step ----
     # Three streams and two sets of device buffers: the copy-in of step s+1 and the copy-out of step s-1 run under
@@ -397,13 +472,13 @@ def run_ours(args):
                 out_done[b_] = torch.cuda.Event(); out_done[b_].record(s_out)
 
         for s in range(2):
-            e2e_step(Wm + K + s)
+            e2e_step(Wm + K + 100000 + s)
         main.wait_stream(s_out)
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for s in range(n_e2e):
-            e2e_step(Wm + K + 2 + s)
+            e2e_step(Wm + K + 100002 + s)
         main.wait_stream(s_in); main.wait_stream(s_out)
         b.record()
         barrier()
@@ -419,21 +494,35 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             v, dt, cores = time_oracle(1, 0)
             cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": SAMPLE_DESC, "seconds": round(dt, 2)}
+        # Denominator from this run's own clock record: a short region at full clocks is compared with the burst
+        # figure of the measured cuBLAS peak, a long or power-capped one with the sustained figure.
+        region_s = total_ms * 1e-3
+        capped = "sw_power_cap" in (clocks.get("reasons") or [])
+        use_burst = region_s < 1.0 and not capped
+        peak = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
+        roofline = {"bound": "tensor", "kernel": "gemm_kernel", "achieved": gemm_tflops, "peak": peak, "unit": "TFLOP/s",
+                    "frac": gemm_tflops / peak,
+                    "peak_source": peaks["source"] + (" (burst: timed region %.3f s, no power cap seen)" % region_s if use_burst
+                                                      else " (sustained: timed region %.3f s%s)" % (region_s, ", sw_power_cap seen" if capped else "")),
+                    "frac_of_burst_peak": gemm_tflops / peaks["bf16_tflops"],
+                    "frac_of_sustained_peak": gemm_tflops / peaks["bf16_tflops_sustained"],
+                    "frac_of_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
+                    "avg_launch_ms": gemm_ms,
+                    "avg_launch_ms_x_sm_mhz": None if not clocks.get("sm_mhz") else round(gemm_ms * clocks["sm_mhz"], 1),
+                    "traffic": GEMM_DRAM_TRAFFIC_BYTES if (M_TOK, K_IN, N_OUT) == (8192, 4096, 16384) else None,
+                    "traffic_unit": "bytes of DRAM read+write per launch (ncu, mean of the three GEMMs)",
+                    "per_gemm_ms": {k: round(per_kernel[k], 4) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}}
+        sweep = None
+        if world == 1 and not args.no_sweep:
+            sweep = quantizer_sweep_cells(dev, peaks)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "tokens_per_gpu": M_TOK, "l2": f"inputs ({2 * (M_TOK * K_IN + N_OUT * K_IN + M_TOK * N_OUT) >> 20} MiB per step) exceed the 126 MB L2",
                        "scale_layout": "tiled" if args.scale_layout else "rowmajor", "amax": "sampled at step 0, held 50 steps"},
-            "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": gemm_tflops,
-                         "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": gemm_tflops / peaks["bf16_tflops_sustained"],
-                         "frac_of_burst_peak": gemm_tflops / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (sustained)",
-                         "avg_launch_ms": gemm_ms,
-                         "traffic": GEMM_DRAM_TRAFFIC_BYTES if (M_TOK, K_IN, N_OUT) == (8192, 4096, 16384) else None,
-                         "traffic_unit": "bytes of DRAM read+write per launch (ncu, mean of the three GEMMs)",
-                         "per_gemm_ms": {k: round(per_kernel[k], 4) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}},
-            "quantizer": quant,
+            "roofline": roofline,
+            "quantizer": quant, "sustained": sustained, "quantizer_sweep": sweep,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -573,6 +662,71 @@ def run_current(args):
                       "tensors": out}), flush=True)
 
 
+def _graph_time(torch, fn, flush, nbytes, warmup, iters):
+    """Median and best time (ms) of one launch replayed from a CUDA graph; L2 flushed before each replay when the
+    tensor would otherwise fit in it."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    # one launch captured in a CUDA graph: the replay keeps the Python/ctypes call (5-10 us of host time)
+    # out of the device timeline, which matters for the small tensors
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fn()
+    ts = []
+    for _ in range(iters):
+        if nbytes < (256 << 20):
+            flush.zero_()                      # inputs that fit in L2: flush it between timed launches
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); graph.replay(); b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    del graph
+    return statistics.median(ts), min(ts)
+
+
+def sweep_row(torch, lib, si, dev, peaks, flush, log2n, warmup, iters):
+    """One size of the quantizer bandwidth sweep: BF16 [rows, 4096]; amax + {1D_ROW, 1D_COL, 2D} x {RNE, SR}, and a plain
+    streaming kernel (elementwise int32 add) moving the same number of bytes as a 1D quantization (what any kernel can
+    reach at this size under this timing)."""
+    rows = (1 << log2n) // 4096
+    x = si.row_scaled_tensor(rows, 4096, seed=log2n, device=dev)
+    g = lib.sample_amax(x)
+    cells = {"amax": (lambda: lib.sample_amax(x, g), rows * 4096 * 2)}
+    for lname, layout in (("1d_row", 0), ("1d_col", 1), ("2d", 2)):
+        for rname, rnd in (("rne", 0), ("sr", 1)):
+            q = lib.quantize(x, layout, rnd, g, seed=1)
+            cells[f"{lname}_{rname}"] = ((lambda layout=layout, rnd=rnd, q=q: lib.quantize(x, layout, rnd, g, seed=1, out=q)),
+                                         _quant_bytes(rows, 4096, layout))
+    half = _quant_bytes(rows, 4096, 0) // 2 // 1024 * 1024
+    src = torch.zeros(half // 4, dtype=torch.int32, device=dev)
+    dst = torch.empty(half // 4, dtype=torch.int32, device=dev)
+    cells["copy_same_bytes"] = (lambda: torch.add(src, 1, out=dst), 2 * half)
+    row = {"log2_elements": log2n}
+    for name, (fn, nbytes) in cells.items():
+        ms, best = _graph_time(torch, fn, flush, rows * 4096 * 2, warmup, iters)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3),
+                     "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3), "best_GB/s": round(nbytes / (best * 1e-3) / 1e9, 1)}
+    return row
+
+
+def quantizer_sweep_cells(dev, peaks, sizes=(25, 27, 29), warmup=20, iters=100):
+    """The part of the bandwidth sweep that goes into the default JSON line: the operand sizes of the benchmark linear
+    (2^25 = X, 2^27 = dY) and a large one."""
+    import torch
+    import paper_2609_02846_b200 as lib
+    import synth_inputs as si
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = {"method": f"CUDA-graph replay of one launch, {warmup} warm-up + {iters} timed, median; L2 flushed before every "
+                     "timed launch; copy_same_bytes = a plain streaming kernel (torch int32 add, read half / write half) moving the "
+                     "bytes a 1D quantization moves: what any kernel reaches at that size under this timing",
+           "sizes": [sweep_row(torch, lib, si, dev, peaks, flush, n, warmup, iters) for n in sizes]}
+    del flush
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_sweep(args):
     """Quantizer-only bandwidth sweep: BF16 [rows, 4096], 2^20 .. 2^30 elements, {1D, 2D} x {RNE, SR} + amax."""
     import torch
@@ -583,41 +737,9 @@ def run_sweep(args):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = []
     for log2n in range(20, 31, args.sweep_stride):
-        rows = (1 << log2n) // 4096
-        x = si.row_scaled_tensor(rows, 4096, seed=log2n, device=dev)
-        g = lib.sample_amax(x)
-        cells = {"amax": (lambda: lib.sample_amax(x, g), rows * 4096 * 2)}
-        for lname, layout in (("1d_row", 0), ("1d_col", 1), ("2d", 2)):
-            for rname, rnd in (("rne", 0), ("sr", 1)):
-                q = lib.quantize(x, layout, rnd, g, seed=1)
-                cells[f"{lname}_{rname}"] = ((lambda layout=layout, rnd=rnd, q=q: lib.quantize(x, layout, rnd, g, seed=1, out=q)),
-                                             _quant_bytes(rows, 4096, layout))
-        row = {"log2_elements": log2n}
-        for name, (fn, nbytes) in cells.items():
-            for _ in range(args.sweep_warmup):
-                fn()
-            torch.cuda.synchronize()
-            # one launch captured in a CUDA graph: the replay keeps the Python/ctypes call (5-10 us of host time)
-            # out of the device timeline, which matters for the small tensors
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
-                fn()
-            ts = []
-            for _ in range(args.sweep_iters):
-                if nbytes < (256 << 20):
-                    flush.zero_()                      # inputs that fit in L2: flush it between timed launches
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(); graph.replay(); b.record()
-                torch.cuda.synchronize()
-                ts.append(a.elapsed_time(b))
-            del graph
-            ms = statistics.median(ts)
-            gbs = nbytes / (ms * 1e-3) / 1e9
-            row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3),
-                         "best_GB/s": round(nbytes / (min(ts) * 1e-3) / 1e9, 1)}
+        row = sweep_row(torch, lib, si, dev, peaks, flush, log2n, args.sweep_warmup, args.sweep_iters)
         out.append(row)
         print(json.dumps(row), flush=True)
-        del x
     return out
 
 
@@ -655,6 +777,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-layout", type=int, default=0, choices=[0, 1])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the two-second sustained leg")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the quantizer sweep cells of the default line")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--stack", action="store_true", help="time the six linears of the 8B-hybrid-shaped layer stack")
     ap.add_argument("--current", action="store_true", help="time the per-batch (D = 1) reference policy")
