@@ -179,7 +179,9 @@ UE5M3_API int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_
  *     FPROP  A = X  (1D_ROW),        B = W   (2D payload, scales)          Mo = tokens, No = out, Kc = in
  *     DGRAD  A = dY (1D_ROW, SR),    B = W^T (2D payload_t, scales_t)      Mo = tokens, No = in,  Kc = out
  *     WGRAD  A = dY^T (1D_COL, SR),  B = X^T (1D_COL)                      Mo = out,    No = in,  Kc = tokens
- *   Mo, No multiples of 128, Kc a multiple of 256 (UE5M3_ERR_SHAPE otherwise).
+ *   Mo, No and Kc multiples of 128 (UE5M3_ERR_SHAPE otherwise).  Kc = 128 * odd costs a little more: the last 256-wide
+ *   stage of the contraction is half empty, and scale rows of 8 * odd bytes (row-major 1D and 2D storage) are read
+ *   with plain loads instead of bulk copies.
  *   a_payload [Mo, Kc/2], b_payload [No, Kc/2]   device, 16-byte aligned.
  *   a_scales, b_scales   device, 16-byte aligned; a_scale_mode / b_scale_mode say how they are
  *                        stored: UE5M3_SCALE_1D ([R, Kc/16] row-major), UE5M3_SCALE_1D_TILED,
@@ -201,7 +203,8 @@ UE5M3_API int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
  *     c_0 = 0,  c_{g+1} = RTZ32(c_g + p_g), g ascending                                       Eq. "issue-rz"
  *     C[m, n] = RNE32( alpha * Q_d(c_G) ),  Q_d(c) = RNE(d c) / d,  alpha = RNE32(d_A * d_B) Eq. "final-grid",
  *                                                                                             Eq. "grid-denominator"
- * Arguments, layouts, shape rules, alignment and error behaviour are those of ue5m3_gemm, plus
+ * Arguments, layouts, alignment and error behaviour are those of ue5m3_gemm (Kc must be a multiple of 256 here, so
+ * that the contraction is a whole number of 64-product groups per 256-wide stage), plus
  *   cross_rounding      0 = toward zero (the model); 1 = nearest even (the paper's control variant).
  *   grid_denominator    d: 0 (no grid step) or a power of two up to 65536; the paper's rule is d = 1024.
  * BF16 output is the FP32 result rounded to nearest even.  The result does not depend on the device's SM count.
@@ -222,7 +225,7 @@ UE5M3_API int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t K
  * context stays usable.
  *   which               0 = the kernel of ue5m3_gemm, 1 = the kernel of ue5m3_gemm_probe_matched.
  *   wait_limit_cycles   1000 .. 4e9 (about 2e6 is one millisecond).
- * All other arguments, and their checks and errors, are those of ue5m3_gemm.
+ * All other arguments, and their checks and errors, are those of ue5m3_gemm (Kc a multiple of 256).
  */
 UE5M3_API int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc,
                const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,

@@ -55,10 +55,12 @@ def _group_rank(group) -> int:
     return 0
 
 
-def _check_dims(M: int, K: int, N: int) -> None:
+def _check_dims(M: int, K: int, N: int, multiple: int = 128) -> None:
+    """Every dimension is an output dimension of one GEMM and the contraction of another: multiples of 128 for
+    ue5m3_gemm, of 256 under the output model (ue5m3_gemm_probe_matched)."""
     for name, v in (("tokens", M), ("in_features", K), ("out_features", N)):
-        if v % 256:
-            raise ValueError(f"{name} = {v}: the three GEMMs of a linear need every dimension to be a multiple of 256")
+        if v % multiple:
+            raise ValueError(f"{name} = {v}: the three GEMMs of this linear need every dimension to be a multiple of {multiple}")
 
 
 class _Ue5m3LinearFn(torch.autograd.Function):
@@ -66,7 +68,7 @@ class _Ue5m3LinearFn(torch.autograd.Function):
     def forward(ctx, x, w, layer, step):
         M, K = x.shape
         N = w.shape[0]
-        _check_dims(M, K, N)
+        _check_dims(M, K, N, 128 if layer.grid_denominator is None else 256)
         ax = layer.scale_x.get(x, step)
         aw = layer.scale_w.get(w, step)
         y, _, qw = B.linear_forward(x, w, ax, aw, layer.target_T, x.dtype, grid_denominator=layer.grid_denominator)

@@ -183,14 +183,14 @@ int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, in
 
 static int check_gemm_args(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
                            int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
-                           int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo) {
+                           int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, int64_t k_multiple) {
     if (op != UE5M3_FPROP && op != UE5M3_DGRAD && op != UE5M3_WGRAD) return UE5M3_ERR_INVALID_ARG;
     if (!a_payload || !a_scales || !a_decode || !b_payload || !b_scales || !b_decode || !out) return UE5M3_ERR_INVALID_ARG;
     if (Mo <= 0 || No <= 0 || Kc <= 0 || ldo < No) return UE5M3_ERR_INVALID_ARG;
     if (out_dtype != UE5M3_F32 && out_dtype != UE5M3_BF16) return UE5M3_ERR_INVALID_ARG;
     for (int m : {a_scale_mode, b_scale_mode})
         if (m != UE5M3_SCALE_1D && m != UE5M3_SCALE_1D_TILED && m != UE5M3_SCALE_2D) return UE5M3_ERR_INVALID_ARG;
-    if ((Mo % 128) || (No % 128) || (Kc % 256)) return UE5M3_ERR_SHAPE;
+    if ((Mo % 128) || (No % 128) || (Kc % k_multiple)) return UE5M3_ERR_SHAPE;
     const int64_t osz = out_dtype == UE5M3_F32 ? 4 : 2;
     if (!aligned16(a_payload) || !aligned16(b_payload) || !aligned16(a_scales) || !aligned16(b_scales) || !aligned16(out) ||
         ((ldo * osz) % 16))
@@ -204,7 +204,7 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
                int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
     const ApiRange range_("ue5m3_gemm");
     const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
-                                    b_scale_mode, b_decode, out, out_dtype, ldo);
+                                    b_scale_mode, b_decode, out, out_dtype, ldo, 128);
     if (bad != UE5M3_OK) return bad;
     const DeviceInfo di = device_info();
     if (!di.ok) return UE5M3_ERR_CUDA;
@@ -220,7 +220,7 @@ int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t Kc, const u
                              void* out, int out_dtype, int64_t ldo, void* stream) {
     const ApiRange range_("ue5m3_gemm_probe_matched");
     const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
-                                    b_scale_mode, b_decode, out, out_dtype, ldo);
+                                    b_scale_mode, b_decode, out, out_dtype, ldo, 256);
     if (bad != UE5M3_OK) return bad;
     if (cross_rounding != 0 && cross_rounding != 1) return UE5M3_ERR_INVALID_ARG;
     if (grid_denominator < 0 || grid_denominator > 65536 || (grid_denominator & (grid_denominator - 1)))
@@ -241,7 +241,7 @@ int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, con
     if (which != 0 && which != 1) return UE5M3_ERR_INVALID_ARG;
     if (wait_limit_cycles < 1000 || wait_limit_cycles > 4000000000LL) return UE5M3_ERR_INVALID_ARG;
     const int bad = check_gemm_args(UE5M3_FPROP, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
-                                    b_scale_mode, b_decode, out, out_dtype, ldo);
+                                    b_scale_mode, b_decode, out, out_dtype, ldo, 256);
     if (bad != UE5M3_OK) return bad;
     const DeviceInfo di = device_info();
     if (!di.ok) return UE5M3_ERR_CUDA;

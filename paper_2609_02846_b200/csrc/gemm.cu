@@ -81,6 +81,12 @@ struct GemmParams {
     int tiles_m, tiles_n;         // 256 x 256 tiles
     long long wait_limit;         // bound of every device-side wait, SM clocks
     int stall_producer;           // self-test: the copy producer issues nothing, so every consumer wait runs out
+    // Kc = 128 * odd: the rows of a row-major scale matrix are then 8 * odd bytes long, which no tensor map can
+    // describe (strides must be multiples of 16 bytes).  Such an operand's scale bytes are read by the dequantizer
+    // threads themselves, four bytes per row and 64-wide slice, one packed stage ahead.
+    const uint8_t* a_scales;
+    const uint8_t* b_scales;
+    int a_direct, b_direct;
 };
 
 // Tile order: groups of kRasterGroup tile rows, and inside a group column by column.  The tiles that are
@@ -125,7 +131,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const uint32_t rank = cluster_rank();                   // 0 = leader of the pair
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_tiles = p.tiles_m * p.tiles_n;
-    const int kchunks = (int)(p.Kc / KCHUNK);
+    const int kchunks = (int)((p.Kc + KCHUNK - 1) / KCHUNK);   // the last chunk is half empty when Kc = 128 * odd
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -156,7 +162,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t it = 0;
             const int a_rows_per_load = (p.a_mode == UE5M3_SCALE_2D) ? 8 : 128;
             const int b_rows_per_load = (p.b_mode == UE5M3_SCALE_2D) ? 8 : 128;
-            const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + a_rows_per_load * 16 + b_rows_per_load * 16;
+            const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + (p.a_direct ? 0 : a_rows_per_load * 16) +
+                                      (p.b_direct ? 0 : b_rows_per_load * 16);
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok && !p.stall_producer; tile += num_pairs) {
                 int tm, tn;
@@ -173,10 +180,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     tma_load_2d(st + PK_A_BYTES, &map_b, full, kc * (KCHUNK / 2), nh * BNH);
                     // scales: the 16 block columns of this K chunk
                     const uint32_t sa = st + PK_A_BYTES + PK_B_BYTES, sb = sa + SC_A_BYTES;
-                    if (p.a_mode == UE5M3_SCALE_1D) tma_load_2d(sa, &map_as, full, kc * 16, mb * BM);
+                    if (p.a_direct) {}
+                    else if (p.a_mode == UE5M3_SCALE_1D) tma_load_2d(sa, &map_as, full, kc * 16, mb * BM);
                     else if (p.a_mode == UE5M3_SCALE_2D) tma_load_2d(sa, &map_as, full, kc * 16, mb * (BM / 16));
                     else tma_load_2d(sa, &map_as, full, 0, (mb * kchunks + kc) * 128);
-                    if (p.b_mode == UE5M3_SCALE_1D) tma_load_2d(sb, &map_bs, full, kc * 16, nh * BNH);
+                    if (p.b_direct) {}
+                    else if (p.b_mode == UE5M3_SCALE_1D) tma_load_2d(sb, &map_bs, full, kc * 16, nh * BNH);
                     else if (p.b_mode == UE5M3_SCALE_2D) tma_load_2d(sb, &map_bs, full, kc * 16, nh * (BNH / 16));
                     else tma_load_2d(sb, &map_bs, full, 0, (nh * kchunks + kc) * 128);
                 }
@@ -309,6 +318,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int pk_off0 = row * 128 + (((2 * grp) ^ r7) << 4), pk_off1 = row * 128 + (((2 * grp + 1) ^ r7) << 4);
         uint32_t it_pk = 0;
         bool ok = true;
+        // Scale bytes read directly from global memory (operands whose scale rows no tensor map can describe):
+        // the four codes of this thread's row and slice for packed stage (tile, kc); 0 beyond the operand.
+        const int64_t kblocks = p.Kc >> 4;
+        auto direct_codes = [&](const uint8_t* scales, int mode, int64_t R, int64_t grow, int kc) -> uint32_t {
+            if (grow >= R || (int64_t)kc * 16 + grp * 4 >= kblocks) return 0u;
+            const int64_t srow = (mode == UE5M3_SCALE_2D) ? (grow >> 4) : grow;
+            return __ldg(reinterpret_cast<const unsigned int*>(scales + srow * kblocks + kc * 16 + grp * 4));
+        };
+        auto prefetch = [&](int tile, int kc, uint32_t& an, uint32_t& bn) {
+            int tm, tn;
+            tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+            if (p.a_direct) an = direct_codes(p.a_scales, p.a_mode, p.Mo, (int64_t)(tm * 2 + (int)rank) * BM + row, kc);
+            if (p.b_direct) bn = direct_codes(p.b_scales, p.b_mode, p.No, (int64_t)(tn * 2 + (int)rank) * BNH + row, kc);
+        };
+        const bool any_direct = p.a_direct || p.b_direct;
+        // slices of the last packed stage that lie beyond Kc (Kc = 128 * odd: slices 2 and 3) hold zero payload
+        // (the copy fills what is out of bounds with zeros); their scale codes are forced to zero as well
+        const bool last_is_partial = (p.Kc % KCHUNK) != 0 && grp * KSUB >= (int)(p.Kc % KCHUNK);
+        uint32_t a_next = 0, b_next = 0;
+        if (any_direct && pair < num_tiles) prefetch(pair, 0, a_next, b_next);
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
             for (int kc = 0; kc < kchunks && ok; ++kc, ++it_pk) {
                 const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
@@ -318,8 +347,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const uint4 a1 = *reinterpret_cast<const uint4*>(st + pk_off1);
                 const uint4 b0 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + pk_off0);
                 const uint4 b1 = *reinterpret_cast<const uint4*>(st + PK_A_BYTES + pk_off1);
-                const uint32_t a_codes = *reinterpret_cast<const uint32_t*>(st + PK_A_BYTES + PK_B_BYTES + a_srow * 16 + grp * 4);
-                const uint32_t b_codes = *reinterpret_cast<const uint32_t*>(st + PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + b_srow * 16 + grp * 4);
+                uint32_t a_codes = p.a_direct ? a_next
+                                              : *reinterpret_cast<const uint32_t*>(st + PK_A_BYTES + PK_B_BYTES + a_srow * 16 + grp * 4);
+                uint32_t b_codes = p.b_direct ? b_next
+                                              : *reinterpret_cast<const uint32_t*>(st + PK_A_BYTES + PK_B_BYTES + SC_A_BYTES + b_srow * 16 + grp * 4);
+                if (last_is_partial && kc == kchunks - 1) a_codes = b_codes = 0;
+                if (any_direct) {
+                    // the codes of the next packed stage, in flight under this stage's arithmetic
+                    const int nkc = (kc + 1 < kchunks) ? kc + 1 : 0;
+                    const int ntile = (kc + 1 < kchunks) ? tile : tile + num_pairs;
+                    if (ntile < num_tiles) prefetch(ntile, nkc, a_next, b_next);
+                }
                 // The packed bytes are in registers: hand the stage back to the producer now, so that the next
                 // copy overlaps the arithmetic (the arrive is a release, ordered after this warp's loads).
                 __syncwarp();
@@ -430,8 +468,15 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
     if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
     if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BNH, true)) return UE5M3_ERR_CUDA;
-    if (!make_scale_map(&mas, g.a_scales, g.a_scale_mode, g.Mo, g.Kc)) return UE5M3_ERR_CUDA;
-    if (!make_scale_map(&mbs, g.b_scales, g.b_scale_mode, g.No, g.Kc)) return UE5M3_ERR_CUDA;
+    // scale rows of Kc/16 bytes fit a tensor map only when that is a multiple of 16 (Kc a multiple of 256); the
+    // tiled layout always does; otherwise the dequantizers read the codes themselves (the map is then a stand-in)
+    const bool pitch_ok = ((g.Kc / 16) % 16) == 0;
+    const bool a_direct = !pitch_ok && g.a_scale_mode != UE5M3_SCALE_1D_TILED;
+    const bool b_direct = !pitch_ok && g.b_scale_mode != UE5M3_SCALE_1D_TILED;
+    if (a_direct) mas = ma;
+    else if (!make_scale_map(&mas, g.a_scales, g.a_scale_mode, g.Mo, g.Kc)) return UE5M3_ERR_CUDA;
+    if (b_direct) mbs = mb;
+    else if (!make_scale_map(&mbs, g.b_scales, g.b_scale_mode, g.No, g.Kc)) return UE5M3_ERR_CUDA;
     CUtensorMap mo;
     if (!make_out_map(&mo, g.out, g.out_dtype == UE5M3_BF16, g.Mo, g.No, g.ldo)) return UE5M3_ERR_CUDA;
 
@@ -444,6 +489,8 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     p.tiles_n = (int)((g.No + BN - 1) / BN);
     p.wait_limit = g.wait_limit_cycles > 0 ? g.wait_limit_cycles : WAIT_LIMIT_CYCLES;
     p.stall_producer = g.stall_producer;
+    p.a_scales = g.a_scales; p.b_scales = g.b_scales;
+    p.a_direct = a_direct ? 1 : 0; p.b_direct = b_direct ? 1 : 0;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int max_pairs = resident_pairs[dev];
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;

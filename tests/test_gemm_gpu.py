@@ -194,6 +194,32 @@ def test_gemm_grouped_tile_order_with_ragged_last_group(shape, out_dtype):
     check_gemm_output(out, y, sa)
 
 
+@pytest.mark.parametrize("Kc", [128, 384, 640, 1152])
+@pytest.mark.parametrize("modes", [(0, 0), (0, 2), (2, 0), (1, 1), (1, 2), (2, 2)])
+def test_gemm_contraction_of_odd_multiples_of_128(Kc, modes):
+    """Kc = 128 * odd: the last 256-wide stage is half empty and row-major scale rows are 8 * odd bytes long, which
+    no bulk copy can fetch (the kernel reads them with plain loads); tiled scale storage keeps its bulk copies and its
+    padding bytes -- filled with non-finite codes here -- must not leak into the sum.  Ragged tile counts included."""
+    Mo, No = 384, 640
+    rng = np.random.default_rng(Kc + 17 * modes[0] + modes[1])
+    qa, ap, asc = _operand(rng, Mo, Kc, modes[0], 0x50, 0xA0, dec=0.5)
+    qb, bp, bsc = _operand(rng, No, Kc, modes[1], 0x50, 0xA0, dec=1.0 / 64.0)
+    for q, sc, R in ((qa, asc, Mo), (qb, bsc, No)):
+        if q.scale_mode == lib.SCALE_1D_TILED:                 # poison the padding of the tiled buffer
+            kb = Kc // 16
+            buf = np.full(q.scales.numel(), 0xFF, np.uint8)
+            r, k = np.meshgrid(np.arange(R), np.arange(kb), indexing="ij")
+            off = ((r >> 7) * ((kb + 15) // 16) + (k >> 4)) * 2048 + (r & 127) * 16 + (k & 15)
+            buf[off.ravel()] = sc.ravel()
+            q.scales.copy_(torch.from_numpy(buf).to(DEV))
+    for out_dtype in (torch.float32, torch.bfloat16):
+        out = lib.gemm(lib.DGRAD, qa, qb, out_dtype)
+        torch.cuda.synchronize()
+        assert lib.last_device_status() == 0
+        y, sa = oracle.gemm(ap, asc, modes[0] == 2, 0.5, bp, bsc, modes[1] == 2, np.float32(1.0 / 64.0))
+        check_gemm_output(out, y, sa)
+
+
 def test_gemm_and_quantizer_are_deterministic():
     """Same inputs, same bytes: three runs of a linear's forward and backward give identical outputs."""
     M, K, N = 512, 1024, 768
@@ -219,8 +245,13 @@ def test_gemm_rejects_bad_shapes():
     with pytest.raises(lib.Ue5m3Error) as e:
         lib.gemm(lib.FPROP, bad, qb)
     assert e.value.status == 2
-    qc, *_ = _operand(rng, 128, 128, 0)
-    qd, *_ = _operand(rng, 128, 128, 0)
+    qc, *_ = _operand(rng, 128, 64, 0)
+    qd, *_ = _operand(rng, 128, 64, 0)
     with pytest.raises(lib.Ue5m3Error) as e:
         lib.gemm(lib.FPROP, qc, qd)
+    assert e.value.status == 2
+    qe, *_ = _operand(rng, 128, 128, 0)
+    qf, *_ = _operand(rng, 128, 128, 0)
+    with pytest.raises(lib.Ue5m3Error) as e:
+        lib.gemm_probe_matched(lib.FPROP, qe, qf)           # the output-model kernel keeps Kc % 256
     assert e.value.status == 2
