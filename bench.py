@@ -3,8 +3,8 @@
 
 One "step" is one pass of the whole path over one batch of synthetic input shaped like the
 8B-hybrid linears: tokens M = 8192, in-features K = 4096, out-features N = 16384, BF16:
-    quantize X (1D rows, RNE), W (2D tiles + transposed copy, RNE), dY (1D rows, SR), dY (1D columns, SR),
-    X (1D columns, RNE);  GEMMs fprop Y = X W^T, dgrad dX = dY W, wgrad dW = dY^T X;
+    quantize X (1D rows and 1D columns, RNE, both from one read), W (2D tiles + transposed copy, RNE), dY (1D rows, SR),
+    dY (1D columns, SR);  GEMMs fprop Y = X W^T, dgrad dX = dY W, wgrad dW = dY^T X;
     tensor maxima are sampled at step 0 and held (re-sampled every 50 steps).
 The reported value is the whole-step rate in TFLOP/s (GEMM flops only: 3 * 2 M K N per step, the
 quantization time is inside the step).  The roofline object covers the dominant kernel (the GEMM);
@@ -34,7 +34,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 M_TOK, K_IN, N_OUT = 8192, 4096, 16384
-WORKLOAD = "linear fwd+bwd M=8192 K=4096 N=16384 bf16 (fprop+dgrad+wgrad, 5 quantizations, SR on dY)"
+WORKLOAD = "linear fwd+bwd M=8192 K=4096 N=16384 bf16 (fprop+dgrad+wgrad, 5 quantized operands from 4 launches, SR on dY)"
 METRIC = "fwd+bwd block-scaled linear throughput (quantize + 3 GEMMs)"
 UNIT = "TFLOP/s"
 FLOPS_PER_STEP = 3 * 2 * M_TOK * K_IN * N_OUT
@@ -211,7 +211,7 @@ class ClockSampler:
 
 class LinearStep:
     """Pre-allocated buffers and the launch sequence of one fwd+bwd step."""
-    KERNELS = ("q_x_row", "q_w_2d", "gemm_fprop", "q_dy_row_sr", "gemm_dgrad", "q_dy_col_sr", "q_x_col", "gemm_wgrad")
+    KERNELS = ("q_x_dual", "q_w_2d", "gemm_fprop", "q_dy_row_sr", "gemm_dgrad", "q_dy_col_sr", "gemm_wgrad")
 
     def __init__(self, device, seed=0, scale_layout=0):
         import torch
@@ -253,8 +253,10 @@ class LinearStep:
         evg = None if per_kernel else ev
 
         def fwd_quant():
-            q["x"] = self._timed("q_x_row", lambda: lib.quantize(self.X, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, gx, 448.0,
-                                                                 scale_layout=sl, out=q.get("x")), evk)
+            # X is needed along K (fprop) and along the tokens (wgrad): both operands come from ONE read of X
+            q["x"], q["xt"] = self._timed("q_x_dual", lambda: lib.quantize_dual(
+                self.X, lib.ROUND_RNE, gx, 448.0, 448.0, scale_layout=sl,
+                out=(q["x"], q["xt"]) if "x" in q else None), evk)
             q["w"] = self._timed("q_w_2d", lambda: lib.quantize(self.W, lib.LAYOUT_2D, lib.ROUND_RNE, gw, 448.0,
                                                                 want_transpose=True, out=q.get("w")), evk)
 
@@ -265,8 +267,6 @@ class LinearStep:
         def wgrad_quant():
             q["gt"] = self._timed("q_dy_col_sr", lambda: lib.quantize(self.dY, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, 448.0,
                                                                       seed=4 * step + 1, scale_layout=sl, out=q.get("gt")), evk)
-            q["xt"] = self._timed("q_x_col", lambda: lib.quantize(self.X, lib.LAYOUT_1D_COL, lib.ROUND_RNE, gx, 448.0,
-                                                                  scale_layout=sl, out=q.get("xt")), evk)
 
         self._timed("quant_fwd", fwd_quant, evg)
         self._timed("gemm_fprop", lambda: lib.gemm(lib.FPROP, q["x"], q["w"], out=self.Y), ev)
@@ -274,10 +274,10 @@ class LinearStep:
         self._timed("gemm_dgrad", lambda: lib.gemm(lib.DGRAD, q["g"], q["w"].transposed(), out=self.dX), ev)
         self._timed("quant_wgrad", wgrad_quant, evg)
         self._timed("gemm_wgrad", lambda: lib.gemm(lib.WGRAD, q["gt"], q["xt"], out=self.dW), ev)
-        self.launches += 8
+        self.launches += 7
 
 
-QUANT_GROUPS = {"quant_fwd": ("q_x_row", "q_w_2d"), "quant_dgrad": ("q_dy_row_sr",), "quant_wgrad": ("q_dy_col_sr", "q_x_col")}
+QUANT_GROUPS = {"quant_fwd": ("q_x_dual", "q_w_2d"), "quant_dgrad": ("q_dy_row_sr",), "quant_wgrad": ("q_dy_col_sr",)}
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 
 
@@ -290,8 +290,9 @@ def _quant_bytes(rows, cols, layout, transposed_copy=False):
 
 
 def kernel_bytes():
+    nx = M_TOK * K_IN
     return {
-        "q_x_row": _quant_bytes(M_TOK, K_IN, 0), "q_x_col": _quant_bytes(M_TOK, K_IN, 1),
+        "q_x_dual": nx * 2 + 2 * (nx // 2 + nx // 16),          # one read of X, row and column operand out
         "q_w_2d": _quant_bytes(N_OUT, K_IN, 2, True),
         "q_dy_row_sr": _quant_bytes(M_TOK, N_OUT, 0), "q_dy_col_sr": _quant_bytes(M_TOK, N_OUT, 1),
     }

@@ -288,7 +288,7 @@ __device__ __forceinline__ void load_row8(const void* x, int64_t off, float f[8]
 // MODE 3: dual layout: MODE 0 plus the 1D_ROW quantization of the same register tile (a row block of 16 is this
 //         lane's 8 columns and lane ^ 1's): the tensor is read once for both operands of a backward pass.
 template <bool IS_BF16, int RND, bool STATS, int MODE, bool TILED, bool WANT_T>
-__global__ void __launch_bounds__(kTileThreads, MODE == 3 ? 1 : 2) quantize_tile_kernel(const __grid_constant__ QuantArgs a) {
+__global__ void __launch_bounds__(kTileThreads, (MODE == 3 && RND != 0) ? 1 : 2) quantize_tile_kernel(const __grid_constant__ QuantArgs a) {
     constexpr bool SR = RND != 0, SMALL = RND == 1;
     static_assert(kTileThreads == 256, "one table entry per thread");
     constexpr bool kDual = MODE == 3;
@@ -579,18 +579,20 @@ constexpr int kAmaxThreads = 512;
 template <bool IS_BF16>
 __global__ void __launch_bounds__(kAmaxThreads) amax_kernel(const void* x, int64_t rows, int64_t cols, int64_t ld,
                                                               float* out) {
-    // work item = 8 consecutive elements (BF16: one 128-bit load; FP32: two)
+    // work item = 8 consecutive elements (BF16: one 128-bit load; FP32: two).  Read-only streaming: a thread keeps
+    // four independent loads in flight per trip (the loop is split so that no bound check sits between them).
     const int64_t per_row = cols >> 3;
     const int64_t total = rows * per_row;
     const int64_t stride = (int64_t)gridDim.x * kAmaxThreads;
     float m = 0.0f;
     uint32_t pm0 = 0, pm1 = 0, pm2 = 0, pm3 = 0;
     const bool flat = (ld == cols);
-#pragma unroll 4
-    for (int64_t i = (int64_t)blockIdx.x * kAmaxThreads + threadIdx.x; i < total; i += stride) {
-        int64_t off;
-        if (flat) off = i * 8;
-        else { const int64_t r = i / per_row; off = r * ld + (i - r * per_row) * 8; }
+    auto offset = [&](int64_t i) -> int64_t {
+        if (flat) return i * 8;
+        const int64_t r = i / per_row;
+        return r * ld + (i - r * per_row) * 8;
+    };
+    auto take = [&](int64_t off) {
         if (IS_BF16) {
             const uint4 v = ldg_nc_v4(reinterpret_cast<const uint16_t*>(x) + off);
             pm0 = bf16x2_absmax(pm0, v.x); pm1 = bf16x2_absmax(pm1, v.y);
@@ -603,7 +605,20 @@ __global__ void __launch_bounds__(kAmaxThreads) amax_kernel(const void* x, int64
             m = fmaxf(m, fmaxf(fmaxf(fabsf(__uint_as_float(v1.x)), fabsf(__uint_as_float(v1.y))),
                                fmaxf(fabsf(__uint_as_float(v1.z)), fabsf(__uint_as_float(v1.w)))));
         }
+    };
+    int64_t i = (int64_t)blockIdx.x * kAmaxThreads + threadIdx.x;
+    if (IS_BF16) {
+        for (; i + 3 * stride < total; i += 4 * stride) {
+            const uint16_t* p = reinterpret_cast<const uint16_t*>(x);
+            const uint4 v0 = ldg_nc_v4(p + offset(i)), v1 = ldg_nc_v4(p + offset(i + stride));
+            const uint4 v2 = ldg_nc_v4(p + offset(i + 2 * stride)), v3 = ldg_nc_v4(p + offset(i + 3 * stride));
+            pm0 = bf16x2_absmax(bf16x2_absmax(pm0, v0.x), v0.y); pm1 = bf16x2_absmax(bf16x2_absmax(pm1, v0.z), v0.w);
+            pm2 = bf16x2_absmax(bf16x2_absmax(pm2, v1.x), v1.y); pm3 = bf16x2_absmax(bf16x2_absmax(pm3, v1.z), v1.w);
+            pm0 = bf16x2_absmax(bf16x2_absmax(pm0, v2.x), v2.y); pm1 = bf16x2_absmax(bf16x2_absmax(pm1, v2.z), v2.w);
+            pm2 = bf16x2_absmax(bf16x2_absmax(pm2, v3.x), v3.y); pm3 = bf16x2_absmax(bf16x2_absmax(pm3, v3.z), v3.w);
+        }
     }
+    for (; i < total; i += stride) take(offset(i));
     if (IS_BF16) {
         const uint32_t p = bf16x2_max(bf16x2_max(bf16x2_magnitudes(pm0), bf16x2_magnitudes(pm1)),
                                       bf16x2_max(bf16x2_magnitudes(pm2), bf16x2_magnitudes(pm3)));
@@ -744,7 +759,7 @@ cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, in
     if (e != cudaSuccess) return e;
     const int64_t items = rows * (cols >> 3);
     int64_t grid = (items + kAmaxThreads - 1) / kAmaxThreads;
-    const int64_t cap = (int64_t)num_sms * 4 * 4;      // 4 resident CTAs per SM, 4 loads in flight per thread
+    const int64_t cap = (int64_t)num_sms * 4;          // one wave of 4 resident CTAs per SM, 4 loads in flight per thread
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
     if (dtype == UE5M3_BF16) amax_kernel<true><<<(unsigned)grid, kAmaxThreads, 0, st>>>(x, rows, cols, ld, out);
