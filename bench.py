@@ -302,7 +302,7 @@ KERNEL_BYTES = kernel_bytes()
 GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the default workload (mean of fprop, dgrad, wgrad;
 # one ncu pass, summary in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt).  Algorithmic bytes: 242 MB per launch.
-GEMM_DRAM_TRAFFIC_BYTES = (151.0e6 + 224.2e6 + 202.8e6 + 48.4e6 + 98.2e6 + 101.9e6) / 3
+GEMM_DRAM_TRAFFIC_BYTES = (150.5e6 + 220.5e6 + 188.9e6 + 47.9e6 + 101.1e6 + 99.5e6) / 3
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -663,30 +663,37 @@ def run_current(args):
                       "tensors": out}), flush=True)
 
 
-def _graph_time(torch, fn, flush, nbytes, warmup, iters):
+def _graph_time(torch, fn, flush, nbytes, warmup, iters, use_graph=True):
     """Median and best time (ms) of one launch replayed from a CUDA graph; L2 flushed before each replay when the
-    tensor would otherwise fit in it."""
+    tensor would otherwise fit in it.  `use_graph=False` launches directly (for captures under a profiler)."""
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
     # one launch captured in a CUDA graph: the replay keeps the Python/ctypes call (5-10 us of host time)
     # out of the device timeline, which matters for the small tensors
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        fn()
+    graph = None
+    if use_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fn()
     ts = []
     for _ in range(iters):
         if nbytes < (256 << 20):
             flush.zero_()                      # inputs that fit in L2: flush it between timed launches
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); graph.replay(); b.record()
+        a.record()
+        if graph is not None:
+            graph.replay()
+        else:
+            fn()
+        b.record()
         torch.cuda.synchronize()
         ts.append(a.elapsed_time(b))
     del graph
     return statistics.median(ts), min(ts)
 
 
-def sweep_row(torch, lib, si, dev, peaks, flush, log2n, warmup, iters):
+def sweep_row(torch, lib, si, dev, peaks, flush, log2n, warmup, iters, use_graph=True):
     """One size of the quantizer bandwidth sweep: BF16 [rows, 4096]; amax + {1D_ROW, 1D_COL, 2D} x {RNE, SR}, and a plain
     streaming kernel (elementwise int32 add) moving the same number of bytes as a 1D quantization (what any kernel can
     reach at this size under this timing)."""
@@ -705,7 +712,7 @@ def sweep_row(torch, lib, si, dev, peaks, flush, log2n, warmup, iters):
     cells["copy_same_bytes"] = (lambda: torch.add(src, 1, out=dst), 2 * half)
     row = {"log2_elements": log2n}
     for name, (fn, nbytes) in cells.items():
-        ms, best = _graph_time(torch, fn, flush, rows * 4096 * 2, warmup, iters)
+        ms, best = _graph_time(torch, fn, flush, rows * 4096 * 2, warmup, iters, use_graph)
         gbs = nbytes / (ms * 1e-3) / 1e9
         row[name] = {"ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 3),
                      "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 3), "best_GB/s": round(nbytes / (best * 1e-3) / 1e9, 1)}
@@ -737,8 +744,9 @@ def run_sweep(args):
     peaks = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = []
-    for log2n in range(20, 31, args.sweep_stride):
-        row = sweep_row(torch, lib, si, dev, peaks, flush, log2n, args.sweep_warmup, args.sweep_iters)
+    lo, hi = args.sweep_log2
+    for log2n in range(lo, hi + 1, args.sweep_stride):
+        row = sweep_row(torch, lib, si, dev, peaks, flush, log2n, args.sweep_warmup, args.sweep_iters, not args.sweep_no_graph)
         out.append(row)
         print(json.dumps(row), flush=True)
     return out
@@ -787,6 +795,10 @@ def main():
     ap.add_argument("--sweep-iters", type=int, default=100)
     ap.add_argument("--sweep-warmup", type=int, default=20)
     ap.add_argument("--sweep-stride", type=int, default=1)
+    ap.add_argument("--sweep-log2", type=int, nargs=2, default=[20, 30], metavar=("LO", "HI"),
+                    help="smallest and largest log2(elements) of --sweep")
+    ap.add_argument("--sweep-no-graph", action="store_true", help="--sweep: launch directly instead of replaying CUDA graphs")
+    ap.add_argument("--sweep-no-oracle", action="store_true", help="--sweep: skip the oracle rows")
     ap.add_argument("--shape", default=None, help="M,K,N override for profiling runs (not the benchmark workload)")
     args = ap.parse_args()
     if args.shape:
@@ -795,7 +807,8 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
-        run_sweep_oracle(args)
+        if not args.sweep_no_oracle:
+            run_sweep_oracle(args)
     elif args.stack:
         run_stack(args)
     elif args.probe:
