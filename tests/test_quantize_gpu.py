@@ -7,6 +7,7 @@ import pytest
 import torch
 
 import oracle
+import paper_2609_02846_b200 as lib
 from helpers import assert_same_quantization, lib_quantize, oracle_quantize
 import synth_inputs as si
 
@@ -24,17 +25,88 @@ def _amax(x):
 @pytest.mark.parametrize("rounding", ROUNDINGS)
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("shape", [(16, 16), (256, 256), (272, 4112), (1040, 208)])
-def test_quantize_matches_oracle(layout, rounding, dtype, shape):
+@pytest.mark.parametrize("with_stats", [True, False])
+def test_quantize_matches_oracle(layout, rounding, dtype, shape, with_stats):
+    """Both kernel families of every cell: with counters and, as the benchmark launches them, without."""
     rows, cols = shape
     x = si.channel_scaled_activation(rows, cols, seed=rows + cols, device=DEV, dtype=dtype)
     x[0, 0] = 0.0
     x[rows - 1, cols - 1] = -0.0
     g = _amax(x) * 0.37                                  # stale reference: some payloads clip
     want_t = layout == oracle.LAYOUT_2D
-    _, got = lib_quantize(x, layout, rounding, g, 448.0, seed=0xC0FFEE12345, want_t=want_t)
+    _, got = lib_quantize(x, layout, rounding, g, 448.0, seed=0xC0FFEE12345, want_t=want_t, with_stats=with_stats)
     want = oracle_quantize(x, layout, rounding, g, 448.0, seed=0xC0FFEE12345, want_t=want_t)
     assert_same_quantization(got, want)
     assert want["stats"]["payload_clipped"] > 0
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("with_stats", [True, False])
+def test_nonfinite_inputs_in_every_kernel_family(dtype, with_stats):
+    """NaN (either sign bit), +-Inf and -0 scattered over a tensor, alone in a block, next to the block maximum and in
+    whole blocks of NaN: NaN is ignored by the block maximum and encodes as +6, +-Inf saturates the block scale and
+    encodes as +-6, in every layout, under both roundings, with and without counters, and in the dual-layout call."""
+    rows, cols = 288, 544
+    x = si.heavy_tailed_gradient(rows, cols, seed=21, device=DEV, dtype=dtype)
+    neg_nan = torch.tensor([0xFFC1], dtype=torch.uint16).view(torch.bfloat16).to(DEV).to(dtype)[0] if dtype == torch.bfloat16 \
+        else torch.tensor([0xFFC00001], dtype=torch.uint32).view(torch.float32).to(DEV)[0]
+    x[0, 0] = float("nan"); x[0, 17] = neg_nan; x[5, 100] = float("inf"); x[6, 101] = float("-inf")
+    x[40, 32:48] = float("nan")                       # a whole row block of NaN
+    x[64:80, 200] = float("nan")                      # a whole column block of NaN
+    x[100, 300] = float("nan"); x[100, 301] = 1e30    # NaN next to a huge value
+    x[rows - 1, cols - 1] = float("nan"); x[rows - 1, 0] = -0.0
+    g = 1e-3
+    xn = si.to_numpy_bits(x)
+    for layout in LAYOUTS:
+        for rounding in ROUNDINGS:
+            _, got = lib_quantize(x, layout, rounding, g, seed=3, want_t=layout == oracle.LAYOUT_2D, with_stats=with_stats)
+            want = oracle.quantize(xn, layout, rounding, g, 448.0, 3, layout == oracle.LAYOUT_2D)
+            assert_same_quantization(got, want)
+    for rounding in ROUNDINGS:
+        g_dev = torch.tensor([g], dtype=torch.float32, device=DEV)
+        st = (torch.zeros(4, dtype=torch.int64, device=DEV), torch.zeros(4, dtype=torch.int64, device=DEV)) if with_stats else (None, None)
+        row, col = lib.quantize_dual(x, rounding, g_dev, seed_row=8, seed_col=9, stats_row=st[0], stats_col=st[1])
+        wr = oracle.quantize(xn, 0, rounding, g, 448.0, 8)
+        wc = oracle.quantize(xn, 1, rounding, g, 448.0, 9)
+        assert np.array_equal(row.payload.cpu().numpy(), wr["payload"]) and np.array_equal(row.scales.cpu().numpy(), wr["scales"])
+        assert np.array_equal(col.payload.cpu().numpy(), wc["payload"]) and np.array_equal(col.scales.cpu().numpy(), wc["scales"])
+        if with_stats:
+            assert dict(zip(oracle.STAT_NAMES, st[0].cpu().tolist())) == wr["stats"]
+            assert dict(zip(oracle.STAT_NAMES, st[1].cpu().tolist())) == wc["stats"]
+
+
+def test_tensor_beyond_2_to_the_35_elements_uses_64_bit_draw_counters():
+    """2^35 BF16 elements (64 GiB): the element index of a draw no longer fits 32 + 3 bits, so the kernels switch to
+    the generator's general routine.  Row bands and column bands far beyond index 2^32 * 8 are compared with the
+    oracle, which quantizes them as windows of the big tensor."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 110 << 30:
+        pytest.skip("needs about 100 GiB of free device memory")
+    rows, cols = 1 << 21, 1 << 14
+    chunk = si.heavy_tailed_gradient(1 << 14, cols, seed=77, device=DEV)            # 2^28 elements
+    x = torch.empty((rows, cols), dtype=torch.bfloat16, device=DEV)
+    for i in range(rows >> 14):
+        x[i << 14:(i + 1) << 14].copy_(chunk)
+        x[(i << 14) + 5, 7] = float(i + 1)                  # make the copies distinguishable
+    g = lib.sample_amax(x)
+    gv = g.item()
+    chunk_np = si.to_numpy_bits(chunk)
+    for rounding in ROUNDINGS:
+        q = lib.quantize(x, lib.LAYOUT_1D_ROW, rounding, g, seed=11)
+        for r0 in (0, (1 << 20) + 16, rows - 16):
+            band = si.to_numpy_bits(x[r0:r0 + 16])
+            o = oracle.quantize(band, 0, rounding, gv, 448.0, 11, window=(cols, r0, 0))
+            assert np.array_equal(q.payload[r0:r0 + 16].cpu().numpy(), o["payload"])
+            assert np.array_equal(q.scales[r0:r0 + 16].cpu().numpy(), o["scales"])
+        del q
+    q = lib.quantize(x, lib.LAYOUT_2D, lib.ROUND_SR, g, seed=12)
+    r0 = rows - 32
+    o = oracle.quantize(si.to_numpy_bits(x[r0:r0 + 32]), 2, 1, gv, 448.0, 12, window=(cols, r0, 0))
+    assert np.array_equal(q.payload[r0:r0 + 32].cpu().numpy(), o["payload"])
+    assert np.array_equal(q.scales[r0 // 16:r0 // 16 + 2].cpu().numpy(), o["scales"])
+    del q, x
+    torch.cuda.empty_cache()
+    assert lib.last_device_status() == 0
 
 
 @pytest.mark.parametrize("layout", [oracle.LAYOUT_1D_ROW, oracle.LAYOUT_1D_COL])
