@@ -124,20 +124,41 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_kernel(const __grid_
     const uint32_t kbpr = (uint32_t)(a.cols >> 4);
     const uint32_t nblocks = (uint32_t)a.rows * kbpr;          // the launcher guarantees < 2^32 - 2^16 blocks
     uint32_t sat = 0, rep = 0, clip = 0, nonf = 0;
-    // all lanes of a warp make the same number of trips (the scale bytes travel through shuffles)
-    for (uint32_t base = blockIdx.x * kRowThreads; base < nblocks; base += gridDim.x * kRowThreads) {
-        const uint32_t idx = base + threadIdx.x;
-        const bool live = idx < nblocks;
+    // Position of a block and (BF16) its 32 bytes.  The loads of the NEXT trip are issued before the current block is
+    // worked on, so that a warp's memory latency lies under its own arithmetic as well as under other warps'
+    // (measured: +5 % for round-to-nearest at 2^26 elements, neutral for stochastic rounding).
+    auto locate = [&](uint32_t base, uint32_t& idx, bool& live, uint32_t& row, uint32_t& kb) {
+        idx = base + threadIdx.x;
+        live = idx < nblocks;
         const uint32_t idc = live ? idx : 0;
         // blocks per row is a power of two for the usual widths: shift instead of divide
-        const uint32_t row = (kb_shift >= 0) ? (idc >> kb_shift) : (idc / kbpr);
-        const uint32_t kb = idc - row * kbpr;
+        row = (kb_shift >= 0) ? (idc >> kb_shift) : (idc / kbpr);
+        kb = idc - row * kbpr;
+    };
+    auto fetch = [&](uint32_t row, uint32_t kb, uint4& v0, uint4& v1) {
+        const uint16_t* p = reinterpret_cast<const uint16_t*>(a.x) + (int64_t)row * a.ld + kb * 16;
+        v0 = ldg_nc_v4(p);
+        v1 = ldg_nc_v4(p + 8);
+    };
+    const uint32_t stride = gridDim.x * kRowThreads;
+    uint32_t idx, row, kb, nidx = 0, nrow = 0, nkb = 0;
+    bool live, nlive = false;
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
+    locate(blockIdx.x * kRowThreads, nidx, nlive, nrow, nkb);
+    if (IS_BF16) fetch(nrow, nkb, n0, n1);
+    // all lanes of a warp make the same number of trips (the scale bytes travel through shuffles)
+    for (uint32_t base = blockIdx.x * kRowThreads; base < nblocks; base += stride) {
+        idx = nidx; live = nlive; row = nrow; kb = nkb;
+        const uint32_t idc = live ? idx : 0;
+        const uint4 v0 = n0, v1 = n1;
+        if (base + stride < nblocks) {
+            locate(base + stride, nidx, nlive, nrow, nkb);
+            if (IS_BF16) fetch(nrow, nkb, n0, n1);
+        }
 
         float f[16];
         float aB = 0.0f;
         if (IS_BF16) {
-            const uint16_t* p = reinterpret_cast<const uint16_t*>(a.x) + (int64_t)row * a.ld + kb * 16;
-            const uint4 v0 = ldg_nc_v4(p), v1 = ldg_nc_v4(p + 8);
             uint32_t raw[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
             uint32_t m = 0;
             if (kRawSanitize) {
@@ -226,11 +247,23 @@ __global__ void __launch_bounds__(kRowThreads) quantize_row_flat_kernel(const __
     if (blockIdx.x == 0 && threadIdx.x == 0 && a.decode_out) *a.decode_out = tab.tc[0].d;
 
     uint32_t sat = 0, rep = 0, clip = 0, nonf = 0;
-    for (uint32_t base = blockIdx.x * kRowThreads; base < nblocks; base += gridDim.x * kRowThreads) {
+    const uint32_t stride = gridDim.x * kRowThreads;
+    // the next trip's block is loaded before the current one is worked on (see quantize_row_kernel)
+    uint32_t nxt[8];
+    {
+        const uint32_t i0 = blockIdx.x * kRowThreads + threadIdx.x;
+        ldg_nc_v8(reinterpret_cast<const uint8_t*>(a.x) + (uint64_t)(i0 < nblocks ? i0 : 0) * 32, nxt);
+    }
+    for (uint32_t base = blockIdx.x * kRowThreads; base < nblocks; base += stride) {
         const uint32_t idx = base + threadIdx.x;
         const bool live = idx < nblocks;
         uint32_t raw[8];
-        ldg_nc_v8(reinterpret_cast<const uint8_t*>(a.x) + (uint64_t)(live ? idx : 0) * 32, raw);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) raw[q] = nxt[q];
+        if (base + stride < nblocks) {
+            const uint32_t in = idx + stride;
+            ldg_nc_v8(reinterpret_cast<const uint8_t*>(a.x) + (uint64_t)(in < nblocks ? in : 0) * 32, nxt);
+        }
         uint32_t m = 0;
 #pragma unroll
         for (int q = 0; q < 8; ++q) m = bf16x2_absmax(m, raw[q]);
