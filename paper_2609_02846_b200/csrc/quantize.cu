@@ -328,7 +328,7 @@ __device__ __forceinline__ void load_row8(const void* x, int64_t off, float f[8]
 // MODE 3: dual layout: MODE 0 plus the 1D_ROW quantization of the same register tile (a row block of 16 is this
 //         lane's 8 columns and lane ^ 1's): the tensor is read once for both operands of a backward pass.
 template <bool IS_BF16, int RND, bool STATS, int MODE, bool TILED, bool WANT_T>
-__global__ void __launch_bounds__(kTileThreads, (MODE == 3 && RND != 0) ? 1 : 2) quantize_tile_kernel(const __grid_constant__ QuantArgs a) {
+__global__ void __launch_bounds__(kTileThreads, 2) quantize_tile_kernel(const __grid_constant__ QuantArgs a) {
     constexpr bool SR = RND != 0, SMALL = RND == 1;
     static_assert(kTileThreads == 256, "one table entry per thread");
     constexpr bool kDual = MODE == 3;
