@@ -483,3 +483,37 @@ def test_current_scaling_call_equals_amax_then_quantize(layout, rounding):
     assert want["stats"]["scale_saturated"] == 0 and int(want["scales"].max()) == oracle.ue5m3_encode(np.float32(448.0))
     with pytest.raises(lib.Ue5m3Error):
         lib.quantize_current(x[:, :520], layout, rounding)          # 520 columns: not a multiple of 16, nothing is launched
+
+
+def test_seeded_sweep_over_shapes_strides_layouts_and_options():
+    """Sixty seeded cases over what the launchers branch on: BF16 / FP32, the three layouts, both roundings, counters
+    on and off, row-major and tiled scales, blocks of 16 and 32, contiguous and strided sources, power-of-two and
+    odd block counts per row, sources that do and do not start on a 32-byte boundary, stale and current references,
+    both targets.  Every byte and counter against the oracle."""
+    rng = np.random.default_rng(20260101)
+    for case in range(60):
+        block = 32 if rng.random() < 0.25 else 16
+        rows = int(rng.integers(1, 12)) * 32
+        cols = int(rng.integers(1, 40)) * 32
+        pad = int(rng.choice([0, 0, 8, 16, 72]))
+        off = int(rng.choice([0, 0, 8])) if pad >= 8 else 0
+        dtype = torch.bfloat16 if rng.random() < 0.7 else torch.float32
+        layout = int(rng.integers(0, 3))
+        rounding = int(rng.integers(0, 2))
+        tiled = layout != oracle.LAYOUT_2D and rng.random() < 0.3
+        with_stats = bool(rng.random() < 0.4)
+        T = 2048.0 if rng.random() < 0.3 else 448.0
+        big = si.heavy_tailed_gradient(rows, cols + pad, seed=1000 + case, device=DEV, dtype=dtype) if case % 2 else \
+            si.channel_scaled_activation(rows, cols + pad, seed=1000 + case, device=DEV, dtype=dtype)
+        x = big[:, off:off + cols]
+        g = _amax(x) * float(rng.choice([1.0, 0.3, 4.0]))
+        seed = int(rng.integers(0, 2 ** 62))
+        want_t = layout == oracle.LAYOUT_2D and rng.random() < 0.5
+        _, got = lib_quantize(x, layout, rounding, g, T, seed=seed, want_t=want_t, with_stats=with_stats,
+                              scale_layout=1 if tiled else 0, block=block)
+        want = oracle.quantize(si.to_numpy_bits(big)[:, off:off + cols], layout, rounding, g, T, seed, want_t, block=block)
+        try:
+            assert_same_quantization(got, want)
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: rows={rows} cols={cols} pad={pad} off={off} {dtype} layout={layout} rounding={rounding} "
+                                 f"tiled={tiled} stats={with_stats} T={T} block={block}: {e}") from e
