@@ -59,6 +59,8 @@ def _load() -> C.CDLL:
         L.ue5m3_quantize_dual.argtypes = [vp, ci, i64, i64, i64, ci, vp, f32, f32, u64, u64, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_gemm.restype = ci
         L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
+        L.ue5m3_gemm_native.restype = ci
+        L.ue5m3_gemm_native.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp, vp]
         L.ue5m3_gemm_probe_matched.restype = ci
         L.ue5m3_gemm_probe_matched.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, ci, ci, vp, ci, i64, vp]
         L.ue5m3_gemm_stall_selftest.restype = ci
@@ -280,6 +282,26 @@ def gemm(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dty
                                   _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
                                   _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
                                   _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)), "ue5m3_gemm")
+    return out
+
+
+def gemm_native(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
+                out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The product of `gemm` on the tensor core's FP4 path (ue5m3_gemm_native).  `workspace` (4 x int32, device) receives
+    the code ranges of the two operands' scales; `out` is left untouched when an operand has no UE4M3 window."""
+    Mo, No, Kc = a.R, b.R, a.Kc
+    if b.Kc != Kc:
+        raise ValueError(f"contraction sizes differ: {Kc} vs {b.Kc}")
+    if out is None:
+        out = torch.empty((Mo, No), dtype=out_dtype, device=a.payload.device)
+    if workspace is None:
+        workspace = torch.empty(4, dtype=torch.int32, device=out.device)
+    with torch.cuda.device(out.device):
+        _check(_load().ue5m3_gemm_native(op, Mo, No, Kc,
+                                         _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
+                                         _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
+                                         _dev_ptr(out), _dtype_code(out), out.stride(0), _dev_ptr(workspace), _stream(out)),
+               "ue5m3_gemm_native")
     return out
 
 

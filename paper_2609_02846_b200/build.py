@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libue5m3.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "gemm_probe.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "gemm_probe.cu", "gemm_native.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

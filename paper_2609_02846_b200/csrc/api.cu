@@ -214,6 +214,27 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
     return launch_gemm(g, di.sms, (cudaStream_t)stream);
 }
 
+int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+                      int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+                      int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, int32_t* workspace,
+                      void* stream) {
+    const ApiRange range_("ue5m3_gemm_native");
+    const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
+                                    b_scale_mode, b_decode, out, out_dtype, ldo, 256);
+    if (bad != UE5M3_OK) return bad;
+    if (!workspace) return UE5M3_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return UE5M3_ERR_ALIGN;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
+               out, out_dtype, ldo};
+    if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
+    const int r = launch_scale_range(g, workspace, di.sms, (cudaStream_t)stream);
+    if (r != UE5M3_OK) return r;
+    return launch_gemm_native(g, workspace, di.sms, (cudaStream_t)stream);
+}
+
 int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
                              int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
                              int b_scale_mode, const float* b_decode, int cross_rounding, int grid_denominator,
@@ -264,7 +285,8 @@ int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t k
 int ue5m3_last_device_status(void) {
     const int a = read_and_clear_device_status();
     const int b = read_and_clear_probe_status();
-    return a != UE5M3_OK ? a : b;
+    const int c = read_and_clear_native_status();
+    return a != UE5M3_OK ? a : (b != UE5M3_OK ? b : c);
 }
 
 }  // extern "C"

@@ -57,6 +57,12 @@ cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, in
 cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, cudaStream_t st);
 int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st);   // returns a UE5M3_* status
 int read_and_clear_device_status();                                  // synchronises the device
+// The same product on the tensor core's FP4 path (gemm_native.cu).  `range` is four words of device workspace:
+// launch_scale_range fills them, the kernel reads them and does nothing when an operand's scale codes have no window.
+bool native_eligible(const GemmArgs& g);
+int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st);
+int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st);
+int read_and_clear_native_status();                                  // synchronises the device
 // The same operands under the output model of Section 6.2 (gemm_probe.cu).
 int launch_gemm_probe(const GemmArgs& g, int cross_rne, int grid_denominator, int num_sms, cudaStream_t st);
 int read_and_clear_probe_status();                                   // synchronises the device
