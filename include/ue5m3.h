@@ -174,8 +174,19 @@ UE5M3_API int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_
  * dW = dY^T X; Section 6.1: y = sum_k a_k b_k on the decoded operands, the tensor-scale product
  * applied after accumulation):
  *     C[Mo, No] = (d_A * d_B) * sum_k (s_hat q)_A[m, k] * (s_hat q)_B[n, k]
- * Both operands are K-major.  Every E2M1 x UE5M3 product (times 2^-4) is exact in FP16, subnormals
- * included; products of two such values are accumulated in FP32 on the tensor cores.  `op` only names the role of the call:
+ * Both operands are K-major.  The call picks one of two kernels on the device, without a host round trip:
+ *   native   the tensor core's own block-scaled FP4 instruction (E2M1 operands, one 8-bit scale per 16 elements).  Its
+ *            scale format is UE4M3 (bias 7); a normal UE5M3 code c and the UE4M3 code c - 8k denote values that differ
+ *            by the constant factor 2^(k-8), so when all non-zero scale codes of an operand fit one window
+ *            8 <= c - 8k <= 126 (largest / smallest block scale < 2^14.8) the product is the native one on shifted
+ *            codes with the two factors folded into d_A * d_B.  Needs Kc % 256 == 0.
+ *   FP16     every E2M1 x UE5M3 product (times 2^-4) is exact in FP16, subnormals included; the operands are
+ *            reconstructed in the kernel and multiplied as FP16.  Used when an operand has no window (UE5M3
+ *            subnormal codes 1..7 included) or Kc = 128 * odd.
+ * Both accumulate in FP32 on the tensor cores and meet the same error bound; their results may differ in the last bits.
+ * Three launches per call when Kc % 256 == 0: a reduction of the scale bytes to their code range (four words of a
+ * per-device workspace ring, allocated at the first call on a device), then both kernels, one of which returns at once.
+ * `op` only names the role of the call:
  *     FPROP  A = X  (1D_ROW),        B = W   (2D payload, scales)          Mo = tokens, No = out, Kc = in
  *     DGRAD  A = dY (1D_ROW, SR),    B = W^T (2D payload_t, scales_t)      Mo = tokens, No = in,  Kc = out
  *     WGRAD  A = dY^T (1D_COL, SR),  B = X^T (1D_COL)                      Mo = out,    No = in,  Kc = tokens
@@ -198,8 +209,18 @@ UE5M3_API int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
                void* out, int out_dtype, int64_t ldo, void* stream);
 
 /*
- * The product of ue5m3_gemm on the tensor core's own FP4 block-scaled path (draft).
+ * The two kernels of ue5m3_gemm on their own (same arguments, layouts, alignment and errors).
+ * ue5m3_gemm_fp16: always the FP16 reconstruction kernel; no workspace is touched.
+ * ue5m3_gemm_native: the range reduction and the native FP4 kernel only.  Kc must be a multiple of 256
+ * (UE5M3_ERR_SHAPE).  `workspace`: device, 4 x int32, 16-byte aligned, owned by the caller; after the call it holds
+ * {largest code of A, 255 - smallest non-zero code of A, the same two for B}.  When an operand has no window the
+ * kernel returns at once and `out` is left untouched: the caller can tell from the workspace.
+ * The paper has no counterpart of the split: its Section 5.3 names the three products, not how a device computes them.
  */
+UE5M3_API int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc,
+               const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
+               const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
+               void* out, int out_dtype, int64_t ldo, void* stream);
 UE5M3_API int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc,
                const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
                const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
@@ -231,7 +252,8 @@ UE5M3_API int ue5m3_gemm_probe_matched(int op, int64_t Mo, int64_t No, int64_t K
  * consumer's first wait expires, all roles drain, tensor memory is released and the kernel returns.  `out` is not
  * written.  Afterwards ue5m3_last_device_status() returns UE5M3_ERR_TIMEOUT once and UE5M3_OK from then on, and the
  * context stays usable.
- *   which               0 = the kernel of ue5m3_gemm, 1 = the kernel of ue5m3_gemm_probe_matched.
+ *   which               0 = the FP16 kernel of ue5m3_gemm, 1 = the kernel of ue5m3_gemm_probe_matched, 2 = the native FP4
+ *                       kernel of ue5m3_gemm (the operands must then have scale windows, see ue5m3_gemm).
  *   wait_limit_cycles   1000 .. 4e9 (about 2e6 is one millisecond).
  * All other arguments, and their checks and errors, are those of ue5m3_gemm (Kc a multiple of 256).
  */

@@ -59,6 +59,8 @@ def _load() -> C.CDLL:
         L.ue5m3_quantize_dual.argtypes = [vp, ci, i64, i64, i64, ci, vp, f32, f32, u64, u64, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_gemm.restype = ci
         L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
+        L.ue5m3_gemm_fp16.restype = ci
+        L.ue5m3_gemm_fp16.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_native.restype = ci
         L.ue5m3_gemm_native.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp, vp]
         L.ue5m3_gemm_probe_matched.restype = ci
@@ -285,6 +287,32 @@ def gemm(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dty
     return out
 
 
+def scale_window(cmin: int, cmax: int) -> Optional[int]:
+    """The rule by which ue5m3_gemm decides between its two kernels, restated on the host: the shift k with
+    8 <= c - 8k <= 126 for all codes cmin..cmax of an operand (then UE5M3 code c and UE4M3 code c - 8k denote values
+    that differ by exactly 2^(k - 8)), or None when the operand has no such window."""
+    if cmin < 8 or cmax > 0xF7 or cmin > cmax:
+        return None
+    k = (cmin - 8) >> 3
+    return k if cmax - 8 * k <= 126 else None
+
+
+def gemm_fp16(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
+              out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The product of `gemm`, always through the FP16 reconstruction kernel (ue5m3_gemm_fp16)."""
+    Mo, No, Kc = a.R, b.R, a.Kc
+    if b.Kc != Kc:
+        raise ValueError(f"contraction sizes differ: {Kc} vs {b.Kc}")
+    if out is None:
+        out = torch.empty((Mo, No), dtype=out_dtype, device=a.payload.device)
+    with torch.cuda.device(out.device):
+        _check(_load().ue5m3_gemm_fp16(op, Mo, No, Kc,
+                                       _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
+                                       _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
+                                       _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)), "ue5m3_gemm_fp16")
+    return out
+
+
 def gemm_native(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
                 out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
     """The product of `gemm` on the tensor core's FP4 path (ue5m3_gemm_native).  `workspace` (4 x int32, device) receives
@@ -327,7 +355,8 @@ def gemm_probe_matched(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dt
 
 def gemm_stall_selftest(which: int, a: QuantizedOperand, b: QuantizedOperand, out: torch.Tensor,
                         wait_limit_cycles: int = 2_000_000) -> None:
-    """ue5m3_gemm_stall_selftest: launches the chosen GEMM kernel (0: ue5m3_gemm, 1: ue5m3_gemm_probe_matched) with its
+    """ue5m3_gemm_stall_selftest: launches the chosen GEMM kernel (0: FP16 kernel of ue5m3_gemm, 1: ue5m3_gemm_probe_matched,
+    2: native FP4 kernel of ue5m3_gemm) with its
     copy producer switched off and every wait bounded by `wait_limit_cycles`; `out` is left untouched and
     `last_device_status()` then reports the timeout once."""
     with torch.cuda.device(out.device):

@@ -211,7 +211,31 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
-    return launch_gemm(g, di.sms, (cudaStream_t)stream);
+    if (!native_eligible(g)) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
+    // Three launches, one of which does the product: the scale-code ranges, the native FP4 kernel (works when both
+    // operands have a UE4M3 window) and the FP16 kernel (works when they do not).
+    int* ws = native_workspace();
+    if (!ws) return UE5M3_ERR_CUDA;
+    int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
+    if (r != UE5M3_OK) return r;
+    r = launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
+    if (r != UE5M3_OK) return r;
+    return launch_gemm(g, ws, di.sms, (cudaStream_t)stream);
+}
+
+int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+                    int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+                    int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
+    const ApiRange range_("ue5m3_gemm_fp16");
+    const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
+                                    b_scale_mode, b_decode, out, out_dtype, ldo, 128);
+    if (bad != UE5M3_OK) return bad;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
+               out, out_dtype, ldo};
+    return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
 }
 
 int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
@@ -259,7 +283,7 @@ int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, con
                                int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo,
                                int64_t wait_limit_cycles, void* stream) {
     const ApiRange range_("ue5m3_gemm_stall_selftest");
-    if (which != 0 && which != 1) return UE5M3_ERR_INVALID_ARG;
+    if (which != 0 && which != 1 && which != 2) return UE5M3_ERR_INVALID_ARG;
     if (wait_limit_cycles < 1000 || wait_limit_cycles > 4000000000LL) return UE5M3_ERR_INVALID_ARG;
     const int bad = check_gemm_args(UE5M3_FPROP, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
                                     b_scale_mode, b_decode, out, out_dtype, ldo, 256);
@@ -271,7 +295,15 @@ int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, con
                out, out_dtype, ldo};
     g.wait_limit_cycles = wait_limit_cycles;
     g.stall_producer = 1;
-    return which == 0 ? launch_gemm(g, di.sms, (cudaStream_t)stream) : launch_gemm_probe(g, 0, 0, di.sms, (cudaStream_t)stream);
+    if (which == 2) {
+        // the native kernel: its workspace is filled by the range kernel as in ue5m3_gemm (the operands must have windows)
+        int* ws = native_workspace();
+        if (!ws) return UE5M3_ERR_CUDA;
+        const int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
+        if (r != UE5M3_OK) return r;
+        return launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
+    }
+    return which == 0 ? launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream) : launch_gemm_probe(g, 0, 0, di.sms, (cudaStream_t)stream);
 }
 
 int ue5m3_unswizzle_scales(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, void* stream) {

@@ -38,6 +38,7 @@
 #include "../../include/ue5m3.h"
 #include "launch.h"
 #include "tcgen05.cuh"
+#include "window.cuh"
 
 namespace ue5m3 {
 
@@ -87,6 +88,7 @@ struct GemmParams {
     const uint8_t* a_scales;
     const uint8_t* b_scales;
     int a_direct, b_direct;
+    const int* range;             // not null: the native FP4 kernel ran first; this one works only if it could not
 };
 
 // Tile order: groups of kRasterGroup tile rows, and inside a group column by column.  The tiles that are
@@ -114,6 +116,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
             const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
+    if (p.range) {
+        int ka, kb;
+        if (native_windows(p.range, ka, kb)) return;        // uniform over the grid
+    }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -444,7 +450,7 @@ bool make_scale_map(CUtensorMap* m, const uint8_t* scales, int mode, int64_t R, 
 
 }  // namespace
 
-int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
+int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st) {
     // CTA pairs that can be resident at once, per device; asked once per device, concurrent first calls serialised
     static int resident_pairs[64];
     static std::once_flag asked[64];
@@ -491,6 +497,7 @@ int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st) {
     p.stall_producer = g.stall_producer;
     p.a_scales = g.a_scales; p.b_scales = g.b_scales;
     p.a_direct = a_direct ? 1 : 0; p.b_direct = b_direct ? 1 : 0;
+    p.range = range;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int max_pairs = resident_pairs[dev];
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;

@@ -14,20 +14,26 @@
 // The window is found on the device: scale_range_kernel reduces both operands' scale bytes to their largest and
 // smallest non-zero code (four words of workspace), gemm_native_kernel reads them and returns at once when an
 // operand has no window (subnormal UE5M3 codes included); the caller then runs the FP16 path, whose kernel
-// evaluates the same predicate the other way round.  A code of 0 (rows beyond the operand, which the copy engine
-// fills with zeros) stays 0.
+// evaluates the same predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.
 //
-// Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 4 stages):
-//   warp 0      copies: packed A rows (128), packed B rows (this CTA's 128), scale bytes of A's rows and of all 256 B rows
+// Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 6 payload stages of 32 KB):
+//   warp 0      copies: packed A rows (128) and packed B rows (this CTA's 128) of a stage
 //   warp 1      (leader CTA) per stage 12 scale copies shared memory -> tensor memory and 4 MMAs of K = 64
 //   warp 2      tensor-memory allocation
+//   warp 3      relay: tells the leader CTA that this CTA's copy of a stage has landed
 //   warps 4-7   epilogue: accumulator -> alpha -> BF16 / FP32 -> shared memory -> bulk tensor store
-//   warps 8-11  scale bytes: window shift and re-layout
+//   warps 8-11  scale bytes: read from global memory four stages ahead (registers), window shift, re-layout into a
+//               ring of two stages in shared memory
+// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 192..447, the
+// scales of the stage in flight in columns 448..495.  Two whole accumulators do not fit beside the scales, so the
+// two overlap in 64 columns: the epilogue drains those 64 first and hands them back, and the MMAs of the next
+// tile run while the other 192 columns are still being stored.
 // Every wait is bounded (SM clocks); on a time-out the role sets the status word, the other roles see the abort
 // flag, in-flight copies and MMAs are drained and the kernel returns.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdint>
+#include <atomic>
 #include <mutex>
 #include "../../include/ue5m3.h"
 #include "launch.h"
@@ -46,34 +52,38 @@ constexpr int BNH = 128;                    // B rows staged by each CTA
 constexpr int KCHUNK = 256;                 // K per stage
 constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks)
 constexpr int MMAS = KCHUNK / KMMA;
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;                   // payload stages
+constexpr int SF_STAGES = 2;                // converted-scale stages
+constexpr int PF = 4;                       // stages the scale bytes are read ahead (registers)
 constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;
 constexpr int NUM_THREADS = 32 * (CONV_WARP0 + CONV_WARPS);
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;           // 16384
 constexpr int PK_B_BYTES = BNH * KCHUNK / 2;          // 16384
-constexpr int RAW_A_BYTES = BM * (KCHUNK / 16);       // 2048: [row][16 block columns]
-constexpr int RAW_B_BYTES = BN * (KCHUNK / 16);       // 4096: all 256 B rows of the tile
-constexpr int SF_A_BYTES = RAW_A_BYTES;               // [mma][32 lanes][4 row groups][4 blocks]
-constexpr int SF_B_BYTES = RAW_B_BYTES;               // [mma][half][32 lanes][4 row groups][4 blocks]
-constexpr int STAGE_BYTES = PK_A_BYTES + PK_B_BYTES + RAW_A_BYTES + RAW_B_BYTES + SF_A_BYTES + SF_B_BYTES;   // 45056
-constexpr int OFF_B = PK_A_BYTES, OFF_RAW_A = OFF_B + PK_B_BYTES, OFF_RAW_B = OFF_RAW_A + RAW_A_BYTES;
-constexpr int OFF_SF_A = OFF_RAW_B + RAW_B_BYTES, OFF_SF_B = OFF_SF_A + SF_A_BYTES;
-constexpr int SMEM_TILES = STAGES * STAGE_BYTES;      // 180224
-constexpr int SMEM_EPI = SMEM_TILES + 1024;           // barriers in between
+constexpr int STAGE_BYTES = PK_A_BYTES + PK_B_BYTES;  // 32768
+constexpr int SF_A_BYTES = BM * (KCHUNK / 16);        // 2048: [mma][32 lanes][4 row groups][4 blocks]
+constexpr int SF_B_BYTES = BN * (KCHUNK / 16);        // 4096: [mma][half][32 lanes][4 row groups][4 blocks]
+constexpr int SF_STAGE_BYTES = SF_A_BYTES + SF_B_BYTES;
+constexpr int SMEM_SF = STAGES * STAGE_BYTES;         // 196608
+constexpr int SMEM_BARS = SMEM_SF + SF_STAGES * SF_STAGE_BYTES;   // 208896
+constexpr int SMEM_EPI = SMEM_BARS + 1024;
 constexpr int EPI_WARP_BYTES = 4096;
-constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;
-constexpr int TMEM_ACC_COL = 0, TMEM_SFA_COL = 256, TMEM_SFB_COL = TMEM_SFA_COL + STAGES * 4 * MMAS;   // 256, 320
+constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 227328
+constexpr int TMEM_ACC_ODD = 192;                     // accumulator base column of odd tiles (even tiles: 0)
+constexpr int TMEM_SFA_COL = 448, TMEM_SFB_COL = 464; // two half-stage slots each: 2 x 8 and 2 x 16 columns
 
 struct NativeParams {
     int64_t Mo, No, Kc;
     const float* a_decode;
     const float* b_decode;
     const int* range;             // {max A, 255 - min nonzero A, max B, 255 - min nonzero B}
+    const uint8_t* a_scales;
+    const uint8_t* b_scales;
     int out_bf16;
     int a_mode, b_mode;
     int tiles_m, tiles_n;
     long long wait_limit;
+    int stall_producer;           // self-test: no copy is issued, so every consumer wait runs out
 };
 
 constexpr int kRasterGroup = 8;
@@ -94,19 +104,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // N = 256, M = 256 (two CTAs), K = 64.
 constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 
-__device__ __forceinline__ void umma_fp4_block16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa,
-                                                 uint32_t sfb, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate) : "memory");
-}
-// 32 rows x 16 bytes of shared memory (in both CTAs of the pair, at the same offset) -> 4 columns of lanes 0..31 of
-// every lane quarter of each CTA's tensor memory.
-__device__ __forceinline__ void tmem_cp_32x128b(uint32_t taddr, uint64_t sdesc) {
-    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
 // Descriptor of 32 rows of 16 bytes stored back to back: no swizzle, 8-row groups 128 bytes apart.
 __device__ __forceinline__ uint64_t sf_smem_desc(uint32_t saddr) {
     uint64_t d = 0;
@@ -116,10 +113,29 @@ __device__ __forceinline__ uint64_t sf_smem_desc(uint32_t saddr) {
     d |= (uint64_t)1 << 46;
     return d;
 }
-
-}  // namespace
-
-namespace {
+// The scale copy and the MMA take their 64-bit shared-memory descriptors as halves: the upper halves are constants of
+// the kernel and the lower halves differ only in the start-address field, so the issuing thread (one thread per CTA
+// pair, every instruction of it on the critical path) adds small constants instead of rebuilding descriptors.
+// Copy: 32 rows x 16 bytes of shared memory (in both CTAs of the pair, at the same offset) -> 4 columns of lanes
+// 0..31 of every lane quarter of each CTA's tensor memory.
+__device__ __forceinline__ void tmem_cp_32x128b(uint32_t taddr, uint32_t lo, uint32_t hi) {
+    asm volatile("{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\ttcgen05.cp.cta_group::2.32x128b.warpx4 [%0], d;\n\t}"
+                 ::"r"(taddr), "r"(lo), "r"(hi) : "memory");
+}
+__device__ __forceinline__ void umma_fp4_block16(uint32_t tmem_d, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc,
+                                                 uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %7, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], da, db, %4, [%5], [%6], p;\n\t}"
+        ::"r"(tmem_d), "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
 
 // ----------------------------------------------------------------------------- range of the scale codes
 __global__ void __launch_bounds__(256) scale_range_kernel(const uint8_t* __restrict__ a, int64_t na, const uint8_t* __restrict__ b,
@@ -159,7 +175,6 @@ __global__ void __launch_bounds__(256) scale_range_kernel(const uint8_t* __restr
 // ----------------------------------------------------------------------------- kernel
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                   const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
                    const __grid_constant__ CUtensorMap map_out, const NativeParams p) {
     int ka, kb;
     if (!native_windows(p.range, ka, kb)) return;            // uniform over the grid: the FP16 kernel does this product
@@ -167,30 +182,38 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t bar_base = smem_base + SMEM_TILES;
-    const uint32_t pk_full = bar_base, pk_empty = bar_base + 32, sf_full = bar_base + 64;
-    const uint32_t acc_full = bar_base + 96, acc_empty = bar_base + 104, drain_bar = bar_base + 112;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_TILES + 120);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_TILES + 128);
+    const uint32_t bar_base = smem_base + SMEM_BARS;
+    // barriers (8 bytes each)
+    const uint32_t pk_full = bar_base, pk_empty = bar_base + 64, pk_ready = bar_base + 128;
+    const uint32_t sf_full = bar_base + 192, sf_empty = bar_base + 256;
+    const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 344);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 352);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int kchunks = (int)(p.Kc / KCHUNK);
+    const int my_tiles = pair < num_tiles ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
+    const uint32_t total = (uint32_t)my_tiles * (uint32_t)kchunks;       // stages this CTA pair works through
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(pk_full + 8 * s, 1);
             mbar_init(pk_empty + 8 * s, 1);
+            mbar_init(pk_ready + 8 * s, 2);                    // the leader's copy collects both CTAs' relays
+        }
+        for (int s = 0; s < SF_STAGES; ++s) {
             mbar_init(sf_full + 8 * s, 2 * CONV_WARPS);        // the leader's copy collects both CTAs' warps
+            mbar_init(sf_empty + 8 * s, 1);
         }
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 8);
         mbar_init(drain_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        prefetch_tmap(&map_a); prefetch_tmap(&map_b); prefetch_tmap(&map_as); prefetch_tmap(&map_bs); prefetch_tmap(&map_out);
+        prefetch_tmap(&map_a); prefetch_tmap(&map_b); prefetch_tmap(&map_out);
     }
     if (warp == 2) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
@@ -203,10 +226,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         // ------------------------------------------------------------------ copies
         if (lane == 0) {
             uint32_t it = 0;
-            const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + (p.a_mode == UE5M3_SCALE_2D ? BM : 16 * BM) +
-                                      (p.b_mode == UE5M3_SCALE_2D ? BN : 16 * BN);
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            for (int tile = pair; tile < num_tiles && ok && !p.stall_producer; tile += num_pairs) {
                 int tm, tn;
                 tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
                 const int mb = tm * 2 + (int)rank, nh = tn * 2 + (int)rank;
@@ -214,47 +235,62 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     if (!mbar_wait(pk_empty + 8 * s, ph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                     const uint32_t st = smem_base + s * STAGE_BYTES, full = pk_full + 8 * s;
-                    mbar_expect_tx(full, tx_bytes);
+                    mbar_expect_tx(full, STAGE_BYTES);
                     tma_load_2d(st, &map_a, full, kc * (KCHUNK / 2), mb * BM);
-                    tma_load_2d(st + OFF_B, &map_b, full, kc * (KCHUNK / 2), nh * BNH);
-                    if (p.a_mode == UE5M3_SCALE_2D) tma_load_2d(st + OFF_RAW_A, &map_as, full, kc * 16, mb * (BM / 16));
-                    else tma_load_2d(st + OFF_RAW_A, &map_as, full, kc * 16, mb * BM);
-                    if (p.b_mode == UE5M3_SCALE_2D) tma_load_2d(st + OFF_RAW_B, &map_bs, full, kc * 16, tn * (BN / 16));
-                    else tma_load_2d(st + OFF_RAW_B, &map_bs, full, kc * 16, tn * BN);
+                    tma_load_2d(st + PK_A_BYTES, &map_b, full, kc * (KCHUNK / 2), nh * BNH);
                 }
             }
+            // let the copies still in flight land before the CTA's shared memory goes away (every one of them was
+            // issued, so it completes: this wait ignores the abort flag)
             for (uint32_t back = 0; back < STAGES && back < it; ++back) {
                 const uint32_t j = it - 1 - back;
                 mbar_wait_drain(pk_full + 8 * (j % STAGES), (j / STAGES) & 1, &g_native_status, p.wait_limit);
             }
         }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ relay: this CTA's stage has landed
+        if (lane == 0) {
+            for (uint32_t it = 0; it < total; ++it) {
+                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                if (!mbar_wait(pk_full + 8 * s, ph, abort_flag, p.wait_limit)) break;
+                mbar_arrive_cluster(pk_ready + 8 * s, 0);
+            }
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
         if (lane == 0 && rank == 0) {
-            uint32_t it = 0, tl = 0;
+            uint32_t tl = 0;
             bool ok = true;
+            // descriptor halves: payload (128-byte swizzle) and scales (no swizzle); only the start address moves
+            const uint64_t d_pk = umma_smem_desc(smem_base), d_sf = sf_smem_desc(smem_base + SMEM_SF);
+            const uint32_t pk_lo0 = (uint32_t)d_pk, pk_hi = (uint32_t)(d_pk >> 32);
+            const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
+            const uint32_t sfa0 = tmem_base + TMEM_SFA_COL, sfb0 = tmem_base + TMEM_SFB_COL;
+            uint32_t s = 0, ph = 0, f = 0, fph = 0;       // payload stage and its phase, scale stage and its phase
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
                 if (!mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t tmem_d = tmem_base + TMEM_ACC_COL;
-                for (int kc = 0; kc < kchunks; ++kc, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                    if (!mbar_wait(sf_full + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
+                const uint32_t tmem_d = tmem_base + ((tl & 1) ? TMEM_ACC_ODD : 0);
+                for (int kc = 0; kc < kchunks; ++kc) {
+                    if (!mbar_wait(sf_full + 8 * f, fph, abort_flag, p.wait_limit)) { ok = false; break; }
+                    if (!mbar_wait(pk_ready + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t st = smem_base + s * STAGE_BYTES;
-                    const uint32_t sfa = tmem_base + TMEM_SFA_COL + s * (4 * MMAS), sfb = tmem_base + TMEM_SFB_COL + s * (8 * MMAS);
+                    const uint32_t a_lo = pk_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (PK_A_BYTES >> 4);
+                    const uint32_t sf_lo = sf_lo0 + f * (SF_STAGE_BYTES >> 4), sfb_lo = sf_lo + (SF_A_BYTES >> 4);
 #pragma unroll
                     for (int j = 0; j < MMAS; ++j) {
-                        tmem_cp_32x128b(sfa + 4 * j, sf_smem_desc(st + OFF_SF_A + j * 512));
-                        tmem_cp_32x128b(sfb + 8 * j, sf_smem_desc(st + OFF_SF_B + j * 1024));
-                        tmem_cp_32x128b(sfb + 8 * j + 4, sf_smem_desc(st + OFF_SF_B + j * 1024 + 512));
+                        // MMA j of a stage has scale columns of its own, so a copy never touches columns an MMA still
+                        // in flight reads (copies and MMAs of one thread execute in issue order)
+                        const uint32_t sfa = sfa0 + 4 * j, sfb = sfb0 + 8 * j;
+                        tmem_cp_32x128b(sfa, sf_lo + j * (512 >> 4), sf_hi);
+                        tmem_cp_32x128b(sfb, sfb_lo + j * (1024 >> 4), sf_hi);
+                        tmem_cp_32x128b(sfb + 4, sfb_lo + j * (1024 >> 4) + (512 >> 4), sf_hi);
+                        umma_fp4_block16(tmem_d, a_lo + 2 * j, b_lo + 2 * j, pk_hi, kInstrDesc, sfa, sfb, (kc | j) != 0 ? 1u : 0u);
                     }
-                    const uint64_t ad = umma_smem_desc(st), bd = umma_smem_desc(st + OFF_B);
-#pragma unroll
-                    for (int j = 0; j < MMAS; ++j)
-                        umma_fp4_block16(tmem_d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), kInstrDesc, sfa + 4 * j, sfb + 8 * j,
-                                         (kc | j) != 0 ? 1u : 0u);
-                    umma_commit_pair(pk_empty + 8 * s);        // both CTAs may refill this stage
+                    umma_commit_pair(pk_empty + 8 * s);        // both CTAs may refill this payload stage
+                    umma_commit_pair(sf_empty + 8 * f);        // ... and this scale stage
+                    if (++s == STAGES) { s = 0; ph ^= 1; }
+                    if (++f == SF_STAGES) { f = 0; fph ^= 1; }
                 }
                 if (ok) umma_commit_pair(acc_full);
             }
@@ -277,17 +313,22 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             if (!mbar_wait(acc_full, tl & 1, abort_flag, p.wait_limit)) { ok = false; break; }
             tc_fence_after();
             const int row0 = mb * BM + q * 32, col0 = nb * BN;
+            const uint32_t odd = tl & 1;
+            const uint32_t acc = tmem_base + ((uint32_t)(q * 32) << 16) + (odd ? TMEM_ACC_ODD : 0);
+            // The 64 columns both accumulators share (the last 64 of an even tile, the first 64 of an odd one) are
+            // read first; once every epilogue warp of the pair has them in registers the next tile's MMAs may start.
             if (p.out_bf16) {
 #pragma unroll 1
-                for (int c = 0; c < BN / 64; ++c) {
+                for (int i = 0; i < BN / 64; ++i) {
+                    const int c = odd ? i : ((i + BN / 64 - 1) & (BN / 64 - 1));
                     uint8_t* mine = stage_gen + lane * 128;
                     const int sw = lane & 7;
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         uint32_t r[32];
-                        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_ACC_COL + c * 64 + half * 32, r);
+                        tmem_ld32(acc + c * 64 + half * 32, r);
                         tmem_ld_wait();
-                        if (c == BN / 64 - 1 && half == 1) {
+                        if (i == 0 && half == 1) {
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -312,11 +353,12 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 }
             } else {
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int i = 0; i < BN / 32; ++i) {
+                    const int c = odd ? i : ((i + BN / 32 - 2) & (BN / 32 - 1));
                     uint32_t r[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + TMEM_ACC_COL + c * 32, r);
+                    tmem_ld32(acc + c * 32, r);
                     tmem_ld_wait();
-                    if (c == BN / 32 - 1) {
+                    if (i == 1) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -339,32 +381,72 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (lane == 0) tma_store_wait_all();
     } else if (warp >= CONV_WARP0) {
         // ------------------------------------------------------------------ scale bytes: window shift and re-layout
-        const int g = warp - CONV_WARP0;               // row group (32 rows) of this warp; lane = row inside the group
-        const int row = g * 32 + lane;
+        // Lane l of warp w handles row g * 32 + dp of A and of both B halves, with dp = 8 w + l / 4 and g = l % 4: the
+        // words a warp stores (index 4 dp + g inside a 512-byte block of 128 rows) are then 32 consecutive ones.
+        const int cw = warp - CONV_WARP0;
+        const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);
         const uint32_t da = (uint32_t)((8 * ka) & 0xFF) * 0x01010101u, db = (uint32_t)((8 * kb) & 0xFF) * 0x01010101u;
-        const int a_raw = (p.a_mode == UE5M3_SCALE_2D ? (row >> 4) : row) * 16;
-        const int b_raw0 = (p.b_mode == UE5M3_SCALE_2D ? (row >> 4) : row) * 16;
-        const int b_raw1 = (p.b_mode == UE5M3_SCALE_2D ? ((row + 128) >> 4) : (row + 128)) * 16;
-        const int dst = (lane * 4 + g) * 4;            // byte offset of this row's word inside a 512-byte block of 128 rows
+        const int dst = (cw * 32 + lane) * 4;          // byte offset of this row's word inside a 512-byte block
+        const int64_t kblocks = p.Kc >> 4;
         auto shift = [](uint32_t v, uint32_t d) { return __vsub4(v, d) & ~__vcmpeq4(v, 0u); };
-        uint32_t it = 0;
+        // Read cursor, PF stages ahead of the stage being written: the addresses of this thread's three rows for the
+        // current stage (nullptr beyond the operand); inside a tile they advance by a constant per stage.
+        const int64_t step_a = p.a_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16, step_b = p.b_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16;
+        const uint8_t *pa = nullptr, *pb0 = nullptr, *pb1 = nullptr;
+        int c_tile = pair, c_kc = 0;
+        auto row_base = [&](const uint8_t* scales, int mode, int64_t R, int64_t grow) -> const uint8_t* {
+            if (grow >= R) return nullptr;
+            if (mode == UE5M3_SCALE_1D_TILED) return scales + (grow >> 7) * kchunks * 2048 + (grow & 127) * 16;
+            return scales + ((mode == UE5M3_SCALE_2D) ? (grow >> 4) : grow) * kblocks;
+        };
+        auto open_tile = [&]() {
+            if (c_tile >= num_tiles) { pa = pb0 = pb1 = nullptr; return; }
+            int tm, tn;
+            tile_coords(c_tile, p.tiles_m, p.tiles_n, tm, tn);
+            pa = row_base(p.a_scales, p.a_mode, p.Mo, (int64_t)(tm * 2 + (int)rank) * BM + row);
+            pb0 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + row);
+            pb1 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + BNH + row);
+        };
+        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            a = pa ? ldg_nc_16(pa) : z;
+            b0 = pb0 ? ldg_nc_16(pb0) : z;
+            b1 = pb1 ? ldg_nc_16(pb1) : z;
+            if (++c_kc == kchunks) {
+                c_kc = 0;
+                c_tile += num_pairs;
+                open_tile();
+            } else {
+                if (pa) pa += step_a;
+                if (pb0) pb0 += step_b;
+                if (pb1) pb1 += step_b;
+            }
+        };
+        open_tile();
+        uint4 ra[PF], rb0[PF], rb1[PF];
+#pragma unroll
+        for (int d = 0; d < PF; ++d) {
+            fetch(ra[d], rb0[d], rb1[d]);
+        }
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-            for (int kc = 0; kc < kchunks && ok; ++kc, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                if (!mbar_wait(pk_full + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
-                uint8_t* st = smem_gen + s * STAGE_BYTES;
-                const uint4 a = *reinterpret_cast<const uint4*>(st + OFF_RAW_A + a_raw);
-                const uint4 b0 = *reinterpret_cast<const uint4*>(st + OFF_RAW_B + b_raw0);
-                const uint4 b1 = *reinterpret_cast<const uint4*>(st + OFF_RAW_B + b_raw1);
-                uint32_t* sa = reinterpret_cast<uint32_t*>(st + OFF_SF_A + dst);
-                uint32_t* sb = reinterpret_cast<uint32_t*>(st + OFF_SF_B + dst);
+        for (uint32_t base = 0; base < total && ok; base += PF) {
+#pragma unroll
+            for (int d = 0; d < PF; ++d) {
+                const uint32_t it = base + d;
+                if (it >= total || !ok) break;
+                const uint32_t f = it % SF_STAGES, fph = (it / SF_STAGES) & 1;
+                if (!mbar_wait(sf_empty + 8 * f, fph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
+                uint8_t* sf = smem_gen + SMEM_SF + f * SF_STAGE_BYTES;
+                uint32_t* sa = reinterpret_cast<uint32_t*>(sf + dst);
+                uint32_t* sb = reinterpret_cast<uint32_t*>(sf + SF_A_BYTES + dst);
+                const uint4 a = ra[d], b0 = rb0[d], b1 = rb1[d];
                 sa[0] = shift(a.x, da); sa[128] = shift(a.y, da); sa[256] = shift(a.z, da); sa[384] = shift(a.w, da);
                 sb[0] = shift(b0.x, db); sb[256] = shift(b0.y, db); sb[512] = shift(b0.z, db); sb[768] = shift(b0.w, db);
                 sb[128] = shift(b1.x, db); sb[384] = shift(b1.y, db); sb[640] = shift(b1.z, db); sb[896] = shift(b1.w, db);
                 fence_proxy_async();                 // the tensor core's scale copy reads what was just written
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(sf_full + 8 * s, 0);
+                if (lane == 0) mbar_arrive_cluster(sf_full + 8 * f, 0);
+                fetch(ra[d], rb0[d], rb1[d]);
             }
         }
     }
@@ -395,9 +477,25 @@ bool make_out_map(CUtensorMap* m, void* out, bool bf16, int64_t Mo, int64_t No, 
 
 bool native_eligible(const GemmArgs& g) {
     if (g.Kc % KCHUNK) return false;
-    for (int m : {g.a_scale_mode, g.b_scale_mode})
-        if (m != UE5M3_SCALE_1D && m != UE5M3_SCALE_2D) return false;
     return true;
+}
+
+// Four words of device workspace for one call: a ring of 256 slots per device, allocated at the first call on that
+// device.  Calls that are in flight at the same time (different streams) use different slots as long as fewer than
+// 256 of them overlap.
+int* native_workspace() {
+    static int* ring[64];
+    static std::once_flag made[64];
+    static std::atomic<unsigned> next{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::call_once(made[dev], [&]() {
+        void* ptr = nullptr;
+        if (cudaMalloc(&ptr, 256 * 4 * sizeof(int)) != cudaSuccess) { (void)cudaGetLastError(); return; }
+        ring[dev] = static_cast<int*>(ptr);
+    });
+    if (!ring[dev]) return nullptr;
+    return ring[dev] + 4 * (next.fetch_add(1) & 255u);
 }
 
 int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st) {
@@ -433,27 +531,26 @@ int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStr
     });
     if (resident_pairs[dev] < 1) return UE5M3_ERR_CUDA;
     if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
-    CUtensorMap ma, mb, mas, mbs, mo;
-    const uint64_t row_bytes = (uint64_t)(g.Kc / 2), kb = (uint64_t)(g.Kc / 16);
+    CUtensorMap ma, mb, mo;
+    const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
     if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
     if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BNH, true)) return UE5M3_ERR_CUDA;
-    const bool a2 = g.a_scale_mode == UE5M3_SCALE_2D, b2 = g.b_scale_mode == UE5M3_SCALE_2D;
-    if (!make_map(&mas, g.a_scales, kb, (uint64_t)(a2 ? g.Mo / 16 : g.Mo), kb, 16, a2 ? BM / 16 : BM, false)) return UE5M3_ERR_CUDA;
-    if (!make_map(&mbs, g.b_scales, kb, (uint64_t)(b2 ? g.No / 16 : g.No), kb, 16, b2 ? BN / 16 : BN, false)) return UE5M3_ERR_CUDA;
     if (!make_out_map(&mo, g.out, g.out_dtype == UE5M3_BF16, g.Mo, g.No, g.ldo)) return UE5M3_ERR_CUDA;
 
     NativeParams p;
     p.Mo = g.Mo; p.No = g.No; p.Kc = g.Kc;
     p.a_decode = g.a_decode; p.b_decode = g.b_decode;
     p.range = range;
+    p.a_scales = g.a_scales; p.b_scales = g.b_scales;
     p.out_bf16 = g.out_dtype == UE5M3_BF16 ? 1 : 0;
     p.a_mode = g.a_scale_mode; p.b_mode = g.b_scale_mode;
     p.tiles_m = (int)((g.Mo + 2 * BM - 1) / (2 * BM));
     p.tiles_n = (int)((g.No + BN - 1) / BN);
     p.wait_limit = g.wait_limit_cycles > 0 ? g.wait_limit_cycles : WAIT_LIMIT_CYCLES;
+    p.stall_producer = g.stall_producer;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int pairs = num_tiles < resident_pairs[dev] ? num_tiles : resident_pairs[dev];
-    gemm_native_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, mo, p);
+    gemm_native_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mo, p);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
@@ -469,3 +566,4 @@ int read_and_clear_native_status() {
 }
 
 }  // namespace ue5m3
+

@@ -55,11 +55,14 @@ cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bo
 cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* out, int num_sms,
                         cudaStream_t st);
 cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, cudaStream_t st);
-int launch_gemm(const GemmArgs& g, int num_sms, cudaStream_t st);   // returns a UE5M3_* status
+// returns a UE5M3_* status; `range` (may be null) is the workspace of the native path: the kernel then does nothing when
+// both operands have a UE4M3 window, because gemm_native_kernel has done the product
+int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st);
 int read_and_clear_device_status();                                  // synchronises the device
 // The same product on the tensor core's FP4 path (gemm_native.cu).  `range` is four words of device workspace:
 // launch_scale_range fills them, the kernel reads them and does nothing when an operand's scale codes have no window.
 bool native_eligible(const GemmArgs& g);
+int* native_workspace();                                             // four words of a per-device ring; null on failure
 int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st);
 int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st);
 int read_and_clear_native_status();                                  // synchronises the device

@@ -1,4 +1,4 @@
-"""Failure detection without a GPU fault: every device-side wait of the two GEMM kernels is bounded, and the
+"""Failure detection without a GPU fault: every device-side wait of the three GEMM kernels is bounded, and the
 self-test entry point makes such a wait run out on purpose (the copy producer is switched off, nothing ever arrives on
 the barrier, the bound is about a millisecond).  The kernel must return by itself, leave the output alone, report
 UE5M3_ERR_TIMEOUT exactly once through the status word and leave the context fit for the next, normal launch."""
@@ -26,7 +26,7 @@ def _operands(rng, Mo, No, Kc):
     return qa, qb, (ap, asc, bp, bsc)
 
 
-@pytest.mark.parametrize("which", [0, 1])
+@pytest.mark.parametrize("which", [0, 1, 2])
 def test_bounded_wait_runs_out_and_is_reported_once(which):
     rng = np.random.default_rng(40 + which)
     Mo = No = 128
@@ -46,11 +46,13 @@ def test_bounded_wait_runs_out_and_is_reported_once(which):
     assert lib.last_device_status() == 0                      # reported once, then cleared
     assert torch.all(out == -3.0)                             # nothing was written
     # the context, the barriers' shared memory and tensor memory are fit for a normal launch
-    fn = lib.gemm if which == 0 else (lambda op, a, b, out: lib.gemm_probe_matched(op, a, b, out=out, grid_denominator=0))
+    fn = {0: lambda op, a, b, out: lib.gemm_fp16(op, a, b, out=out),
+          1: lambda op, a, b, out: lib.gemm_probe_matched(op, a, b, out=out, grid_denominator=0),
+          2: lambda op, a, b, out: lib.gemm_native(op, a, b, out=out)}[which]
     fn(lib.FPROP, qa, qb, out=out)
     torch.cuda.synchronize()
     assert lib.last_device_status() == 0
-    if which == 0:
+    if which != 1:
         y, sa = oracle.gemm(ap, asc, False, 1.0, bp, bsc, False, 1.0)
         check_gemm_output(out, y, sa)
     else:
@@ -63,7 +65,7 @@ def test_selftest_rejects_bad_arguments():
     qa, qb, _ = _operands(rng, 128, 128, 256)
     out = torch.zeros((128, 128), dtype=torch.float32, device=DEV)
     with pytest.raises(lib.Ue5m3Error):
-        lib.gemm_stall_selftest(2, qa, qb, out)
+        lib.gemm_stall_selftest(3, qa, qb, out)
     with pytest.raises(lib.Ue5m3Error):
         lib.gemm_stall_selftest(0, qa, qb, out, wait_limit_cycles=10)
     torch.cuda.synchronize()

@@ -1,0 +1,177 @@
+"""The native FP4 path of ue5m3_gemm: UE5M3 scale codes shifted into a UE4M3 window, the tensor core's own block-scaled
+instruction.  Parity with the exact-integer oracle under the same bound as the FP16 path (FP32: |y - y*| <= 1e-5 *
+sum_k |a_k b_k| + 1e-30, BF16: 1 ulp), the window's edges, the fallback when there is no window, and the dispatch."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_02846_b200 as lib
+from helpers import check_gemm_output
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _tiled(scales, R, Kc):
+    kb = Kc // 16
+    buf = np.zeros(((R + 127) // 128) * ((kb + 15) // 16) * 2048, np.uint8)
+    r, k = np.meshgrid(np.arange(R), np.arange(kb), indexing="ij")
+    off = ((r >> 7) * ((kb + 15) // 16) + (k >> 4)) * 2048 + (r & 127) * 16 + (k & 15)
+    buf[off.ravel()] = scales.ravel()
+    return buf
+
+
+def _operand(rng, R, Kc, mode, lo, hi, dec=1.0, scales=None):
+    payload = rng.integers(0, 256, (R, Kc // 2), dtype=np.uint8)
+    shape = (R // 16, Kc // 16) if mode == lib.SCALE_2D else (R, Kc // 16)
+    if scales is None:
+        scales = rng.integers(lo, hi, shape, dtype=np.uint8)
+    stored = _tiled(scales, R, Kc) if mode == lib.SCALE_1D_TILED else scales
+    q = lib.QuantizedOperand(torch.from_numpy(payload).to(DEV), torch.from_numpy(stored).to(DEV),
+                             torch.tensor([dec], dtype=torch.float32, device=DEV), mode)
+    return q, payload, scales
+
+
+def _native(qa, qb, dtype, Mo, No):
+    """Runs ue5m3_gemm_native on an output pre-filled with NaN; returns (out, workspace as a list)."""
+    out = torch.full((Mo, No), float("nan"), dtype=dtype, device=DEV)
+    ws = torch.zeros(4, dtype=torch.int32, device=DEV)
+    lib.gemm_native(lib.FPROP, qa, qb, dtype, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    return out, ws.tolist()
+
+
+# (Mo, No, Kc): one tile and one stage; several stages; ragged tile counts (a CTA of a pair without rows, a tile
+# narrower than 256); more tile rows than one raster group (8) and not a multiple of it; an odd number of tiles per
+# CTA pair is reached by every shape with more tiles than pairs
+SHAPES = [(128, 128, 256), (256, 256, 256), (256, 384, 512), (384, 640, 1024), (2432, 384, 256), (512, 256, 4096)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("modes", [(0, 0), (0, 2), (1, 1), (2, 0), (1, 2)])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_native_matches_oracle(shape, modes, out_dtype):
+    Mo, No, Kc = shape
+    rng = np.random.default_rng(Mo + 3 * No + 5 * Kc + 7 * modes[0] + modes[1])
+    lo = int(rng.integers(0x20, 0x70))
+    qa, ap, asc = _operand(rng, Mo, Kc, modes[0], lo, lo + 0x50, dec=0.37)
+    qb, bp, bsc = _operand(rng, No, Kc, modes[1], 0x40, 0xA0, dec=1.0 / 2688.0)
+    out, ws = _native(qa, qb, out_dtype, Mo, No)
+    assert ws == [int(asc.max()), 255 - int(asc.min()), int(bsc.max()), 255 - int(bsc.min())]
+    y, sa = oracle.gemm(ap, asc, modes[0] == 2, 0.37, bp, bsc, modes[1] == 2, np.float32(1.0 / 2688.0))
+    check_gemm_output(out, y, sa)
+
+
+def test_native_many_tiles_per_pair():
+    """More tiles than resident CTA pairs, so that every pair alternates between its two accumulators and hands the
+    shared columns back while the rest of the previous tile is still being stored."""
+    Mo, No, Kc = 4096, 3072, 512                      # 16 x 12 = 192 tiles
+    rng = np.random.default_rng(77)
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x60, 0x90, dec=1.0)
+    qb, bp, bsc = _operand(rng, No, Kc, 2, 0x60, 0x90, dec=1.0)
+    out, _ = _native(qa, qb, torch.float32, Mo, No)
+    ci = rng.integers(0, Mo, 6000)
+    cj = rng.integers(0, No, 6000)
+    for r in (0, 127, 128, 255, 256, Mo - 1):        # full rows and columns through tile corners
+        ci = np.concatenate([ci, np.full(No, r)]); cj = np.concatenate([cj, np.arange(No)])
+    for c in (0, 255, 256, No - 1):
+        ci = np.concatenate([ci, np.arange(Mo)]); cj = np.concatenate([cj, np.full(Mo, c)])
+    y, sa = oracle.gemm_cells(ap, asc, False, 1.0, bp, bsc, True, 1.0, ci, cj)
+    got = out.cpu().numpy().astype(np.float64)[ci, cj]
+    assert np.all(np.abs(got - y) <= 1e-5 * sa + 1e-30)
+
+
+@pytest.mark.parametrize("k", [0, 1, 7, 14, 15])
+def test_window_edges(k):
+    """Every code of the window 8k + 8 .. 8k + 126 (the widest one: 119 codes) in both operands, zero codes mixed in."""
+    Mo, No, Kc = 128, 256, 256
+    rng = np.random.default_rng(100 + k)
+    lo, hi = 8 * k + 8, min(8 * k + 126, 0xF7)
+    codes = np.arange(lo, hi + 1, dtype=np.uint8)
+    asc = rng.choice(codes, (Mo, Kc // 16)); asc[0, :2] = (lo, hi); asc[5, 3] = 0
+    bsc = rng.choice(codes, (No, Kc // 16)); bsc[1, :2] = (hi, lo); bsc[7, 0] = 0
+    dec = float(2.0 ** (10 - 2 * k))                  # keeps the products inside FP32 for the high windows
+    qa, ap, _ = _operand(rng, Mo, Kc, 0, 0, 0, dec=dec, scales=asc)
+    qb, bp, _ = _operand(rng, No, Kc, 0, 0, 0, dec=dec, scales=bsc)
+    out, ws = _native(qa, qb, torch.float32, Mo, No)
+    assert ws == [hi, 255 - lo, hi, 255 - lo]
+    y, sa = oracle.gemm(ap, asc, False, dec, bp, bsc, False, np.float32(dec))
+    check_gemm_output(out, y, sa)
+
+
+@pytest.mark.parametrize("case", ["too_wide", "subnormal", "a_only"])
+def test_no_window_leaves_output_alone_and_gemm_falls_back(case):
+    Mo, No, Kc = 256, 256, 512
+    rng = np.random.default_rng(len(case))
+    if case == "too_wide":
+        a_rng, b_rng = (0x20, 0x98), (0x40, 0x80)      # 0x20 .. 0x97: 120 codes, one more than a window holds
+    elif case == "subnormal":
+        a_rng, b_rng = (0x01, 0x40), (0x40, 0x80)      # UE5M3 subnormal codes have no UE4M3 counterpart in any window
+    else:
+        a_rng, b_rng = (0x08, 0xF8), (0x50, 0x60)
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, *a_rng)
+    qb, bp, bsc = _operand(rng, No, Kc, 0, *b_rng, dec=2.0 ** -20)
+    asc[0, 0], asc[0, 1] = a_rng[0], a_rng[1] - 1
+    qa.scales.copy_(torch.from_numpy(asc))
+    out, ws = _native(qa, qb, torch.float32, Mo, No)
+    assert ws[0] == a_rng[1] - 1 and ws[1] == 255 - a_rng[0]
+    assert bool(torch.isnan(out).all())               # the native kernel declined
+    got = lib.gemm(lib.FPROP, qa, qb, torch.float32)
+    ref = lib.gemm_fp16(lib.FPROP, qa, qb, torch.float32)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    assert torch.equal(got, ref)                      # the same kernel did the work
+    y, sa = oracle.gemm(ap, asc, False, 1.0, bp, bsc, False, np.float32(2.0 ** -20))
+    check_gemm_output(got, y, sa)
+
+
+def test_gemm_dispatches_to_the_native_kernel_when_there_is_a_window():
+    Mo, No, Kc = 384, 512, 1024
+    rng = np.random.default_rng(9)
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x58, 0x98, dec=0.5)
+    qb, bp, bsc = _operand(rng, No, Kc, 2, 0x58, 0x98, dec=0.25)
+    got = lib.gemm(lib.FPROP, qa, qb, torch.float32)
+    nat, _ = _native(qa, qb, torch.float32, Mo, No)
+    assert torch.equal(got, nat)
+    # Kc = 128 * odd is not eligible: the FP16 kernel does it
+    qa, _, _ = _operand(rng, 128, 384, 0, 0x58, 0x98)
+    qb, _, _ = _operand(rng, 128, 384, 0, 0x58, 0x98)
+    assert torch.equal(lib.gemm(lib.FPROP, qa, qb, torch.float32), lib.gemm_fp16(lib.FPROP, qa, qb, torch.float32))
+    with pytest.raises(lib.Ue5m3Error):
+        lib.gemm_native(lib.FPROP, qa, qb, torch.float32)
+
+
+def test_every_operand_value_pair_of_a_window_multiplies_exactly():
+    """All 119 scale codes of a window x 14 nonzero payload codes of A against the same set for B, one product per
+    output: the shifted codes and the tensor core's product are exact for every operand value, so the FP32 output
+    equals the rational product bit for bit."""
+    lo = 0x48
+    pairs = [(sc, q) for sc in range(lo, lo + 119) for q in list(range(1, 8)) + list(range(9, 16))]
+    R = ((len(pairs) + 127) // 128) * 128
+    Kc = 256
+    payload = np.zeros((R, Kc // 2), np.uint8)
+    scales = np.full((R, Kc // 16), lo + 60, np.uint8)
+    for i, (sc, q) in enumerate(pairs):
+        payload[i, 0] = q
+        scales[i, 0] = sc
+    scales[0, 1], scales[1, 1] = lo, lo + 118         # the window's ends are present whatever the first column holds
+    one = torch.ones(1, dtype=torch.float32, device=DEV)
+    q = lib.QuantizedOperand(torch.from_numpy(payload).to(DEV), torch.from_numpy(scales).to(DEV), one, lib.SCALE_1D)
+    out, ws = _native(q, q, torch.float32, R, R)
+    assert ws == [lo + 118, 255 - lo, lo + 118, 255 - lo]
+    y, _ = oracle.gemm(payload, scales, False, 1.0, payload, scales, False, np.float32(1.0))
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), y)
+
+
+def test_native_is_deterministic_and_independent_of_the_workspace_contents():
+    Mo, No, Kc = 512, 512, 2048
+    rng = np.random.default_rng(3)
+    qa, _, _ = _operand(rng, Mo, Kc, 0, 0x60, 0xA0)
+    qb, _, _ = _operand(rng, No, Kc, 0, 0x60, 0xA0, dec=2.0 ** -12)
+    first, _ = _native(qa, qb, torch.bfloat16, Mo, No)
+    ws = torch.full((4,), 12345, dtype=torch.int32, device=DEV)     # stale contents: the call clears them itself
+    again = lib.gemm_native(lib.FPROP, qa, qb, torch.bfloat16, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(first, again)
