@@ -213,7 +213,7 @@ class LinearStep:
     """Pre-allocated buffers and the launch sequence of one fwd+bwd step."""
     KERNELS = ("q_x_dual", "q_w_2d", "gemm_fprop", "q_dy_row_sr", "gemm_dgrad", "q_dy_col_sr", "gemm_wgrad")
 
-    def __init__(self, device, seed=0, scale_layout=0):
+    def __init__(self, device, seed=0, scale_layout=0, gemm_path="auto"):
         import torch
         import paper_2609_02846_b200 as lib
         import synth_inputs as si
@@ -228,6 +228,10 @@ class LinearStep:
         self.dX = torch.empty((M_TOK, K_IN), dtype=torch.bfloat16, device=device)
         self.dW = torch.empty((N_OUT, K_IN), dtype=torch.bfloat16, device=device)
         self.launches = 0
+        # auto: ue5m3_gemm (range reduction, native FP4 kernel, FP16 kernel: three launches, one does the product);
+        # fp16: ue5m3_gemm_fp16 (the FP16 reconstruction kernel alone)
+        self.gemm = lib.gemm if gemm_path == "auto" else lib.gemm_fp16
+        self.gemm_launches = 3 if gemm_path == "auto" else 1
 
     def _timed(self, name, fn, ev):
         if ev is None:
@@ -269,12 +273,32 @@ class LinearStep:
                                                                       seed=4 * step + 1, scale_layout=sl, out=q.get("gt")), evk)
 
         self._timed("quant_fwd", fwd_quant, evg)
-        self._timed("gemm_fprop", lambda: lib.gemm(lib.FPROP, q["x"], q["w"], out=self.Y), ev)
+        self._timed("gemm_fprop", lambda: self.gemm(lib.FPROP, q["x"], q["w"], out=self.Y), ev)
         self._timed("quant_dgrad", dgrad_quant, evg)
-        self._timed("gemm_dgrad", lambda: lib.gemm(lib.DGRAD, q["g"], q["w"].transposed(), out=self.dX), ev)
+        self._timed("gemm_dgrad", lambda: self.gemm(lib.DGRAD, q["g"], q["w"].transposed(), out=self.dX), ev)
         self._timed("quant_wgrad", wgrad_quant, evg)
-        self._timed("gemm_wgrad", lambda: lib.gemm(lib.WGRAD, q["gt"], q["xt"], out=self.dW), ev)
-        self.launches += 7
+        self._timed("gemm_wgrad", lambda: self.gemm(lib.WGRAD, q["gt"], q["xt"], out=self.dW), ev)
+        self.launches += 4 + 3 * self.gemm_launches
+
+
+    def gemm_kernels(self):
+        """Which kernel ue5m3_gemm uses for each of the three products of the step just run: the code ranges of the
+        operands' scales (ue5m3_gemm_native writes them to its workspace) decide, by the same rule as on the device."""
+        lib, q, torch = self.lib, self.q, self.torch
+        from paper_2609_02846_b200.binding import scale_window
+        out = {}
+        for name, a, b, c in (("gemm_fprop", q["x"], q["w"], self.Y), ("gemm_dgrad", q["g"], q["w"].transposed(), self.dX),
+                              ("gemm_wgrad", q["gt"], q["xt"], self.dW)):
+            if self.gemm_launches == 1 or a.Kc % 256:
+                out[name] = "gemm_kernel"
+                continue
+            ws = torch.zeros(4, dtype=torch.int32, device=c.device)
+            lib.gemm_native(lib.FPROP, a, b, out=c, workspace=ws)
+            torch.cuda.synchronize()
+            r = ws.tolist()
+            ok = all(hi == 0 or scale_window(255 - inv, hi) is not None for hi, inv in ((r[0], r[1]), (r[2], r[3])))
+            out[name] = "gemm_native_kernel" if ok else "gemm_kernel"
+        return out
 
 
 QUANT_GROUPS = {"quant_fwd": ("q_x_dual", "q_w_2d"), "quant_dgrad": ("q_dy_row_sr",), "quant_wgrad": ("q_dy_col_sr",)}
@@ -301,8 +325,11 @@ def kernel_bytes():
 KERNEL_BYTES = kernel_bytes()
 GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the default workload (mean of fprop, dgrad, wgrad;
-# one ncu pass, summary in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt).  Algorithmic bytes: 242 MB per launch.
-GEMM_DRAM_TRAFFIC_BYTES = (150.5e6 + 220.5e6 + 188.9e6 + 47.9e6 + 101.1e6 + 99.5e6) / 3
+# one ncu pass each; summaries in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt and
+# profiles/gemm_native_kernel_linear_M8192_K4096_N16384_ncu_full.txt).  Algorithmic bytes: 238 MB per launch.
+GEMM_DRAM_TRAFFIC_BYTES = {"gemm_kernel": (150.5e6 + 220.5e6 + 188.9e6 + 47.9e6 + 101.1e6 + 99.5e6) / 3,
+                           "gemm_native_kernel": (150.8e6 + 220.2e6 + 195.9e6 + 51.1e6 + 101.0e6 + 102.7e6) / 3}
+NOMINAL_FP4_OVER_BF16 = 4.0      # dense tensor peaks of the part: 9 PFLOP/s FP4, 2.25 PFLOP/s BF16
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -348,7 +375,7 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
     peaks = measured_peaks()
-    step = LinearStep(dev, seed=rank, scale_layout=args.scale_layout)
+    step = LinearStep(dev, seed=rank, scale_layout=args.scale_layout, gemm_path=args.gemm_path)
     K, Wm = args.steps, max(args.warmup, 3)
 
     sampler = ClockSampler(dev)
@@ -377,6 +404,7 @@ def run_ours(args):
     ms_per_step = total_ms / K
     value = job_value(ms_per_step, world)
     gpu_launches = step.launches - launches0
+    gemm_kernels = step.gemm_kernels()          # after the timed region: it launches each product once more
 
     per_kernel = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in ev.items()}
     gemm_ms = statistics.mean(per_kernel[k] for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad"))
@@ -433,9 +461,11 @@ def run_ours(args):
         sustained = {"seconds": round(sus_ms * n_sus * 1e-3, 2), "steps": n_sus, "ms_per_step": round(sus_ms, 4),
                      "tflops_per_step": round(FLOPS_PER_STEP / (sus_ms * 1e-3) / 1e12, 1),
                      "gemm_tflops_per_launch": round(sus_gemm, 1), "gemm_avg_launch_ms": round(sus_gemm_ms, 4),
-                     "gemm_frac_of_sustained_peak": round(sus_gemm / peaks["bf16_tflops_sustained"], 3),
-                     "gemm_frac_of_burst_peak": round(sus_gemm / peaks["bf16_tflops"], 3),
-                     "gemm_frac_of_nominal_2250": round(sus_gemm / NOMINAL_BF16_TFLOPS, 3),
+                     "gemm_over_bf16_sustained_peak": round(sus_gemm / peaks["bf16_tflops_sustained"], 3),
+                     "gemm_over_bf16_burst_peak": round(sus_gemm / peaks["bf16_tflops"], 3),
+                     "gemm_over_bf16_nominal_2250": round(sus_gemm / NOMINAL_BF16_TFLOPS, 3),
+                     "gemm_frac_of_own_pipe_sustained": round(sus_gemm / (peaks["bf16_tflops_sustained"] * (
+                         NOMINAL_FP4_OVER_BF16 if all(v == "gemm_native_kernel" for v in gemm_kernels.values()) else 1.0)), 3),
                      "clocks": clk2,
                      "gemm_launch_ms_x_sm_mhz": None if not clk2.get("sm_mhz") else round(sus_gemm_ms * clk2["sm_mhz"], 1)}
 
@@ -496,21 +526,30 @@ def run_ours(args):
             v, dt, cores = time_oracle(1, 0)
             cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": SAMPLE_DESC, "seconds": round(dt, 2)}
         # Denominator from this run's own clock record: a short region at full clocks is compared with the burst
-        # figure of the measured cuBLAS peak, a long or power-capped one with the sustained figure.
+        # figure of the measured cuBLAS BF16 peak, a long or power-capped one with the sustained figure.  When the three
+        # products ran on the native FP4 kernel the peak is that of its own pipe: the measured BF16 figure times the
+        # nominal dense FP4 : BF16 ratio (9 : 2.25 PFLOP/s).
         region_s = total_ms * 1e-3
         capped = "sw_power_cap" in (clocks.get("reasons") or [])
         use_burst = region_s < 1.0 and not capped
-        peak = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
-        roofline = {"bound": "tensor", "kernel": "gemm_kernel", "achieved": gemm_tflops, "peak": peak, "unit": "TFLOP/s",
-                    "frac": gemm_tflops / peak,
-                    "peak_source": peaks["source"] + (" (burst: timed region %.3f s, no power cap seen)" % region_s if use_burst
-                                                      else " (sustained: timed region %.3f s%s)" % (region_s, ", sw_power_cap seen" if capped else "")),
-                    "frac_of_burst_peak": gemm_tflops / peaks["bf16_tflops"],
-                    "frac_of_sustained_peak": gemm_tflops / peaks["bf16_tflops_sustained"],
-                    "frac_of_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
+        native = all(v == "gemm_native_kernel" for v in gemm_kernels.values())
+        ratio = NOMINAL_FP4_OVER_BF16 if native else 1.0
+        peak = ratio * (peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"])
+        kernel = "gemm_native_kernel" if native else "gemm_kernel"
+        roofline = {"bound": "tensor", "kernel": kernel, "kernel_per_gemm": gemm_kernels,
+                    "achieved": gemm_tflops, "peak": peak, "unit": "TFLOP/s", "frac": gemm_tflops / peak,
+                    "peak_source": peaks["source"] + " cuBLAS BF16" + (" x 4 (nominal dense FP4 : BF16), " if native else ", ") +
+                                   ("burst: timed region %.3f s, no power cap seen" % region_s if use_burst
+                                    else "sustained: timed region %.3f s%s" % (region_s, ", sw_power_cap seen" if capped else "")),
+                    "achieved_over_bf16_burst_peak": gemm_tflops / peaks["bf16_tflops"],
+                    "achieved_over_bf16_sustained_peak": gemm_tflops / peaks["bf16_tflops_sustained"],
+                    "achieved_over_bf16_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
+                    "achieved_over_fp4_nominal_9000": gemm_tflops / (NOMINAL_BF16_TFLOPS * NOMINAL_FP4_OVER_BF16),
                     "avg_launch_ms": gemm_ms,
+                    "avg_launch_ms_note": "one ue5m3_gemm call: with --gemm-path auto that is the range reduction, the kernel "
+                                          "that does the product and the other kernel's immediate return",
                     "avg_launch_ms_x_sm_mhz": None if not clocks.get("sm_mhz") else round(gemm_ms * clocks["sm_mhz"], 1),
-                    "traffic": GEMM_DRAM_TRAFFIC_BYTES if (M_TOK, K_IN, N_OUT) == (8192, 4096, 16384) else None,
+                    "traffic": GEMM_DRAM_TRAFFIC_BYTES.get(kernel) if (M_TOK, K_IN, N_OUT) == (8192, 4096, 16384) else None,
                     "traffic_unit": "bytes of DRAM read+write per launch (ncu, mean of the three GEMMs)",
                     "per_gemm_ms": {k: round(per_kernel[k], 4) for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}}
         sweep = None
@@ -519,8 +558,9 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "tokens_per_gpu": M_TOK, "l2": f"inputs ({2 * (M_TOK * K_IN + N_OUT * K_IN + M_TOK * N_OUT) >> 20} MiB per step) exceed the 126 MB L2",
+            "dtype": "fp4 (e2m1 operands, 8-bit block scales, f32 accumulate)" if native else "f16 (exact reconstruction of e2m1 x ue5m3, f32 accumulate)",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "gemm_path": args.gemm_path, "tokens_per_gpu": M_TOK, "l2": f"inputs ({2 * (M_TOK * K_IN + N_OUT * K_IN + M_TOK * N_OUT) >> 20} MiB per step) exceed the 126 MB L2",
                        "scale_layout": "tiled" if args.scale_layout else "rowmajor", "amax": "sampled at step 0, held 50 steps"},
             "roofline": roofline,
             "quantizer": quant, "sustained": sustained, "quantizer_sweep": sweep,
@@ -785,6 +825,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-layout", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--gemm-path", default="auto", choices=["auto", "fp16"],
+                    help="auto: ue5m3_gemm picks the native FP4 kernel when the scale codes allow; fp16: the FP16 kernel alone")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the two-second sustained leg")
     ap.add_argument("--no-sweep", action="store_true", help="skip the quantizer sweep cells of the default line")
