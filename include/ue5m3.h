@@ -209,6 +209,22 @@ UE5M3_API int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
                void* out, int out_dtype, int64_t ldo, void* stream);
 
 /*
+ * ue5m3_gemm with a workspace that is never allocated (the paper has no counterpart: this is about how a library
+ * holds four words of device scratch, not about the method).  Same arguments, results (bit for bit), checks and errors
+ * as ue5m3_gemm.  The range words live in a file-scope device array of 256 bytes inside the library instead of the
+ * allocated per-device ring; a call needs 16 of them whatever Mo, No and Kc are, and a need above 256 bytes would be
+ * refused with UE5M3_ERR_UNSUPPORTED.  The call allocates and frees nothing, on the host or the device; the array's
+ * address is looked up once per device, at the first call there, so make that first call outside any stream capture.
+ * All calls on a device share the array.  Each call clears its words before use, so calls that follow one another
+ * on one stream are independent; two calls that can run at the same time (different streams without an ordering
+ * between them) race on the words and may each pick the wrong kernel's answer: order them, or use ue5m3_gemm.
+ */
+UE5M3_API int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc,
+               const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
+               const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
+               void* out, int out_dtype, int64_t ldo, void* stream);
+
+/*
  * The two kernels of ue5m3_gemm on their own (same arguments, layouts, alignment and errors).
  * ue5m3_gemm_fp16: always the FP16 reconstruction kernel; no workspace is touched.
  * ue5m3_gemm_native: the range reduction and the native FP4 kernel only.  Kc must be a multiple of 256

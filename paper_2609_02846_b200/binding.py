@@ -59,6 +59,8 @@ def _load() -> C.CDLL:
         L.ue5m3_quantize_dual.argtypes = [vp, ci, i64, i64, i64, ci, vp, f32, f32, u64, u64, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         L.ue5m3_gemm.restype = ci
         L.ue5m3_gemm.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
+        L.ue5m3_gemm_static.restype = ci
+        L.ue5m3_gemm_static.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_fp16.restype = ci
         L.ue5m3_gemm_fp16.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_native.restype = ci
@@ -284,6 +286,23 @@ def gemm(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dty
                                   _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
                                   _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
                                   _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)), "ue5m3_gemm")
+    return out
+
+
+def gemm_static(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """`gemm` with the library's file-scope workspace instead of its allocated one (ue5m3_gemm_static): nothing is
+    allocated by the call; calls that may overlap in time must be ordered by the caller."""
+    Mo, No, Kc = a.R, b.R, a.Kc
+    if b.Kc != Kc:
+        raise ValueError(f"contraction sizes differ: {Kc} vs {b.Kc}")
+    if out is None:
+        out = torch.empty((Mo, No), dtype=out_dtype, device=a.payload.device)
+    with torch.cuda.device(out.device):
+        _check(_load().ue5m3_gemm_static(op, Mo, No, Kc,
+                                         _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),
+                                         _dev_ptr(b.payload), _dev_ptr(b.scales), b.scale_mode, _dev_ptr(b.decode),
+                                         _dev_ptr(out), _dtype_code(out), out.stride(0), _stream(out)), "ue5m3_gemm_static")
     return out
 
 

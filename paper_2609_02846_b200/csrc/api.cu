@@ -223,6 +223,29 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
     return launch_gemm(g, ws, di.sms, (cudaStream_t)stream);
 }
 
+int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
+                      int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
+                      int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {
+    const ApiRange range_("ue5m3_gemm_static");
+    const int bad = check_gemm_args(op, Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales,
+                                    b_scale_mode, b_decode, out, out_dtype, ldo, 128);
+    if (bad != UE5M3_OK) return bad;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return UE5M3_ERR_CUDA;
+    if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
+    GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
+               out, out_dtype, ldo};
+    if (!native_eligible(g)) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
+    const size_t need = 4 * sizeof(int);              // the four range words; does not grow with the problem
+    int* ws = static_workspace(need);
+    if (!ws) return UE5M3_ERR_UNSUPPORTED;
+    int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
+    if (r != UE5M3_OK) return r;
+    r = launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
+    if (r != UE5M3_OK) return r;
+    return launch_gemm(g, ws, di.sms, (cudaStream_t)stream);
+}
+
 int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
                     int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
                     int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, void* stream) {

@@ -498,6 +498,28 @@ int* native_workspace() {
     return ring[dev] + 4 * (next.fetch_add(1) & 255u);
 }
 
+// Workspace of ue5m3_gemm_static: a file-scope device array instead of allocated memory.  One call needs 16 bytes
+// (the four range words), whatever the problem size; the array holds kStaticWorkspaceBytes.  Its address is asked for
+// once per device; nothing is allocated, here or later.  All calls on a device share the array: the four words are
+// cleared by every call before its range kernel runs, so two calls may follow one another on a stream, but two calls
+// in flight at the same time (different streams) would read each other's ranges.
+constexpr size_t kStaticWorkspaceBytes = 256;
+static __device__ __align__(256) int g_static_workspace[kStaticWorkspaceBytes / sizeof(int)];
+
+int* static_workspace(size_t need_bytes) {
+    if (need_bytes > kStaticWorkspaceBytes) return nullptr;
+    static int* addr[64];
+    static std::once_flag asked[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::call_once(asked[dev], [&]() {
+        int* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_static_workspace) != cudaSuccess) { (void)cudaGetLastError(); return; }
+        addr[dev] = ptr;
+    });
+    return addr[dev];
+}
+
 int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st) {
     const int64_t kb = g.Kc / 16;
     const int64_t na = (g.a_scale_mode == UE5M3_SCALE_2D ? g.Mo / 16 : g.Mo) * kb;

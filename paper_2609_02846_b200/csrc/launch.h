@@ -63,6 +63,7 @@ int read_and_clear_device_status();                                  // synchron
 // launch_scale_range fills them, the kernel reads them and does nothing when an operand's scale codes have no window.
 bool native_eligible(const GemmArgs& g);
 int* native_workspace();                                             // four words of a per-device ring; null on failure
+int* static_workspace(size_t need_bytes);                            // file-scope device array; null if the need exceeds it
 int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st);
 int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st);
 int read_and_clear_native_status();                                  // synchronises the device

@@ -1,0 +1,53 @@
+"""ue5m3_gemm_static: the GEMM whose four words of scratch live in a file-scope device array.  Compared bit for bit with
+ue5m3_gemm on two calls in a row (the second call finds the words the first one left), on operands that take the native
+kernel and on operands that fall back to the FP16 kernel, and checked not to move the device allocator."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_02846_b200 as lib
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _operand(rng, R, Kc, lo, hi, dec):
+    payload = rng.integers(0, 256, (R, Kc // 2), dtype=np.uint8)
+    scales = rng.integers(lo, hi, (R, Kc // 16), dtype=np.uint8)
+    return lib.QuantizedOperand(torch.from_numpy(payload).to(DEV), torch.from_numpy(scales).to(DEV),
+                                torch.tensor([dec], dtype=torch.float32, device=DEV), lib.SCALE_1D)
+
+
+def test_static_workspace_gemm_equals_gemm_on_two_calls_in_a_row():
+    rng = np.random.default_rng(2026)
+    Mo, No, Kc = 384, 512, 1024
+    windowed = (_operand(rng, Mo, Kc, 0x50, 0x90, 0.5), _operand(rng, No, Kc, 0x60, 0xA0, 2.0 ** -9))
+    wide = (_operand(rng, Mo, Kc, 0x01, 0xF0, 2.0 ** -12), _operand(rng, No, Kc, 0x40, 0x60, 2.0 ** -12))     # no window
+    want = [lib.gemm(lib.FPROP, a, b, torch.float32) for a, b in (windowed, wide)]
+    torch.cuda.synchronize()
+    lib.gemm_static(lib.FPROP, *windowed, torch.float32)            # first call on the device: looks the array up
+    torch.cuda.synchronize()
+    out = [torch.full((Mo, No), float("nan"), dtype=torch.float32, device=DEV) for _ in range(4)]
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    # two calls in a row, no synchronisation in between; then the other kernel's case twice: the words a call finds
+    # are those of the call before it, with the opposite verdict
+    lib.gemm_static(lib.FPROP, *windowed, out=out[0])
+    lib.gemm_static(lib.FPROP, *wide, out=out[1])
+    lib.gemm_static(lib.FPROP, *wide, out=out[2])
+    lib.gemm_static(lib.FPROP, *windowed, out=out[3])
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert lib.last_device_status() == 0
+    assert free1 == free0                                           # the calls took no device memory
+    assert torch.equal(out[0], want[0]) and torch.equal(out[3], want[0])
+    assert torch.equal(out[1], want[1]) and torch.equal(out[2], want[1])
+
+
+def test_static_workspace_gemm_checks_arguments_like_gemm():
+    rng = np.random.default_rng(1)
+    a, b = _operand(rng, 128, 256, 0x60, 0x70, 1.0), _operand(rng, 128, 512, 0x60, 0x70, 1.0)
+    with pytest.raises(ValueError):
+        lib.gemm_static(lib.FPROP, a, b)
+    a = _operand(rng, 128, 384, 0x60, 0x70, 1.0); b = _operand(rng, 128, 384, 0x60, 0x70, 1.0)      # Kc = 128 * 3: FP16 kernel
+    assert torch.equal(lib.gemm_static(lib.FPROP, a, b, torch.float32), lib.gemm(lib.FPROP, a, b, torch.float32))
