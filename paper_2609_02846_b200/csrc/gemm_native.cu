@@ -8,8 +8,8 @@
 // exactly.  When all scale codes of an operand lie in one such window of 119 codes (a ratio of 2^14.8 between the
 // largest and the smallest block scale), the GEMM is the native one on the shifted codes and the two powers of two
 // go into alpha.  The packed payload reaches the tensor core as the copy engine delivered it: no conversion, no
-// second staging.  The shifted scale bytes are written by four warps per CTA (three integer operations per four
-// codes) in the layout the scale copy into tensor memory expects.
+// second staging.  The shifted scale bytes (three integer operations per four codes) are written into tensor memory
+// by four warps per CTA, in the layout the block-scaled MMA reads.
 //
 // The window is found on the device: scale_range_kernel reduces both operands' scale bytes to their largest and
 // smallest non-zero code (four words of workspace), gemm_native_kernel reads them and returns at once when an
@@ -18,16 +18,20 @@
 //
 // Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 6 payload stages of 32 KB):
 //   warp 0      copies: packed A rows (128) and packed B rows (this CTA's 128) of a stage
-//   warp 1      (leader CTA) per stage 12 scale copies shared memory -> tensor memory and 4 MMAs of K = 64
+//   warp 1      (leader CTA) 4 MMAs of K = 64 per stage
 //   warp 2      tensor-memory allocation
 //   warp 3      relay: tells the leader CTA that this CTA's copy of a stage has landed
 //   warps 4-7   epilogue: accumulator -> alpha -> BF16 / FP32 -> shared memory -> bulk tensor store
-//   warps 8-11  scale bytes: read from global memory four stages ahead (registers), window shift, re-layout into a
-//               ring of two stages in shared memory
-// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 192..447, the
-// scales of the stage in flight in columns 448..495.  Two whole accumulators do not fit beside the scales, so the
-// two overlap in 64 columns: the epilogue drains those 64 first and hands them back, and the MMAs of the next
-// tile run while the other 192 columns are still being stored.
+//   warps 8-11  scale bytes: read from global memory two stages ahead (registers), window shift, written straight
+//               into tensor memory (tcgen05.st), one warp per lane quarter, two stages of scales resident
+// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 160..415, two
+// stages of scales in columns 416..511.  Two whole accumulators do not fit beside the scales, so the two overlap in
+// 96 columns: the epilogue drains those 96 first and hands them back, and the MMAs of the next tile run while the
+// other 160 columns are still being stored.
+// One thread issues a tensor instruction every 50-60 clocks at best (measured: 12 scale copies 578 clocks, 4 MMAs
+// 258 clocks into an idle pipe), so the issuing thread does nothing but the four MMAs and one commit per stage;
+// an earlier version that copied the scales from shared memory with tcgen05.cp (12 copies per stage, same thread)
+// spent 950 clocks per stage issuing.
 // Every wait is bounded (SM clocks); on a time-out the role sets the status word, the other roles see the abort
 // flag, in-flight copies and MMAs are drained and the kernel returns.
 #include <cuda.h>
@@ -53,24 +57,24 @@ constexpr int KCHUNK = 256;                 // K per stage
 constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks)
 constexpr int MMAS = KCHUNK / KMMA;
 constexpr int STAGES = 6;                   // payload stages
-constexpr int SF_STAGES = 2;                // converted-scale stages
-constexpr int PF = 4;                       // stages the scale bytes are read ahead (registers)
-constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;
-constexpr int NUM_THREADS = 32 * (CONV_WARP0 + CONV_WARPS);
+constexpr int SF_SLOTS = 2;                 // stages whose scales are in tensor memory at a time
+constexpr int PF = 2;                       // group-stages (= 4 stages) the scale bytes are read ahead (registers)
+constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;    // CONV_WARPS per group, two groups
+constexpr int NUM_THREADS = 32 * (CONV_WARP0 + 2 * CONV_WARPS);
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;           // 16384
 constexpr int PK_B_BYTES = BNH * KCHUNK / 2;          // 16384
 constexpr int STAGE_BYTES = PK_A_BYTES + PK_B_BYTES;  // 32768
-constexpr int SF_A_BYTES = BM * (KCHUNK / 16);        // 2048: [mma][32 lanes][4 row groups][4 blocks]
-constexpr int SF_B_BYTES = BN * (KCHUNK / 16);        // 4096: [mma][half][32 lanes][4 row groups][4 blocks]
-constexpr int SF_STAGE_BYTES = SF_A_BYTES + SF_B_BYTES;
-constexpr int SMEM_SF = STAGES * STAGE_BYTES;         // 196608
-constexpr int SMEM_BARS = SMEM_SF + SF_STAGES * SF_STAGE_BYTES;   // 208896
+constexpr int XCH_A_BYTES = BM * (KCHUNK / 16), XCH_BYTES = XCH_A_BYTES + BN * (KCHUNK / 16);   // 2048 + 4096 per group
+constexpr int SMEM_XCH = STAGES * STAGE_BYTES;        // 196608
+constexpr int SMEM_BARS = SMEM_XCH + 2 * XCH_BYTES;   // 208896
 constexpr int SMEM_EPI = SMEM_BARS + 1024;
 constexpr int EPI_WARP_BYTES = 4096;
-constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 227328
-constexpr int TMEM_ACC_ODD = 192;                     // accumulator base column of odd tiles (even tiles: 0)
-constexpr int TMEM_SFA_COL = 448, TMEM_SFB_COL = 464; // two half-stage slots each: 2 x 8 and 2 x 16 columns
+constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 215040
+// Tensor memory (512 columns): accumulator of even tiles 0..255, of odd tiles 160..415 (they share 96 columns), then two
+// scale slots of 48 columns: 16 for A (column 4 j + g: rows 32 g + lane, MMA j) and 32 for B (column 8 j + 4 h + g).
+constexpr int TMEM_ACC_ODD = 160;
+constexpr int TMEM_SF_COL = 416, TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
 
 struct NativeParams {
     int64_t Mo, No, Kc;
@@ -104,24 +108,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // N = 256, M = 256 (two CTAs), K = 64.
 constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 
-// Descriptor of 32 rows of 16 bytes stored back to back: no swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t sf_smem_desc(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(128 >> 4) << 16;
-    d |= (uint64_t)(128 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    return d;
-}
-// The scale copy and the MMA take their 64-bit shared-memory descriptors as halves: the upper halves are constants of
-// the kernel and the lower halves differ only in the start-address field, so the issuing thread (one thread per CTA
-// pair, every instruction of it on the critical path) adds small constants instead of rebuilding descriptors.
-// Copy: 32 rows x 16 bytes of shared memory (in both CTAs of the pair, at the same offset) -> 4 columns of lanes
-// 0..31 of every lane quarter of each CTA's tensor memory.
-__device__ __forceinline__ void tmem_cp_32x128b(uint32_t taddr, uint32_t lo, uint32_t hi) {
-    asm volatile("{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\ttcgen05.cp.cta_group::2.32x128b.warpx4 [%0], d;\n\t}"
-                 ::"r"(taddr), "r"(lo), "r"(hi) : "memory");
-}
+// The MMA takes its 64-bit shared-memory descriptors as halves: the upper half is a constant of the kernel and the
+// lower halves differ only in the start-address field, so the issuing thread (one thread per CTA pair, every
+// instruction of it on the critical path) adds small constants instead of rebuilding descriptors.
 __device__ __forceinline__ void umma_fp4_block16(uint32_t tmem_d, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc,
                                                  uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
     asm volatile(
@@ -130,6 +119,15 @@ __device__ __forceinline__ void umma_fp4_block16(uint32_t tmem_d, uint32_t alo, 
         "setp.ne.b32 p, %7, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], da, db, %4, [%5], [%6], p;\n\t}"
         ::"r"(tmem_d), "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate) : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t r[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
 }
 __device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
     uint4 v;
@@ -185,7 +183,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const uint32_t bar_base = smem_base + SMEM_BARS;
     // barriers (8 bytes each)
     const uint32_t pk_full = bar_base, pk_empty = bar_base + 64, pk_ready = bar_base + 128;
-    const uint32_t sf_full = bar_base + 192, sf_empty = bar_base + 256;
+    const uint32_t sf_full = bar_base + 192;
     const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 344);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 352);
@@ -205,10 +203,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             mbar_init(pk_empty + 8 * s, 1);
             mbar_init(pk_ready + 8 * s, 2);                    // the leader's copy collects both CTAs' relays
         }
-        for (int s = 0; s < SF_STAGES; ++s) {
-            mbar_init(sf_full + 8 * s, 2 * CONV_WARPS);        // the leader's copy collects both CTAs' warps
-            mbar_init(sf_empty + 8 * s, 1);
-        }
+        for (int s = 0; s < SF_SLOTS; ++s) mbar_init(sf_full + 8 * s, 2 * CONV_WARPS);   // the leader's copy collects both CTAs' warps
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 8);
         mbar_init(drain_bar, 1);
@@ -261,36 +256,29 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (lane == 0 && rank == 0) {
             uint32_t tl = 0;
             bool ok = true;
-            // descriptor halves: payload (128-byte swizzle) and scales (no swizzle); only the start address moves
-            const uint64_t d_pk = umma_smem_desc(smem_base), d_sf = sf_smem_desc(smem_base + SMEM_SF);
+            // descriptor halves of the payload stages (128-byte swizzle); only the start address moves
+            const uint64_t d_pk = umma_smem_desc(smem_base);
             const uint32_t pk_lo0 = (uint32_t)d_pk, pk_hi = (uint32_t)(d_pk >> 32);
-            const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
-            const uint32_t sfa0 = tmem_base + TMEM_SFA_COL, sfb0 = tmem_base + TMEM_SFB_COL;
-            uint32_t s = 0, ph = 0, f = 0, fph = 0;       // payload stage and its phase, scale stage and its phase
+            uint32_t s = 0, ph = 0, u = 0, uph = 0;       // payload stage and its phase, scale slot and its phase
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
                 if (!mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + ((tl & 1) ? TMEM_ACC_ODD : 0);
                 for (int kc = 0; kc < kchunks; ++kc) {
-                    if (!mbar_wait(sf_full + 8 * f, fph, abort_flag, p.wait_limit)) { ok = false; break; }
+                    if (!mbar_wait(sf_full + 8 * u, uph, abort_flag, p.wait_limit)) { ok = false; break; }
                     if (!mbar_wait(pk_ready + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_lo = pk_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (PK_A_BYTES >> 4);
-                    const uint32_t sf_lo = sf_lo0 + f * (SF_STAGE_BYTES >> 4), sfb_lo = sf_lo + (SF_A_BYTES >> 4);
+                    const uint32_t sfa = tmem_base + TMEM_SF_COL + u * TMEM_SF_SLOT_COLS, sfb = sfa + TMEM_SFB_OFF;
 #pragma unroll
-                    for (int j = 0; j < MMAS; ++j) {
-                        // MMA j of a stage has scale columns of its own, so a copy never touches columns an MMA still
-                        // in flight reads (copies and MMAs of one thread execute in issue order)
-                        const uint32_t sfa = sfa0 + 4 * j, sfb = sfb0 + 8 * j;
-                        tmem_cp_32x128b(sfa, sf_lo + j * (512 >> 4), sf_hi);
-                        tmem_cp_32x128b(sfb, sfb_lo + j * (1024 >> 4), sf_hi);
-                        tmem_cp_32x128b(sfb + 4, sfb_lo + j * (1024 >> 4) + (512 >> 4), sf_hi);
-                        umma_fp4_block16(tmem_d, a_lo + 2 * j, b_lo + 2 * j, pk_hi, kInstrDesc, sfa, sfb, (kc | j) != 0 ? 1u : 0u);
-                    }
-                    umma_commit_pair(pk_empty + 8 * s);        // both CTAs may refill this payload stage
-                    umma_commit_pair(sf_empty + 8 * f);        // ... and this scale stage
+                    for (int j = 0; j < MMAS; ++j)
+                        umma_fp4_block16(tmem_d, a_lo + 2 * j, b_lo + 2 * j, pk_hi, kInstrDesc, sfa + 4 * j, sfb + 8 * j,
+                                         (kc | j) != 0 ? 1u : 0u);
+                    // both CTAs may refill this payload stage; their scale warps read the same barrier to learn that
+                    // the scale slot of this stage is free again
+                    umma_commit_pair(pk_empty + 8 * s);
                     if (++s == STAGES) { s = 0; ph ^= 1; }
-                    if (++f == SF_STAGES) { f = 0; fph ^= 1; }
+                    if (++u == SF_SLOTS) { u = 0; uph ^= 1; }
                 }
                 if (ok) umma_commit_pair(acc_full);
             }
@@ -315,25 +303,29 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             const int row0 = mb * BM + q * 32, col0 = nb * BN;
             const uint32_t odd = tl & 1;
             const uint32_t acc = tmem_base + ((uint32_t)(q * 32) << 16) + (odd ? TMEM_ACC_ODD : 0);
-            // The 64 columns both accumulators share (the last 64 of an even tile, the first 64 of an odd one) are
-            // read first; once every epilogue warp of the pair has them in registers the next tile's MMAs may start.
+            // The 96 columns both accumulators share (the last 96 of an even tile, the first 96 of an odd one) are read
+            // first; once every epilogue warp of the pair has them in registers the next tile's MMAs may start.  Units
+            // of 32 columns: an even tile goes 6 7 | 5 4 | 0 1 | 2 3, an odd one 0 1 | 2 3 | 4 5 | 6 7, and the hand-back
+            // comes after the third unit.
             if (p.out_bf16) {
 #pragma unroll 1
                 for (int i = 0; i < BN / 64; ++i) {
-                    const int c = odd ? i : ((i + BN / 64 - 1) & (BN / 64 - 1));
+                    const int cc = odd ? i : (i == 0 ? 3 : i == 1 ? 2 : i - 2);      // chunk of 64 columns: 3 2 0 1 | 0 1 2 3
                     uint8_t* mine = stage_gen + lane * 128;
                     const int sw = lane & 7;
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
+                    for (int hh = 0; hh < 2; ++hh) {
+                        // inside the second chunk the shared unit comes first (even: unit 5 before 4)
+                        const int half = (!odd && i == 1) ? (hh ^ 1) : hh;
                         uint32_t r[32];
-                        tmem_ld32(acc + c * 64 + half * 32, r);
+                        tmem_ld32(acc + cc * 64 + half * 32, r);
                         tmem_ld_wait();
-                        if (i == 0 && half == 1) {
+                        if (i == 1 && hh == 0) {
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
                         }
-                        if (half == 0) {
+                        if (hh == 0) {
                             if (lane == 0) tma_store_wait_read<0>();
                             __syncwarp();
                         }
@@ -349,16 +341,17 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     }
                     fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) tma_store_2d(&map_out, stage, col0 + c * 64, row0);
+                    if (lane == 0) tma_store_2d(&map_out, stage, col0 + cc * 64, row0);
                 }
             } else {
 #pragma unroll 1
                 for (int i = 0; i < BN / 32; ++i) {
-                    const int c = odd ? i : ((i + BN / 32 - 2) & (BN / 32 - 1));
+                    // units of 32 columns: even 6 7 5 4 0 1 2 3, odd 0 1 2 3 4 5 6 7
+                    const int c = odd ? i : (i < 2 ? 6 + i : i == 2 ? 5 : i == 3 ? 4 : i - 4);
                     uint32_t r[32];
                     tmem_ld32(acc + c * 32, r);
                     tmem_ld_wait();
-                    if (i == 1) {
+                    if (i == 2) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -380,17 +373,18 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         }
         if (lane == 0) tma_store_wait_all();
     } else if (warp >= CONV_WARP0) {
-        // ------------------------------------------------------------------ scale bytes: window shift and re-layout
-        // Lane l of warp w handles row g * 32 + dp of A and of both B halves, with dp = 8 w + l / 4 and g = l % 4: the
-        // words a warp stores (index 4 dp + g inside a 512-byte block of 128 rows) are then 32 consecutive ones.
-        const int cw = warp - CONV_WARP0;
-        const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);
+        // ------------------------------------------------------------------ scale bytes: window shift, into tensor memory
+        // The tensor core wants the scales of row 32 g + r in lane r (of every lane quarter), one column per (MMA, g) with
+        // the MMA's four block scales as its bytes.  Two groups of four warps take the stages in turn (group = stage
+        // parity = scale slot).  A group's 128 threads read one row each of A and of the two B halves (16 bytes per row
+        // and stage, PF group-stages ahead in registers), shift the codes, and exchange them through shared memory in
+        // the order [MMA][lane][g] (32 consecutive words per warp store); then warp w reads the 12 x 16 bytes of its lane
+        // and writes lane quarter w of the slot with two tcgen05.st.
+        const int cg = (warp - CONV_WARP0) >> 2, cw = warp & 3;
+        const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);            // the row this thread reads
         const uint32_t da = (uint32_t)((8 * ka) & 0xFF) * 0x01010101u, db = (uint32_t)((8 * kb) & 0xFF) * 0x01010101u;
-        const int dst = (cw * 32 + lane) * 4;          // byte offset of this row's word inside a 512-byte block
         const int64_t kblocks = p.Kc >> 4;
         auto shift = [](uint32_t v, uint32_t d) { return __vsub4(v, d) & ~__vcmpeq4(v, 0u); };
-        // Read cursor, PF stages ahead of the stage being written: the addresses of this thread's three rows for the
-        // current stage (nullptr beyond the operand); inside a tile they advance by a constant per stage.
         const int64_t step_a = p.a_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16, step_b = p.b_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16;
         const uint8_t *pa = nullptr, *pb0 = nullptr, *pb1 = nullptr;
         int c_tile = pair, c_kc = 0;
@@ -407,11 +401,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             pb0 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + row);
             pb1 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + BNH + row);
         };
-        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            a = pa ? ldg_nc_16(pa) : z;
-            b0 = pb0 ? ldg_nc_16(pb0) : z;
-            b1 = pb1 ? ldg_nc_16(pb1) : z;
+        auto advance = [&]() {                       // the cursor moves on by one stage
             if (++c_kc == kchunks) {
                 c_kc = 0;
                 c_tile += num_pairs;
@@ -422,31 +412,62 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 if (pb1) pb1 += step_b;
             }
         };
+        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {     // this group's next stage; the other group's is skipped
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            a = pa ? ldg_nc_16(pa) : z;
+            b0 = pb0 ? ldg_nc_16(pb0) : z;
+            b1 = pb1 ? ldg_nc_16(pb1) : z;
+            advance();
+            advance();
+        };
         open_tile();
+        if (cg) advance();
         uint4 ra[PF], rb0[PF], rb1[PF];
 #pragma unroll
-        for (int d = 0; d < PF; ++d) {
-            fetch(ra[d], rb0[d], rb1[d]);
-        }
+        for (int d = 0; d < PF; ++d) fetch(ra[d], rb0[d], rb1[d]);
         bool ok = true;
-        for (uint32_t base = 0; base < total && ok; base += PF) {
+        uint8_t* xch = smem_gen + SMEM_XCH + cg * XCH_BYTES;
+        uint32_t* xa = reinterpret_cast<uint32_t*>(xch) + cw * 32 + lane;            // + 128 j
+        uint32_t* xb = reinterpret_cast<uint32_t*>(xch + XCH_A_BYTES) + cw * 32 + lane;   // + 256 j + 128 h
+        const uint4* ya = reinterpret_cast<const uint4*>(xch) + lane;                 // + 32 j
+        const uint4* yb = reinterpret_cast<const uint4*>(xch + XCH_A_BYTES) + lane;   // + 64 j + 32 h
+        const uint32_t slot = tmem_base + ((uint32_t)(cw * 32) << 16) + TMEM_SF_COL + cg * TMEM_SF_SLOT_COLS;
+        const int bar_id = 1 + cg;
+        for (uint32_t base = cg; base < total && ok; base += 2 * PF) {
 #pragma unroll
             for (int d = 0; d < PF; ++d) {
-                const uint32_t it = base + d;
+                const uint32_t it = base + 2 * d;
                 if (it >= total || !ok) break;
-                const uint32_t f = it % SF_STAGES, fph = (it / SF_STAGES) & 1;
-                if (!mbar_wait(sf_empty + 8 * f, fph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
-                uint8_t* sf = smem_gen + SMEM_SF + f * SF_STAGE_BYTES;
-                uint32_t* sa = reinterpret_cast<uint32_t*>(sf + dst);
-                uint32_t* sb = reinterpret_cast<uint32_t*>(sf + SF_A_BYTES + dst);
                 const uint4 a = ra[d], b0 = rb0[d], b1 = rb1[d];
-                sa[0] = shift(a.x, da); sa[128] = shift(a.y, da); sa[256] = shift(a.z, da); sa[384] = shift(a.w, da);
-                sb[0] = shift(b0.x, db); sb[256] = shift(b0.y, db); sb[512] = shift(b0.z, db); sb[768] = shift(b0.w, db);
-                sb[128] = shift(b1.x, db); sb[384] = shift(b1.y, db); sb[640] = shift(b1.z, db); sb[896] = shift(b1.w, db);
-                fence_proxy_async();                 // the tensor core's scale copy reads what was just written
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(sf_full + 8 * f, 0);
+                xa[0] = shift(a.x, da); xa[128] = shift(a.y, da); xa[256] = shift(a.z, da); xa[384] = shift(a.w, da);
+                xb[0] = shift(b0.x, db); xb[256] = shift(b0.y, db); xb[512] = shift(b0.z, db); xb[768] = shift(b0.w, db);
+                xb[128] = shift(b1.x, db); xb[384] = shift(b1.y, db); xb[640] = shift(b1.z, db); xb[896] = shift(b1.w, db);
                 fetch(ra[d], rb0[d], rb1[d]);
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // the group's 128 rows are in place
+                uint32_t ca[16], cb[32];
+#pragma unroll
+                for (int j = 0; j < MMAS; ++j) {
+                    const uint4 va = ya[32 * j], v0 = yb[64 * j], v1 = yb[64 * j + 32];
+                    ca[4 * j] = va.x; ca[4 * j + 1] = va.y; ca[4 * j + 2] = va.z; ca[4 * j + 3] = va.w;
+                    cb[8 * j] = v0.x; cb[8 * j + 1] = v0.y; cb[8 * j + 2] = v0.z; cb[8 * j + 3] = v0.w;
+                    cb[8 * j + 4] = v1.x; cb[8 * j + 5] = v1.y; cb[8 * j + 6] = v1.z; cb[8 * j + 7] = v1.w;
+                }
+                // the slot held the scales of stage it - 2: free once that stage's MMAs have retired, which is what the
+                // payload barrier of that stage says
+                if (it >= SF_SLOTS) {
+                    const uint32_t prev = it - SF_SLOTS;
+                    if (!mbar_wait(pk_empty + 8 * (prev % STAGES), (prev / STAGES) & 1, abort_flag, p.wait_limit)) ok = false;
+                    tc_fence_after();
+                }
+                if (ok) {
+                    tmem_st16(slot, ca);
+                    tmem_st32(slot + TMEM_SFB_OFF, cb);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(sf_full + 8 * cg, 0);
+                }
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // everyone has read: the exchange buffer is free
             }
         }
     }
