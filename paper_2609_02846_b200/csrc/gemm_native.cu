@@ -129,6 +129,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t r[16]) 
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
     uint4 v;
     asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
@@ -136,20 +142,29 @@ __device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
 }
 
 // ----------------------------------------------------------------------------- range of the scale codes
-__global__ void __launch_bounds__(256) scale_range_kernel(const uint8_t* __restrict__ a, int64_t na, const uint8_t* __restrict__ b,
+__global__ void __launch_bounds__(512) scale_range_kernel(const uint8_t* __restrict__ a, int64_t na, const uint8_t* __restrict__ b,
                                                           int64_t nb, int* __restrict__ range) {
-    uint32_t mx[2] = {0u, 0u}, inv[2] = {0u, 0u};
+    __shared__ uint32_t part[16][4];
+    uint32_t red[4];                                      // max A, 255 - min nonzero A, max B, 255 - min nonzero B
     for (int op = 0; op < 2; ++op) {
         const uint8_t* s = op ? b : a;
         const int64_t n = op ? nb : na, words = n >> 4;
         uint32_t m = 0u, iv = 0u;
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (int64_t)gridDim.x * blockDim.x) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(s) + i);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        // four independent 16-byte loads per trip
+        const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += 4 * stride) {
+            uint4 v[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                m = __vmaxu4(m, w[j]);
-                iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));      // 255 - c, and 0 for c = 0
+            for (int t = 0; t < 4; ++t)
+                v[t] = (i + t * stride < words) ? __ldg(reinterpret_cast<const uint4*>(s) + i + t * stride) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const uint32_t w[4] = {v[t].x, v[t].y, v[t].z, v[t].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    m = __vmaxu4(m, w[j]);
+                    iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));      // 255 - c, and 0 for c = 0
+                }
             }
         }
         if (blockIdx.x == 0 && threadIdx.x < (n & 15)) {
@@ -159,14 +174,24 @@ __global__ void __launch_bounds__(256) scale_range_kernel(const uint8_t* __restr
         }
         m = max(max(m & 0xFFu, (m >> 8) & 0xFFu), max((m >> 16) & 0xFFu, m >> 24));
         iv = max(max(iv & 0xFFu, (iv >> 8) & 0xFFu), max((iv >> 16) & 0xFFu, iv >> 24));
-        mx[op] = __reduce_max_sync(0xFFFFFFFFu, m);
-        inv[op] = __reduce_max_sync(0xFFFFFFFFu, iv);
+        red[2 * op] = __reduce_max_sync(0xFFFFFFFFu, m);
+        red[2 * op + 1] = __reduce_max_sync(0xFFFFFFFFu, iv);
     }
-    if ((threadIdx.x & 31) == 0) {
-        if (mx[0]) atomicMax(range + 0, (int)mx[0]);
-        if (inv[0]) atomicMax(range + 1, (int)inv[0]);
-        if (mx[1]) atomicMax(range + 2, (int)mx[1]);
-        if (inv[1]) atomicMax(range + 3, (int)inv[1]);
+    // one set of atomics per CTA: thousands of warps hitting four words one after the other would cost more than the read
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane < 4) part[warp][lane] = lane == 0 ? red[0] : lane == 1 ? red[1] : lane == 2 ? red[2] : red[3];
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t v = lane < 16 ? part[lane][0] : 0u, w = lane < 16 ? part[lane][1] : 0u;
+        const uint32_t x = lane < 16 ? part[lane][2] : 0u, y = lane < 16 ? part[lane][3] : 0u;
+        const uint32_t r0 = __reduce_max_sync(0xFFFFFFFFu, v), r1 = __reduce_max_sync(0xFFFFFFFFu, w);
+        const uint32_t r2 = __reduce_max_sync(0xFFFFFFFFu, x), r3 = __reduce_max_sync(0xFFFFFFFFu, y);
+        if (lane == 0) {
+            if (r0) atomicMax(range + 0, (int)r0);
+            if (r1) atomicMax(range + 1, (int)r1);
+            if (r2) atomicMax(range + 2, (int)r2);
+            if (r3) atomicMax(range + 3, (int)r3);
+        }
     }
 }
 
@@ -183,7 +208,6 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const uint32_t bar_base = smem_base + SMEM_BARS;
     // barriers (8 bytes each)
     const uint32_t pk_full = bar_base, pk_empty = bar_base + 64, pk_ready = bar_base + 128;
-    const uint32_t sf_full = bar_base + 192;
     const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 344);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 352);
@@ -201,9 +225,10 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(pk_full + 8 * s, 1);
             mbar_init(pk_empty + 8 * s, 1);
-            mbar_init(pk_ready + 8 * s, 2);                    // the leader's copy collects both CTAs' relays
+            // the leader's copy collects, for the stage that lives here, both CTAs' relays (payload landed) and both CTAs'
+            // scale warps (the stage's scales are in tensor memory)
+            mbar_init(pk_ready + 8 * s, 2 + 2 * CONV_WARPS);
         }
-        for (int s = 0; s < SF_SLOTS; ++s) mbar_init(sf_full + 8 * s, 2 * CONV_WARPS);   // the leader's copy collects both CTAs' warps
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 8);
         mbar_init(drain_bar, 1);
@@ -253,37 +278,51 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
-        if (lane == 0 && rank == 0) {
+        // The whole warp runs the loop and one elected lane issues: the operands of the tensor instructions (descriptors,
+        // tensor-memory addresses) are then warp-uniform values that the compiler keeps in uniform registers, where the
+        // instructions want them; computed by a single lane they would be moved there one by one before every issue
+        // (measured: 80 clocks per MMA that way).
+        if (rank == 0) {
             uint32_t tl = 0;
             bool ok = true;
+            const bool elected = elect_one();
             // descriptor halves of the payload stages (128-byte swizzle); only the start address moves
             const uint64_t d_pk = umma_smem_desc(smem_base);
             const uint32_t pk_lo0 = (uint32_t)d_pk, pk_hi = (uint32_t)(d_pk >> 32);
-            uint32_t s = 0, ph = 0, u = 0, uph = 0;       // payload stage and its phase, scale slot and its phase
+            const uint32_t tm0 = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
+            uint32_t s = 0, ph = 0, u = 0;                // payload stage and its phase, scale slot
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
-                if (!mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit));
+                if (!ok) break;
                 tc_fence_after();
-                const uint32_t tmem_d = tmem_base + ((tl & 1) ? TMEM_ACC_ODD : 0);
+                const uint32_t tmem_d = tm0 + ((tl & 1) ? TMEM_ACC_ODD : 0);
                 for (int kc = 0; kc < kchunks; ++kc) {
-                    if (!mbar_wait(sf_full + 8 * u, uph, abort_flag, p.wait_limit)) { ok = false; break; }
-                    if (!mbar_wait(pk_ready + 8 * s, ph, abort_flag, p.wait_limit)) { ok = false; break; }
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(pk_ready + 8 * s, ph, abort_flag, p.wait_limit));
+                    if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_lo = pk_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (PK_A_BYTES >> 4);
-                    const uint32_t sfa = tmem_base + TMEM_SF_COL + u * TMEM_SF_SLOT_COLS, sfb = sfa + TMEM_SFB_OFF;
+                    const uint32_t sfa = tm0 + TMEM_SF_COL + u * TMEM_SF_SLOT_COLS, sfb = sfa + TMEM_SFB_OFF;
+                    if (elected) {
 #pragma unroll
-                    for (int j = 0; j < MMAS; ++j)
-                        umma_fp4_block16(tmem_d, a_lo + 2 * j, b_lo + 2 * j, pk_hi, kInstrDesc, sfa + 4 * j, sfb + 8 * j,
-                                         (kc | j) != 0 ? 1u : 0u);
-                    // both CTAs may refill this payload stage; their scale warps read the same barrier to learn that
-                    // the scale slot of this stage is free again
-                    umma_commit_pair(pk_empty + 8 * s);
+                        for (int j = 0; j < MMAS; ++j)
+                            umma_fp4_block16(tmem_d, a_lo + 2 * j, b_lo + 2 * j, pk_hi, kInstrDesc, sfa + 4 * j, sfb + 8 * j,
+                                             (kc | j) != 0 ? 1u : 0u);
+                        // both CTAs may refill this payload stage; their scale warps read the same barrier to learn that
+                        // the scale slot of this stage is free again
+                        umma_commit_pair(pk_empty + 8 * s);
+                    }
+                    __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1; }
-                    if (++u == SF_SLOTS) { u = 0; uph ^= 1; }
+                    u ^= 1;
                 }
-                if (ok) umma_commit_pair(acc_full);
+                if (ok && elected) umma_commit_pair(acc_full);
+                __syncwarp();
             }
-            umma_commit_local(drain_bar);
-            mbar_wait_drain(drain_bar, 0, &g_native_status, p.wait_limit);
+            if (elected) {
+                umma_commit_local(drain_bar);
+                mbar_wait_drain(drain_bar, 0, &g_native_status, p.wait_limit);
+            }
+            __syncwarp();
         }
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------------------------ epilogue
@@ -465,7 +504,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(sf_full + 8 * cg, 0);
+                    if (lane == 0) mbar_arrive_cluster(pk_ready + 8 * (it % STAGES), 0);
                 }
                 asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // everyone has read: the exchange buffer is free
             }
@@ -547,10 +586,10 @@ int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t 
     const int64_t nb = (g.b_scale_mode == UE5M3_SCALE_2D ? g.No / 16 : g.No) * kb;
     if (cudaMemsetAsync(range, 0, 4 * sizeof(int), st) != cudaSuccess) return UE5M3_ERR_CUDA;
     const int64_t words = (na > nb ? na : nb) >> 4;
-    int64_t grid = (words + 256 * 4 - 1) / (256 * 4);
-    if (grid > 4 * num_sms) grid = 4 * num_sms;
+    int64_t grid = (words + 512 * 4 - 1) / (512 * 4);
+    if (grid > 2 * num_sms) grid = 2 * num_sms;
     if (grid < 1) grid = 1;
-    scale_range_kernel<<<(unsigned)grid, 256, 0, st>>>(g.a_scales, na, g.b_scales, nb, range);
+    scale_range_kernel<<<(unsigned)grid, 512, 0, st>>>(g.a_scales, na, g.b_scales, nb, range);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
