@@ -8,30 +8,31 @@
 // exactly.  When all scale codes of an operand lie in one such window of 119 codes (a ratio of 2^14.8 between the
 // largest and the smallest block scale), the GEMM is the native one on the shifted codes and the two powers of two
 // go into alpha.  The packed payload reaches the tensor core as the copy engine delivered it: no conversion, no
-// second staging.  The shifted scale bytes (three integer operations per four codes) are written into tensor memory
-// by four warps per CTA, in the layout the block-scaled MMA reads.
+// second staging.  The shifted scale bytes (three integer operations per four codes) take their own route into
+// tensor memory, in the layout the block-scaled MMA reads.
 //
 // The window is found on the device: scale_range_kernel reduces both operands' scale bytes to their largest and
 // smallest non-zero code (four words of workspace), gemm_native_kernel reads them and returns at once when an
 // operand has no window (subnormal UE5M3 codes included); the caller then runs the FP16 path, whose kernel
 // evaluates the same predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.
 //
-// Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 6 payload stages of 32 KB):
+// Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 5 payload stages of 32 KB):
 //   warp 0      copies: packed A rows (128) and packed B rows (this CTA's 128) of a stage
-//   warp 1      (leader CTA) 4 MMAs of K = 64 per stage
-//   warp 2      tensor-memory allocation
-//   warp 3      relay: tells the leader CTA that this CTA's copy of a stage has landed
+//   warp 1      (leader CTA) MMA issuer: 4 MMAs of K = 64 and one commit per stage
+//   warp 2      tensor-memory allocation; relay: tells the leader CTA that this CTA's copy of a stage has landed
+//   warp 3      (leader CTA) scale copier: 12 tcgen05.cp per stage, shared memory -> tensor memory of both CTAs
 //   warps 4-7   epilogue: accumulator -> alpha -> BF16 / FP32 -> shared memory -> bulk tensor store
-//   warps 8-11  scale bytes: read from global memory two stages ahead (registers), window shift, written straight
-//               into tensor memory (tcgen05.st), one warp per lane quarter, two stages of scales resident
-// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 160..415, two
-// stages of scales in columns 416..511.  Two whole accumulators do not fit beside the scales, so the two overlap in
-// 96 columns: the epilogue drains those 96 first and hands them back, and the MMAs of the next tile run while the
-// other 160 columns are still being stored.
-// One thread issues a tensor instruction every 50-60 clocks at best (measured: 12 scale copies 578 clocks, 4 MMAs
-// 258 clocks into an idle pipe), so the issuing thread does nothing but the four MMAs and one commit per stage;
-// an earlier version that copied the scales from shared memory with tcgen05.cp (12 copies per stage, same thread)
-// spent 950 clocks per stage issuing.
+//   warps 8-11  scale bytes: read from global memory four stages ahead (registers), window shift, stored in the order
+//               the scale copy wants into a ring of six stages in shared memory
+// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 64..319, four
+// stages of scales in columns 320..511.  Two whole accumulators do not fit beside the scales, so the two overlap in
+// 192 columns: the epilogue drains those first and hands them back, and the MMAs of the next tile run while the
+// last 64 columns are still being stored.
+// The two issuing warps run their loops warp-uniformly and let one elected lane issue: the operands of the tensor
+// instructions are then uniform-register values.  Issued from a single lane's registers an instruction costs 50-80
+// clocks (measured into an idle pipe: 12 scale copies 578 clocks, 4 MMAs 258; with uniform operands 4 MMAs 82), and an
+// earlier version in which one such lane issued copies and MMAs spent 950 clocks per stage issuing, against 512
+// clocks of MMA work.
 // Every wait is bounded (SM clocks); on a time-out the role sets the status word, the other roles see the abort
 // flag, in-flight copies and MMAs are drained and the kernel returns.
 #include <cuda.h>
@@ -56,25 +57,28 @@ constexpr int BNH = 128;                    // B rows staged by each CTA
 constexpr int KCHUNK = 256;                 // K per stage
 constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks)
 constexpr int MMAS = KCHUNK / KMMA;
-constexpr int STAGES = 6;                   // payload stages
-constexpr int SF_SLOTS = 2;                 // stages whose scales are in tensor memory at a time
-constexpr int PF = 2;                       // group-stages (= 4 stages) the scale bytes are read ahead (registers)
-constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;    // CONV_WARPS per group, two groups
-constexpr int NUM_THREADS = 32 * (CONV_WARP0 + 2 * CONV_WARPS);
+constexpr int STAGES = 5;                   // payload stages
+constexpr int SF_SLOTS = 4;                 // stages whose scales are in tensor memory at a time
+constexpr int PF = 4;                       // stages the scale bytes are read ahead (registers)
+constexpr int SF_RING = 6;                  // stages of shifted scales in shared memory, on their way to tensor memory
+constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;
+constexpr int NUM_THREADS = 32 * (CONV_WARP0 + CONV_WARPS);
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;           // 16384
 constexpr int PK_B_BYTES = BNH * KCHUNK / 2;          // 16384
 constexpr int STAGE_BYTES = PK_A_BYTES + PK_B_BYTES;  // 32768
-constexpr int XCH_A_BYTES = BM * (KCHUNK / 16), XCH_BYTES = XCH_A_BYTES + BN * (KCHUNK / 16);   // 2048 + 4096 per group
-constexpr int SMEM_XCH = STAGES * STAGE_BYTES;        // 196608
-constexpr int SMEM_BARS = SMEM_XCH + 2 * XCH_BYTES;   // 208896
+constexpr int XCH_A_BYTES = BM * (KCHUNK / 16), XCH_BYTES = XCH_A_BYTES + BN * (KCHUNK / 16);   // 2048 + 4096 per stage
+constexpr int SMEM_XCH = STAGES * STAGE_BYTES;        // 163840
+constexpr int SMEM_BARS = SMEM_XCH + SF_RING * XCH_BYTES;   // 200704
 constexpr int SMEM_EPI = SMEM_BARS + 1024;
 constexpr int EPI_WARP_BYTES = 4096;
-constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 215040
-// Tensor memory (512 columns): accumulator of even tiles 0..255, of odd tiles 160..415 (they share 96 columns), then two
+constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 219136
+// Tensor memory (512 columns): accumulator of even tiles 0..255, of odd tiles 64..319 (they share 192 columns), then four
 // scale slots of 48 columns: 16 for A (column 4 j + g: rows 32 g + lane, MMA j) and 32 for B (column 8 j + 4 h + g).
-constexpr int TMEM_ACC_ODD = 160;
-constexpr int TMEM_SF_COL = 416, TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
+// A slot is written again only after the MMAs that read it have retired; four slots cover that turn-around (commit,
+// barrier, copies, commit, barrier, issue).
+constexpr int TMEM_ACC_ODD = 64;
+constexpr int TMEM_SF_COL = 320, TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
 
 struct NativeParams {
     int64_t Mo, No, Kc;
@@ -119,6 +123,21 @@ __device__ __forceinline__ void umma_fp4_block16(uint32_t tmem_d, uint32_t alo, 
         "setp.ne.b32 p, %7, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], da, db, %4, [%5], [%6], p;\n\t}"
         ::"r"(tmem_d), "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate) : "memory");
+}
+// 32 rows x 16 bytes of shared memory (in both CTAs of the pair, at the same offset) -> 4 columns of lanes 0..31 of every
+// lane quarter of each CTA's tensor memory; the descriptor is given as halves (see the MMA above).
+__device__ __forceinline__ void tmem_cp_32x128b(uint32_t taddr, uint32_t lo, uint32_t hi) {
+    asm volatile("{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\ttcgen05.cp.cta_group::2.32x128b.warpx4 [%0], d;\n\t}"
+                 ::"r"(taddr), "r"(lo), "r"(hi) : "memory");
+}
+// Descriptor of 32 rows of 16 bytes stored back to back: no swizzle, 8-row groups 128 bytes apart.
+__device__ __forceinline__ uint64_t sf_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(128 >> 4) << 16;
+    d |= (uint64_t)(128 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
 }
 // 16 consecutive 32-bit columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t r[16]) {
@@ -208,7 +227,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const uint32_t bar_base = smem_base + SMEM_BARS;
     // barriers (8 bytes each)
     const uint32_t pk_full = bar_base, pk_empty = bar_base + 64, pk_ready = bar_base + 128;
-    const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336;
+    const uint32_t sf_full = bar_base + 192, sf_empty = bar_base + 256;
+    const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336, drain_bar2 = bar_base + 360;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 344);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 352);
 
@@ -225,10 +245,15 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(pk_full + 8 * s, 1);
             mbar_init(pk_empty + 8 * s, 1);
-            // the leader's copy collects, for the stage that lives here, both CTAs' relays (payload landed) and both CTAs'
-            // scale warps (the stage's scales are in tensor memory)
-            mbar_init(pk_ready + 8 * s, 2 + 2 * CONV_WARPS);
+            // the leader's copy collects, for the stage that lives here, both CTAs' relays (payload landed) and the commit
+            // of the scale copies (the stage's scales are in tensor memory)
+            mbar_init(pk_ready + 8 * s, 3);
         }
+        for (int s = 0; s < SF_RING; ++s) {
+            mbar_init(sf_full + 8 * s, 2 * CONV_WARPS);        // the leader's copy collects both CTAs' scale warps
+            mbar_init(sf_empty + 8 * s, 1);
+        }
+        mbar_init(drain_bar2, 1);
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 8);
         mbar_init(drain_bar, 1);
@@ -267,7 +292,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 mbar_wait_drain(pk_full + 8 * (j % STAGES), (j / STAGES) & 1, &g_native_status, p.wait_limit);
             }
         }
-    } else if (warp == 3) {
+    } else if (warp == 2) {
         // ------------------------------------------------------------------ relay: this CTA's stage has landed
         if (lane == 0) {
             for (uint32_t it = 0; it < total; ++it) {
@@ -275,6 +300,53 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 if (!mbar_wait(pk_full + 8 * s, ph, abort_flag, p.wait_limit)) break;
                 mbar_arrive_cluster(pk_ready + 8 * s, 0);
             }
+        }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ scale copier (leader CTA)
+        // Shared memory -> tensor memory, for both CTAs at once: 12 copies per stage (A: one per MMA, B: two), each of
+        // which the hardware replicates to the four lane quarters.  Warp-uniform loop, one elected lane issues (see the
+        // MMA issuer).  The commit after the copies tells the MMA issuer that the stage's scales are in place and both
+        // CTAs' scale warps that the shared-memory stage may be rewritten.
+        if (rank == 0) {
+            bool ok = true;
+            const bool elected = elect_one();
+            const uint64_t d_sf = sf_smem_desc(smem_base + SMEM_XCH);
+            const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
+            const uint32_t tm0 = __shfl_sync(0xFFFFFFFFu, tmem_base, 0) + TMEM_SF_COL;
+            uint32_t s = 0, f = 0, fph = 0, u = 0;        // payload stage, shared-memory scale stage and phase, tensor-memory slot
+            for (uint32_t it = 0; it < total && ok; ++it) {
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(sf_full + 8 * f, fph, abort_flag, p.wait_limit));
+                if (!ok) break;
+                // the slot held the scales of stage it - SF_SLOTS: free once that stage's MMAs have retired, which is what
+                // the payload barrier of that stage says
+                if (it >= SF_SLOTS) {
+                    const uint32_t prev = it - SF_SLOTS;
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(pk_empty + 8 * (prev % STAGES), (prev / STAGES) & 1, abort_flag, p.wait_limit));
+                    if (!ok) break;
+                }
+                tc_fence_after();
+                const uint32_t lo = sf_lo0 + f * (XCH_BYTES >> 4), lob = lo + (XCH_A_BYTES >> 4);
+                const uint32_t sfa = tm0 + u * TMEM_SF_SLOT_COLS, sfb = sfa + TMEM_SFB_OFF;
+                if (elected) {
+#pragma unroll
+                    for (int j = 0; j < MMAS; ++j) {
+                        tmem_cp_32x128b(sfa + 4 * j, lo + j * (512 >> 4), sf_hi);
+                        tmem_cp_32x128b(sfb + 8 * j, lob + j * (1024 >> 4), sf_hi);
+                        tmem_cp_32x128b(sfb + 8 * j + 4, lob + j * (1024 >> 4) + (512 >> 4), sf_hi);
+                    }
+                    umma_commit_local(pk_ready + 8 * s);
+                    umma_commit_pair(sf_empty + 8 * f);
+                }
+                __syncwarp();
+                if (++s == STAGES) s = 0;
+                if (++f == SF_RING) { f = 0; fph ^= 1; }
+                u = (u + 1) & (SF_SLOTS - 1);
+            }
+            if (elected) {
+                umma_commit_local(drain_bar2);
+                mbar_wait_drain(drain_bar2, 0, &g_native_status, p.wait_limit);
+            }
+            __syncwarp();
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
@@ -313,7 +385,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     }
                     __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1; }
-                    u ^= 1;
+                    u = (u + 1) & (SF_SLOTS - 1);
                 }
                 if (ok && elected) umma_commit_pair(acc_full);
                 __syncwarp();
@@ -342,24 +414,22 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             const int row0 = mb * BM + q * 32, col0 = nb * BN;
             const uint32_t odd = tl & 1;
             const uint32_t acc = tmem_base + ((uint32_t)(q * 32) << 16) + (odd ? TMEM_ACC_ODD : 0);
-            // The 96 columns both accumulators share (the last 96 of an even tile, the first 96 of an odd one) are read
-            // first; once every epilogue warp of the pair has them in registers the next tile's MMAs may start.  Units
-            // of 32 columns: an even tile goes 6 7 | 5 4 | 0 1 | 2 3, an odd one 0 1 | 2 3 | 4 5 | 6 7, and the hand-back
-            // comes after the third unit.
+            // The 192 columns both accumulators share (the last 192 of an even tile, the first 192 of an odd one) are read
+            // first; once every epilogue warp of the pair has read them the next tile's MMAs may start.  Chunks of 64
+            // columns: an even tile goes 3 2 1 | 0, an odd one 0 1 2 | 3, and the hand-back comes after the third chunk.
             if (p.out_bf16) {
 #pragma unroll 1
                 for (int i = 0; i < BN / 64; ++i) {
-                    const int cc = odd ? i : (i == 0 ? 3 : i == 1 ? 2 : i - 2);      // chunk of 64 columns: 3 2 0 1 | 0 1 2 3
+                    const int cc = odd ? i : 3 - i;                                  // chunk of 64 columns: 3 2 1 | 0 or 0 1 2 | 3
                     uint8_t* mine = stage_gen + lane * 128;
                     const int sw = lane & 7;
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
-                        // inside the second chunk the shared unit comes first (even: unit 5 before 4)
-                        const int half = (!odd && i == 1) ? (hh ^ 1) : hh;
+                        const int half = hh;
                         uint32_t r[32];
                         tmem_ld32(acc + cc * 64 + half * 32, r);
                         tmem_ld_wait();
-                        if (i == 1 && hh == 0) {
+                        if (i == 2 && hh == 1) {
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -385,12 +455,12 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             } else {
 #pragma unroll 1
                 for (int i = 0; i < BN / 32; ++i) {
-                    // units of 32 columns: even 6 7 5 4 0 1 2 3, odd 0 1 2 3 4 5 6 7
-                    const int c = odd ? i : (i < 2 ? 6 + i : i == 2 ? 5 : i == 3 ? 4 : i - 4);
+                    // units of 32 columns: even 7 6 5 4 3 2 | 1 0, odd 0 1 2 3 4 5 | 6 7
+                    const int c = odd ? i : 7 - i;
                     uint32_t r[32];
                     tmem_ld32(acc + c * 32, r);
                     tmem_ld_wait();
-                    if (i == 2) {
+                    if (i == 5) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -412,14 +482,13 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         }
         if (lane == 0) tma_store_wait_all();
     } else if (warp >= CONV_WARP0) {
-        // ------------------------------------------------------------------ scale bytes: window shift, into tensor memory
+        // ------------------------------------------------------------------ scale bytes: window shift and re-layout
         // The tensor core wants the scales of row 32 g + r in lane r (of every lane quarter), one column per (MMA, g) with
-        // the MMA's four block scales as its bytes.  Two groups of four warps take the stages in turn (group = stage
-        // parity = scale slot).  A group's 128 threads read one row each of A and of the two B halves (16 bytes per row
-        // and stage, PF group-stages ahead in registers), shift the codes, and exchange them through shared memory in
-        // the order [MMA][lane][g] (32 consecutive words per warp store); then warp w reads the 12 x 16 bytes of its lane
-        // and writes lane quarter w of the slot with two tcgen05.st.
-        const int cg = (warp - CONV_WARP0) >> 2, cw = warp & 3;
+        // the MMA's four block scales as its bytes; the scale copy (32 rows x 16 bytes -> 4 columns) makes that from
+        // shared memory laid out [MMA][r][g] in 4-byte words.  The 128 threads read one row each of A and of the two B
+        // halves (16 bytes per row and stage, PF stages ahead in registers), shift the codes and store them there; the
+        // lane assignment makes a warp's 32 stores consecutive words.
+        const int cw = warp - CONV_WARP0;
         const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);            // the row this thread reads
         const uint32_t da = (uint32_t)((8 * ka) & 0xFF) * 0x01010101u, db = (uint32_t)((8 * kb) & 0xFF) * 0x01010101u;
         const int64_t kblocks = p.Kc >> 4;
@@ -440,7 +509,11 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             pb0 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + row);
             pb1 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + BNH + row);
         };
-        auto advance = [&]() {                       // the cursor moves on by one stage
+        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            a = pa ? ldg_nc_16(pa) : z;
+            b0 = pb0 ? ldg_nc_16(pb0) : z;
+            b1 = pb1 ? ldg_nc_16(pb1) : z;
             if (++c_kc == kchunks) {
                 c_kc = 0;
                 c_tile += num_pairs;
@@ -451,62 +524,29 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 if (pb1) pb1 += step_b;
             }
         };
-        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {     // this group's next stage; the other group's is skipped
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            a = pa ? ldg_nc_16(pa) : z;
-            b0 = pb0 ? ldg_nc_16(pb0) : z;
-            b1 = pb1 ? ldg_nc_16(pb1) : z;
-            advance();
-            advance();
-        };
         open_tile();
-        if (cg) advance();
         uint4 ra[PF], rb0[PF], rb1[PF];
 #pragma unroll
         for (int d = 0; d < PF; ++d) fetch(ra[d], rb0[d], rb1[d]);
         bool ok = true;
-        uint8_t* xch = smem_gen + SMEM_XCH + cg * XCH_BYTES;
-        uint32_t* xa = reinterpret_cast<uint32_t*>(xch) + cw * 32 + lane;            // + 128 j
-        uint32_t* xb = reinterpret_cast<uint32_t*>(xch + XCH_A_BYTES) + cw * 32 + lane;   // + 256 j + 128 h
-        const uint4* ya = reinterpret_cast<const uint4*>(xch) + lane;                 // + 32 j
-        const uint4* yb = reinterpret_cast<const uint4*>(xch + XCH_A_BYTES) + lane;   // + 64 j + 32 h
-        const uint32_t slot = tmem_base + ((uint32_t)(cw * 32) << 16) + TMEM_SF_COL + cg * TMEM_SF_SLOT_COLS;
-        const int bar_id = 1 + cg;
-        for (uint32_t base = cg; base < total && ok; base += 2 * PF) {
+        uint32_t f = 0, fph = 0;
+        for (uint32_t base = 0; base < total && ok; base += PF) {
 #pragma unroll
             for (int d = 0; d < PF; ++d) {
-                const uint32_t it = base + 2 * d;
+                const uint32_t it = base + d;
                 if (it >= total || !ok) break;
+                if (!mbar_wait(sf_empty + 8 * f, fph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
+                uint32_t* xa = reinterpret_cast<uint32_t*>(smem_gen + SMEM_XCH + f * XCH_BYTES) + cw * 32 + lane;     // + 128 j
+                uint32_t* xb = xa + XCH_A_BYTES / 4;                                                                  // + 256 j + 128 h
                 const uint4 a = ra[d], b0 = rb0[d], b1 = rb1[d];
                 xa[0] = shift(a.x, da); xa[128] = shift(a.y, da); xa[256] = shift(a.z, da); xa[384] = shift(a.w, da);
                 xb[0] = shift(b0.x, db); xb[256] = shift(b0.y, db); xb[512] = shift(b0.z, db); xb[768] = shift(b0.w, db);
                 xb[128] = shift(b1.x, db); xb[384] = shift(b1.y, db); xb[640] = shift(b1.z, db); xb[896] = shift(b1.w, db);
+                fence_proxy_async();                 // the tensor core's scale copy reads what was just written
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(sf_full + 8 * f, 0);
                 fetch(ra[d], rb0[d], rb1[d]);
-                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // the group's 128 rows are in place
-                uint32_t ca[16], cb[32];
-#pragma unroll
-                for (int j = 0; j < MMAS; ++j) {
-                    const uint4 va = ya[32 * j], v0 = yb[64 * j], v1 = yb[64 * j + 32];
-                    ca[4 * j] = va.x; ca[4 * j + 1] = va.y; ca[4 * j + 2] = va.z; ca[4 * j + 3] = va.w;
-                    cb[8 * j] = v0.x; cb[8 * j + 1] = v0.y; cb[8 * j + 2] = v0.z; cb[8 * j + 3] = v0.w;
-                    cb[8 * j + 4] = v1.x; cb[8 * j + 5] = v1.y; cb[8 * j + 6] = v1.z; cb[8 * j + 7] = v1.w;
-                }
-                // the slot held the scales of stage it - 2: free once that stage's MMAs have retired, which is what the
-                // payload barrier of that stage says
-                if (it >= SF_SLOTS) {
-                    const uint32_t prev = it - SF_SLOTS;
-                    if (!mbar_wait(pk_empty + 8 * (prev % STAGES), (prev / STAGES) & 1, abort_flag, p.wait_limit)) ok = false;
-                    tc_fence_after();
-                }
-                if (ok) {
-                    tmem_st16(slot, ca);
-                    tmem_st32(slot + TMEM_SFB_OFF, cb);
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(pk_ready + 8 * (it % STAGES), 0);
-                }
-                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // everyone has read: the exchange buffer is free
+                if (++f == SF_RING) { f = 0; fph ^= 1; }
             }
         }
     }
