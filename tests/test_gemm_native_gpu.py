@@ -175,3 +175,30 @@ def test_native_is_deterministic_and_independent_of_the_workspace_contents():
     again = lib.gemm_native(lib.FPROP, qa, qb, torch.bfloat16, workspace=ws)
     torch.cuda.synchronize()
     assert torch.equal(first, again)
+
+
+def test_quantized_operands_of_the_workload_recipe_take_the_native_kernel():
+    """Operands quantized against a fresh tensor reference with T = 448 (channel-scaled activations, N(0, 0.02^2) weights,
+    heavy-tailed gradients with stochastic rounding) have scale codes inside one window, so the three products of a
+    linear run on the native kernel; the outputs match the exact oracle on the same operand bytes."""
+    import synth_inputs as si
+    M, K, N = 512, 768, 1024
+    x = si.channel_scaled_activation(M, K, seed=11, device=DEV)
+    w = si.weight(N, K, seed=12, device=DEV)
+    dy = si.heavy_tailed_gradient(M, N, seed=13, device=DEV)
+    gx, gw, gg = (lib.sample_amax(t) for t in (x, w, dy))
+    qx = lib.quantize(x, lib.LAYOUT_1D_ROW, lib.ROUND_RNE, gx, 448.0)
+    qxt = lib.quantize(x, lib.LAYOUT_1D_COL, lib.ROUND_RNE, gx, 448.0)
+    qw = lib.quantize(w, lib.LAYOUT_2D, lib.ROUND_RNE, gw, 448.0, want_transpose=True)
+    qg = lib.quantize(dy, lib.LAYOUT_1D_ROW, lib.ROUND_SR, gg, 448.0, seed=4)
+    qgt = lib.quantize(dy, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, 448.0, seed=5)
+    for a, b, Mo, No in ((qx, qw, M, N), (qg, qw.transposed(), M, K), (qgt, qxt, N, K)):
+        out, ws = _native(a, b, torch.float32, Mo, No)
+        assert not bool(torch.isnan(out).any())                       # the native kernel did the product
+        for hi, inv in ((ws[0], ws[1]), (ws[2], ws[3])):
+            from paper_2609_02846_b200.binding import scale_window
+            assert scale_window(255 - inv, hi) is not None
+        a2d, b2d = a.scale_mode == lib.SCALE_2D, b.scale_mode == lib.SCALE_2D
+        y, sa = oracle.gemm(a.payload.cpu().numpy(), a.scales.cpu().numpy(), a2d, float(a.decode.item()),
+                            b.payload.cpu().numpy(), b.scales.cpu().numpy(), b2d, np.float32(b.decode.item()))
+        check_gemm_output(out, y, sa)
