@@ -164,6 +164,7 @@ __device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
 __global__ void __launch_bounds__(512) scale_range_kernel(const uint8_t* __restrict__ a, int64_t na, const uint8_t* __restrict__ b,
                                                           int64_t nb, int* __restrict__ range) {
     __shared__ uint32_t part[16][4];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the GEMM's prologue may run beside this kernel
     uint32_t red[4];                                      // max A, 255 - min nonzero A, max B, 255 - min nonzero B
     for (int op = 0; op < 2; ++op) {
         const uint8_t* s = op ? b : a;
@@ -218,9 +219,6 @@ __global__ void __launch_bounds__(512) scale_range_kernel(const uint8_t* __restr
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_out, const NativeParams p) {
-    int ka, kb;
-    if (!native_windows(p.range, ka, kb)) return;            // uniform over the grid: the FP16 kernel does this product
-
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -266,8 +264,14 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above touched only this CTA pair's shared and tensor memory and may have run while the range kernel was
+    // still at work (programmatic dependent launch); its four words are read from here on.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    int ka, kb;
+    const bool work = native_windows(p.range, ka, kb);       // uniform over the grid; false: the FP16 kernel does this product
 
-    if (warp == 0) {
+    if (!work) {
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ copies
         if (lane == 0) {
             uint32_t it = 0;
@@ -672,8 +676,19 @@ int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStr
     p.stall_producer = g.stall_producer;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int pairs = num_tiles < resident_pairs[dev] ? num_tiles : resident_pairs[dev];
-    gemm_native_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mo, p);
-    return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
+    // Programmatic dependent launch: the kernel's prologue (barriers, tensor-memory allocation, cluster barrier) runs
+    // beside the range kernel, which releases its dependents at once; the kernel waits for it before reading the range.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_native_kernel, ma, mb, mo, p) == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
 int read_and_clear_native_status() {
