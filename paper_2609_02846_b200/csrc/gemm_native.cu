@@ -22,8 +22,9 @@
 //   warp 2      tensor-memory allocation; relay: tells the leader CTA that this CTA's copy of a stage has landed
 //   warp 3      (leader CTA) scale copier: 12 tcgen05.cp per stage, shared memory -> tensor memory of both CTAs
 //   warps 4-7   epilogue: accumulator -> alpha -> BF16 / FP32 -> shared memory -> bulk tensor store
-//   warps 8-11  scale bytes: read from global memory four stages ahead (registers), window shift, stored in the order
-//               the scale copy wants into a ring of six stages in shared memory
+//   warps 8-15  scale bytes, two groups of four warps taking the stages in turn: read from global memory four stages
+//               ahead (registers), window shift, stored in the order the scale copy wants into a ring of six stages
+//               in shared memory
 // Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 64..319, four
 // stages of scales in columns 320..511.  Two whole accumulators do not fit beside the scales, so the two overlap in
 // 192 columns: the epilogue drains those first and hands them back, and the MMAs of the next tile run while the
@@ -59,10 +60,11 @@ constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks
 constexpr int MMAS = KCHUNK / KMMA;
 constexpr int STAGES = 5;                   // payload stages
 constexpr int SF_SLOTS = 4;                 // stages whose scales are in tensor memory at a time
-constexpr int PF = 4;                       // stages the scale bytes are read ahead (registers)
+constexpr int PF = 2;                       // group-stages (= 4 stages) the scale bytes are read ahead (registers)
 constexpr int SF_RING = 6;                  // stages of shifted scales in shared memory, on their way to tensor memory
-constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;
-constexpr int NUM_THREADS = 32 * (CONV_WARP0 + CONV_WARPS);
+constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;    // CONV_WARPS per group; two groups take the stages in turn
+constexpr int NUM_THREADS = 32 * (CONV_WARP0 + 2 * CONV_WARPS);
+static_assert(SF_RING % 2 == 0, "each scale group owns every other ring stage");
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;           // 16384
 constexpr int PK_B_BYTES = BNH * KCHUNK / 2;          // 16384
@@ -77,8 +79,10 @@ constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 219136
 // scale slots of 48 columns: 16 for A (column 4 j + g: rows 32 g + lane, MMA j) and 32 for B (column 8 j + 4 h + g).
 // A slot is written again only after the MMAs that read it have retired; four slots cover that turn-around (commit,
 // barrier, copies, commit, barrier, issue).
-constexpr int TMEM_ACC_ODD = 64;
-constexpr int TMEM_SF_COL = 320, TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
+constexpr int TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
+constexpr int OVERLAP_UNITS = (SF_SLOTS * TMEM_SF_SLOT_COLS + 31) / 32;       // 32-column units the two accumulators share
+constexpr int TMEM_ACC_ODD = 256 - 32 * OVERLAP_UNITS;
+constexpr int TMEM_SF_COL = TMEM_ACC_ODD + 256;
 
 struct NativeParams {
     int64_t Mo, No, Kc;
@@ -344,7 +348,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 __syncwarp();
                 if (++s == STAGES) s = 0;
                 if (++f == SF_RING) { f = 0; fph ^= 1; }
-                u = (u + 1) & (SF_SLOTS - 1);
+                if (++u == SF_SLOTS) u = 0;
             }
             if (elected) {
                 umma_commit_local(drain_bar2);
@@ -389,7 +393,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     }
                     __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1; }
-                    u = (u + 1) & (SF_SLOTS - 1);
+                    if (++u == SF_SLOTS) u = 0;
                 }
                 if (ok && elected) umma_commit_pair(acc_full);
                 __syncwarp();
@@ -424,16 +428,16 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             if (p.out_bf16) {
 #pragma unroll 1
                 for (int i = 0; i < BN / 64; ++i) {
-                    const int cc = odd ? i : 3 - i;                                  // chunk of 64 columns: 3 2 1 | 0 or 0 1 2 | 3
+                    const int cc = odd ? i : 3 - i;                                  // chunk of 64 columns, shared ones first
                     uint8_t* mine = stage_gen + lane * 128;
                     const int sw = lane & 7;
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
-                        const int half = hh;
+                        const int half = odd ? hh : hh ^ 1;                           // inside a chunk too: the shared unit first
                         uint32_t r[32];
                         tmem_ld32(acc + cc * 64 + half * 32, r);
                         tmem_ld_wait();
-                        if (i == 2 && hh == 1) {
+                        if (2 * i + hh == OVERLAP_UNITS - 1) {
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -464,7 +468,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     uint32_t r[32];
                     tmem_ld32(acc + c * 32, r);
                     tmem_ld_wait();
-                    if (i == 5) {
+                    if (i == OVERLAP_UNITS - 1) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
@@ -489,10 +493,10 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         // ------------------------------------------------------------------ scale bytes: window shift and re-layout
         // The tensor core wants the scales of row 32 g + r in lane r (of every lane quarter), one column per (MMA, g) with
         // the MMA's four block scales as its bytes; the scale copy (32 rows x 16 bytes -> 4 columns) makes that from
-        // shared memory laid out [MMA][r][g] in 4-byte words.  The 128 threads read one row each of A and of the two B
-        // halves (16 bytes per row and stage, PF stages ahead in registers), shift the codes and store them there; the
-        // lane assignment makes a warp's 32 stores consecutive words.
-        const int cw = warp - CONV_WARP0;
+        // shared memory laid out [MMA][r][g] in 4-byte words.  Two groups of four warps take the stages in turn; a group's
+        // 128 threads read one row each of A and of the two B halves (16 bytes per row and stage, PF group-stages ahead in
+        // registers), shift the codes and store them there; the lane assignment makes a warp's 32 stores consecutive words.
+        const int cg = (warp - CONV_WARP0) >> 2, cw = warp & 3;          // group (= stage parity), warp inside the group
         const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);            // the row this thread reads
         const uint32_t da = (uint32_t)((8 * ka) & 0xFF) * 0x01010101u, db = (uint32_t)((8 * kb) & 0xFF) * 0x01010101u;
         const int64_t kblocks = p.Kc >> 4;
@@ -513,11 +517,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             pb0 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + row);
             pb1 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + BNH + row);
         };
-        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            a = pa ? ldg_nc_16(pa) : z;
-            b0 = pb0 ? ldg_nc_16(pb0) : z;
-            b1 = pb1 ? ldg_nc_16(pb1) : z;
+        auto advance = [&]() {                       // the cursor moves on by one stage
             if (++c_kc == kchunks) {
                 c_kc = 0;
                 c_tile += num_pairs;
@@ -528,16 +528,25 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 if (pb1) pb1 += step_b;
             }
         };
+        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {     // this group's next stage; the other group's is skipped
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            a = pa ? ldg_nc_16(pa) : z;
+            b0 = pb0 ? ldg_nc_16(pb0) : z;
+            b1 = pb1 ? ldg_nc_16(pb1) : z;
+            advance();
+            advance();
+        };
         open_tile();
+        if (cg) advance();
         uint4 ra[PF], rb0[PF], rb1[PF];
 #pragma unroll
         for (int d = 0; d < PF; ++d) fetch(ra[d], rb0[d], rb1[d]);
         bool ok = true;
-        uint32_t f = 0, fph = 0;
-        for (uint32_t base = 0; base < total && ok; base += PF) {
+        uint32_t f = cg, fph = 0;
+        for (uint32_t base = cg; base < total && ok; base += 2 * PF) {
 #pragma unroll
             for (int d = 0; d < PF; ++d) {
-                const uint32_t it = base + d;
+                const uint32_t it = base + 2 * d;
                 if (it >= total || !ok) break;
                 if (!mbar_wait(sf_empty + 8 * f, fph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 uint32_t* xa = reinterpret_cast<uint32_t*>(smem_gen + SMEM_XCH + f * XCH_BYTES) + cw * 32 + lane;     // + 128 j
@@ -550,7 +559,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(sf_full + 8 * f, 0);
                 fetch(ra[d], rb0[d], rb1[d]);
-                if (++f == SF_RING) { f = 0; fph ^= 1; }
+                f += 2;
+                if (f >= SF_RING) { f -= SF_RING; fph ^= 1; }
             }
         }
     }
