@@ -202,3 +202,36 @@ def test_quantized_operands_of_the_workload_recipe_take_the_native_kernel():
         y, sa = oracle.gemm(a.payload.cpu().numpy(), a.scales.cpu().numpy(), a2d, float(a.decode.item()),
                             b.payload.cpu().numpy(), b.scales.cpu().numpy(), b2d, np.float32(b.decode.item()))
         check_gemm_output(out, y, sa)
+
+
+def test_native_seeded_sweep_over_shapes_modes_windows_and_strides():
+    """Forty seeded cases: Mo, No multiples of 128 up to 1152, Kc multiples of 256 up to 2048, every pair of scale layouts, a
+    random window position and width per operand, FP32 or BF16 output written into a wider buffer (ldo > No)."""
+    rng = np.random.default_rng(20261125)
+    for case in range(40):
+        Mo, No = (int(rng.integers(1, 10)) * 128 for _ in range(2))
+        Kc = int(rng.integers(1, 9)) * 256
+        ma, mb = int(rng.integers(0, 3)), int(rng.integers(0, 3))
+        wins = []
+        for _ in range(2):
+            k = int(rng.integers(0, 16))
+            lo = 8 * k + 8 + int(rng.integers(0, 8))
+            hi = min(lo + int(rng.integers(1, 8 * k + 127 - lo)), 8 * k + 126, 0xF7)
+            wins.append((lo, hi + 1))
+        # decode factors that bring the products near 1 whatever the windows are
+        mid = [2.0 ** ((w[0] + w[1]) // 16 - 15) for w in wins]
+        da, db = float(2.0 ** -round(np.log2(mid[0]))), float(2.0 ** -round(np.log2(mid[1])) / 64)
+        qa, ap, asc = _operand(rng, Mo, Kc, ma, *wins[0], dec=da)
+        qb, bp, bsc = _operand(rng, No, Kc, mb, *wins[1], dec=db)
+        dtype = torch.float32 if case % 2 else torch.bfloat16
+        ldo = No + 64 * int(rng.integers(0, 3))
+        buf = torch.full((Mo, ldo), float("nan"), dtype=dtype, device=DEV)
+        out = buf[:, :No]
+        lib.gemm_native(lib.FPROP, qa, qb, dtype, out=out)
+        torch.cuda.synchronize()
+        assert lib.last_device_status() == 0
+        assert not bool(torch.isnan(out).any()), (case, Mo, No, Kc, ma, mb, wins)
+        if ldo > No:
+            assert bool(torch.isnan(buf[:, No:]).all())               # nothing beyond the output's columns
+        y, sa = oracle.gemm(ap, asc, ma == 2, da, bp, bsc, mb == 2, np.float32(db))
+        check_gemm_output(out.contiguous(), y, sa)

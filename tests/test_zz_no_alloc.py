@@ -31,7 +31,7 @@ def test_static_workspace_gemm_equals_gemm_on_two_calls_in_a_row():
     torch.cuda.synchronize()
     free0, _ = torch.cuda.mem_get_info()
     # two calls in a row, no synchronisation in between; then the other kernel's case twice: the words a call finds
-    # are those of the call before it, with the opposite verdict
+    # are those of the call before it, with the opposite outcome
     lib.gemm_static(lib.FPROP, *windowed, out=out[0])
     lib.gemm_static(lib.FPROP, *wide, out=out[1])
     lib.gemm_static(lib.FPROP, *wide, out=out[2])
