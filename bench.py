@@ -327,7 +327,7 @@ GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the default workload (mean of fprop, dgrad, wgrad;
 # one ncu pass each; summaries in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt and
 # profiles/gemm_native_kernel_linear_M8192_K4096_N16384_ncu_full.txt).  Algorithmic bytes: 238 MB per launch.
-GEMM_DRAM_TRAFFIC_BYTES = {"gemm_kernel": (150.5e6 + 220.5e6 + 188.9e6 + 47.9e6 + 101.1e6 + 99.5e6) / 3,
+GEMM_DRAM_TRAFFIC_BYTES = {"gemm_kernel": (150.3e6 + 220.9e6 + 195.0e6 + 48.0e6 + 100.7e6 + 99.1e6) / 3,
                            "gemm_native_kernel": (151.5e6 + 221.6e6 + 195.8e6 + 51.1e6 + 100.1e6 + 104.7e6) / 3}
 NOMINAL_FP4_OVER_BF16 = 4.0      # dense tensor peaks of the part: 9 PFLOP/s FP4, 2.25 PFLOP/s BF16
 
