@@ -282,21 +282,19 @@ class LinearStep:
 
 
     def gemm_kernels(self):
-        """Which kernel ue5m3_gemm uses for each of the three products of the step just run: the code ranges of the
-        operands' scales (ue5m3_gemm_native writes them to its workspace) decide, by the same rule as on the device."""
+        """Which kernel ue5m3_gemm uses for each of the three products of the step just run: ue5m3_gemm_native says in its
+        workspace whether every scale row of the two operands had a window (then it did the product)."""
         lib, q, torch = self.lib, self.q, self.torch
-        from paper_2609_02846_b200.binding import scale_window
         out = {}
         for name, a, b, c in (("gemm_fprop", q["x"], q["w"], self.Y), ("gemm_dgrad", q["g"], q["w"].transposed(), self.dX),
                               ("gemm_wgrad", q["gt"], q["xt"], self.dW)):
             if self.gemm_launches == 1 or a.Kc % 256:
                 out[name] = "gemm_kernel"
                 continue
-            ws = torch.zeros(4, dtype=torch.int32, device=c.device)
+            ws = lib.gemm_native_workspace(a, b)
             lib.gemm_native(lib.FPROP, a, b, out=c, workspace=ws)
             torch.cuda.synchronize()
-            r = ws.tolist()
-            ok = all(hi == 0 or scale_window(255 - inv, hi) is not None for hi, inv in ((r[0], r[1]), (r[2], r[3])))
+            ok = lib.native_windows(ws, a, b)[0]
             out[name] = "gemm_native_kernel" if ok else "gemm_kernel"
         return out
 

@@ -63,6 +63,8 @@ def _load() -> C.CDLL:
         L.ue5m3_gemm_static.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_fp16.restype = ci
         L.ue5m3_gemm_fp16.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
+        L.ue5m3_gemm_native_workspace_bytes.restype = C.c_size_t
+        L.ue5m3_gemm_native_workspace_bytes.argtypes = [i64, i64, ci, ci]
         L.ue5m3_gemm_native.restype = ci
         L.ue5m3_gemm_native.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp, vp]
         L.ue5m3_gemm_probe_matched.restype = ci
@@ -308,12 +310,15 @@ def gemm_static(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: to
 
 def scale_window(cmin: int, cmax: int) -> Optional[int]:
     """The rule by which ue5m3_gemm decides between its two kernels, restated on the host: the shift k with
-    8 <= c - 8k <= 126 for all codes cmin..cmax of an operand (then UE5M3 code c and UE4M3 code c - 8k denote values
-    that differ by exactly 2^(k - 8)), or None when the operand has no such window."""
+    8 <= c - 8k <= 126 for all non-zero codes cmin..cmax of a scale row (then UE5M3 code c and UE4M3 code c - 8k denote
+    values that differ by exactly 2^(k - 8)), or None when the row has no such window."""
     if cmin < 8 or cmax > 0xF7 or cmin > cmax:
         return None
-    k = (cmin - 8) >> 3
-    return k if cmax - 8 * k <= 126 else None
+    k_lo = (cmax - 126 + 7) >> 3 if cmax > 126 else 0   # the smallest shift that brings cmax down to 126
+    k_hi = (cmin - 8) >> 3                              # the largest one that keeps cmin at 8 or above
+    if k_lo > k_hi:
+        return None
+    return 2 if k_lo <= 2 <= k_hi else k_lo             # rows agree on 2 where they can
 
 
 def gemm_fp16(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
@@ -332,17 +337,32 @@ def gemm_fp16(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torc
     return out
 
 
+def gemm_native_workspace(a: QuantizedOperand, b: QuantizedOperand) -> torch.Tensor:
+    """A workspace of the size ue5m3_gemm_native wants for these operands (uint8, device)."""
+    n = _load().ue5m3_gemm_native_workspace_bytes(a.R, b.R, a.scale_mode, b.scale_mode)
+    return torch.empty(int(n), dtype=torch.uint8, device=a.payload.device)
+
+
+def native_windows(workspace: torch.Tensor, a: QuantizedOperand, b: QuantizedOperand):
+    """Reads a workspace back: (all rows have windows, k of A's scale rows, k of B's scale rows) as numpy arrays."""
+    w = workspace.cpu().numpy()
+    ra = a.R // 16 if a.scale_mode == SCALE_2D else a.R
+    rb = b.R // 16 if b.scale_mode == SCALE_2D else b.R
+    off_b = 16 + ((ra + 15) // 16) * 16
+    return int(w[:4].view("int32")[0]) == 0, w[16:16 + ra].copy(), w[off_b:off_b + rb].copy()
+
+
 def gemm_native(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torch.dtype = torch.bfloat16,
                 out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """The product of `gemm` on the tensor core's FP4 path (ue5m3_gemm_native).  `workspace` (4 x int32, device) receives
-    the code ranges of the two operands' scales; `out` is left untouched when an operand has no UE4M3 window."""
+    """The product of `gemm` on the tensor core's FP4 path (ue5m3_gemm_native).  `workspace` (see gemm_native_workspace)
+    receives the window shift of every scale row; `out` is left untouched when some row has no UE4M3 window."""
     Mo, No, Kc = a.R, b.R, a.Kc
     if b.Kc != Kc:
         raise ValueError(f"contraction sizes differ: {Kc} vs {b.Kc}")
     if out is None:
         out = torch.empty((Mo, No), dtype=out_dtype, device=a.payload.device)
     if workspace is None:
-        workspace = torch.empty(4, dtype=torch.int32, device=out.device)
+        workspace = gemm_native_workspace(a, b)
     with torch.cuda.device(out.device):
         _check(_load().ue5m3_gemm_native(op, Mo, No, Kc,
                                          _dev_ptr(a.payload), _dev_ptr(a.scales), a.scale_mode, _dev_ptr(a.decode),

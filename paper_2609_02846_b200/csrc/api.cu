@@ -212,9 +212,9 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
     if (!native_eligible(g)) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
-    // Three launches, one of which does the product: the scale-code ranges, the native FP4 kernel (works when both
-    // operands have a UE4M3 window) and the FP16 kernel (works when they do not).
-    int* ws = native_workspace();
+    // Three launches, one of which does the product: the windows of the scale rows, the native FP4 kernel (works when
+    // every scale row of both operands has a UE4M3 window) and the FP16 kernel (works when one does not).
+    int* ws = native_workspace(native_workspace_bytes(g));
     if (!ws) return UE5M3_ERR_CUDA;
     int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
@@ -235,10 +235,9 @@ int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t*
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
-    if (!native_eligible(g)) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
-    const size_t need = 4 * sizeof(int);              // the four range words; does not grow with the problem
-    int* ws = static_workspace(need);
-    if (!ws) return UE5M3_ERR_UNSUPPORTED;
+    if (Kc % 256) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);      // the FP16 kernel alone: no workspace
+    int* ws = static_workspace(native_workspace_bytes(g));    // 16 bytes + one per scale row of the two operands
+    if (!ws) return UE5M3_ERR_UNSUPPORTED;            // more rows than the file-scope array holds
     int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
     r = launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
@@ -261,6 +260,13 @@ int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a
     return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
 }
 
+size_t ue5m3_gemm_native_workspace_bytes(int64_t Mo, int64_t No, int a_scale_mode, int b_scale_mode) {
+    if (Mo <= 0 || No <= 0) return 0;
+    GemmArgs g{};
+    g.Mo = Mo; g.No = No; g.a_scale_mode = a_scale_mode; g.b_scale_mode = b_scale_mode;
+    return native_workspace_bytes(g);
+}
+
 int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
                       int a_scale_mode, const float* a_decode, const uint8_t* b_payload, const uint8_t* b_scales,
                       int b_scale_mode, const float* b_decode, void* out, int out_dtype, int64_t ldo, int32_t* workspace,
@@ -276,7 +282,7 @@ int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t*
     if (di.major != 10) return UE5M3_ERR_UNSUPPORTED;
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
-    if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
+    if (Kc % 256) return UE5M3_ERR_UNSUPPORTED;
     const int r = launch_scale_range(g, workspace, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
     return launch_gemm_native(g, workspace, di.sms, (cudaStream_t)stream);
@@ -320,7 +326,8 @@ int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, con
     g.stall_producer = 1;
     if (which == 2) {
         // the native kernel: its workspace is filled by the range kernel as in ue5m3_gemm (the operands must have windows)
-        int* ws = native_workspace();
+        if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
+        int* ws = native_workspace(native_workspace_bytes(g));
         if (!ws) return UE5M3_ERR_CUDA;
         const int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
         if (r != UE5M3_OK) return r;

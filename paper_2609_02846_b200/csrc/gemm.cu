@@ -116,10 +116,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
             const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
-    if (p.range) {
-        int ka, kb;
-        if (native_windows(p.range, ka, kb)) return;        // uniform over the grid
-    }
+    if (p.range && native_all_rows_have_windows(p.range)) return;      // uniform over the grid
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));

@@ -88,7 +88,9 @@ struct NativeParams {
     int64_t Mo, No, Kc;
     const float* a_decode;
     const float* b_decode;
-    const int* range;             // {max A, 255 - min nonzero A, max B, 255 - min nonzero B}
+    const int* workspace;         // word 0: 0 when every scale row has a window (layout in window.cuh)
+    const uint8_t* ka_rows;       // shift k of every scale row of A
+    const uint8_t* kb_rows;       // ... of B
     const uint8_t* a_scales;
     const uint8_t* b_scales;
     int out_bf16;
@@ -158,58 +160,44 @@ __device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
     return v;
 }
 
-// ----------------------------------------------------------------------------- range of the scale codes
-__global__ void __launch_bounds__(512) scale_range_kernel(const uint8_t* __restrict__ a, int64_t na, const uint8_t* __restrict__ b,
-                                                          int64_t nb, int* __restrict__ range) {
-    __shared__ uint32_t part[16][4];
+// ----------------------------------------------------------------------------- windows of the scale rows
+// One warp per scale row of A and then of B: the row's largest and smallest non-zero code -> its shift k (a byte of
+// the workspace), or the workspace's first word set when the row has no window.  `tiled`: the row's 16-byte pieces lie
+// 2048 bytes apart (128 x 16 tiles) instead of back to back.
+__global__ void __launch_bounds__(512) scale_range_kernel(const uint8_t* __restrict__ a, int64_t rows_a, int a_tiled,
+                                                          const uint8_t* __restrict__ b, int64_t rows_b, int b_tiled,
+                                                          int64_t kblocks, int* __restrict__ workspace) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the GEMM's prologue may run beside this kernel
-    uint32_t red[4];                                      // max A, 255 - min nonzero A, max B, 255 - min nonzero B
-    for (int op = 0; op < 2; ++op) {
-        const uint8_t* s = op ? b : a;
-        const int64_t n = op ? nb : na, words = n >> 4;
-        uint32_t m = 0u, iv = 0u;
-        // four independent 16-byte loads per trip
-        const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += 4 * stride) {
-            uint4 v[4];
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows_a + rows_b) return;
+    const bool is_b = row >= rows_a;
+    const int64_t r = is_b ? row - rows_a : row;
+    const uint8_t* s = is_b ? b : a;
+    const bool tiled = is_b ? b_tiled : a_tiled;
+    const int64_t pieces = kblocks >> 4;                                 // 16-byte pieces of the row (Kc is a multiple of 256)
+    const uint8_t* base = tiled ? s + (r >> 7) * pieces * 2048 + (r & 127) * 16 : s + r * kblocks;
+    const int64_t pstride = tiled ? 2048 : 16;
+    uint32_t m = 0u, iv = 0u;
+    for (int64_t i = lane; i < pieces; i += 32) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + i * pstride));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
-                v[t] = (i + t * stride < words) ? __ldg(reinterpret_cast<const uint4*>(s) + i + t * stride) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const uint32_t w[4] = {v[t].x, v[t].y, v[t].z, v[t].w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    m = __vmaxu4(m, w[j]);
-                    iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));      // 255 - c, and 0 for c = 0
-                }
-            }
+        for (int j = 0; j < 4; ++j) {
+            m = __vmaxu4(m, w[j]);
+            iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));              // 255 - c, and 0 for c = 0
         }
-        if (blockIdx.x == 0 && threadIdx.x < (n & 15)) {
-            const uint32_t c = s[(words << 4) + threadIdx.x];
-            m = __vmaxu4(m, c);
-            if (c) iv = __vmaxu4(iv, 255u - c);
-        }
-        m = max(max(m & 0xFFu, (m >> 8) & 0xFFu), max((m >> 16) & 0xFFu, m >> 24));
-        iv = max(max(iv & 0xFFu, (iv >> 8) & 0xFFu), max((iv >> 16) & 0xFFu, iv >> 24));
-        red[2 * op] = __reduce_max_sync(0xFFFFFFFFu, m);
-        red[2 * op + 1] = __reduce_max_sync(0xFFFFFFFFu, iv);
     }
-    // one set of atomics per CTA: thousands of warps hitting four words one after the other would cost more than the read
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane < 4) part[warp][lane] = lane == 0 ? red[0] : lane == 1 ? red[1] : lane == 2 ? red[2] : red[3];
-    __syncthreads();
-    if (warp == 0) {
-        const uint32_t v = lane < 16 ? part[lane][0] : 0u, w = lane < 16 ? part[lane][1] : 0u;
-        const uint32_t x = lane < 16 ? part[lane][2] : 0u, y = lane < 16 ? part[lane][3] : 0u;
-        const uint32_t r0 = __reduce_max_sync(0xFFFFFFFFu, v), r1 = __reduce_max_sync(0xFFFFFFFFu, w);
-        const uint32_t r2 = __reduce_max_sync(0xFFFFFFFFu, x), r3 = __reduce_max_sync(0xFFFFFFFFu, y);
-        if (lane == 0) {
-            if (r0) atomicMax(range + 0, (int)r0);
-            if (r1) atomicMax(range + 1, (int)r1);
-            if (r2) atomicMax(range + 2, (int)r2);
-            if (r3) atomicMax(range + 3, (int)r3);
-        }
+    m = max(max(m & 0xFFu, (m >> 8) & 0xFFu), max((m >> 16) & 0xFFu, m >> 24));
+    iv = max(max(iv & 0xFFu, (iv >> 8) & 0xFFu), max((iv >> 16) & 0xFFu, iv >> 24));
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    iv = __reduce_max_sync(0xFFFFFFFFu, iv);
+    if (lane == 0) {
+        int k;
+        const bool ok = pick_window((int)m, (int)iv, k);
+        uint8_t* kbytes = reinterpret_cast<uint8_t*>(workspace) + 16 + (is_b ? ((rows_a + 15) / 16) * 16 : 0);
+        kbytes[r] = (uint8_t)k;
+        if (!ok) atomicOr(workspace, 1);
     }
 }
 
@@ -263,10 +251,9 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // Everything above touched only this CTA pair's shared and tensor memory and may have run while the range kernel was
-    // still at work (programmatic dependent launch); its four words are read from here on.
+    // still at work (programmatic dependent launch); the workspace it fills is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    int ka, kb;
-    const bool work = native_windows(p.range, ka, kb);       // uniform over the grid; false: the FP16 kernel does this product
+    const bool work = native_all_rows_have_windows(p.workspace);      // uniform over the grid; false: the FP16 kernel does this product
 
     if (!work) {
     } else if (warp == 0) {
@@ -401,8 +388,10 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;
-        // value5 = value4 * 2^(k - 8) for each operand
-        const float alpha = __fmul_rn(__fmul_rn(__ldg(p.a_decode), __ldg(p.b_decode)), __int_as_float((127 + ka + kb - 16) << 23));
+        // value5 = value4 * 2^(k - 8) for every scale row: output (m, n) takes 2^(k_m - 8) from its A row and 2^(k_n - 8) from
+        // its B row, both exact, before the one rounding of the product with d_A * d_B
+        const float alpha0 = __fmul_rn(__ldg(p.a_decode), __ldg(p.b_decode));
+        const bool a2d = p.a_mode == UE5M3_SCALE_2D, b2d = p.b_mode == UE5M3_SCALE_2D;
         const uint32_t stage = smem_base + SMEM_EPI + q * EPI_WARP_BYTES;
         uint8_t* stage_gen = smem_gen + SMEM_EPI + q * EPI_WARP_BYTES;
         uint32_t tl = 0;
@@ -411,9 +400,49 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             int tm, nb;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, nb);
             const int mb = tm * 2 + (int)rank;
-            if (!mbar_wait(acc_full, tl & 1, abort_flag, p.wait_limit)) { ok = false; break; }
-            tc_fence_after();
             const int row0 = mb * BM + q * 32, col0 = nb * BN;
+            // This lane's row shift and, for the tile's 256 columns, eight column shifts per lane (lane j: columns 8 j .. 8 j + 7),
+            // asked for before the accumulator is waited for, so that the loads are long done when they are needed.
+            uint32_t ka_row = 8u;
+            uint2 kcol = make_uint2(0x08080808u, 0x08080808u);
+            if (row0 + lane < p.Mo) {
+                const int64_t ar = row0 + lane;
+                ka_row = __ldg(p.ka_rows + (a2d ? (ar >> 4) : ar));
+            }
+            if (col0 + 8 * lane < p.No) {
+                if (b2d) kcol.x = kcol.y = (uint32_t)__ldg(p.kb_rows + ((col0 + 8 * lane) >> 4)) * 0x01010101u;
+                else kcol = __ldg(reinterpret_cast<const uint2*>(p.kb_rows + col0 + 8 * lane));
+            }
+            // While the accumulator is still being computed: which of the eight 32-column units have one shift for all
+            // their columns (bit u of `usame`; unit u's columns sit in lanes 4 u .. 4 u + 3), and this row's factor.
+            const uint32_t kbyte = kcol.x & 0xFFu;
+            const uint32_t kfirst = __shfl_sync(0xFFFFFFFFu, kbyte, lane & ~3);       // every lane takes part: no short circuit
+            const bool lane_same = (kcol.x == kbyte * 0x01010101u) & (kcol.y == kcol.x) & (kbyte == kfirst);
+            const uint32_t lanes_same = __ballot_sync(0xFFFFFFFFu, lane_same);
+            uint32_t usame = 0u;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) usame |= (((lanes_same >> (4 * u)) & 0xFu) == 0xFu) ? (1u << u) : 0u;
+            const float alpha = alpha0 * __int_as_float((119 + (int)ka_row) << 23);
+            // the same answer in every lane: the lanes meet in shuffles below
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_full, tl & 1, abort_flag, p.wait_limit));
+            if (!ok) break;
+            tc_fence_after();
+            // the shifts of 32 consecutive output columns (unit u of the tile), four per word
+            auto col_shifts = [&](int n0, uint32_t (&w)[8]) {
+                const int u = (n0 - col0) >> 5;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    w[2 * t] = __shfl_sync(0xFFFFFFFFu, kcol.x, 4 * u + t);
+                    w[2 * t + 1] = __shfl_sync(0xFFFFFFFFu, kcol.y, 4 * u + t);
+                }
+            };
+            auto colf = [](const uint32_t (&w)[8], int j) {
+                return __int_as_float((int)((((w[j >> 2] >> (8 * (j & 3))) & 0xFFu) + 119u) << 23));
+            };
+            // the factor of unit u when all its columns share one shift (the usual case): folded into the row's factor
+            auto unit_factor = [&](int u) {
+                return alpha * __int_as_float((int)((__shfl_sync(0xFFFFFFFFu, kbyte, 4 * u) + 119u) << 23));
+            };
             const uint32_t odd = tl & 1;
             const uint32_t acc = tmem_base + ((uint32_t)(q * 32) << 16) + (odd ? TMEM_ACC_ODD : 0);
             // The 192 columns both accumulators share (the last 192 of an even tile, the first 192 of an odd one) are read
@@ -429,8 +458,19 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     for (int hh = 0; hh < 2; ++hh) {
                         const int half = odd ? hh : hh ^ 1;                           // inside a chunk too: the shared unit first
                         uint32_t r[32];
-                        tmem_ld32(acc + cc * 64 + half * 32, r);
+                        const int unit = cc * 2 + half;
+                        tmem_ld32(acc + unit * 32, r);
                         tmem_ld_wait();
+                        // the column factors: one for all 32 columns (the usual case, folded into the row's factor), or each
+                        // applied to its accumulator first -- powers of two, so nothing is rounded before the product with alpha
+                        float au = unit_factor(unit);
+                        if (!((usame >> unit) & 1u)) {
+                            uint32_t ks[8];
+                            col_shifts(col0 + unit * 32, ks);
+                            au = alpha;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * colf(ks, j));
+                        }
                         if (2 * i + hh == OVERLAP_UNITS - 1) {
                             tc_fence_before();
                             __syncwarp();
@@ -443,10 +483,10 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {
                             uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * alpha, __uint_as_float(r[8 * v + 1]) * alpha);
-                            o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * alpha, __uint_as_float(r[8 * v + 3]) * alpha);
-                            o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * alpha, __uint_as_float(r[8 * v + 5]) * alpha);
-                            o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * alpha, __uint_as_float(r[8 * v + 7]) * alpha);
+                            o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * au, __uint_as_float(r[8 * v + 1]) * au);
+                            o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * au, __uint_as_float(r[8 * v + 3]) * au);
+                            o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * au, __uint_as_float(r[8 * v + 5]) * au);
+                            o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * au, __uint_as_float(r[8 * v + 7]) * au);
                             *reinterpret_cast<uint4*>(mine + (((half * 4 + v) ^ sw) << 4)) = o;
                         }
                     }
@@ -462,6 +502,14 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     uint32_t r[32];
                     tmem_ld32(acc + c * 32, r);
                     tmem_ld_wait();
+                    float au = unit_factor(c);
+                    if (!((usame >> c) & 1u)) {
+                        uint32_t ks[8];
+                        col_shifts(col0 + c * 32, ks);
+                        au = alpha;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * colf(ks, j));
+                    }
                     if (i == OVERLAP_UNITS - 1) {
                         tc_fence_before();
                         __syncwarp();
@@ -474,8 +522,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 #pragma unroll
                     for (int v = 0; v < 8; ++v)
                         *reinterpret_cast<float4*>(mine + ((v ^ sw) << 4)) =
-                            make_float4(__uint_as_float(r[4 * v + 0]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
-                                        __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+                            make_float4(__uint_as_float(r[4 * v + 0]) * au, __uint_as_float(r[4 * v + 1]) * au,
+                                        __uint_as_float(r[4 * v + 2]) * au, __uint_as_float(r[4 * v + 3]) * au);
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) tma_store_2d(&map_out, stage, col0 + c * 32, row0);
@@ -492,8 +540,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         // registers), shift the codes and store them there; the lane assignment makes a warp's 32 stores consecutive words.
         const int cg = (warp - CONV_WARP0) >> 2, cw = warp & 3;          // group (= stage parity), warp inside the group
         const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);            // the row this thread reads
-        const uint32_t da = (uint32_t)((8 * ka) & 0xFF) * 0x01010101u, db = (uint32_t)((8 * kb) & 0xFF) * 0x01010101u;
         const int64_t kblocks = p.Kc >> 4;
+        uint32_t cda = 0u, cdb0 = 0u, cdb1 = 0u;      // 8 k in every byte, for the three rows of the cursor's tile
         auto shift = [](uint32_t v, uint32_t d) { return __vsub4(v, d) & ~__vcmpeq4(v, 0u); };
         const int64_t step_a = p.a_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16, step_b = p.b_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16;
         const uint8_t *pa = nullptr, *pb0 = nullptr, *pb1 = nullptr;
@@ -503,13 +551,31 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             if (mode == UE5M3_SCALE_1D_TILED) return scales + (grow >> 7) * kchunks * 2048 + (grow & 127) * 16;
             return scales + ((mode == UE5M3_SCALE_2D) ? (grow >> 4) : grow) * kblocks;
         };
+        // the three rows' shift bytes of a tile, asked for one tile ahead (raw bytes; 0 beyond the operands)
+        uint32_t nka = 0u, nkb0 = 0u, nkb1 = 0u;
+        auto ask_shifts = [&](int tile) {
+            nka = nkb0 = nkb1 = 0u;
+            if (tile >= num_tiles) return;
+            int tm, tn;
+            tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+            const int64_t ga = (int64_t)(tm * 2 + (int)rank) * BM + row, gb0 = (int64_t)tn * BN + row, gb1 = gb0 + BNH;
+            if (ga < p.Mo) nka = __ldg(p.ka_rows + (p.a_mode == UE5M3_SCALE_2D ? (ga >> 4) : ga));
+            if (gb0 < p.No) nkb0 = __ldg(p.kb_rows + (p.b_mode == UE5M3_SCALE_2D ? (gb0 >> 4) : gb0));
+            if (gb1 < p.No) nkb1 = __ldg(p.kb_rows + (p.b_mode == UE5M3_SCALE_2D ? (gb1 >> 4) : gb1));
+        };
         auto open_tile = [&]() {
             if (c_tile >= num_tiles) { pa = pb0 = pb1 = nullptr; return; }
             int tm, tn;
             tile_coords(c_tile, p.tiles_m, p.tiles_n, tm, tn);
-            pa = row_base(p.a_scales, p.a_mode, p.Mo, (int64_t)(tm * 2 + (int)rank) * BM + row);
-            pb0 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + row);
-            pb1 = row_base(p.b_scales, p.b_mode, p.No, (int64_t)tn * BN + BNH + row);
+            const int64_t ga = (int64_t)(tm * 2 + (int)rank) * BM + row, gb0 = (int64_t)tn * BN + row, gb1 = gb0 + BNH;
+            pa = row_base(p.a_scales, p.a_mode, p.Mo, ga);
+            pb0 = row_base(p.b_scales, p.b_mode, p.No, gb0);
+            pb1 = row_base(p.b_scales, p.b_mode, p.No, gb1);
+            // this tile's shifts were asked for when the previous tile was opened; now ask for the next tile's
+            cda = ((8u * nka) & 0xFFu) * 0x01010101u;
+            cdb0 = ((8u * nkb0) & 0xFFu) * 0x01010101u;
+            cdb1 = ((8u * nkb1) & 0xFFu) * 0x01010101u;
+            ask_shifts(c_tile + num_pairs);
         };
         auto advance = [&]() {                       // the cursor moves on by one stage
             if (++c_kc == kchunks) {
@@ -522,19 +588,22 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 if (pb1) pb1 += step_b;
             }
         };
-        auto fetch = [&](uint4& a, uint4& b0, uint4& b1) {     // this group's next stage; the other group's is skipped
+        auto fetch = [&](uint4& a, uint4& b0, uint4& b1, uint32_t (&d)[3]) {     // this group's next stage; the other group's is skipped
             const uint4 z = make_uint4(0u, 0u, 0u, 0u);
             a = pa ? ldg_nc_16(pa) : z;
             b0 = pb0 ? ldg_nc_16(pb0) : z;
             b1 = pb1 ? ldg_nc_16(pb1) : z;
+            d[0] = cda; d[1] = cdb0; d[2] = cdb1;
             advance();
             advance();
         };
+        ask_shifts(pair);
         open_tile();
         if (cg) advance();
         uint4 ra[PF], rb0[PF], rb1[PF];
+        uint32_t rd[PF][3];
 #pragma unroll
-        for (int d = 0; d < PF; ++d) fetch(ra[d], rb0[d], rb1[d]);
+        for (int d = 0; d < PF; ++d) fetch(ra[d], rb0[d], rb1[d], rd[d]);
         bool ok = true;
         uint32_t f = cg, fph = 0;
         for (uint32_t base = cg; base < total && ok; base += 2 * PF) {
@@ -546,13 +615,14 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 uint32_t* xa = reinterpret_cast<uint32_t*>(smem_gen + SMEM_XCH + f * XCH_BYTES) + cw * 32 + lane;     // + 128 j
                 uint32_t* xb = xa + XCH_A_BYTES / 4;                                                                  // + 256 j + 128 h
                 const uint4 a = ra[d], b0 = rb0[d], b1 = rb1[d];
+                const uint32_t da = rd[d][0], db0 = rd[d][1], db1 = rd[d][2];
                 xa[0] = shift(a.x, da); xa[128] = shift(a.y, da); xa[256] = shift(a.z, da); xa[384] = shift(a.w, da);
-                xb[0] = shift(b0.x, db); xb[256] = shift(b0.y, db); xb[512] = shift(b0.z, db); xb[768] = shift(b0.w, db);
-                xb[128] = shift(b1.x, db); xb[384] = shift(b1.y, db); xb[640] = shift(b1.z, db); xb[896] = shift(b1.w, db);
+                xb[0] = shift(b0.x, db0); xb[256] = shift(b0.y, db0); xb[512] = shift(b0.z, db0); xb[768] = shift(b0.w, db0);
+                xb[128] = shift(b1.x, db1); xb[384] = shift(b1.y, db1); xb[640] = shift(b1.z, db1); xb[896] = shift(b1.w, db1);
                 fence_proxy_async();                 // the tensor core's scale copy reads what was just written
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(sf_full + 8 * f, 0);
-                fetch(ra[d], rb0[d], rb1[d]);
+                fetch(ra[d], rb0[d], rb1[d], rd[d]);
                 f += 2;
                 if (f >= SF_RING) { f -= SF_RING; fph ^= 1; }
             }
@@ -584,38 +654,39 @@ bool make_out_map(CUtensorMap* m, void* out, bool bf16, int64_t Mo, int64_t No, 
 }  // namespace
 
 bool native_eligible(const GemmArgs& g) {
-    if (g.Kc % KCHUNK) return false;
-    return true;
+    return g.Kc % KCHUNK == 0 && native_workspace_bytes(g) <= kNativeWorkspaceSlotBytes;
 }
 
-// Four words of device workspace for one call: a ring of 256 slots per device, allocated at the first call on that
-// device.  Calls that are in flight at the same time (different streams) use different slots as long as fewer than
-// 256 of them overlap.
-int* native_workspace() {
-    static int* ring[64];
+// Device workspace for one call: a ring of 64 slots of kNativeWorkspaceSlotBytes per device, allocated at the first call
+// on that device.  Calls that are in flight at the same time (different streams) use different slots as long as fewer
+// than 64 of them overlap.
+int* native_workspace(size_t need_bytes) {
+    constexpr unsigned kSlots = 64;
+    static uint8_t* ring[64];
     static std::once_flag made[64];
     static std::atomic<unsigned> next{0};
+    if (need_bytes > kNativeWorkspaceSlotBytes) return nullptr;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     std::call_once(made[dev], [&]() {
         void* ptr = nullptr;
-        if (cudaMalloc(&ptr, 256 * 4 * sizeof(int)) != cudaSuccess) { (void)cudaGetLastError(); return; }
-        ring[dev] = static_cast<int*>(ptr);
+        if (cudaMalloc(&ptr, kSlots * kNativeWorkspaceSlotBytes) != cudaSuccess) { (void)cudaGetLastError(); return; }
+        ring[dev] = static_cast<uint8_t*>(ptr);
     });
     if (!ring[dev]) return nullptr;
-    return ring[dev] + 4 * (next.fetch_add(1) & 255u);
+    return reinterpret_cast<int*>(ring[dev] + (size_t)(next.fetch_add(1) % kSlots) * kNativeWorkspaceSlotBytes);
 }
 
-// Workspace of ue5m3_gemm_static: a file-scope device array instead of allocated memory.  One call needs 16 bytes
-// (the four range words), whatever the problem size; the array holds kStaticWorkspaceBytes.  Its address is asked for
-// once per device; nothing is allocated, here or later.  All calls on a device share the array: the four words are
-// cleared by every call before its range kernel runs, so two calls may follow one another on a stream, but two calls
-// in flight at the same time (different streams) would read each other's ranges.
-constexpr size_t kStaticWorkspaceBytes = 256;
-static __device__ __align__(256) int g_static_workspace[kStaticWorkspaceBytes / sizeof(int)];
+// Workspace of ue5m3_gemm_static: a file-scope device array instead of allocated memory.  A call needs 16 bytes plus
+// one byte per scale row of the two operands; the array holds kNativeWorkspaceSlotBytes, and a call that needs more is
+// refused.  Its address is asked for once per device; nothing is allocated, here or later.  All calls on a device
+// share the array: the first word is cleared and every row byte written by every call before its GEMM kernels run,
+// so two calls may follow one another on a stream, but two calls in flight at the same time (different streams) would
+// read each other's windows.
+static __device__ __align__(256) unsigned char g_static_workspace[kNativeWorkspaceSlotBytes];
 
 int* static_workspace(size_t need_bytes) {
-    if (need_bytes > kStaticWorkspaceBytes) return nullptr;
+    if (need_bytes > kNativeWorkspaceSlotBytes) return nullptr;
     static int* addr[64];
     static std::once_flag asked[64];
     int dev = 0;
@@ -628,20 +699,18 @@ int* static_workspace(size_t need_bytes) {
     return addr[dev];
 }
 
-int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st) {
-    const int64_t kb = g.Kc / 16;
-    const int64_t na = (g.a_scale_mode == UE5M3_SCALE_2D ? g.Mo / 16 : g.Mo) * kb;
-    const int64_t nb = (g.b_scale_mode == UE5M3_SCALE_2D ? g.No / 16 : g.No) * kb;
-    if (cudaMemsetAsync(range, 0, 4 * sizeof(int), st) != cudaSuccess) return UE5M3_ERR_CUDA;
-    const int64_t words = (na > nb ? na : nb) >> 4;
-    int64_t grid = (words + 512 * 4 - 1) / (512 * 4);
-    if (grid > 2 * num_sms) grid = 2 * num_sms;
-    if (grid < 1) grid = 1;
-    scale_range_kernel<<<(unsigned)grid, 512, 0, st>>>(g.a_scales, na, g.b_scales, nb, range);
+int launch_scale_range(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st) {
+    (void)num_sms;
+    const int64_t ra = native_scale_rows(g.Mo, g.a_scale_mode), rb = native_scale_rows(g.No, g.b_scale_mode);
+    if (cudaMemsetAsync(workspace, 0, sizeof(int), st) != cudaSuccess) return UE5M3_ERR_CUDA;
+    const int64_t grid = (ra + rb + 15) / 16;                     // 16 warps per CTA, one row each
+    scale_range_kernel<<<(unsigned)grid, 512, 0, st>>>(g.a_scales, ra, g.a_scale_mode == UE5M3_SCALE_1D_TILED ? 1 : 0,
+                                                       g.b_scales, rb, g.b_scale_mode == UE5M3_SCALE_1D_TILED ? 1 : 0,
+                                                       g.Kc / 16, workspace);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
-int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st) {
+int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st) {
     static int resident_pairs[64];
     static std::once_flag asked[64];
     int dev = 0;
@@ -670,7 +739,9 @@ int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStr
     NativeParams p;
     p.Mo = g.Mo; p.No = g.No; p.Kc = g.Kc;
     p.a_decode = g.a_decode; p.b_decode = g.b_decode;
-    p.range = range;
+    p.workspace = workspace;
+    p.ka_rows = reinterpret_cast<const uint8_t*>(workspace) + 16;
+    p.kb_rows = p.ka_rows + ((native_scale_rows(g.Mo, g.a_scale_mode) + 15) / 16) * 16;
     p.a_scales = g.a_scales; p.b_scales = g.b_scales;
     p.out_bf16 = g.out_dtype == UE5M3_BF16 ? 1 : 0;
     p.a_mode = g.a_scale_mode; p.b_mode = g.b_scale_mode;
@@ -681,7 +752,7 @@ int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStr
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int pairs = num_tiles < resident_pairs[dev] ? num_tiles : resident_pairs[dev];
     // Programmatic dependent launch: the kernel's prologue (barriers, tensor-memory allocation, cluster barrier) runs
-    // beside the range kernel, which releases its dependents at once; the kernel waits for it before reading the range.
+    // beside the range kernel, which releases its dependents at once; the kernel waits for it before reading the workspace.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);

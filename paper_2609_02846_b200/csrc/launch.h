@@ -55,17 +55,24 @@ cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bo
 cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* out, int num_sms,
                         cudaStream_t st);
 cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, cudaStream_t st);
-// returns a UE5M3_* status; `range` (may be null) is the workspace of the native path: the kernel then does nothing when
-// both operands have a UE4M3 window, because gemm_native_kernel has done the product
-int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st);
+// returns a UE5M3_* status; `workspace` (may be null) is the workspace of the native path: the kernel then does nothing
+// when every scale row has a UE4M3 window, because gemm_native_kernel has done the product
+int launch_gemm(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st);
 int read_and_clear_device_status();                                  // synchronises the device
-// The same product on the tensor core's FP4 path (gemm_native.cu).  `range` is four words of device workspace:
-// launch_scale_range fills them, the kernel reads them and does nothing when an operand's scale codes have no window.
-bool native_eligible(const GemmArgs& g);
-int* native_workspace();                                             // four words of a per-device ring; null on failure
+// The same product on the tensor core's FP4 path (gemm_native.cu).  `workspace` is device memory of
+// native_workspace_bytes(g) bytes (layout in window.cuh): launch_scale_range fills it, the native kernel reads it and does
+// nothing when some scale row has no window, and the FP16 kernel (launch_gemm with the same workspace) then does the product.
+inline int64_t native_scale_rows(int64_t R, int mode) { return mode == 2 /* UE5M3_SCALE_2D */ ? R / 16 : R; }
+inline size_t native_workspace_bytes(const GemmArgs& g) {
+    const int64_t ra = native_scale_rows(g.Mo, g.a_scale_mode), rb = native_scale_rows(g.No, g.b_scale_mode);
+    return (size_t)(16 + ((ra + 15) / 16) * 16 + ((rb + 15) / 16) * 16);
+}
+constexpr size_t kNativeWorkspaceSlotBytes = 64 * 1024;             // largest workspace the library's own rings hold
+bool native_eligible(const GemmArgs& g);                             // Kc % 256 == 0 and the workspace fits a ring slot
+int* native_workspace(size_t need_bytes);                            // a slot of the per-device ring; null on failure
 int* static_workspace(size_t need_bytes);                            // file-scope device array; null if the need exceeds it
-int launch_scale_range(const GemmArgs& g, int* range, int num_sms, cudaStream_t st);
-int launch_gemm_native(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st);
+int launch_scale_range(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st);
+int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st);
 int read_and_clear_native_status();                                  // synchronises the device
 // The same operands under the output model of Section 6.2 (gemm_probe.cu).
 int launch_gemm_probe(const GemmArgs& g, int cross_rne, int grid_denominator, int num_sms, cudaStream_t st);

@@ -1,29 +1,33 @@
-// The UE4M3 window of an operand's UE5M3 scale codes, shared by the native FP4 GEMM (which runs when both operands
-// have one) and the FP16 GEMM (which runs when they do not).
+// The UE4M3 window of a row of UE5M3 scale codes, shared by the native FP4 GEMM (which runs when every scale row of both
+// operands has one) and the FP16 GEMM (which runs when one does not).
 #pragma once
 #include <cstdint>
 
 namespace ue5m3 {
 
-// k with 8 <= c - 8k <= 126 for every non-zero code c of the operand, if there is one: then
+// k with 8 <= c - 8k <= 126 for every non-zero code c of the row, if there is one: then
 // value5(c) = value4(c - 8k) * 2^(k - 8) exactly.  `cmax` is the largest code, `inv_min` is 255 - the smallest
-// non-zero code (both 0 when every code is 0).
+// non-zero code (both 0 when every code is 0).  The shift may differ from row to row: row m of A and row n of B
+// contribute the factor 2^(k_m - 8) * 2^(k_n - 8) to output (m, n), which the epilogue applies.
 __device__ __forceinline__ bool pick_window(int cmax, int inv_min, int& k) {
     k = 8;
     if (cmax == 0) return true;                       // no non-zero code at all
     const int cmin = 255 - inv_min;
     if (cmin < 8 || cmax > 0xF7) return false;        // subnormal or invalid codes
-    const int k_hi = (cmin - 8) >> 3;
-    if (cmax - 8 * k_hi > 126) return false;
-    k = k_hi;
+    // Any k between the smallest one that brings the largest code down to 126 and the largest one that keeps the smallest
+    // code at 8 or above is exact.  Rows should agree on k where they can (the epilogue then has one factor per 32 output
+    // columns instead of 32): k = 2 is taken whenever it is valid -- it is for every row of a tensor quantized with
+    // T = 448 against a current reference whose block scales stay above 2^-12 -- and the smallest valid k otherwise.
+    const int k_lo = cmax > 126 ? (cmax - 126 + 7) >> 3 : 0, k_hi = (cmin - 8) >> 3;
+    if (k_lo > k_hi) return false;
+    k = (k_lo <= 2 && 2 <= k_hi) ? 2 : k_lo;
     return true;
 }
 
-// range = {max A, 255 - min nonzero A, max B, 255 - min nonzero B}, 16-byte aligned
-__device__ __forceinline__ bool native_windows(const int* range, int& ka, int& kb) {
-    const int4 r = *reinterpret_cast<const int4*>(range);
-    const bool a = pick_window(r.x, r.y, ka), b = pick_window(r.z, r.w, kb);
-    return a && b;
-}
+// Workspace of one ue5m3_gemm call on the native path:
+//   word 0          0 when every scale row of both operands has a window, non-zero otherwise (the FP16 kernel then works)
+//   bytes 16 ...    the shift k of every scale row of A (one byte per row; rows of a 2D operand are its 16-row groups),
+//                   padded to a multiple of 16; then the same for B
+__device__ __forceinline__ bool native_all_rows_have_windows(const int* workspace) { return *workspace == 0; }
 
 }  // namespace ue5m3

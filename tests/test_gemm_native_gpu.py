@@ -1,5 +1,5 @@
-"""The native FP4 path of ue5m3_gemm: UE5M3 scale codes shifted into a UE4M3 window, the tensor core's own block-scaled
-instruction.  Parity with the exact-integer oracle under the same bound as the FP16 path (FP32: |y - y*| <= 1e-5 *
+"""The native FP4 path of ue5m3_gemm: the UE5M3 scale codes of every scale row shifted into a UE4M3 window, the tensor core's
+own block-scaled instruction.  Parity with the exact-integer oracle under the same bound as the FP16 path (FP32: |y - y*| <= 1e-5 *
 sum_k |a_k b_k| + 1e-30, BF16: 1 ulp), the window's edges, the fallback when there is no window, and the dispatch."""
 import numpy as np
 import pytest
@@ -34,13 +34,26 @@ def _operand(rng, R, Kc, mode, lo, hi, dec=1.0, scales=None):
 
 
 def _native(qa, qb, dtype, Mo, No):
-    """Runs ue5m3_gemm_native on an output pre-filled with NaN; returns (out, workspace as a list)."""
+    """Runs ue5m3_gemm_native on an output pre-filled with NaN; returns (out, every row has a window, k of A's scale rows,
+    k of B's scale rows)."""
     out = torch.full((Mo, No), float("nan"), dtype=dtype, device=DEV)
-    ws = torch.zeros(4, dtype=torch.int32, device=DEV)
+    ws = lib.gemm_native_workspace(qa, qb)
+    ws.fill_(0xEE)                                     # stale contents: the call writes what it reads
     lib.gemm_native(lib.FPROP, qa, qb, dtype, out=out, workspace=ws)
     torch.cuda.synchronize()
     assert lib.last_device_status() == 0
-    return out, ws.tolist()
+    ok, ka, kb = lib.native_windows(ws, qa, qb)
+    return out, ok, ka, kb
+
+
+def _row_k(scales):
+    """The shift the library must have chosen for every scale row (None where a row has no window)."""
+    from paper_2609_02846_b200.binding import scale_window
+    ks = []
+    for row in scales:
+        nz = row[row != 0]
+        ks.append(8 if nz.size == 0 else scale_window(int(nz.min()), int(nz.max())))
+    return ks
 
 
 # (Mo, No, Kc): one tile and one stage; several stages; ragged tile counts (a CTA of a pair without rows, a tile
@@ -58,8 +71,8 @@ def test_native_matches_oracle(shape, modes, out_dtype):
     lo = int(rng.integers(0x20, 0x70))
     qa, ap, asc = _operand(rng, Mo, Kc, modes[0], lo, lo + 0x50, dec=0.37)
     qb, bp, bsc = _operand(rng, No, Kc, modes[1], 0x40, 0xA0, dec=1.0 / 2688.0)
-    out, ws = _native(qa, qb, out_dtype, Mo, No)
-    assert ws == [int(asc.max()), 255 - int(asc.min()), int(bsc.max()), 255 - int(bsc.min())]
+    out, ok, ka, kb = _native(qa, qb, out_dtype, Mo, No)
+    assert ok and list(ka) == _row_k(asc) and list(kb) == _row_k(bsc)
     y, sa = oracle.gemm(ap, asc, modes[0] == 2, 0.37, bp, bsc, modes[1] == 2, np.float32(1.0 / 2688.0))
     check_gemm_output(out, y, sa)
 
@@ -71,7 +84,8 @@ def test_native_many_tiles_per_pair():
     rng = np.random.default_rng(77)
     qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x60, 0x90, dec=1.0)
     qb, bp, bsc = _operand(rng, No, Kc, 2, 0x60, 0x90, dec=1.0)
-    out, _ = _native(qa, qb, torch.float32, Mo, No)
+    out, ok, _, _ = _native(qa, qb, torch.float32, Mo, No)
+    assert ok
     ci = rng.integers(0, Mo, 6000)
     cj = rng.integers(0, No, 6000)
     for r in (0, 127, 128, 255, 256, Mo - 1):        # full rows and columns through tile corners
@@ -95,8 +109,8 @@ def test_window_edges(k):
     dec = float(2.0 ** (10 - 2 * k))                  # keeps the products inside FP32 for the high windows
     qa, ap, _ = _operand(rng, Mo, Kc, 0, 0, 0, dec=dec, scales=asc)
     qb, bp, _ = _operand(rng, No, Kc, 0, 0, 0, dec=dec, scales=bsc)
-    out, ws = _native(qa, qb, torch.float32, Mo, No)
-    assert ws == [hi, 255 - lo, hi, 255 - lo]
+    out, ok, ka, kb = _native(qa, qb, torch.float32, Mo, No)
+    assert ok and ka[0] == k and kb[1] == k and list(ka) == _row_k(asc) and list(kb) == _row_k(bsc)
     y, sa = oracle.gemm(ap, asc, False, dec, bp, bsc, False, np.float32(dec))
     check_gemm_output(out, y, sa)
 
@@ -113,11 +127,10 @@ def test_no_window_leaves_output_alone_and_gemm_falls_back(case):
         a_rng, b_rng = (0x08, 0xF8), (0x50, 0x60)
     qa, ap, asc = _operand(rng, Mo, Kc, 0, *a_rng)
     qb, bp, bsc = _operand(rng, No, Kc, 0, *b_rng, dec=2.0 ** -20)
-    asc[0, 0], asc[0, 1] = a_rng[0], a_rng[1] - 1
+    asc[0, 0], asc[0, 1] = a_rng[0], a_rng[1] - 1     # both ends of the range inside one scale row
     qa.scales.copy_(torch.from_numpy(asc))
-    out, ws = _native(qa, qb, torch.float32, Mo, No)
-    assert ws[0] == a_rng[1] - 1 and ws[1] == 255 - a_rng[0]
-    assert bool(torch.isnan(out).all())               # the native kernel declined
+    out, ok, _, _ = _native(qa, qb, torch.float32, Mo, No)
+    assert not ok and bool(torch.isnan(out).all())    # row 0 of A has no window: the native kernel declined
     got = lib.gemm(lib.FPROP, qa, qb, torch.float32)
     ref = lib.gemm_fp16(lib.FPROP, qa, qb, torch.float32)
     torch.cuda.synchronize()
@@ -133,8 +146,8 @@ def test_gemm_dispatches_to_the_native_kernel_when_there_is_a_window():
     qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x58, 0x98, dec=0.5)
     qb, bp, bsc = _operand(rng, No, Kc, 2, 0x58, 0x98, dec=0.25)
     got = lib.gemm(lib.FPROP, qa, qb, torch.float32)
-    nat, _ = _native(qa, qb, torch.float32, Mo, No)
-    assert torch.equal(got, nat)
+    nat, ok, _, _ = _native(qa, qb, torch.float32, Mo, No)
+    assert ok and torch.equal(got, nat)
     # Kc = 128 * odd is not eligible: the FP16 kernel does it
     qa, _, _ = _operand(rng, 128, 384, 0, 0x58, 0x98)
     qb, _, _ = _operand(rng, 128, 384, 0, 0x58, 0x98)
@@ -159,8 +172,8 @@ def test_every_operand_value_pair_of_a_window_multiplies_exactly():
     scales[0, 1], scales[1, 1] = lo, lo + 118         # the window's ends are present whatever the first column holds
     one = torch.ones(1, dtype=torch.float32, device=DEV)
     q = lib.QuantizedOperand(torch.from_numpy(payload).to(DEV), torch.from_numpy(scales).to(DEV), one, lib.SCALE_1D)
-    out, ws = _native(q, q, torch.float32, R, R)
-    assert ws == [lo + 118, 255 - lo, lo + 118, 255 - lo]
+    out, ok, ka, _ = _native(q, q, torch.float32, R, R)
+    assert ok and list(ka) == _row_k(scales)
     y, _ = oracle.gemm(payload, scales, False, 1.0, payload, scales, False, np.float32(1.0))
     assert np.array_equal(out.cpu().numpy().astype(np.float64), y)
 
@@ -170,8 +183,10 @@ def test_native_is_deterministic_and_independent_of_the_workspace_contents():
     rng = np.random.default_rng(3)
     qa, _, _ = _operand(rng, Mo, Kc, 0, 0x60, 0xA0)
     qb, _, _ = _operand(rng, No, Kc, 0, 0x60, 0xA0, dec=2.0 ** -12)
-    first, _ = _native(qa, qb, torch.bfloat16, Mo, No)
-    ws = torch.full((4,), 12345, dtype=torch.int32, device=DEV)     # stale contents: the call clears them itself
+    first, ok, _, _ = _native(qa, qb, torch.bfloat16, Mo, No)
+    assert ok
+    ws = lib.gemm_native_workspace(qa, qb)
+    ws.fill_(0x5A)                                                  # stale contents: the call writes what it reads
     again = lib.gemm_native(lib.FPROP, qa, qb, torch.bfloat16, workspace=ws)
     torch.cuda.synchronize()
     assert torch.equal(first, again)
@@ -193,11 +208,8 @@ def test_quantized_operands_of_the_workload_recipe_take_the_native_kernel():
     qg = lib.quantize(dy, lib.LAYOUT_1D_ROW, lib.ROUND_SR, gg, 448.0, seed=4)
     qgt = lib.quantize(dy, lib.LAYOUT_1D_COL, lib.ROUND_SR, gg, 448.0, seed=5)
     for a, b, Mo, No in ((qx, qw, M, N), (qg, qw.transposed(), M, K), (qgt, qxt, N, K)):
-        out, ws = _native(a, b, torch.float32, Mo, No)
-        assert not bool(torch.isnan(out).any())                       # the native kernel did the product
-        for hi, inv in ((ws[0], ws[1]), (ws[2], ws[3])):
-            from paper_2609_02846_b200.binding import scale_window
-            assert scale_window(255 - inv, hi) is not None
+        out, ok, _, _ = _native(a, b, torch.float32, Mo, No)
+        assert ok and not bool(torch.isnan(out).any())                # the native kernel did the product
         a2d, b2d = a.scale_mode == lib.SCALE_2D, b.scale_mode == lib.SCALE_2D
         y, sa = oracle.gemm(a.payload.cpu().numpy(), a.scales.cpu().numpy(), a2d, float(a.decode.item()),
                             b.payload.cpu().numpy(), b.scales.cpu().numpy(), b2d, np.float32(b.decode.item()))
@@ -235,3 +247,31 @@ def test_native_seeded_sweep_over_shapes_modes_windows_and_strides():
             assert bool(torch.isnan(buf[:, No:]).all())               # nothing beyond the output's columns
         y, sa = oracle.gemm(ap, asc, ma == 2, da, bp, bsc, mb == 2, np.float32(db))
         check_gemm_output(out.contiguous(), y, sa)
+
+
+def test_every_row_has_its_own_window():
+    """Scale rows whose codes sit in different windows: the operand as a whole spans every code from 0x08 to 0xF7 and has no
+    common window, each row has one, and the native kernel does the product with a shift per row of A and of B (1D rows and
+    the 16-row groups of 2D scales)."""
+    Mo, No, Kc = 512, 768, 1024
+    rng = np.random.default_rng(4242)
+    for modes in ((0, 0), (0, 2), (2, 1)):
+        def rows(n):
+            lo = rng.integers(8, 0xF8 - 60, n)
+            width = rng.integers(1, 60, n)
+            sc = (lo[:, None] + rng.integers(0, 1 << 30, (n, Kc // 16)) % width[:, None]).astype(np.uint8)
+            sc[0, :] = rng.choice(np.array([8, 8 + 118], np.uint8), Kc // 16)            # the widest window there is, at the bottom ...
+            sc[1, :] = rng.choice(np.array([0xF7 - 110, 0xF7], np.uint8), Kc // 16)     # ... and one at the top
+            sc[2, :] = 0                               # a row of zero scales
+            return sc
+        asc = rows(Mo // 16 if modes[0] == 2 else Mo)
+        bsc = rows(No // 16 if modes[1] == 2 else No)
+        # decode factors per operand cannot follow the rows; keep the products finite by small payloads on large-scale rows
+        qa, ap, _ = _operand(rng, Mo, Kc, modes[0], 0, 0, dec=2.0 ** -8, scales=asc)
+        qb, bp, _ = _operand(rng, No, Kc, modes[1], 0, 0, dec=2.0 ** -8, scales=bsc)
+        out, ok, ka, kb = _native(qa, qb, torch.float32, Mo, No)
+        assert ok and list(ka) == _row_k(asc) and list(kb) == _row_k(bsc)
+        assert len(set(ka)) > 5 and len(set(kb)) > 5              # many different shifts in one product
+        y, sa = oracle.gemm(ap, asc, modes[0] == 2, 2.0 ** -8, bp, bsc, modes[1] == 2, np.float32(2.0 ** -8))
+        check_gemm_output(out, y, sa)
+        assert torch.equal(lib.gemm(lib.FPROP, qa, qb, torch.float32), out)      # ue5m3_gemm takes the same kernel

@@ -40,4 +40,6 @@ def test_window_rule_finds_a_window_whenever_one_exists():
             else:
                 assert k is None, (cmin, cmax)
     assert B.scale_window(0x20, 0x96) == 3 and B.scale_window(0x20, 0x97) is None      # 119 codes fit, 120 do not
+    assert B.scale_window(0x30, 0x7E) == 2 and B.scale_window(0x30, 0x7F) == 2 and B.scale_window(0x30, 0x8E) == 2
+    assert B.scale_window(0x10, 0x7E) == 0 and B.scale_window(0x10, 0x7F) == 1 and B.scale_window(0x70, 0xD0) == 11
     assert B.scale_window(1, 0x40) is None and B.scale_window(8, 0xF8) is None

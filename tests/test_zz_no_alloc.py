@@ -1,4 +1,4 @@
-"""ue5m3_gemm_static: the GEMM whose four words of scratch live in a file-scope device array.  Compared bit for bit with
+"""ue5m3_gemm_static: the GEMM whose device scratch (a flag and one byte per scale row) lives in a file-scope device array.  Compared bit for bit with
 ue5m3_gemm on two calls in a row (the second call finds the words the first one left), on operands that take the native
 kernel and on operands that fall back to the FP16 kernel, and checked not to move the device allocator."""
 import numpy as np
@@ -22,7 +22,7 @@ def test_static_workspace_gemm_equals_gemm_on_two_calls_in_a_row():
     rng = np.random.default_rng(2026)
     Mo, No, Kc = 384, 512, 1024
     windowed = (_operand(rng, Mo, Kc, 0x50, 0x90, 0.5), _operand(rng, No, Kc, 0x60, 0xA0, 2.0 ** -9))
-    wide = (_operand(rng, Mo, Kc, 0x01, 0xF0, 2.0 ** -12), _operand(rng, No, Kc, 0x40, 0x60, 2.0 ** -12))     # no window
+    wide = (_operand(rng, Mo, Kc, 0x01, 0xF0, 2.0 ** -12), _operand(rng, No, Kc, 0x40, 0x60, 2.0 ** -12))     # rows without a window
     want = [lib.gemm(lib.FPROP, a, b, torch.float32) for a, b in (windowed, wide)]
     torch.cuda.synchronize()
     lib.gemm_static(lib.FPROP, *windowed, torch.float32)            # first call on the device: looks the array up
@@ -51,3 +51,27 @@ def test_static_workspace_gemm_checks_arguments_like_gemm():
         lib.gemm_static(lib.FPROP, a, b)
     a = _operand(rng, 128, 384, 0x60, 0x70, 1.0); b = _operand(rng, 128, 384, 0x60, 0x70, 1.0)      # Kc = 128 * 3: FP16 kernel
     assert torch.equal(lib.gemm_static(lib.FPROP, a, b, torch.float32), lib.gemm(lib.FPROP, a, b, torch.float32))
+
+
+def test_static_workspace_gemm_refuses_operands_with_more_scale_rows_than_the_array_holds():
+    """65,536 bytes hold 16 + one byte per scale row (each operand's rows padded to a multiple of 16): 65,408 + 128 rows need
+    65,552.  The call is refused before anything is launched; ue5m3_gemm takes the same operands (on its FP16 kernel)."""
+    Ra, Rb, Kc = 65408, 128, 256
+    one = torch.ones(1, dtype=torch.float32, device=DEV)
+    def zeros_operand(R):
+        return lib.QuantizedOperand(torch.zeros((R, Kc // 2), dtype=torch.uint8, device=DEV),
+                                    torch.full((R, Kc // 16), 0x78, dtype=torch.uint8, device=DEV), one, lib.SCALE_1D)
+    a, b = zeros_operand(Ra), zeros_operand(Rb)
+    out = torch.full((Ra, Rb), 7.0, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(lib.Ue5m3Error):
+        lib.gemm_static(lib.FPROP, a, b, out=out)
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())
+    lib.gemm(lib.FPROP, a, b, out=out)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0 and bool((out == 0.0).all())
+    # one row block fewer fits: 65,280 + 128 rows need 65,424 bytes
+    a2 = zeros_operand(Ra - 128)
+    out2 = lib.gemm_static(lib.FPROP, a2, b, torch.bfloat16)
+    torch.cuda.synchronize()
+    assert bool((out2 == 0.0).all())
