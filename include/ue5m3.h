@@ -183,11 +183,12 @@ UE5M3_API int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_
  *            exact factors 2^(k_m - 8) 2^(k_n - 8) together with d_A * d_B.  k is chosen per row.  Needs Kc % 256 == 0.
  *   FP16     every E2M1 x UE5M3 product (times 2^-4) is exact in FP16, subnormals included; the operands are
  *            reconstructed in the kernel and multiplied as FP16.  Used when some scale row has no window (UE5M3
- *            subnormal codes 1..7 included), Kc = 128 * odd, or the operands have more than 65,520 scale rows together.
+ *            subnormal codes 1..7 included) or Kc = 128 * odd.
  * Both accumulate in FP32 on the tensor cores and meet the same error bound; their results may differ in the last bits.
- * Three launches per call when Kc % 256 == 0: a pass over the scale bytes that writes every row's k (one byte per row, in a
- * slot of a per-device workspace ring allocated at the first call on a device), then both kernels, one of which returns
- * at once.
+ * Three launches per call when Kc % 256 == 0: a pass over the scale bytes that writes every row's k and the shifted codes in
+ * the order the tensor core reads them (one byte per block, i.e. (Mo + No) * Kc / 16 bytes with Mo and No rounded up to 256,
+ * into a workspace the library keeps per device and stream and grows with cudaMalloc when a call needs more: make the first
+ * call of a shape on a stream outside any stream capture), then both kernels, one of which returns at once.
  * `op` only names the role of the call:
  *     FPROP  A = X  (1D_ROW),        B = W   (2D payload, scales)          Mo = tokens, No = out, Kc = in
  *     DGRAD  A = dY (1D_ROW, SR),    B = W^T (2D payload_t, scales_t)      Mo = tokens, No = in,  Kc = out
@@ -213,14 +214,14 @@ UE5M3_API int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc,
 /*
  * ue5m3_gemm with a workspace that is never allocated (the paper has no counterpart: this is about how a library
  * holds its device scratch, not about the method).  Same arguments, results (bit for bit), checks and errors as
- * ue5m3_gemm.  The workspace (16 bytes + one byte per scale row of A and of B) lives in a file-scope device array of
- * 65,536 bytes inside the library instead of the allocated per-device ring; operands with more scale rows than that
- * are refused with UE5M3_ERR_UNSUPPORTED (ue5m3_gemm would run them on the FP16 kernel).  The call allocates and frees
+ * ue5m3_gemm.  The workspace (ue5m3_gemm_native_workspace_bytes: about one byte per 16 operand elements) lives in a
+ * file-scope device array of 16 MiB inside the library instead of the allocated per-stream buffer; calls that need more
+ * (e.g. Mo + No > 16,384 at Kc = 16,384) are refused with UE5M3_ERR_UNSUPPORTED.  The call allocates and frees
  * nothing, on the host or the device; the array's address is looked up once per device, at the first call there, so
  * make that first call outside any stream capture.
  * All calls on a device share the array.  Each call rewrites what it reads before its GEMM kernels run, so calls that
  * follow one another on one stream are independent; two calls that can run at the same time (different streams
- * without an ordering between them) race on it and may each use the other's windows: order them, or use ue5m3_gemm.
+ * without an ordering between them) race on it and may each use the other's scales: order them, or use ue5m3_gemm.
  */
 UE5M3_API int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc,
                const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
@@ -232,16 +233,17 @@ UE5M3_API int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc,
  * ue5m3_gemm_fp16: always the FP16 reconstruction kernel; no workspace is touched.
  * ue5m3_gemm_native: the pass over the scale bytes and the native FP4 kernel only.  Kc must be a multiple of 256
  * (UE5M3_ERR_UNSUPPORTED).  `workspace`: device, ue5m3_gemm_native_workspace_bytes(...) bytes, 16-byte aligned, owned by
- * the caller.  After the call its first int32 is 0 when every scale row had a window, and then bytes 16.. hold k for every
- * scale row of A (padded to a multiple of 16) followed by every scale row of B; otherwise the first int32 is non-zero, the
- * kernel has returned at once and `out` is left untouched.
+ * the caller (0 is returned for a Kc that is not a multiple of 256).  After the call its first int32 is 0 when every scale
+ * row had a window, and then bytes 16.. hold k for every scale row of A (padded to a multiple of 16) followed by every scale
+ * row of B (the rest is the kernel's copy of the shifted scales); otherwise the first int32 is non-zero, the kernel has
+ * returned at once and `out` is left untouched.
  * The paper has no counterpart of the split: its Section 5.3 names the three products, not how a device computes them.
  */
 UE5M3_API int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc,
                const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
                const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,
                void* out, int out_dtype, int64_t ldo, void* stream);
-UE5M3_API size_t ue5m3_gemm_native_workspace_bytes(int64_t Mo, int64_t No, int a_scale_mode, int b_scale_mode);
+UE5M3_API size_t ue5m3_gemm_native_workspace_bytes(int64_t Mo, int64_t No, int64_t Kc, int a_scale_mode, int b_scale_mode);
 UE5M3_API int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc,
                const uint8_t* a_payload, const uint8_t* a_scales, int a_scale_mode, const float* a_decode,
                const uint8_t* b_payload, const uint8_t* b_scales, int b_scale_mode, const float* b_decode,

@@ -64,7 +64,7 @@ def _load() -> C.CDLL:
         L.ue5m3_gemm_fp16.restype = ci
         L.ue5m3_gemm_fp16.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp]
         L.ue5m3_gemm_native_workspace_bytes.restype = C.c_size_t
-        L.ue5m3_gemm_native_workspace_bytes.argtypes = [i64, i64, ci, ci]
+        L.ue5m3_gemm_native_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
         L.ue5m3_gemm_native.restype = ci
         L.ue5m3_gemm_native.argtypes = [ci, i64, i64, i64, vp, vp, ci, vp, vp, vp, ci, vp, vp, ci, i64, vp, vp]
         L.ue5m3_gemm_probe_matched.restype = ci
@@ -339,16 +339,16 @@ def gemm_fp16(op: int, a: QuantizedOperand, b: QuantizedOperand, out_dtype: torc
 
 def gemm_native_workspace(a: QuantizedOperand, b: QuantizedOperand) -> torch.Tensor:
     """A workspace of the size ue5m3_gemm_native wants for these operands (uint8, device)."""
-    n = _load().ue5m3_gemm_native_workspace_bytes(a.R, b.R, a.scale_mode, b.scale_mode)
-    return torch.empty(int(n), dtype=torch.uint8, device=a.payload.device)
+    n = _load().ue5m3_gemm_native_workspace_bytes(a.R, b.R, a.Kc, a.scale_mode, b.scale_mode)
+    return torch.empty(max(int(n), 16), dtype=torch.uint8, device=a.payload.device)     # 0: a Kc the call will refuse
 
 
 def native_windows(workspace: torch.Tensor, a: QuantizedOperand, b: QuantizedOperand):
     """Reads a workspace back: (all rows have windows, k of A's scale rows, k of B's scale rows) as numpy arrays."""
-    w = workspace.cpu().numpy()
     ra = a.R // 16 if a.scale_mode == SCALE_2D else a.R
     rb = b.R // 16 if b.scale_mode == SCALE_2D else b.R
     off_b = 16 + ((ra + 15) // 16) * 16
+    w = workspace[:off_b + rb].cpu().numpy()          # the shifted scales that follow are the kernel's own business
     return int(w[:4].view("int32")[0]) == 0, w[16:16 + ra].copy(), w[off_b:off_b + rb].copy()
 
 

@@ -214,9 +214,9 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
     if (!native_eligible(g)) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
     // Three launches, one of which does the product: the windows of the scale rows, the native FP4 kernel (works when
     // every scale row of both operands has a UE4M3 window) and the FP16 kernel (works when one does not).
-    int* ws = native_workspace(native_workspace_bytes(g));
+    int* ws = native_workspace(native_layout(g).bytes, (cudaStream_t)stream);
     if (!ws) return UE5M3_ERR_CUDA;
-    int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
+    int r = launch_scale_prepare(g, ws, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
     r = launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
@@ -236,9 +236,9 @@ int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t*
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
     if (Kc % 256) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);      // the FP16 kernel alone: no workspace
-    int* ws = static_workspace(native_workspace_bytes(g));    // 16 bytes + one per scale row of the two operands
-    if (!ws) return UE5M3_ERR_UNSUPPORTED;            // more rows than the file-scope array holds
-    int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
+    int* ws = static_workspace(native_layout(g).bytes);
+    if (!ws) return UE5M3_ERR_UNSUPPORTED;            // larger operands than the file-scope array has room for
+    int r = launch_scale_prepare(g, ws, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
     r = launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
@@ -260,11 +260,11 @@ int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a
     return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
 }
 
-size_t ue5m3_gemm_native_workspace_bytes(int64_t Mo, int64_t No, int a_scale_mode, int b_scale_mode) {
-    if (Mo <= 0 || No <= 0) return 0;
+size_t ue5m3_gemm_native_workspace_bytes(int64_t Mo, int64_t No, int64_t Kc, int a_scale_mode, int b_scale_mode) {
+    if (Mo <= 0 || No <= 0 || Kc <= 0 || Kc % 256) return 0;
     GemmArgs g{};
-    g.Mo = Mo; g.No = No; g.a_scale_mode = a_scale_mode; g.b_scale_mode = b_scale_mode;
-    return native_workspace_bytes(g);
+    g.Mo = Mo; g.No = No; g.Kc = Kc; g.a_scale_mode = a_scale_mode; g.b_scale_mode = b_scale_mode;
+    return native_layout(g).bytes;
 }
 
 int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payload, const uint8_t* a_scales,
@@ -283,7 +283,7 @@ int ue5m3_gemm_native(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t*
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
     if (Kc % 256) return UE5M3_ERR_UNSUPPORTED;
-    const int r = launch_scale_range(g, workspace, di.sms, (cudaStream_t)stream);
+    const int r = launch_scale_prepare(g, workspace, di.sms, (cudaStream_t)stream);
     if (r != UE5M3_OK) return r;
     return launch_gemm_native(g, workspace, di.sms, (cudaStream_t)stream);
 }
@@ -327,9 +327,9 @@ int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, con
     if (which == 2) {
         // the native kernel: its workspace is filled by the range kernel as in ue5m3_gemm (the operands must have windows)
         if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
-        int* ws = native_workspace(native_workspace_bytes(g));
+        int* ws = native_workspace(native_layout(g).bytes, (cudaStream_t)stream);
         if (!ws) return UE5M3_ERR_CUDA;
-        const int r = launch_scale_range(g, ws, di.sms, (cudaStream_t)stream);
+        const int r = launch_scale_prepare(g, ws, di.sms, (cudaStream_t)stream);
         if (r != UE5M3_OK) return r;
         return launch_gemm_native(g, ws, di.sms, (cudaStream_t)stream);
     }

@@ -5,25 +5,30 @@
 // the signed format's unsigned half, UE4M3 (bias 7, codes 0x08 .. 0x7E normal).  A normal UE5M3 code c (bias 15)
 // and the UE4M3 code c - 8k have the same three fraction bits and exponents that differ by the constant k - 8:
 //     value5(c) = value4(c - 8k) * 2^(k - 8)      for every c with 8 <= c - 8k <= 126,
-// exactly.  When all scale codes of an operand lie in one such window of 119 codes (a ratio of 2^14.8 between the
-// largest and the smallest block scale), the GEMM is the native one on the shifted codes and the two powers of two
-// go into alpha.  The packed payload reaches the tensor core as the copy engine delivered it: no conversion, no
-// second staging.  The shifted scale bytes (three integer operations per four codes) take their own route into
-// tensor memory, in the layout the block-scaled MMA reads.
+// exactly.  The shift k may differ from one scale row to the next (an output row m for A, an output column n for B):
+// the tensor core sums value4 products along K for one (m, n), and the two constant factors 2^(k_m - 8) and
+// 2^(k_n - 8) come out of the sum.  So when the codes of every scale row lie in one such window of 119 codes (a ratio
+// of 2^14.8 between the largest and the smallest block scale of that row), the GEMM is the native one on the shifted
+// codes and the epilogue multiplies each output by its two powers of two, which is exact.  The packed payload reaches
+// the tensor core as the copy engine delivered it: no conversion, no second staging.  The shifted scale bytes (three
+// integer operations per four codes) take their own route into tensor memory, in the layout the block-scaled MMA reads.
 //
-// The window is found on the device: scale_range_kernel reduces both operands' scale bytes to their largest and
-// smallest non-zero code (four words of workspace), gemm_native_kernel reads them and returns at once when an
-// operand has no window (subnormal UE5M3 codes included); the caller then runs the FP16 path, whose kernel
-// evaluates the same predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.
+// The windows are found on the device: scale_range_kernel gives each scale row of both operands to one warp, which
+// reduces the row's codes to the largest and the smallest non-zero one and writes the row's k (one byte) into the
+// workspace, or sets the workspace's first word when the row has no window (subnormal UE5M3 codes included).
+// gemm_native_kernel reads that word and returns at once when it is set; the caller then runs the FP16 path, whose
+// kernel evaluates the same predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.  Where a
+// row allows it k is 2, so that the rows of ordinary data share one shift and the epilogue takes its uniform path.
 //
 // Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 5 payload stages of 32 KB):
 //   warp 0      copies: packed A rows (128) and packed B rows (this CTA's 128) of a stage
 //   warp 1      (leader CTA) MMA issuer: 4 MMAs of K = 64 and one commit per stage
 //   warp 2      tensor-memory allocation; relay: tells the leader CTA that this CTA's copy of a stage has landed
 //   warp 3      (leader CTA) scale copier: 12 tcgen05.cp per stage, shared memory -> tensor memory of both CTAs
-//   warps 4-7   epilogue: accumulator -> alpha -> BF16 / FP32 -> shared memory -> bulk tensor store
+//   warps 4-7   epilogue: accumulator -> alpha and the row's and column's window factors -> BF16 / FP32 -> shared
+//               memory -> bulk tensor store
 //   warps 8-15  scale bytes, two groups of four warps taking the stages in turn: read from global memory four stages
-//               ahead (registers), window shift, stored in the order the scale copy wants into a ring of six stages
+//               ahead (registers), each row's window shift, stored in the order the scale copy wants into a ring of six stages
 //               in shared memory
 // Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 64..319, four
 // stages of scales in columns 320..511.  Two whole accumulators do not fit beside the scales, so the two overlap in
@@ -39,8 +44,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdint>
-#include <atomic>
 #include <mutex>
+#include <vector>
 #include "../../include/ue5m3.h"
 #include "launch.h"
 #include "tcgen05.cuh"
@@ -58,27 +63,26 @@ constexpr int BNH = 128;                    // B rows staged by each CTA
 constexpr int KCHUNK = 256;                 // K per stage
 constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks)
 constexpr int MMAS = KCHUNK / KMMA;
-constexpr int STAGES = 5;                   // payload stages
-constexpr int SF_SLOTS = 4;                 // stages whose scales are in tensor memory at a time
-constexpr int PF = 2;                       // group-stages (= 4 stages) the scale bytes are read ahead (registers)
-constexpr int SF_RING = 6;                  // stages of shifted scales in shared memory, on their way to tensor memory
-constexpr int CONV_WARP0 = 8, CONV_WARPS = 4, EPI_WARP0 = 4;    // CONV_WARPS per group; two groups take the stages in turn
-constexpr int NUM_THREADS = 32 * (CONV_WARP0 + 2 * CONV_WARPS);
-static_assert(SF_RING % 2 == 0, "each scale group owns every other ring stage");
+constexpr int STAGES = 5;                   // stages of payload and scales
+constexpr int SF_SLOTS = 2;                 // stages whose scales have room in tensor memory
+constexpr int EPI_WARP0 = 4;
+constexpr int NUM_THREADS = 256;
 
 constexpr int PK_A_BYTES = BM * KCHUNK / 2;           // 16384
 constexpr int PK_B_BYTES = BNH * KCHUNK / 2;          // 16384
-constexpr int STAGE_BYTES = PK_A_BYTES + PK_B_BYTES;  // 32768
-constexpr int XCH_A_BYTES = BM * (KCHUNK / 16), XCH_BYTES = XCH_A_BYTES + BN * (KCHUNK / 16);   // 2048 + 4096 per stage
-constexpr int SMEM_XCH = STAGES * STAGE_BYTES;        // 163840
-constexpr int SMEM_BARS = SMEM_XCH + SF_RING * XCH_BYTES;   // 200704
+constexpr int SF_A_BYTES = BM * (KCHUNK / 16);        // 2048: this CTA's 128 rows of A
+constexpr int SF_B_BYTES = BN * (KCHUNK / 16);        // 4096: all 256 rows of B (each CTA's MMA half reads all of them)
+constexpr int SF_OFF = PK_A_BYTES + PK_B_BYTES;       // the stage's scales follow its payload
+constexpr int STAGE_BYTES = SF_OFF + SF_A_BYTES + SF_B_BYTES;     // 38912, a multiple of 1024 (128-byte swizzle)
+constexpr int SMEM_BARS = STAGES * STAGE_BYTES;       // 194560
 constexpr int SMEM_EPI = SMEM_BARS + 1024;
 constexpr int EPI_WARP_BYTES = 4096;
-constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 219136
-// Tensor memory (512 columns): accumulator of even tiles 0..255, of odd tiles 64..319 (they share 192 columns), then four
-// scale slots of 48 columns: 16 for A (column 4 j + g: rows 32 g + lane, MMA j) and 32 for B (column 8 j + 4 h + g).
-// A slot is written again only after the MMAs that read it have retired; four slots cover that turn-around (commit,
-// barrier, copies, commit, barrier, issue).
+constexpr int SMEM_BYTES = SMEM_EPI + 4 * EPI_WARP_BYTES + 1024;  // 212992
+static_assert(STAGE_BYTES % 1024 == 0, "payload stages must stay 1024-byte aligned");
+// Tensor memory (512 columns): accumulator of even tiles from column 0, of odd tiles from TMEM_ACC_ODD (they share
+// 32 * OVERLAP_UNITS columns), then SF_SLOTS scale slots of 48 columns: 16 for A (column 4 j + g: rows 32 g + lane, MMA j)
+// and 32 for B (column 8 j + 4 h + g).  Scale copies and MMAs are issued by one thread and run in issue order, so a
+// slot may be written again as soon as the MMAs that read it have been issued.
 constexpr int TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
 constexpr int OVERLAP_UNITS = (SF_SLOTS * TMEM_SF_SLOT_COLS + 31) / 32;       // 32-column units the two accumulators share
 constexpr int TMEM_ACC_ODD = 256 - 32 * OVERLAP_UNITS;
@@ -91,8 +95,8 @@ struct NativeParams {
     const int* workspace;         // word 0: 0 when every scale row has a window (layout in window.cuh)
     const uint8_t* ka_rows;       // shift k of every scale row of A
     const uint8_t* kb_rows;       // ... of B
-    const uint8_t* a_scales;
-    const uint8_t* b_scales;
+    const uint8_t* sfa;           // shifted scales of A in the order the scale copy wants: [128-row group][stage][2048]
+    const uint8_t* sfb;           // ... of B: [256-row tile][stage][4096]
     int out_bf16;
     int a_mode, b_mode;
     int tiles_m, tiles_n;
@@ -145,59 +149,130 @@ __device__ __forceinline__ uint64_t sf_smem_desc(uint32_t saddr) {
     d |= (uint64_t)1 << 46;
     return d;
 }
-// 16 consecutive 32-bit columns of this thread's tensor-memory lane.
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t r[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-__device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+// Plain bulk copy global -> shared memory of this CTA (addresses and size multiples of 16), completion on `bar`.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-// ----------------------------------------------------------------------------- windows of the scale rows
-// One warp per scale row of A and then of B: the row's largest and smallest non-zero code -> its shift k (a byte of
-// the workspace), or the workspace's first word set when the row has no window.  `tiled`: the row's 16-byte pieces lie
-// 2048 bytes apart (128 x 16 tiles) instead of back to back.
-__global__ void __launch_bounds__(512) scale_range_kernel(const uint8_t* __restrict__ a, int64_t rows_a, int a_tiled,
-                                                          const uint8_t* __restrict__ b, int64_t rows_b, int b_tiled,
-                                                          int64_t kblocks, int* __restrict__ workspace) {
+// ----------------------------------------------------------------------------- windows and scale layout
+// One CTA per group of 128 operand rows (first A's groups, then B's).  First the window of every scale row of the
+// group: largest and smallest non-zero code -> shift k (a byte of the workspace, for the epilogue's factors), or the
+// workspace's first word set when a row has no window.  Then the group's scale bytes, shifted by 8 k, are written in
+// the order the tensor core's scale copy reads them: per stage of 256 K and MMA j, 32 pieces of 16 bytes, piece dp
+// holding the four block scales of MMA j for rows dp, 32 + dp, 64 + dp, 96 + dp.  A's groups lie one after the other
+// ([group][stage][j][dp]); B's two groups of a 256-row tile are interleaved per MMA ([tile][stage][j][half][dp]).
+// Rows beyond the operand get zeros.  Source layouts: one row after the other (1D), 16-byte pieces of 128 rows
+// interleaved (1D tiled: piece p of row r at (r / 128 * pieces + p) * 2048 + r % 128 * 16), one row per 16 operand
+// rows (2D).
+struct PrepareParams {
+    const uint8_t* src[2];
+    int64_t rows[2];              // operand rows (Mo, No)
+    int mode[2];
+    int groups_a;                 // 128-row groups of A (2 per row of tiles)
+    int64_t kblocks;              // Kc / 16
+    int* workspace;
+    uint8_t* k_rows[2];
+    uint8_t* sf[2];
+};
+
+// The group's scale bytes pass through shared memory (rows of `cblocks` bytes + one word, so that the 32 rows a warp
+// gathers from lie in 32 banks): read once from global memory, 64 bytes per row at a time, when the rows have at most
+// kPrepChunkBlocks bytes; longer rows are read twice, chunk by chunk (first for the windows, then for the re-ordering).
+constexpr int kPrepChunkBlocks = 1536;
+constexpr int kPrepSmemBytes = 128 * (kPrepChunkBlocks + 4);
+
+__global__ void __launch_bounds__(512) scale_prepare_kernel(const PrepareParams q) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the GEMM's prologue may run beside this kernel
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= rows_a + rows_b) return;
-    const bool is_b = row >= rows_a;
-    const int64_t r = is_b ? row - rows_a : row;
-    const uint8_t* s = is_b ? b : a;
-    const bool tiled = is_b ? b_tiled : a_tiled;
-    const int64_t pieces = kblocks >> 4;                                 // 16-byte pieces of the row (Kc is a multiple of 256)
-    const uint8_t* base = tiled ? s + (r >> 7) * pieces * 2048 + (r & 127) * 16 : s + r * kblocks;
-    const int64_t pstride = tiled ? 2048 : 16;
+    extern __shared__ uint32_t rows_smem[];
+    __shared__ uint32_t shift8[128];                                     // 8 k in every byte, per scale row of the group
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int is_b = (int)blockIdx.x >= q.groups_a;
+    const int group = is_b ? (int)blockIdx.x - q.groups_a : (int)blockIdx.x;
+    const uint8_t* __restrict__ src = is_b ? q.src[1] : q.src[0];
+    const int mode = is_b ? q.mode[1] : q.mode[0];
+    uint8_t* k_rows = is_b ? q.k_rows[1] : q.k_rows[0];
+    const int64_t R = is_b ? q.rows[1] : q.rows[0], r0 = (int64_t)group * 128;
+    const int pieces = (int)(q.kblocks >> 4);                            // 16-byte pieces (= stages) of a row
+    const bool two_d = mode == UE5M3_SCALE_2D, tiled = mode == UE5M3_SCALE_1D_TILED;
+    const int64_t srows = two_d ? R / 16 : R, s0 = two_d ? r0 / 16 : r0;  // scale rows: all of them, first of the group
+    const int nrows = two_d ? 8 : 128;
+    const int chunk_pieces = min(pieces, kPrepChunkBlocks / 16);
+    const int nchunks = (pieces + chunk_pieces - 1) / chunk_pieces;
+    const int pitch = chunk_pieces * 4 + 1;                              // words per row in shared memory
+    auto piece_ptr = [&](int64_t srow, int piece) -> const uint8_t* {
+        return tiled ? src + ((srow >> 7) * pieces + piece) * 2048 + (srow & 127) * 16 : src + srow * q.kblocks + (int64_t)piece * 16;
+    };
+    // a warp takes 8 scale rows, four lanes per row
+    const int i = warp * 8 + (lane >> 2);
+    const int64_t srow = s0 + i;
+    const bool have_row = i < nrows && srow < srows;
     uint32_t m = 0u, iv = 0u;
-    for (int64_t i = lane; i < pieces; i += 32) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + i * pstride));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    auto load_chunk = [&](int c, bool keep, bool reduce) {
+        const int first = c * chunk_pieces, n = min(chunk_pieces, pieces - first);
+        if (!have_row) return;
+        uint32_t* mine = rows_smem + i * pitch;
+        for (int pc0 = lane & 3; pc0 < n; pc0 += 32) {                   // eight loads in flight per thread
+            uint4 v[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            m = __vmaxu4(m, w[j]);
-            iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));              // 255 - c, and 0 for c = 0
+            for (int t = 0; t < 8; ++t)
+                v[t] = pc0 + 4 * t < n ? __ldg(reinterpret_cast<const uint4*>(piece_ptr(srow, first + pc0 + 4 * t))) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const int pc = pc0 + 4 * t;
+                const uint32_t w[4] = {v[t].x, v[t].y, v[t].z, v[t].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (reduce) {
+                        m = __vmaxu4(m, w[j]);
+                        iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));  // 255 - c, and 0 for c = 0
+                    }
+                    if (keep && pc < n) mine[4 * pc + j] = w[j];
+                }
+            }
         }
-    }
+    };
+    for (int c = 0; c < nchunks; ++c) load_chunk(c, nchunks == 1, true);
     m = max(max(m & 0xFFu, (m >> 8) & 0xFFu), max((m >> 16) & 0xFFu, m >> 24));
     iv = max(max(iv & 0xFFu, (iv >> 8) & 0xFFu), max((iv >> 16) & 0xFFu, iv >> 24));
-    m = __reduce_max_sync(0xFFFFFFFFu, m);
-    iv = __reduce_max_sync(0xFFFFFFFFu, iv);
-    if (lane == 0) {
-        int k;
-        const bool ok = pick_window((int)m, (int)iv, k);
-        uint8_t* kbytes = reinterpret_cast<uint8_t*>(workspace) + 16 + (is_b ? ((rows_a + 15) / 16) * 16 : 0);
-        kbytes[r] = (uint8_t)k;
-        if (!ok) atomicOr(workspace, 1);
+#pragma unroll
+    for (int d = 1; d <= 2; d <<= 1) {
+        m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+        iv = max(iv, __shfl_xor_sync(0xFFFFFFFFu, iv, d));
+    }
+    if ((lane & 3) == 0 && i < nrows) {
+        int k = 8;
+        const bool ok = !have_row || pick_window((int)m, (int)iv, k);
+        shift8[i] = ok ? (uint32_t)(8 * k) * 0x01010101u : 0u;
+        if (have_row) k_rows[srow] = (uint8_t)k;
+        if (!ok) atomicOr(q.workspace, 1);
+    }
+    __syncthreads();
+    // shifted bytes in the scale copy's order: thread -> one 16-byte piece (stage s, MMA j, lane dp), rows 32 g + dp
+    uint8_t* out = is_b ? q.sf[1] + (int64_t)(group >> 1) * pieces * 4096 + (group & 1) * 512 : q.sf[0] + (int64_t)group * pieces * 2048;
+    const int64_t stride_s = is_b ? 4096 : 2048, stride_j = is_b ? 1024 : 512;
+    for (int c = 0; c < nchunks; ++c) {
+        const int first = c * chunk_pieces, n = min(chunk_pieces, pieces - first);
+        if (nchunks > 1) {
+            __syncthreads();                                             // the previous chunk has been read out
+            load_chunk(c, true, false);
+            __syncthreads();
+        }
+        for (int u = threadIdx.x; u < n * 128; u += blockDim.x) {
+            const int dp = u & 31, j = (u >> 5) & 3, sl = u >> 7;
+            uint32_t w[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const int row = 32 * g + dp;
+                w[g] = 0u;
+                if (r0 + row < R) {
+                    const int ri = two_d ? row >> 4 : row;
+                    const uint32_t v = rows_smem[ri * pitch + 4 * sl + j];
+                    w[g] = __vsub4(v, shift8[ri]) & ~__vcmpeq4(v, 0u);    // a code of 0 stays 0
+                }
+            }
+            *reinterpret_cast<uint4*>(out + (int64_t)(first + sl) * stride_s + j * stride_j + dp * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
     }
 }
 
@@ -211,8 +286,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const uint32_t bar_base = smem_base + SMEM_BARS;
     // barriers (8 bytes each)
     const uint32_t pk_full = bar_base, pk_empty = bar_base + 64, pk_ready = bar_base + 128;
-    const uint32_t sf_full = bar_base + 192, sf_empty = bar_base + 256;
-    const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336, drain_bar2 = bar_base + 360;
+    const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 344);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 352);
 
@@ -229,15 +303,9 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(pk_full + 8 * s, 1);
             mbar_init(pk_empty + 8 * s, 1);
-            // the leader's copy collects, for the stage that lives here, both CTAs' relays (payload landed) and the commit
-            // of the scale copies (the stage's scales are in tensor memory)
-            mbar_init(pk_ready + 8 * s, 3);
+            // the leader's copy collects both CTAs' relays: the stage's payload and scales have landed in both
+            mbar_init(pk_ready + 8 * s, 2);
         }
-        for (int s = 0; s < SF_RING; ++s) {
-            mbar_init(sf_full + 8 * s, 2 * CONV_WARPS);        // the leader's copy collects both CTAs' scale warps
-            mbar_init(sf_empty + 8 * s, 1);
-        }
-        mbar_init(drain_bar2, 1);
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 8);
         mbar_init(drain_bar, 1);
@@ -272,6 +340,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     mbar_expect_tx(full, STAGE_BYTES);
                     tma_load_2d(st, &map_a, full, kc * (KCHUNK / 2), mb * BM);
                     tma_load_2d(st + PK_A_BYTES, &map_b, full, kc * (KCHUNK / 2), nh * BNH);
+                    bulk_load(st + SF_OFF, p.sfa + ((int64_t)mb * kchunks + kc) * SF_A_BYTES, SF_A_BYTES, full);
+                    bulk_load(st + SF_OFF + SF_A_BYTES, p.sfb + ((int64_t)tn * kchunks + kc) * SF_B_BYTES, SF_B_BYTES, full);
                 }
             }
             // let the copies still in flight land before the CTA's shared memory goes away (every one of them was
@@ -290,53 +360,6 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 mbar_arrive_cluster(pk_ready + 8 * s, 0);
             }
         }
-    } else if (warp == 3) {
-        // ------------------------------------------------------------------ scale copier (leader CTA)
-        // Shared memory -> tensor memory, for both CTAs at once: 12 copies per stage (A: one per MMA, B: two), each of
-        // which the hardware replicates to the four lane quarters.  Warp-uniform loop, one elected lane issues (see the
-        // MMA issuer).  The commit after the copies tells the MMA issuer that the stage's scales are in place and both
-        // CTAs' scale warps that the shared-memory stage may be rewritten.
-        if (rank == 0) {
-            bool ok = true;
-            const bool elected = elect_one();
-            const uint64_t d_sf = sf_smem_desc(smem_base + SMEM_XCH);
-            const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
-            const uint32_t tm0 = __shfl_sync(0xFFFFFFFFu, tmem_base, 0) + TMEM_SF_COL;
-            uint32_t s = 0, f = 0, fph = 0, u = 0;        // payload stage, shared-memory scale stage and phase, tensor-memory slot
-            for (uint32_t it = 0; it < total && ok; ++it) {
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(sf_full + 8 * f, fph, abort_flag, p.wait_limit));
-                if (!ok) break;
-                // the slot held the scales of stage it - SF_SLOTS: free once that stage's MMAs have retired, which is what
-                // the payload barrier of that stage says
-                if (it >= SF_SLOTS) {
-                    const uint32_t prev = it - SF_SLOTS;
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(pk_empty + 8 * (prev % STAGES), (prev / STAGES) & 1, abort_flag, p.wait_limit));
-                    if (!ok) break;
-                }
-                tc_fence_after();
-                const uint32_t lo = sf_lo0 + f * (XCH_BYTES >> 4), lob = lo + (XCH_A_BYTES >> 4);
-                const uint32_t sfa = tm0 + u * TMEM_SF_SLOT_COLS, sfb = sfa + TMEM_SFB_OFF;
-                if (elected) {
-#pragma unroll
-                    for (int j = 0; j < MMAS; ++j) {
-                        tmem_cp_32x128b(sfa + 4 * j, lo + j * (512 >> 4), sf_hi);
-                        tmem_cp_32x128b(sfb + 8 * j, lob + j * (1024 >> 4), sf_hi);
-                        tmem_cp_32x128b(sfb + 8 * j + 4, lob + j * (1024 >> 4) + (512 >> 4), sf_hi);
-                    }
-                    umma_commit_local(pk_ready + 8 * s);
-                    umma_commit_pair(sf_empty + 8 * f);
-                }
-                __syncwarp();
-                if (++s == STAGES) s = 0;
-                if (++f == SF_RING) { f = 0; fph ^= 1; }
-                if (++u == SF_SLOTS) u = 0;
-            }
-            if (elected) {
-                umma_commit_local(drain_bar2);
-                mbar_wait_drain(drain_bar2, 0, &g_native_status, p.wait_limit);
-            }
-            __syncwarp();
-        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
         // The whole warp runs the loop and one elected lane issues: the operands of the tensor instructions (descriptors,
@@ -347,11 +370,13 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             uint32_t tl = 0;
             bool ok = true;
             const bool elected = elect_one();
-            // descriptor halves of the payload stages (128-byte swizzle); only the start address moves
-            const uint64_t d_pk = umma_smem_desc(smem_base);
+            // descriptor halves of the payload stages (128-byte swizzle) and of the scale pieces (no swizzle); only the
+            // start address moves
+            const uint64_t d_pk = umma_smem_desc(smem_base), d_sf = sf_smem_desc(smem_base + SF_OFF);
             const uint32_t pk_lo0 = (uint32_t)d_pk, pk_hi = (uint32_t)(d_pk >> 32);
+            const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
             const uint32_t tm0 = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
-            uint32_t s = 0, ph = 0, u = 0;                // payload stage and its phase, scale slot
+            uint32_t s = 0, ph = 0, u = 0;                // stage and its phase, scale slot
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit));
                 if (!ok) break;
@@ -362,15 +387,21 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_lo = pk_lo0 + s * (STAGE_BYTES >> 4), b_lo = a_lo + (PK_A_BYTES >> 4);
+                    const uint32_t xa_lo = sf_lo0 + s * (STAGE_BYTES >> 4), xb_lo = xa_lo + (SF_A_BYTES >> 4);
                     const uint32_t sfa = tm0 + TMEM_SF_COL + u * TMEM_SF_SLOT_COLS, sfb = sfa + TMEM_SFB_OFF;
                     if (elected) {
+                        // Per MMA of K = 64: its scales, shared memory -> tensor memory of both CTAs (32 rows x 16 bytes -> 4
+                        // columns, replicated by the hardware to the four lane quarters; one copy for A's 128 rows per CTA, two
+                        // for B's 256), then the MMA.  Copies and MMAs run in the order they are issued.
 #pragma unroll
-                        for (int j = 0; j < MMAS; ++j)
+                        for (int j = 0; j < MMAS; ++j) {
+                            tmem_cp_32x128b(sfa + 4 * j, xa_lo + j * (512 >> 4), sf_hi);
+                            tmem_cp_32x128b(sfb + 8 * j, xb_lo + j * (1024 >> 4), sf_hi);
+                            tmem_cp_32x128b(sfb + 8 * j + 4, xb_lo + j * (1024 >> 4) + (512 >> 4), sf_hi);
                             umma_fp4_block16(tmem_d, a_lo + 2 * j, b_lo + 2 * j, pk_hi, kInstrDesc, sfa + 4 * j, sfb + 8 * j,
                                              (kc | j) != 0 ? 1u : 0u);
-                        // both CTAs may refill this payload stage; their scale warps read the same barrier to learn that
-                        // the scale slot of this stage is free again
-                        umma_commit_pair(pk_empty + 8 * s);
+                        }
+                        umma_commit_pair(pk_empty + 8 * s);        // both CTAs may refill this stage
                     }
                     __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1; }
@@ -531,102 +562,6 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             }
         }
         if (lane == 0) tma_store_wait_all();
-    } else if (warp >= CONV_WARP0) {
-        // ------------------------------------------------------------------ scale bytes: window shift and re-layout
-        // The tensor core wants the scales of row 32 g + r in lane r (of every lane quarter), one column per (MMA, g) with
-        // the MMA's four block scales as its bytes; the scale copy (32 rows x 16 bytes -> 4 columns) makes that from
-        // shared memory laid out [MMA][r][g] in 4-byte words.  Two groups of four warps take the stages in turn; a group's
-        // 128 threads read one row each of A and of the two B halves (16 bytes per row and stage, PF group-stages ahead in
-        // registers), shift the codes and store them there; the lane assignment makes a warp's 32 stores consecutive words.
-        const int cg = (warp - CONV_WARP0) >> 2, cw = warp & 3;          // group (= stage parity), warp inside the group
-        const int row = (lane & 3) * 32 + cw * 8 + (lane >> 2);            // the row this thread reads
-        const int64_t kblocks = p.Kc >> 4;
-        uint32_t cda = 0u, cdb0 = 0u, cdb1 = 0u;      // 8 k in every byte, for the three rows of the cursor's tile
-        auto shift = [](uint32_t v, uint32_t d) { return __vsub4(v, d) & ~__vcmpeq4(v, 0u); };
-        const int64_t step_a = p.a_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16, step_b = p.b_mode == UE5M3_SCALE_1D_TILED ? 2048 : 16;
-        const uint8_t *pa = nullptr, *pb0 = nullptr, *pb1 = nullptr;
-        int c_tile = pair, c_kc = 0;
-        auto row_base = [&](const uint8_t* scales, int mode, int64_t R, int64_t grow) -> const uint8_t* {
-            if (grow >= R) return nullptr;
-            if (mode == UE5M3_SCALE_1D_TILED) return scales + (grow >> 7) * kchunks * 2048 + (grow & 127) * 16;
-            return scales + ((mode == UE5M3_SCALE_2D) ? (grow >> 4) : grow) * kblocks;
-        };
-        // the three rows' shift bytes of a tile, asked for one tile ahead (raw bytes; 0 beyond the operands)
-        uint32_t nka = 0u, nkb0 = 0u, nkb1 = 0u;
-        auto ask_shifts = [&](int tile) {
-            nka = nkb0 = nkb1 = 0u;
-            if (tile >= num_tiles) return;
-            int tm, tn;
-            tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
-            const int64_t ga = (int64_t)(tm * 2 + (int)rank) * BM + row, gb0 = (int64_t)tn * BN + row, gb1 = gb0 + BNH;
-            if (ga < p.Mo) nka = __ldg(p.ka_rows + (p.a_mode == UE5M3_SCALE_2D ? (ga >> 4) : ga));
-            if (gb0 < p.No) nkb0 = __ldg(p.kb_rows + (p.b_mode == UE5M3_SCALE_2D ? (gb0 >> 4) : gb0));
-            if (gb1 < p.No) nkb1 = __ldg(p.kb_rows + (p.b_mode == UE5M3_SCALE_2D ? (gb1 >> 4) : gb1));
-        };
-        auto open_tile = [&]() {
-            if (c_tile >= num_tiles) { pa = pb0 = pb1 = nullptr; return; }
-            int tm, tn;
-            tile_coords(c_tile, p.tiles_m, p.tiles_n, tm, tn);
-            const int64_t ga = (int64_t)(tm * 2 + (int)rank) * BM + row, gb0 = (int64_t)tn * BN + row, gb1 = gb0 + BNH;
-            pa = row_base(p.a_scales, p.a_mode, p.Mo, ga);
-            pb0 = row_base(p.b_scales, p.b_mode, p.No, gb0);
-            pb1 = row_base(p.b_scales, p.b_mode, p.No, gb1);
-            // this tile's shifts were asked for when the previous tile was opened; now ask for the next tile's
-            cda = ((8u * nka) & 0xFFu) * 0x01010101u;
-            cdb0 = ((8u * nkb0) & 0xFFu) * 0x01010101u;
-            cdb1 = ((8u * nkb1) & 0xFFu) * 0x01010101u;
-            ask_shifts(c_tile + num_pairs);
-        };
-        auto advance = [&]() {                       // the cursor moves on by one stage
-            if (++c_kc == kchunks) {
-                c_kc = 0;
-                c_tile += num_pairs;
-                open_tile();
-            } else {
-                if (pa) pa += step_a;
-                if (pb0) pb0 += step_b;
-                if (pb1) pb1 += step_b;
-            }
-        };
-        auto fetch = [&](uint4& a, uint4& b0, uint4& b1, uint32_t (&d)[3]) {     // this group's next stage; the other group's is skipped
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            a = pa ? ldg_nc_16(pa) : z;
-            b0 = pb0 ? ldg_nc_16(pb0) : z;
-            b1 = pb1 ? ldg_nc_16(pb1) : z;
-            d[0] = cda; d[1] = cdb0; d[2] = cdb1;
-            advance();
-            advance();
-        };
-        ask_shifts(pair);
-        open_tile();
-        if (cg) advance();
-        uint4 ra[PF], rb0[PF], rb1[PF];
-        uint32_t rd[PF][3];
-#pragma unroll
-        for (int d = 0; d < PF; ++d) fetch(ra[d], rb0[d], rb1[d], rd[d]);
-        bool ok = true;
-        uint32_t f = cg, fph = 0;
-        for (uint32_t base = cg; base < total && ok; base += 2 * PF) {
-#pragma unroll
-            for (int d = 0; d < PF; ++d) {
-                const uint32_t it = base + 2 * d;
-                if (it >= total || !ok) break;
-                if (!mbar_wait(sf_empty + 8 * f, fph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
-                uint32_t* xa = reinterpret_cast<uint32_t*>(smem_gen + SMEM_XCH + f * XCH_BYTES) + cw * 32 + lane;     // + 128 j
-                uint32_t* xb = xa + XCH_A_BYTES / 4;                                                                  // + 256 j + 128 h
-                const uint4 a = ra[d], b0 = rb0[d], b1 = rb1[d];
-                const uint32_t da = rd[d][0], db0 = rd[d][1], db1 = rd[d][2];
-                xa[0] = shift(a.x, da); xa[128] = shift(a.y, da); xa[256] = shift(a.z, da); xa[384] = shift(a.w, da);
-                xb[0] = shift(b0.x, db0); xb[256] = shift(b0.y, db0); xb[512] = shift(b0.z, db0); xb[768] = shift(b0.w, db0);
-                xb[128] = shift(b1.x, db1); xb[384] = shift(b1.y, db1); xb[640] = shift(b1.z, db1); xb[896] = shift(b1.w, db1);
-                fence_proxy_async();                 // the tensor core's scale copy reads what was just written
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(sf_full + 8 * f, 0);
-                fetch(ra[d], rb0[d], rb1[d], rd[d]);
-                f += 2;
-                if (f >= SF_RING) { f -= SF_RING; fph ^= 1; }
-            }
-        }
     }
 
     tc_fence_before();
@@ -653,40 +588,41 @@ bool make_out_map(CUtensorMap* m, void* out, bool bf16, int64_t Mo, int64_t No, 
 
 }  // namespace
 
-bool native_eligible(const GemmArgs& g) {
-    return g.Kc % KCHUNK == 0 && native_workspace_bytes(g) <= kNativeWorkspaceSlotBytes;
-}
-
-// Device workspace for one call: a ring of 64 slots of kNativeWorkspaceSlotBytes per device, allocated at the first call
-// on that device.  Calls that are in flight at the same time (different streams) use different slots as long as fewer
-// than 64 of them overlap.
-int* native_workspace(size_t need_bytes) {
-    constexpr unsigned kSlots = 64;
-    static uint8_t* ring[64];
-    static std::once_flag made[64];
-    static std::atomic<unsigned> next{0};
-    if (need_bytes > kNativeWorkspaceSlotBytes) return nullptr;
+// Device workspace of one call: one buffer per (device, stream), grown (never shrunk, never freed) when a call needs
+// more.  Calls on one stream run one after the other, so they may share a buffer; calls on different streams have
+// different buffers.  Growing allocates: a call made while its stream is being captured must find a buffer that an
+// earlier call on that stream has made large enough.
+int* native_workspace(size_t need_bytes, cudaStream_t st) {
+    struct Buffer { int dev; cudaStream_t st; uint8_t* ptr; size_t bytes; };
+    static std::mutex mu;
+    static std::vector<Buffer> buffers;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    std::call_once(made[dev], [&]() {
-        void* ptr = nullptr;
-        if (cudaMalloc(&ptr, kSlots * kNativeWorkspaceSlotBytes) != cudaSuccess) { (void)cudaGetLastError(); return; }
-        ring[dev] = static_cast<uint8_t*>(ptr);
-    });
-    if (!ring[dev]) return nullptr;
-    return reinterpret_cast<int*>(ring[dev] + (size_t)(next.fetch_add(1) % kSlots) * kNativeWorkspaceSlotBytes);
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    Buffer* mine = nullptr;
+    for (Buffer& b : buffers)
+        if (b.dev == dev && b.st == st) { mine = &b; break; }
+    if (mine && mine->bytes >= need_bytes) return reinterpret_cast<int*>(mine->ptr);
+    const size_t bytes = (need_bytes + (need_bytes >> 2) + ((1u << 20) - 1)) >> 20 << 20;      // a quarter spare, whole MiB
+    void* ptr = nullptr;
+    if (cudaMalloc(&ptr, bytes) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    // the old buffer stays allocated: launches that read it may still be queued
+    if (mine) { mine->ptr = static_cast<uint8_t*>(ptr); mine->bytes = bytes; }
+    else buffers.push_back(Buffer{dev, st, static_cast<uint8_t*>(ptr), bytes});
+    return static_cast<int*>(ptr);
 }
 
-// Workspace of ue5m3_gemm_static: a file-scope device array instead of allocated memory.  A call needs 16 bytes plus
-// one byte per scale row of the two operands; the array holds kNativeWorkspaceSlotBytes, and a call that needs more is
-// refused.  Its address is asked for once per device; nothing is allocated, here or later.  All calls on a device
-// share the array: the first word is cleared and every row byte written by every call before its GEMM kernels run,
-// so two calls may follow one another on a stream, but two calls in flight at the same time (different streams) would
-// read each other's windows.
-static __device__ __align__(256) unsigned char g_static_workspace[kNativeWorkspaceSlotBytes];
+// Workspace of ue5m3_gemm_static: a file-scope device array instead of allocated memory.  A call needs what
+// native_layout() says (16 bytes, a byte per scale row, and one byte per operand row and 16 K for the re-ordered
+// scales, rows padded to whole tiles); the array holds kStaticWorkspaceBytes, and a call that needs more is refused.
+// Its address is asked for once per device; nothing is allocated, here or later.  All calls on a device share the
+// array: every byte a call's GEMM kernels read is written by that call's preparing kernel before they run (and the
+// first word cleared), so two calls may follow one another on a stream, but two calls in flight at the same time
+// (different streams) would read each other's scales.
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
 
 int* static_workspace(size_t need_bytes) {
-    if (need_bytes > kNativeWorkspaceSlotBytes) return nullptr;
+    if (need_bytes > kStaticWorkspaceBytes) return nullptr;
     static int* addr[64];
     static std::once_flag asked[64];
     int dev = 0;
@@ -699,14 +635,32 @@ int* static_workspace(size_t need_bytes) {
     return addr[dev];
 }
 
-int launch_scale_range(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st) {
+int launch_scale_prepare(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st) {
     (void)num_sms;
-    const int64_t ra = native_scale_rows(g.Mo, g.a_scale_mode), rb = native_scale_rows(g.No, g.b_scale_mode);
+    if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
+    const NativeLayout l = native_layout(g);
     if (cudaMemsetAsync(workspace, 0, sizeof(int), st) != cudaSuccess) return UE5M3_ERR_CUDA;
-    const int64_t grid = (ra + rb + 15) / 16;                     // 16 warps per CTA, one row each
-    scale_range_kernel<<<(unsigned)grid, 512, 0, st>>>(g.a_scales, ra, g.a_scale_mode == UE5M3_SCALE_1D_TILED ? 1 : 0,
-                                                       g.b_scales, rb, g.b_scale_mode == UE5M3_SCALE_1D_TILED ? 1 : 0,
-                                                       g.Kc / 16, workspace);
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+    PrepareParams q;
+    q.src[0] = g.a_scales; q.src[1] = g.b_scales;
+    q.rows[0] = g.Mo; q.rows[1] = g.No;
+    q.mode[0] = g.a_scale_mode; q.mode[1] = g.b_scale_mode;
+    q.groups_a = l.groups_a;
+    q.kblocks = g.Kc / 16;
+    q.workspace = workspace;
+    q.k_rows[0] = ws + l.k_a; q.k_rows[1] = ws + l.k_b;
+    q.sf[0] = ws + l.sf_a; q.sf[1] = ws + l.sf_b;
+    static std::once_flag asked[64];
+    static bool attr_ok[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return UE5M3_ERR_CUDA;
+    std::call_once(asked[dev], [&]() {
+        attr_ok[dev] = cudaFuncSetAttribute(scale_prepare_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepSmemBytes) == cudaSuccess;
+    });
+    if (!attr_ok[dev]) return UE5M3_ERR_CUDA;
+    const int64_t cblocks = q.kblocks < kPrepChunkBlocks ? q.kblocks : kPrepChunkBlocks;
+    const size_t smem = 128 * (size_t)(cblocks + 4);
+    scale_prepare_kernel<<<(unsigned)(l.groups_a + 2 * l.tiles_n), 512, smem, st>>>(q);
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
@@ -739,10 +693,13 @@ int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cud
     NativeParams p;
     p.Mo = g.Mo; p.No = g.No; p.Kc = g.Kc;
     p.a_decode = g.a_decode; p.b_decode = g.b_decode;
+    const NativeLayout l = native_layout(g);
+    const uint8_t* ws = reinterpret_cast<const uint8_t*>(workspace);
     p.workspace = workspace;
-    p.ka_rows = reinterpret_cast<const uint8_t*>(workspace) + 16;
-    p.kb_rows = p.ka_rows + ((native_scale_rows(g.Mo, g.a_scale_mode) + 15) / 16) * 16;
-    p.a_scales = g.a_scales; p.b_scales = g.b_scales;
+    p.ka_rows = ws + l.k_a;
+    p.kb_rows = ws + l.k_b;
+    p.sfa = ws + l.sf_a;
+    p.sfb = ws + l.sf_b;
     p.out_bf16 = g.out_dtype == UE5M3_BF16 ? 1 : 0;
     p.a_mode = g.a_scale_mode; p.b_mode = g.b_scale_mode;
     p.tiles_m = (int)((g.Mo + 2 * BM - 1) / (2 * BM));

@@ -60,18 +60,33 @@ cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t
 int launch_gemm(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st);
 int read_and_clear_device_status();                                  // synchronises the device
 // The same product on the tensor core's FP4 path (gemm_native.cu).  `workspace` is device memory of
-// native_workspace_bytes(g) bytes (layout in window.cuh): launch_scale_range fills it, the native kernel reads it and does
+// native_layout(g).bytes bytes (layout in window.cuh): launch_scale_prepare fills it, the native kernel reads it and does
 // nothing when some scale row has no window, and the FP16 kernel (launch_gemm with the same workspace) then does the product.
 inline int64_t native_scale_rows(int64_t R, int mode) { return mode == 2 /* UE5M3_SCALE_2D */ ? R / 16 : R; }
-inline size_t native_workspace_bytes(const GemmArgs& g) {
+struct NativeLayout {
+    size_t k_a, k_b;              // byte offsets of the rows' shifts
+    size_t sf_a, sf_b;            // ... of the shifted scales in the tensor core's order
+    size_t bytes;
+    int groups_a, tiles_n;        // 128-row groups of A, 256-row tiles of B
+};
+inline NativeLayout native_layout(const GemmArgs& g) {
     const int64_t ra = native_scale_rows(g.Mo, g.a_scale_mode), rb = native_scale_rows(g.No, g.b_scale_mode);
-    return (size_t)(16 + ((ra + 15) / 16) * 16 + ((rb + 15) / 16) * 16);
+    const int64_t stages = g.Kc / 256;
+    NativeLayout l;
+    l.groups_a = (int)(2 * ((g.Mo + 255) / 256));
+    l.tiles_n = (int)((g.No + 255) / 256);
+    l.k_a = 16;
+    l.k_b = l.k_a + (size_t)((ra + 15) / 16) * 16;
+    l.sf_a = (l.k_b + (size_t)((rb + 15) / 16) * 16 + 127) / 128 * 128;
+    l.sf_b = l.sf_a + (size_t)l.groups_a * (size_t)stages * 2048;
+    l.bytes = l.sf_b + (size_t)l.tiles_n * (size_t)stages * 4096;
+    return l;
 }
-constexpr size_t kNativeWorkspaceSlotBytes = 64 * 1024;             // largest workspace the library's own rings hold
-bool native_eligible(const GemmArgs& g);                             // Kc % 256 == 0 and the workspace fits a ring slot
-int* native_workspace(size_t need_bytes);                            // a slot of the per-device ring; null on failure
+constexpr size_t kStaticWorkspaceBytes = 16u << 20;                  // the file-scope array of ue5m3_gemm_static
+inline bool native_eligible(const GemmArgs& g) { return g.Kc % 256 == 0; }
+int* native_workspace(size_t need_bytes, cudaStream_t st);           // this stream's buffer, grown when needed; null on failure
 int* static_workspace(size_t need_bytes);                            // file-scope device array; null if the need exceeds it
-int launch_scale_range(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st);
+int launch_scale_prepare(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st);
 int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st);
 int read_and_clear_native_status();                                  // synchronises the device
 // The same operands under the output model of Section 6.2 (gemm_probe.cu).

@@ -275,3 +275,23 @@ def test_every_row_has_its_own_window():
         y, sa = oracle.gemm(ap, asc, modes[0] == 2, 2.0 ** -8, bp, bsc, modes[1] == 2, np.float32(2.0 ** -8))
         check_gemm_output(out, y, sa)
         assert torch.equal(lib.gemm(lib.FPROP, qa, qb, torch.float32), out)      # ue5m3_gemm takes the same kernel
+
+
+@pytest.mark.parametrize("modes", [(0, 1), (1, 2), (2, 0)])
+def test_rows_longer_than_the_preparing_kernels_shared_memory(modes):
+    """Kc = 28,672: 1,792 scale bytes per row, more than the kernel that finds the windows and re-orders the scales keeps in
+    shared memory at once (1,536), so it reads the rows in two chunks (96 + 16 stages) and twice.  The windows differ from
+    row to row and are decided by codes in the second chunk."""
+    Mo, No, Kc = 256, 128, 28672
+    rng = np.random.default_rng(911 + modes[0])
+    sa = rng.integers(0x60, 0x7F, (Mo // 16 if modes[0] == 2 else Mo, Kc // 16), dtype=np.uint8)
+    sb = rng.integers(0x60, 0x7F, (No // 16 if modes[1] == 2 else No, Kc // 16), dtype=np.uint8)
+    sa[1::3, -5] = 0xC8                                # k = 10 for these rows, from a code in the last stages
+    sb[::2, 1700] = 0x0B                               # k = 0
+    qa, ap, asc = _operand(rng, Mo, Kc, modes[0], 0, 0, dec=0.5, scales=sa)
+    qb, bp, bsc = _operand(rng, No, Kc, modes[1], 0, 0, dec=2.0, scales=sb)
+    out, ok, ka, kb = _native(qa, qb, torch.float32, Mo, No)
+    assert ok and list(ka) == _row_k(asc) and list(kb) == _row_k(bsc)
+    assert {10, 2} <= set(ka.tolist()) and {0, 2} <= set(kb.tolist())
+    y, sabs = oracle.gemm(ap, asc, modes[0] == 2, 0.5, bp, bsc, modes[1] == 2, 2.0)
+    check_gemm_output(out, y, sabs)

@@ -53,15 +53,17 @@ def test_static_workspace_gemm_checks_arguments_like_gemm():
     assert torch.equal(lib.gemm_static(lib.FPROP, a, b, torch.float32), lib.gemm(lib.FPROP, a, b, torch.float32))
 
 
-def test_static_workspace_gemm_refuses_operands_with_more_scale_rows_than_the_array_holds():
-    """65,536 bytes hold 16 + one byte per scale row (each operand's rows padded to a multiple of 16): 65,408 + 128 rows need
-    65,552.  The call is refused before anything is launched; ue5m3_gemm takes the same operands (on its FP16 kernel)."""
-    Ra, Rb, Kc = 65408, 128, 256
+def test_static_workspace_gemm_refuses_operands_larger_than_the_array_holds():
+    """The array holds 16 MiB; a call needs 16 bytes, a byte per scale row and a byte per 16 operand elements (rows padded to
+    256): 65,280 + 256 rows of Kc = 4096 need 16,777,216 bytes for the scales alone.  The call is refused before anything is
+    launched; ue5m3_gemm takes the same operands."""
+    Ra, Rb, Kc = 65280, 256, 4096
     one = torch.ones(1, dtype=torch.float32, device=DEV)
     def zeros_operand(R):
         return lib.QuantizedOperand(torch.zeros((R, Kc // 2), dtype=torch.uint8, device=DEV),
                                     torch.full((R, Kc // 16), 0x78, dtype=torch.uint8, device=DEV), one, lib.SCALE_1D)
     a, b = zeros_operand(Ra), zeros_operand(Rb)
+    assert lib.gemm_native_workspace(a, b).numel() > 16 << 20
     out = torch.full((Ra, Rb), 7.0, dtype=torch.bfloat16, device=DEV)
     with pytest.raises(lib.Ue5m3Error):
         lib.gemm_static(lib.FPROP, a, b, out=out)
@@ -70,8 +72,9 @@ def test_static_workspace_gemm_refuses_operands_with_more_scale_rows_than_the_ar
     lib.gemm(lib.FPROP, a, b, out=out)
     torch.cuda.synchronize()
     assert lib.last_device_status() == 0 and bool((out == 0.0).all())
-    # one row block fewer fits: 65,280 + 128 rows need 65,424 bytes
-    a2 = zeros_operand(Ra - 128)
+    # one row tile fewer fits: 65,024 + 256 rows need 16,777,088 bytes
+    a2 = zeros_operand(Ra - 256)
+    assert lib.gemm_native_workspace(a2, b).numel() == 16777088
     out2 = lib.gemm_static(lib.FPROP, a2, b, torch.bfloat16)
     torch.cuda.synchronize()
     assert bool((out2 == 0.0).all())
