@@ -116,7 +116,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
             const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
-    if (p.range && native_all_rows_have_windows(p.range)) return;      // uniform over the grid
+    if (p.range) {
+        // Launched as a programmatic dependent of the native kernel, i.e. possibly while that kernel is still at work; the
+        // workspace was complete before it started.  Uniform over the grid: nothing to do when the native kernel does the
+        // product, and otherwise (it has returned at once) wait until it is gone for good.
+        if (native_all_rows_have_windows(p.range)) return;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -515,8 +521,18 @@ int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t s
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int max_pairs = resident_pairs[dev];
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
-    gemm_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(ma, mb, mas, mbs, mo, p);
-    return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    // behind the native kernel: launched while that kernel runs, so that a launch with nothing to do costs nothing
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = range ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gemm_kernel, ma, mb, mas, mbs, mo, p) == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
 int read_and_clear_device_status() {

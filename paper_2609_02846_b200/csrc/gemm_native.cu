@@ -64,7 +64,7 @@ constexpr int KCHUNK = 256;                 // K per stage
 constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks)
 constexpr int MMAS = KCHUNK / KMMA;
 constexpr int STAGES = 5;                   // stages of payload and scales
-constexpr int SF_SLOTS = 2;                 // stages whose scales have room in tensor memory
+constexpr int SF_SLOTS = 1;                 // stages whose scales have room in tensor memory
 constexpr int EPI_WARP0 = 4;
 constexpr int NUM_THREADS = 256;
 
@@ -321,6 +321,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     // Everything above touched only this CTA pair's shared and tensor memory and may have run while the range kernel was
     // still at work (programmatic dependent launch); the workspace it fills is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // the FP16 kernel queued behind this one may be launched from here on: it reads the same word and returns
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const bool work = native_all_rows_have_windows(p.workspace);      // uniform over the grid; false: the FP16 kernel does this product
 
     if (!work) {
