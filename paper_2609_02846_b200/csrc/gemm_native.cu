@@ -13,32 +13,34 @@
 // the tensor core as the copy engine delivered it: no conversion, no second staging.  The shifted scale bytes (three
 // integer operations per four codes) take their own route into tensor memory, in the layout the block-scaled MMA reads.
 //
-// The windows are found on the device: scale_range_kernel gives each scale row of both operands to one warp, which
-// reduces the row's codes to the largest and the smallest non-zero one and writes the row's k (one byte) into the
-// workspace, or sets the workspace's first word when the row has no window (subnormal UE5M3 codes included).
-// gemm_native_kernel reads that word and returns at once when it is set; the caller then runs the FP16 path, whose
-// kernel evaluates the same predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.  Where a
-// row allows it k is 2, so that the rows of ordinary data share one shift and the epilogue takes its uniform path.
+// The windows are found on the device: scale_prepare_kernel gives each group of 128 operand rows to one CTA, which
+// reduces every scale row's codes to the largest and the smallest non-zero one, writes the row's k (one byte) into the
+// workspace, or sets the workspace's first word when the row has no window (subnormal UE5M3 codes included), and
+// writes the group's codes, shifted, in the order the tensor core's scale copy reads them.  gemm_native_kernel reads
+// that word and returns at once when it is set; the caller then runs the FP16 path, whose kernel evaluates the same
+// predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.  Where a row allows it k is 2, so
+// that the rows of ordinary data share one shift and the epilogue takes its uniform path.
 //
-// Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 5 payload stages of 32 KB):
-//   warp 0      copies: packed A rows (128) and packed B rows (this CTA's 128) of a stage
-//   warp 1      (leader CTA) MMA issuer: 4 MMAs of K = 64 and one commit per stage
-//   warp 2      tensor-memory allocation; relay: tells the leader CTA that this CTA's copy of a stage has landed
-//   warp 3      (leader CTA) scale copier: 12 tcgen05.cp per stage, shared memory -> tensor memory of both CTAs
+// Roles per CTA of a pair (cta_group::2, tile 256 x 256, 256 K per stage, 5 stages of 38 KB):
+//   warp 0      copies: packed A rows (128) and packed B rows (this CTA's 128) of a stage as tensor copies, the stage's
+//               prepared scales (2 KB for A's 128 rows, 4 KB for B's 256) as two plain bulk copies, all on one barrier
+//   warp 1      (leader CTA) issuer: per MMA of K = 64 three scale copies shared memory -> tensor memory of both CTAs
+//               (tcgen05.cp) and the MMA; one commit per stage.  Copies and MMAs run in issue order, so one scale
+//               slot in tensor memory is enough.
+//   warp 2      tensor-memory allocation; relay: tells the leader CTA that this CTA's copies of a stage have landed
 //   warps 4-7   epilogue: accumulator -> alpha and the row's and column's window factors -> BF16 / FP32 -> shared
 //               memory -> bulk tensor store
-//   warps 8-15  scale bytes, two groups of four warps taking the stages in turn: read from global memory four stages
-//               ahead (registers), each row's window shift, stored in the order the scale copy wants into a ring of six stages
-//               in shared memory
-// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 64..319, four
-// stages of scales in columns 320..511.  Two whole accumulators do not fit beside the scales, so the two overlap in
-// 192 columns: the epilogue drains those first and hands them back, and the MMAs of the next tile run while the
-// last 64 columns are still being stored.
-// The two issuing warps run their loops warp-uniformly and let one elected lane issue: the operands of the tensor
+// (warp 3 idles.)
+// Tensor memory: the accumulators of even tiles sit in columns 0..255, those of odd tiles in columns 192..447, the
+// scales in columns 448..495.  Two whole accumulators do not fit beside the scales, so the two overlap in 64 columns:
+// the epilogue drains those first and hands them back, and the MMAs of the next tile run while the other 192 columns
+// are still being stored.
+// The issuing warp runs its loop warp-uniformly and lets one elected lane issue: the operands of the tensor
 // instructions are then uniform-register values.  Issued from a single lane's registers an instruction costs 50-80
-// clocks (measured into an idle pipe: 12 scale copies 578 clocks, 4 MMAs 258; with uniform operands 4 MMAs 82), and an
-// earlier version in which one such lane issued copies and MMAs spent 950 clocks per stage issuing, against 512
-// clocks of MMA work.
+// clocks (measured into an idle pipe: 12 scale copies 578 clocks, 4 MMAs 258; with uniform operands 4 MMAs 82).
+// An earlier version shifted and re-ordered the scale bytes inside this kernel (eight warps loading them from global
+// memory, a ring in shared memory, a second issuing warp for the copies): that path shared the shared-memory / L1 unit
+// with the copy engine's feed, which bounds the kernel, and cost 20-35 % of its time.
 // Every wait is bounded (SM clocks); on a time-out the role sets the status word, the other roles see the abort
 // flag, in-flight copies and MMAs are drained and the kernel returns.
 #include <cuda.h>

@@ -24,10 +24,12 @@ __device__ __forceinline__ bool pick_window(int cmax, int inv_min, int& k) {
     return true;
 }
 
-// Workspace of one ue5m3_gemm call on the native path:
+// Workspace of one ue5m3_gemm call on the native path (offsets by native_layout() in launch.h):
 //   word 0          0 when every scale row of both operands has a window, non-zero otherwise (the FP16 kernel then works)
 //   bytes 16 ...    the shift k of every scale row of A (one byte per row; rows of a 2D operand are its 16-row groups),
 //                   padded to a multiple of 16; then the same for B
+//   then, 128-byte aligned, the scale codes shifted by 8 k in the order the tensor core's scale copy reads them: for
+//   every 128-row group of A and stage of 256 K 2048 bytes, for every 256-row tile of B and stage 4096 bytes
 __device__ __forceinline__ bool native_all_rows_have_windows(const int* workspace) { return *workspace == 0; }
 
 }  // namespace ue5m3
