@@ -295,3 +295,56 @@ def test_rows_longer_than_the_preparing_kernels_shared_memory(modes):
     assert {10, 2} <= set(ka.tolist()) and {0, 2} <= set(kb.tolist())
     y, sabs = oracle.gemm(ap, asc, modes[0] == 2, 0.5, bp, bsc, modes[1] == 2, 2.0)
     check_gemm_output(out, y, sabs)
+
+
+def test_calls_on_two_streams_have_their_own_workspaces():
+    """ue5m3_gemm keeps one workspace per stream: products of different shapes queued on two streams without an ordering
+    between them (so that they may overlap) equal the same products computed one after the other."""
+    rng = np.random.default_rng(4242)
+    cases = []
+    for (Mo, No, Kc, ma, mb) in [(1024, 768, 2048, 0, 2), (512, 1280, 1024, 1, 1)]:
+        qa, _, _ = _operand(rng, Mo, Kc, ma, 0x50, 0x90, dec=0.5)
+        qb, _, _ = _operand(rng, No, Kc, mb, 0x48, 0x88, dec=0.25)
+        cases.append((qa, qb, lib.gemm(lib.FPROP, qa, qb, torch.float32)))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[], []]
+    for rep in range(6):
+        for i, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                qa, qb, _ = cases[i]
+                outs[i].append(lib.gemm(lib.FPROP, qa, qb, torch.float32))
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    for i in range(2):
+        for o in outs[i]:
+            assert torch.equal(o, cases[i][2])
+
+
+def test_gemm_replays_from_a_cuda_graph():
+    """After one call on the stream (which sizes the stream's workspace) the three launches of ue5m3_gemm, the two
+    programmatic dependencies between them included, can be captured and replayed; new operand contents in the same
+    buffers are picked up, a window that disappears too."""
+    Mo, No, Kc = 512, 768, 1024
+    rng = np.random.default_rng(515)
+    qa, ap, asc = _operand(rng, Mo, Kc, 0, 0x50, 0x90, dec=0.5)
+    qb, bp, bsc = _operand(rng, No, Kc, 2, 0x50, 0x90, dec=0.25)
+    out = torch.zeros((Mo, No), dtype=torch.float32, device=DEV)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        lib.gemm(lib.FPROP, qa, qb, out=out)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            lib.gemm(lib.FPROP, qa, qb, out=out)
+        for trial in range(3):
+            asc2 = rng.integers(0x50, 0x90, asc.shape, dtype=np.uint8)
+            if trial == 2:
+                asc2[5, 7] = 0x03                     # a subnormal code: no window, the FP16 kernel must do this replay
+            qa.scales.copy_(torch.from_numpy(asc2).to(DEV))
+            out.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            assert lib.last_device_status() == 0
+            y, sabs = oracle.gemm(ap, asc2, False, 0.5, bp, bsc, True, 0.25)
+            check_gemm_output(out, y, sabs)
