@@ -88,6 +88,7 @@ static_assert(STAGE_BYTES % 1024 == 0, "payload stages must stay 1024-byte align
 constexpr int TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
 constexpr int OVERLAP_UNITS = (SF_SLOTS * TMEM_SF_SLOT_COLS + 31) / 32;       // 32-column units the two accumulators share
 constexpr int TMEM_ACC_ODD = 256 - 32 * OVERLAP_UNITS;
+static_assert(OVERLAP_UNITS % 2 == 0, "the BF16 epilogue hands the shared columns back in chunks of two units");
 constexpr int TMEM_SF_COL = TMEM_ACC_ODD + 256;
 
 struct NativeParams {
@@ -489,13 +490,22 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     const int cc = odd ? i : 3 - i;                                  // chunk of 64 columns, shared ones first
                     uint8_t* mine = stage_gen + lane * 128;
                     const int sw = lane & 7;
+                    // both units of the chunk are on their way before either is looked at: the hand-back below then comes one
+                    // load latency and one conversion earlier
+                    uint32_t r[2][32];
+                    tmem_ld32(acc + cc * 64, r[0]);
+                    tmem_ld32(acc + cc * 64 + 32, r[1]);
+                    tmem_ld_wait();
+                    if (2 * i + 1 == OVERLAP_UNITS - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
+                    }
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        const int half = odd ? hh : hh ^ 1;                           // inside a chunk too: the shared unit first
-                        uint32_t r[32];
+                    for (int half = 0; half < 2; ++half) {
                         const int unit = cc * 2 + half;
-                        tmem_ld32(acc + unit * 32, r);
-                        tmem_ld_wait();
                         // the column factors: one for all 32 columns (the usual case, folded into the row's factor), or each
                         // applied to its accumulator first -- powers of two, so nothing is rounded before the product with alpha
                         float au = unit_factor(unit);
@@ -504,24 +514,15 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                             col_shifts(col0 + unit * 32, ks);
                             au = alpha;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * colf(ks, j));
-                        }
-                        if (2 * i + hh == OVERLAP_UNITS - 1) {
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive_cluster(acc_empty, 0);
-                        }
-                        if (hh == 0) {
-                            if (lane == 0) tma_store_wait_read<0>();
-                            __syncwarp();
+                            for (int j = 0; j < 32; ++j) r[half][j] = __float_as_uint(__uint_as_float(r[half][j]) * colf(ks, j));
                         }
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {
                             uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * au, __uint_as_float(r[8 * v + 1]) * au);
-                            o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * au, __uint_as_float(r[8 * v + 3]) * au);
-                            o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * au, __uint_as_float(r[8 * v + 5]) * au);
-                            o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * au, __uint_as_float(r[8 * v + 7]) * au);
+                            o.x = pack_bf16x2(__uint_as_float(r[half][8 * v + 0]) * au, __uint_as_float(r[half][8 * v + 1]) * au);
+                            o.y = pack_bf16x2(__uint_as_float(r[half][8 * v + 2]) * au, __uint_as_float(r[half][8 * v + 3]) * au);
+                            o.z = pack_bf16x2(__uint_as_float(r[half][8 * v + 4]) * au, __uint_as_float(r[half][8 * v + 5]) * au);
+                            o.w = pack_bf16x2(__uint_as_float(r[half][8 * v + 6]) * au, __uint_as_float(r[half][8 * v + 7]) * au);
                             *reinterpret_cast<uint4*>(mine + (((half * 4 + v) ^ sw) << 4)) = o;
                         }
                     }
