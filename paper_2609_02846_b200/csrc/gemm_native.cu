@@ -62,11 +62,13 @@ namespace {
 constexpr int BM = 128;                     // A rows per CTA (256 per pair)
 constexpr int BN = 256;                     // output columns per tile
 constexpr int BNH = 128;                    // B rows staged by each CTA
-constexpr int KCHUNK = 256;                 // K per stage
+constexpr int KCHUNK = 256;                 // K per stage: rows of 128 bytes, 128-byte swizzle.  128 (rows of 64 bytes, 64-byte
+                                            // swizzle, 11 stages of 19 KB) also works and keeps more bytes in flight, but the copy
+                                            // engine delivers 64-byte rows at half the rate: 300 us per call against 200
 constexpr int KMMA = 64;                    // K per MMA (four 16-element blocks)
 constexpr int MMAS = KCHUNK / KMMA;
-constexpr int STAGES = 5;                   // stages of payload and scales
-constexpr int SF_SLOTS = 1;                 // stages whose scales have room in tensor memory
+constexpr int STAGES = KCHUNK == 128 ? 11 : 5;     // stages of payload and scales
+constexpr int ROW_BYTES = KCHUNK / 2;        // a payload row of a stage
 constexpr int EPI_WARP0 = 4;
 constexpr int NUM_THREADS = 256;
 
@@ -85,7 +87,8 @@ static_assert(STAGE_BYTES % 1024 == 0, "payload stages must stay 1024-byte align
 // 32 * OVERLAP_UNITS columns), then SF_SLOTS scale slots of 48 columns: 16 for A (column 4 j + g: rows 32 g + lane, MMA j)
 // and 32 for B (column 8 j + 4 h + g).  Scale copies and MMAs are issued by one thread and run in issue order, so a
 // slot may be written again as soon as the MMAs that read it have been issued.
-constexpr int TMEM_SF_SLOT_COLS = 48, TMEM_SFB_OFF = 16;
+constexpr int TMEM_SF_SLOT_COLS = 12 * MMAS, TMEM_SFB_OFF = 4 * MMAS;
+constexpr int SF_SLOTS = 48 / TMEM_SF_SLOT_COLS;       // stages whose scales have room in tensor memory (used in turn)
 constexpr int OVERLAP_UNITS = (SF_SLOTS * TMEM_SF_SLOT_COLS + 31) / 32;       // 32-column units the two accumulators share
 constexpr int TMEM_ACC_ODD = 256 - 32 * OVERLAP_UNITS;
 static_assert(OVERLAP_UNITS % 2 == 0, "the BF16 epilogue hands the shared columns back in chunks of two units");
@@ -142,6 +145,17 @@ __device__ __forceinline__ void umma_fp4_block16(uint32_t tmem_d, uint32_t alo, 
 __device__ __forceinline__ void tmem_cp_32x128b(uint32_t taddr, uint32_t lo, uint32_t hi) {
     asm volatile("{\n\t.reg .b64 d;\n\tmov.b64 d, {%1, %2};\n\ttcgen05.cp.cta_group::2.32x128b.warpx4 [%0], d;\n\t}"
                  ::"r"(taddr), "r"(lo), "r"(hi) : "memory");
+}
+// Descriptor of a K-major packed-FP4 tile whose rows are ROW_BYTES long, swizzled over its own row length: 8-row groups
+// are 8 * ROW_BYTES apart.
+__device__ __forceinline__ uint64_t payload_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                                        // leading byte offset (ignored for swizzled K-major)
+    d |= (uint64_t)((8 * ROW_BYTES) >> 4) << 32;                   // stride byte offset
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)(ROW_BYTES == 128 ? 2 : 4) << 61;               // 128-byte / 64-byte swizzle
+    return d;
 }
 // Descriptor of 32 rows of 16 bytes stored back to back: no swizzle, 8-row groups 128 bytes apart.
 __device__ __forceinline__ uint64_t sf_smem_desc(uint32_t saddr) {
@@ -288,10 +302,11 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t bar_base = smem_base + SMEM_BARS;
     // barriers (8 bytes each)
-    const uint32_t pk_full = bar_base, pk_empty = bar_base + 64, pk_ready = bar_base + 128;
-    const uint32_t acc_full = bar_base + 320, acc_empty = bar_base + 328, drain_bar = bar_base + 336;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 344);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 352);
+    const uint32_t pk_full = bar_base, pk_empty = bar_base + 128, pk_ready = bar_base + 256;
+    const uint32_t acc_full = bar_base + 384, acc_empty = bar_base + 392, drain_bar = bar_base + 400;
+    static_assert(STAGES <= 16, "room for 16 barriers per array");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BARS + 408);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + SMEM_BARS + 416);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();
@@ -377,7 +392,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             const bool elected = elect_one();
             // descriptor halves of the payload stages (128-byte swizzle) and of the scale pieces (no swizzle); only the
             // start address moves
-            const uint64_t d_pk = umma_smem_desc(smem_base), d_sf = sf_smem_desc(smem_base + SF_OFF);
+            const uint64_t d_pk = payload_smem_desc(smem_base), d_sf = sf_smem_desc(smem_base + SF_OFF);
             const uint32_t pk_lo0 = (uint32_t)d_pk, pk_hi = (uint32_t)(d_pk >> 32);
             const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
             const uint32_t tm0 = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
@@ -578,6 +593,19 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     }
 }
 
+// Packed payload [rows, row_bytes]: boxes of box_rows rows x ROW_BYTES, swizzled over the box row.
+bool make_payload_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {ROW_BYTES, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              ROW_BYTES == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_out_map(CUtensorMap* m, void* out, bool bf16, int64_t Mo, int64_t No, int64_t ldo) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
@@ -691,8 +719,8 @@ int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cud
     if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
     CUtensorMap ma, mb, mo;
     const uint64_t row_bytes = (uint64_t)(g.Kc / 2);
-    if (!make_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, row_bytes, KCHUNK / 2, BM, true)) return UE5M3_ERR_CUDA;
-    if (!make_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, row_bytes, KCHUNK / 2, BNH, true)) return UE5M3_ERR_CUDA;
+    if (!make_payload_map(&ma, g.a_payload, row_bytes, (uint64_t)g.Mo, BM)) return UE5M3_ERR_CUDA;
+    if (!make_payload_map(&mb, g.b_payload, row_bytes, (uint64_t)g.No, BNH)) return UE5M3_ERR_CUDA;
     if (!make_out_map(&mo, g.out, g.out_dtype == UE5M3_BF16, g.Mo, g.No, g.ldo)) return UE5M3_ERR_CUDA;
 
     NativeParams p;
