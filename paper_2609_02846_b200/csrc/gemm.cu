@@ -118,10 +118,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
     if (p.range) {
         // Launched as a programmatic dependent of the native kernel, i.e. possibly while that kernel is still at work; the
-        // workspace was complete before it started.  Uniform over the grid: nothing to do when the native kernel does the
-        // product, and otherwise (it has returned at once) wait until it is gone for good.
-        if (native_all_rows_have_windows(p.range)) return;
+        // workspace was complete before it started.  Either way this grid ends only after the native kernel has: what
+        // follows on the stream is then ordered behind both by construction.  Uniform over the grid: nothing else to do
+        // when the native kernel does the product.
+        const bool native_works = native_all_rows_have_windows(p.range);
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (native_works) return;
     }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
