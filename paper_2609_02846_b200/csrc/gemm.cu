@@ -88,7 +88,8 @@ struct GemmParams {
     const uint8_t* a_scales;
     const uint8_t* b_scales;
     int a_direct, b_direct;
-    const int* range;             // not null: the native FP4 kernel ran first; this one works only if it could not
+    const uint8_t* flags;         // not null: the native FP4 kernel was launched first; this one works only if that one does not
+    int n_flags;                  // (one byte per 128-row group of the operands, layout in window.cuh)
 };
 
 // Tile order: groups of kRasterGroup tile rows, and inside a group column by column.  The tiles that are
@@ -116,12 +117,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_as, const __grid_constant__ CUtensorMap map_bs,
             const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
-    if (p.range) {
+    if (p.flags) {
         // Launched as a programmatic dependent of the native kernel, i.e. possibly while that kernel is still at work; the
         // workspace was complete before it started.  Either way this grid ends only after the native kernel has: what
         // follows on the stream is then ordered behind both by construction.  Uniform over the grid: nothing else to do
         // when the native kernel does the product.
-        const bool native_works = native_all_rows_have_windows(p.range);
+        const bool native_works = native_all_rows_have_windows(p.flags, p.n_flags);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if (native_works) return;
     }
@@ -519,7 +520,12 @@ int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t s
     p.stall_producer = g.stall_producer;
     p.a_scales = g.a_scales; p.b_scales = g.b_scales;
     p.a_direct = a_direct ? 1 : 0; p.b_direct = b_direct ? 1 : 0;
-    p.range = range;
+    p.flags = nullptr; p.n_flags = 0;
+    if (range) {
+        const NativeLayout l = native_layout(g);
+        p.flags = reinterpret_cast<const uint8_t*>(range) + l.flags;
+        p.n_flags = l.n_flags;
+    }
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int max_pairs = resident_pairs[dev];
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;

@@ -15,9 +15,9 @@
 //
 // The windows are found on the device: scale_prepare_kernel gives each group of 128 operand rows to one CTA, which
 // reduces every scale row's codes to the largest and the smallest non-zero one, writes the row's k (one byte) into the
-// workspace, or sets the workspace's first word when the row has no window (subnormal UE5M3 codes included), and
+// workspace, says in the group's flag byte whether a row has no window (subnormal UE5M3 codes included), and
 // writes the group's codes, shifted, in the order the tensor core's scale copy reads them.  gemm_native_kernel reads
-// that word and returns at once when it is set; the caller then runs the FP16 path, whose kernel evaluates the same
+// the flags and returns at once when one is set; the caller then runs the FP16 path, whose kernel evaluates the same
 // predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.  Where a row allows it k is 2, so
 // that the rows of ordinary data share one shift and the epilogue takes its uniform path.
 //
@@ -98,7 +98,9 @@ struct NativeParams {
     int64_t Mo, No, Kc;
     const float* a_decode;
     const float* b_decode;
-    const int* workspace;         // word 0: 0 when every scale row has a window (layout in window.cuh)
+    int* result;                  // word 0 of the workspace: written with 0 when every scale row has a window, 1 otherwise
+    const uint8_t* flags;         // one byte per 128-row group: a row of the group has no window (layout in window.cuh)
+    int n_flags;
     const uint8_t* ka_rows;       // shift k of every scale row of A
     const uint8_t* kb_rows;       // ... of B
     const uint8_t* sfa;           // shifted scales of A in the order the scale copy wants: [128-row group][stage][2048]
@@ -174,8 +176,8 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 
 // ----------------------------------------------------------------------------- windows and scale layout
 // One CTA per group of 128 operand rows (first A's groups, then B's).  First the window of every scale row of the
-// group: largest and smallest non-zero code -> shift k (a byte of the workspace, for the epilogue's factors), or the
-// workspace's first word set when a row has no window.  Then the group's scale bytes, shifted by 8 k, are written in
+// group: largest and smallest non-zero code -> shift k (a byte of the workspace, for the epilogue's factors), and the
+// group's flag byte: non-zero when a row has no window (written either way: no atomics, nothing to clear).  Then the group's scale bytes, shifted by 8 k, are written in
 // the order the tensor core's scale copy reads them: per stage of 256 K and MMA j, 32 pieces of 16 bytes, piece dp
 // holding the four block scales of MMA j for rows dp, 32 + dp, 64 + dp, 96 + dp.  A's groups lie one after the other
 // ([group][stage][j][dp]); B's two groups of a 256-row tile are interleaved per MMA ([tile][stage][j][half][dp]).
@@ -188,7 +190,7 @@ struct PrepareParams {
     int mode[2];
     int groups_a;                 // 128-row groups of A (2 per row of tiles)
     int64_t kblocks;              // Kc / 16
-    int* workspace;
+    uint8_t* flags;               // one byte per CTA of the grid
     uint8_t* k_rows[2];
     uint8_t* sf[2];
 };
@@ -257,14 +259,15 @@ __global__ void __launch_bounds__(512) scale_prepare_kernel(const PrepareParams 
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
         iv = max(iv, __shfl_xor_sync(0xFFFFFFFFu, iv, d));
     }
+    bool ok = true;
     if ((lane & 3) == 0 && i < nrows) {
         int k = 8;
-        const bool ok = !have_row || pick_window((int)m, (int)iv, k);
+        ok = !have_row || pick_window((int)m, (int)iv, k);
         shift8[i] = ok ? (uint32_t)(8 * k) * 0x01010101u : 0u;
         if (have_row) k_rows[srow] = (uint8_t)k;
-        if (!ok) atomicOr(q.workspace, 1);
     }
-    __syncthreads();
+    const int group_bad = __syncthreads_or(ok ? 0 : 1);          // also orders shift8 before the second part
+    if (threadIdx.x == 0) q.flags[blockIdx.x] = group_bad ? 1 : 0;
     // shifted bytes in the scale copy's order: thread -> one 16-byte piece (stage s, MMA j, lane dp), rows 32 g + dp
     uint8_t* out = is_b ? q.sf[1] + (int64_t)(group >> 1) * pieces * 4096 + (group & 1) * 512 : q.sf[0] + (int64_t)group * pieces * 2048;
     const int64_t stride_s = is_b ? 4096 : 2048, stride_j = is_b ? 1024 : 512;
@@ -341,7 +344,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // the FP16 kernel queued behind this one may be launched from here on: it reads the same word and returns
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const bool work = native_all_rows_have_windows(p.workspace);      // uniform over the grid; false: the FP16 kernel does this product
+    const bool work = native_all_rows_have_windows(p.flags, p.n_flags);      // uniform over the grid; false: the FP16 kernel does this product
+    if (blockIdx.x == 0 && threadIdx.x == 0) *p.result = work ? 0 : 1;
 
     if (!work) {
     } else if (warp == 0) {
@@ -649,8 +653,8 @@ int* native_workspace(size_t need_bytes, cudaStream_t st) {
 // native_layout() says (16 bytes, a byte per scale row, and one byte per operand row and 16 K for the re-ordered
 // scales, rows padded to whole tiles); the array holds kStaticWorkspaceBytes, and a call that needs more is refused.
 // Its address is asked for once per device; nothing is allocated, here or later.  All calls on a device share the
-// array: every byte a call's GEMM kernels read is written by that call's preparing kernel before they run (and the
-// first word cleared), so two calls may follow one another on a stream, but two calls in flight at the same time
+// array: every byte a call's GEMM kernels read is written by that call's preparing kernel before they run -- nothing
+// has to start at zero --, so two calls may follow one another on a stream, but two calls in flight at the same time
 // (different streams) would read each other's scales.
 static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
 
@@ -672,7 +676,6 @@ int launch_scale_prepare(const GemmArgs& g, int* workspace, int num_sms, cudaStr
     (void)num_sms;
     if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
     const NativeLayout l = native_layout(g);
-    if (cudaMemsetAsync(workspace, 0, sizeof(int), st) != cudaSuccess) return UE5M3_ERR_CUDA;
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
     PrepareParams q;
     q.src[0] = g.a_scales; q.src[1] = g.b_scales;
@@ -680,7 +683,7 @@ int launch_scale_prepare(const GemmArgs& g, int* workspace, int num_sms, cudaStr
     q.mode[0] = g.a_scale_mode; q.mode[1] = g.b_scale_mode;
     q.groups_a = l.groups_a;
     q.kblocks = g.Kc / 16;
-    q.workspace = workspace;
+    q.flags = ws + l.flags;
     q.k_rows[0] = ws + l.k_a; q.k_rows[1] = ws + l.k_b;
     q.sf[0] = ws + l.sf_a; q.sf[1] = ws + l.sf_b;
     static std::once_flag asked[64];
@@ -697,7 +700,7 @@ int launch_scale_prepare(const GemmArgs& g, int* workspace, int num_sms, cudaStr
     return cudaGetLastError() == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 
-int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st) {
+int launch_gemm_native(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st) {
     static int resident_pairs[64];
     static std::once_flag asked[64];
     int dev = 0;
@@ -728,7 +731,9 @@ int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cud
     p.a_decode = g.a_decode; p.b_decode = g.b_decode;
     const NativeLayout l = native_layout(g);
     const uint8_t* ws = reinterpret_cast<const uint8_t*>(workspace);
-    p.workspace = workspace;
+    p.result = workspace;
+    p.flags = ws + l.flags;
+    p.n_flags = l.n_flags;
     p.ka_rows = ws + l.k_a;
     p.kb_rows = ws + l.k_b;
     p.sfa = ws + l.sf_a;

@@ -65,9 +65,11 @@ int read_and_clear_device_status();                                  // synchron
 inline int64_t native_scale_rows(int64_t R, int mode) { return mode == 2 /* UE5M3_SCALE_2D */ ? R / 16 : R; }
 struct NativeLayout {
     size_t k_a, k_b;              // byte offsets of the rows' shifts
+    size_t flags;                 // ... of one byte per 128-row group (A's groups, then B's): non-zero = a row without a window
     size_t sf_a, sf_b;            // ... of the shifted scales in the tensor core's order
     size_t bytes;
-    int groups_a, tiles_n;        // 128-row groups of A, 256-row tiles of B
+    int groups_a, tiles_n;        // 128-row groups of A, 256-row tiles of B (two groups each)
+    int n_flags;
 };
 inline NativeLayout native_layout(const GemmArgs& g) {
     const int64_t ra = native_scale_rows(g.Mo, g.a_scale_mode), rb = native_scale_rows(g.No, g.b_scale_mode);
@@ -77,7 +79,9 @@ inline NativeLayout native_layout(const GemmArgs& g) {
     l.tiles_n = (int)((g.No + 255) / 256);
     l.k_a = 16;
     l.k_b = l.k_a + (size_t)((ra + 15) / 16) * 16;
-    l.sf_a = (l.k_b + (size_t)((rb + 15) / 16) * 16 + 127) / 128 * 128;
+    l.flags = l.k_b + (size_t)((rb + 15) / 16) * 16;
+    l.n_flags = l.groups_a + 2 * l.tiles_n;
+    l.sf_a = (l.flags + (size_t)l.n_flags + 127) / 128 * 128;
     l.sf_b = l.sf_a + (size_t)l.groups_a * (size_t)stages * 2048;
     l.bytes = l.sf_b + (size_t)l.tiles_n * (size_t)stages * 4096;
     return l;
@@ -87,7 +91,7 @@ inline bool native_eligible(const GemmArgs& g) { return g.Kc % 256 == 0; }
 int* native_workspace(size_t need_bytes, cudaStream_t st);           // this stream's buffer, grown when needed; null on failure
 int* static_workspace(size_t need_bytes);                            // file-scope device array; null if the need exceeds it
 int launch_scale_prepare(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st);
-int launch_gemm_native(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st);
+int launch_gemm_native(const GemmArgs& g, int* workspace, int num_sms, cudaStream_t st);
 int read_and_clear_native_status();                                  // synchronises the device
 // The same operands under the output model of Section 6.2 (gemm_probe.cu).
 int launch_gemm_probe(const GemmArgs& g, int cross_rne, int grid_denominator, int num_sms, cudaStream_t st);

@@ -25,11 +25,19 @@ __device__ __forceinline__ bool pick_window(int cmax, int inv_min, int& k) {
 }
 
 // Workspace of one ue5m3_gemm call on the native path (offsets by native_layout() in launch.h):
-//   word 0          0 when every scale row of both operands has a window, non-zero otherwise (the FP16 kernel then works)
+//   word 0          written by the native kernel for the host: 0 when every scale row of both operands has a window
 //   bytes 16 ...    the shift k of every scale row of A (one byte per row; rows of a 2D operand are its 16-row groups),
 //                   padded to a multiple of 16; then the same for B
+//   then            one byte per 128-row group of A and then of B: non-zero when a row of the group has no window
 //   then, 128-byte aligned, the scale codes shifted by 8 k in the order the tensor core's scale copy reads them: for
 //   every 128-row group of A and stage of 256 K 2048 bytes, for every 256-row tile of B and stage 4096 bytes
-__device__ __forceinline__ bool native_all_rows_have_windows(const int* workspace) { return *workspace == 0; }
+// Every byte the GEMM kernels read is written by the preparing kernel of the same call: nothing has to be cleared.
+//
+// Called by every thread of a CTA (it contains a barrier); the same answer in every CTA of both GEMM kernels.
+__device__ __forceinline__ bool native_all_rows_have_windows(const uint8_t* group_flags, int n) {
+    int bad = 0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) bad |= group_flags[i];
+    return __syncthreads_or(bad) == 0;
+}
 
 }  // namespace ue5m3
