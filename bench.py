@@ -544,7 +544,7 @@ def run_ours(args):
                     "achieved_over_bf16_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
                     "achieved_over_fp4_nominal_9000": gemm_tflops / (NOMINAL_BF16_TFLOPS * NOMINAL_FP4_OVER_BF16),
                     "avg_launch_ms": gemm_ms,
-                    "avg_launch_ms_note": "one ue5m3_gemm call: with --gemm-path auto that is the range reduction, the kernel "
+                    "avg_launch_ms_note": "one ue5m3_gemm call: with --gemm-path auto that is the kernel that prepares the scales, the kernel "
                                           "that does the product and the other kernel's immediate return",
                     "avg_launch_ms_x_sm_mhz": None if not clocks.get("sm_mhz") else round(gemm_ms * clocks["sm_mhz"], 1),
                     "traffic": GEMM_DRAM_TRAFFIC_BYTES.get(kernel) if (M_TOK, K_IN, N_OUT) == (8192, 4096, 16384) else None,

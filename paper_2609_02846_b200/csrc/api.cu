@@ -325,7 +325,7 @@ int ue5m3_gemm_stall_selftest(int which, int64_t Mo, int64_t No, int64_t Kc, con
     g.wait_limit_cycles = wait_limit_cycles;
     g.stall_producer = 1;
     if (which == 2) {
-        // the native kernel: its workspace is filled by the range kernel as in ue5m3_gemm (the operands must have windows)
+        // the native kernel: its workspace is filled by the preparing kernel as in ue5m3_gemm (the operands must have windows)
         if (!native_eligible(g)) return UE5M3_ERR_UNSUPPORTED;
         int* ws = native_workspace(native_layout(g).bytes, (cudaStream_t)stream);
         if (!ws) return UE5M3_ERR_CUDA;

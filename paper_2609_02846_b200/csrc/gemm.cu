@@ -473,7 +473,7 @@ bool make_scale_map(CUtensorMap* m, const uint8_t* scales, int mode, int64_t R, 
 
 }  // namespace
 
-int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t st) {
+int launch_gemm(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st) {
     // CTA pairs that can be resident at once, per device; asked once per device, concurrent first calls serialised
     static int resident_pairs[64];
     static std::once_flag asked[64];
@@ -521,9 +521,9 @@ int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t s
     p.a_scales = g.a_scales; p.b_scales = g.b_scales;
     p.a_direct = a_direct ? 1 : 0; p.b_direct = b_direct ? 1 : 0;
     p.flags = nullptr; p.n_flags = 0;
-    if (range) {
+    if (workspace) {
         const NativeLayout l = native_layout(g);
-        p.flags = reinterpret_cast<const uint8_t*>(range) + l.flags;
+        p.flags = reinterpret_cast<const uint8_t*>(workspace) + l.flags;
         p.n_flags = l.n_flags;
     }
     const int num_tiles = p.tiles_m * p.tiles_n;
@@ -539,7 +539,7 @@ int launch_gemm(const GemmArgs& g, const int* range, int num_sms, cudaStream_t s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = range ? 1 : 0;
+    cfg.numAttrs = workspace ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, gemm_kernel, ma, mb, mas, mbs, mo, p) == cudaSuccess ? UE5M3_OK : UE5M3_ERR_CUDA;
 }
 

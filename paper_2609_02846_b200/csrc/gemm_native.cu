@@ -339,7 +339,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // Everything above touched only this CTA pair's shared and tensor memory and may have run while the range kernel was
+    // Everything above touched only this CTA pair's shared and tensor memory and may have run while the preparing kernel was
     // still at work (programmatic dependent launch); the workspace it fills is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // the FP16 kernel queued behind this one may be launched from here on: it reads the same word and returns
@@ -747,7 +747,7 @@ int launch_gemm_native(const GemmArgs& g, int* workspace, int num_sms, cudaStrea
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int pairs = num_tiles < resident_pairs[dev] ? num_tiles : resident_pairs[dev];
     // Programmatic dependent launch: the kernel's prologue (barriers, tensor-memory allocation, cluster barrier) runs
-    // beside the range kernel, which releases its dependents at once; the kernel waits for it before reading the workspace.
+    // beside the preparing kernel, which releases its dependents at once; the kernel waits for it before reading the workspace.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
