@@ -326,7 +326,7 @@ GEMM_FLOPS = 2 * M_TOK * K_IN * N_OUT
 # one ncu pass each; summaries in profiles/gemm_kernel_M9472_K4096_N1024_ncu_full.txt and
 # profiles/gemm_native_kernel_linear_M8192_K4096_N16384_ncu_full.txt).  Algorithmic bytes: 238 MB per launch.
 GEMM_DRAM_TRAFFIC_BYTES = {"gemm_kernel": (150.3e6 + 220.9e6 + 195.0e6 + 48.0e6 + 100.7e6 + 99.1e6) / 3,
-                           "gemm_native_kernel": (167.6e6 + 224.4e6 + 220.4e6 + 51.6e6 + 100.1e6 + 101.5e6) / 3}
+                           "gemm_native_kernel": (167.7e6 + 221.7e6 + 219.4e6 + 51.6e6 + 100.3e6 + 101.6e6) / 3}
 NOMINAL_FP4_OVER_BF16 = 4.0      # dense tensor peaks of the part: 9 PFLOP/s FP4, 2.25 PFLOP/s BF16
 
 
