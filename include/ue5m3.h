@@ -174,7 +174,8 @@ UE5M3_API int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_
  * dW = dY^T X; Section 6.1: y = sum_k a_k b_k on the decoded operands, the tensor-scale product
  * applied after accumulation):
  *     C[Mo, No] = (d_A * d_B) * sum_k (s_hat q)_A[m, k] * (s_hat q)_B[n, k]
- * Both operands are K-major.  The call picks one of two kernels on the device, without a host round trip:
+ * Both operands are K-major.  Two kernels share the work, decided on the device for every 256 x 256 tile of the output,
+ * without a host round trip:
  *   native   the tensor core's own block-scaled FP4 instruction (E2M1 operands, one 8-bit scale per 16 elements).  Its
  *            scale format is UE4M3 (bias 7); a normal UE5M3 code c and the UE4M3 code c - 8k denote values that differ
  *            by the constant factor 2^(k-8).  A scale row (the block scales of one operand row along the contraction;
@@ -182,13 +183,14 @@ UE5M3_API int ue5m3_quantize_dual(const void* x, int dtype, int64_t rows, int64_
  *            block scale of the row < 2^14.8) is therefore a native row on shifted codes, and output (m, n) takes the two
  *            exact factors 2^(k_m - 8) 2^(k_n - 8) together with d_A * d_B.  k is chosen per row.  Needs Kc % 256 == 0.
  *   FP16     every E2M1 x UE5M3 product (times 2^-4) is exact in FP16, subnormals included; the operands are
- *            reconstructed in the kernel and multiplied as FP16.  Used when some scale row has no window (UE5M3
- *            subnormal codes 1..7 included) or Kc = 128 * odd.
+ *            reconstructed in the kernel and multiplied as FP16.  Used for the tiles in which some scale row (of the
+ *            tile's 256 rows of A or 256 rows of B) has no window (UE5M3 subnormal codes 1..7 included), and for Kc = 128 * odd.
  * Both accumulate in FP32 on the tensor cores and meet the same error bound; their results may differ in the last bits.
  * Three launches per call when Kc % 256 == 0: a pass over the scale bytes that writes every row's k and the shifted codes in
  * the order the tensor core reads them (one byte per block, i.e. (Mo + No) * Kc / 16 bytes with Mo and No rounded up to 256,
  * into a workspace the library keeps per device and stream and grows with cudaMalloc when a call needs more: make the first
- * call of a shape on a stream outside any stream capture), then both kernels, one of which returns at once.
+ * call of a shape on a stream outside any stream capture), then both kernels; normally every tile is a native one and the
+ * FP16 kernel returns at once.
  * `op` only names the role of the call:
  *     FPROP  A = X  (1D_ROW),        B = W   (2D payload, scales)          Mo = tokens, No = out, Kc = in
  *     DGRAD  A = dY (1D_ROW, SR),    B = W^T (2D payload_t, scales_t)      Mo = tokens, No = in,  Kc = out
@@ -235,8 +237,9 @@ UE5M3_API int ue5m3_gemm_static(int op, int64_t Mo, int64_t No, int64_t Kc,
  * (UE5M3_ERR_UNSUPPORTED).  `workspace`: device, ue5m3_gemm_native_workspace_bytes(...) bytes, 16-byte aligned, owned by
  * the caller (0 is returned for a Kc that is not a multiple of 256).  After the call its first int32 is 0 when every scale
  * row had a window, and then bytes 16.. hold k for every scale row of A (padded to a multiple of 16) followed by every scale
- * row of B (the rest is the kernel's copy of the shifted scales); otherwise the first int32 is non-zero, the kernel has
- * returned at once and `out` is left untouched.
+ * row of B (the rest is the kernel's copy of the shifted scales); otherwise the first int32 is non-zero and the kernel has
+ * left untouched every 256 x 256 tile of `out` (tile (i, j): rows 256 i .., columns 256 j ..) that has a scale row without
+ * a window among its rows of A or B, and computed the others.
  * The paper has no counterpart of the split: its Section 5.3 names the three products, not how a device computes them.
  */
 UE5M3_API int ue5m3_gemm_fp16(int op, int64_t Mo, int64_t No, int64_t Kc,

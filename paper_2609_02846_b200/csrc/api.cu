@@ -212,8 +212,8 @@ int ue5m3_gemm(int op, int64_t Mo, int64_t No, int64_t Kc, const uint8_t* a_payl
     GemmArgs g{Mo, No, Kc, a_payload, a_scales, a_scale_mode, a_decode, b_payload, b_scales, b_scale_mode, b_decode,
                out, out_dtype, ldo};
     if (!native_eligible(g)) return launch_gemm(g, nullptr, di.sms, (cudaStream_t)stream);
-    // Three launches, one of which does the product: the windows of the scale rows, the native FP4 kernel (works when
-    // every scale row of both operands has a UE4M3 window) and the FP16 kernel (works when one does not).
+    // Three launches: the windows of the scale rows and the re-ordered scales, the native FP4 kernel (the tiles all of
+    // whose scale rows have a UE4M3 window: normally all) and the FP16 kernel (the other tiles: normally none).
     int* ws = native_workspace(native_layout(g).bytes, (cudaStream_t)stream);
     if (!ws) return UE5M3_ERR_CUDA;
     int r = launch_scale_prepare(g, ws, di.sms, (cudaStream_t)stream);

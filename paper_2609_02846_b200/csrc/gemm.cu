@@ -126,6 +126,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if (native_works) return;
     }
+    // Behind the native kernel this one computes the tiles that have a scale row without a window; alone, every tile.
+    // Every role walks this CTA pair's tiles with the same function.
+    auto next_mine = [&](int tile) {
+        if (p.flags) {
+            for (; tile < p.tiles_m * p.tiles_n; tile += (int)(gridDim.x >> 1)) {
+                int tm, tn;
+                tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+                if (!tile_is_native(p.flags, 2 * p.tiles_m, tm, tn)) break;
+            }
+        }
+        return tile;
+    };
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;      // same offset in both CTAs of the pair
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -177,7 +189,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint32_t tx_bytes = PK_A_BYTES + PK_B_BYTES + (p.a_direct ? 0 : a_rows_per_load * 16) +
                                       (p.b_direct ? 0 : b_rows_per_load * 16);
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok && !p.stall_producer; tile += num_pairs) {
+            for (int tile = next_mine(pair); tile < num_tiles && ok && !p.stall_producer; tile = next_mine(tile + num_pairs)) {
                 int tm, tn;
                 tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
                 const int mb = tm * 2 + (int)rank;                       // 128-row block of A
@@ -222,7 +234,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint64_t bd0 = umma_smem_desc(bf_base);
             const uint32_t bd_lo0 = (uint32_t)bd0, bd_hi = (uint32_t)(bd0 >> 32);
             uint32_t s = 0, ph = 0;                          // FP16 stage of the next slice and its phase
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
+            for (int tile = next_mine(pair); tile < num_tiles && ok; tile = next_mine(tile + num_pairs), ++tl) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit));   // epilogues have read tile tl-1
                 if (!ok) break;
                 tc_fence_after();
@@ -264,7 +276,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint8_t* stage_gen = smem_gen + SMEM_EPI + q * EPI_WARP_BYTES;
         uint32_t tl = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
+        for (int tile = next_mine(pair); tile < num_tiles && ok; tile = next_mine(tile + num_pairs), ++tl) {
             int tm, nb;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, nb);
             const int mb = tm * 2 + (int)rank;
@@ -366,8 +378,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // (the copy fills what is out of bounds with zeros); their scale codes are forced to zero as well
         const bool last_is_partial = (p.Kc % KCHUNK) != 0 && grp * KSUB >= (int)(p.Kc % KCHUNK);
         uint32_t a_next = 0, b_next = 0;
-        if (any_direct && pair < num_tiles) prefetch(pair, 0, a_next, b_next);
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        if (any_direct && next_mine(pair) < num_tiles) prefetch(next_mine(pair), 0, a_next, b_next);
+        for (int tile = next_mine(pair); tile < num_tiles && ok; tile = next_mine(tile + num_pairs)) {
             for (int kc = 0; kc < kchunks && ok; ++kc, ++it_pk) {
                 const uint32_t ps = it_pk % PK_STAGES, pph = (it_pk / PK_STAGES) & 1;
                 if (!mbar_wait(pk_full + 8 * ps, pph, abort_flag, p.wait_limit)) { ok = false; break; }
@@ -384,7 +396,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (any_direct) {
                     // the codes of the next packed stage, in flight under this stage's arithmetic
                     const int nkc = (kc + 1 < kchunks) ? kc + 1 : 0;
-                    const int ntile = (kc + 1 < kchunks) ? tile : tile + num_pairs;
+                    const int ntile = (kc + 1 < kchunks) ? tile : next_mine(tile + num_pairs);
                     if (ntile < num_tiles) prefetch(ntile, nkc, a_next, b_next);
                 }
                 // The packed bytes are in registers: hand the stage back to the producer now, so that the next

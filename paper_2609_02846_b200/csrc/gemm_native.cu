@@ -17,7 +17,8 @@
 // reduces every scale row's codes to the largest and the smallest non-zero one, writes the row's k (one byte) into the
 // workspace, says in the group's flag byte whether a row has no window (subnormal UE5M3 codes included), and
 // writes the group's codes, shifted, in the order the tensor core's scale copy reads them.  gemm_native_kernel reads
-// the flags and returns at once when one is set; the caller then runs the FP16 path, whose kernel evaluates the same
+// the flags and computes the 256 x 256 tiles none of whose four row groups is flagged -- normally all of them --; the
+// caller then runs the FP16 path, whose kernel computes the other tiles: it evaluates the same
 // predicate the other way round.  A code of 0 (rows beyond the operand) stays 0.  Where a row allows it k is 2, so
 // that the rows of ordinary data share one shift and the epilogue takes its uniform path.
 //
@@ -316,8 +317,6 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int kchunks = (int)(p.Kc / KCHUNK);
-    const int my_tiles = pair < num_tiles ? (num_tiles - pair + num_pairs - 1) / num_pairs : 0;
-    const uint32_t total = (uint32_t)my_tiles * (uint32_t)kchunks;       // stages this CTA pair works through
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -344,16 +343,27 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // the FP16 kernel queued behind this one may be launched from here on: it reads the same word and returns
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const bool work = native_all_rows_have_windows(p.flags, p.n_flags);      // uniform over the grid; false: the FP16 kernel does this product
-    if (blockIdx.x == 0 && threadIdx.x == 0) *p.result = work ? 0 : 1;
+    const bool all_native = native_all_rows_have_windows(p.flags, p.n_flags);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *p.result = all_native ? 0 : 1;
+    // This kernel computes the tiles all of whose scale rows have windows; the FP16 kernel computes the others.  Every
+    // role walks this CTA pair's tiles with the same two functions.
+    auto mine = [&](int tile) {
+        int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        return tile_is_native(p.flags, 2 * p.tiles_m, tm, tn);
+    };
+    auto next_mine = [&](int tile) {
+        if (!all_native)
+            while (tile < num_tiles && !mine(tile)) tile += num_pairs;
+        return tile;
+    };
 
-    if (!work) {
-    } else if (warp == 0) {
+    if (warp == 0) {
         // ------------------------------------------------------------------ copies
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok && !p.stall_producer; tile += num_pairs) {
+            for (int tile = next_mine(pair); tile < num_tiles && ok && !p.stall_producer; tile = next_mine(tile + num_pairs)) {
                 int tm, tn;
                 tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
                 const int mb = tm * 2 + (int)rank, nh = tn * 2 + (int)rank;
@@ -378,6 +388,8 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     } else if (warp == 2) {
         // ------------------------------------------------------------------ relay: this CTA's stage has landed
         if (lane == 0) {
+            uint32_t total = 0;                          // stages this CTA pair works through
+            for (int tile = next_mine(pair); tile < num_tiles; tile = next_mine(tile + num_pairs)) total += (uint32_t)kchunks;
             for (uint32_t it = 0; it < total; ++it) {
                 const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                 if (!mbar_wait(pk_full + 8 * s, ph, abort_flag, p.wait_limit)) break;
@@ -401,7 +413,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             const uint32_t sf_lo0 = (uint32_t)d_sf, sf_hi = (uint32_t)(d_sf >> 32);
             const uint32_t tm0 = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
             uint32_t s = 0, ph = 0, u = 0;                // stage and its phase, scale slot
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
+            for (int tile = next_mine(pair); tile < num_tiles && ok; tile = next_mine(tile + num_pairs), ++tl) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty, (tl & 1) ^ 1, abort_flag, p.wait_limit));
                 if (!ok) break;
                 tc_fence_after();
@@ -451,7 +463,7 @@ gemm_native_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         uint8_t* stage_gen = smem_gen + SMEM_EPI + q * EPI_WARP_BYTES;
         uint32_t tl = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tl) {
+        for (int tile = next_mine(pair); tile < num_tiles && ok; tile = next_mine(tile + num_pairs), ++tl) {
             int tm, nb;
             tile_coords(tile, p.tiles_m, p.tiles_n, tm, nb);
             const int mb = tm * 2 + (int)rank;

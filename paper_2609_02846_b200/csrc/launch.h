@@ -55,13 +55,13 @@ cudaError_t launch_quantize_dual(const QuantArgs& a, int dtype, int rounding, bo
 cudaError_t launch_amax(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* out, int num_sms,
                         cudaStream_t st);
 cudaError_t launch_unswizzle(const uint8_t* in, uint8_t* out, int64_t R, int64_t kblocks, cudaStream_t st);
-// returns a UE5M3_* status; `workspace` (may be null) is the workspace of the native path: the kernel then does nothing
-// when every scale row has a UE4M3 window, because gemm_native_kernel has done the product
+// returns a UE5M3_* status; `workspace` (may be null) is the workspace of the native path: the kernel then computes only
+// the tiles that have a scale row without a UE4M3 window, because gemm_native_kernel does the others
 int launch_gemm(const GemmArgs& g, const int* workspace, int num_sms, cudaStream_t st);
 int read_and_clear_device_status();                                  // synchronises the device
 // The same product on the tensor core's FP4 path (gemm_native.cu).  `workspace` is device memory of
-// native_layout(g).bytes bytes (layout in window.cuh): launch_scale_prepare fills it, the native kernel reads it and does
-// nothing when some scale row has no window, and the FP16 kernel (launch_gemm with the same workspace) then does the product.
+// native_layout(g).bytes bytes (layout in window.cuh): launch_scale_prepare fills it, the native kernel reads it and skips
+// the tiles in which some scale row has no window, and the FP16 kernel (launch_gemm with the same workspace) does those.
 inline int64_t native_scale_rows(int64_t R, int mode) { return mode == 2 /* UE5M3_SCALE_2D */ ? R / 16 : R; }
 struct NativeLayout {
     size_t k_a, k_b;              // byte offsets of the rows' shifts

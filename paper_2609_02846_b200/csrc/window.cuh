@@ -40,4 +40,13 @@ __device__ __forceinline__ bool native_all_rows_have_windows(const uint8_t* grou
     return __syncthreads_or(bad) == 0;
 }
 
+// Tile (tm, tn) of the output covers the 128-row groups 2 tm, 2 tm + 1 of A and 2 tn, 2 tn + 1 of B (A's groups come first
+// in the flags, `groups_a` of them).  The native kernel computes the tiles for which this is true, the FP16 kernel the
+// others; both walk the same tile sequence, so together they write every tile exactly once.
+__device__ __forceinline__ bool tile_is_native(const uint8_t* group_flags, int groups_a, int tm, int tn) {
+    const uint8_t* fa = group_flags + 2 * tm;
+    const uint8_t* fb = group_flags + groups_a + 2 * tn;
+    return (fa[0] | fa[1] | fb[0] | fb[1]) == 0;
+}
+
 }  // namespace ue5m3

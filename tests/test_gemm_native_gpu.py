@@ -348,3 +348,36 @@ def test_gemm_replays_from_a_cuda_graph():
             assert lib.last_device_status() == 0
             y, sabs = oracle.gemm(ap, asc2, False, 0.5, bp, bsc, True, 0.25)
             check_gemm_output(out, y, sabs)
+
+
+@pytest.mark.parametrize("modes", [(0, 0), (1, 2)])
+def test_tiles_with_a_row_without_a_window_go_to_the_fp16_kernel_and_the_others_stay_native(modes):
+    """3 x 2 tiles of 256 x 256.  One scale row of A in tile row 1 holds a UE5M3 subnormal code, one of B in tile column 1
+    spans more than a window: ue5m3_gemm_native computes tiles (0, 0) and (2, 0) and leaves the rest alone, ue5m3_gemm
+    computes those two on the native kernel (bit for bit the same) and the other four on the FP16 kernel (bit for bit what
+    ue5m3_gemm_fp16 gives), and the whole output meets the bound against the oracle."""
+    Mo, No, Kc = 768, 512, 512
+    rng = np.random.default_rng(31 + modes[0])
+    sa = rng.integers(0x50, 0x90, (Mo, Kc // 16), dtype=np.uint8)
+    sb = rng.integers(0x50, 0x90, (No // 16 if modes[1] == 2 else No, Kc // 16), dtype=np.uint8)
+    sa[300, 3] = 0x05                                  # subnormal: row 300 of A (tile row 1) has no window
+    rb = 400 // 16 if modes[1] == 2 else 400
+    sb[rb, 0], sb[rb, 1] = 0x10, 0xE0                  # row 400 of B (tile column 1): 209 codes apart
+    qa, ap, asc = _operand(rng, Mo, Kc, modes[0], 0, 0, dec=0.5, scales=sa)
+    qb, bp, bsc = _operand(rng, No, Kc, modes[1], 0, 0, dec=0.125, scales=sb)
+    nat, ok, ka, kb = _native(qa, qb, torch.float32, Mo, No)
+    assert not ok
+    native_tile = np.zeros((Mo, No), bool)
+    native_tile[0:256, 0:256] = True
+    native_tile[512:768, 0:256] = True
+    mask = torch.from_numpy(native_tile).to(DEV)
+    assert bool(torch.isnan(nat[~mask]).all()) and bool(torch.isfinite(nat[mask]).all())
+    got = lib.gemm(lib.FPROP, qa, qb, torch.float32)
+    f16 = lib.gemm_fp16(lib.FPROP, qa, qb, torch.float32)
+    torch.cuda.synchronize()
+    assert lib.last_device_status() == 0
+    assert torch.equal(got[mask], nat[mask]) and torch.equal(got[~mask], f16[~mask])
+    y, sabs = oracle.gemm(ap, asc, False, 0.5, bp, bsc, modes[1] == 2, 0.125)
+    check_gemm_output(got, y, sabs)
+    # the same through the no-allocation entry point
+    assert torch.equal(lib.gemm_static(lib.FPROP, qa, qb, torch.float32), got)
