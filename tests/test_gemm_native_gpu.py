@@ -381,3 +381,40 @@ def test_tiles_with_a_row_without_a_window_go_to_the_fp16_kernel_and_the_others_
     check_gemm_output(got, y, sabs)
     # the same through the no-allocation entry point
     assert torch.equal(lib.gemm_static(lib.FPROP, qa, qb, torch.float32), got)
+
+
+def test_mixed_dispatch_seeded_sweep():
+    """Random shapes, scale layouts and output types with a few rows without a window sprinkled over A and B (none, one
+    operand, both; subnormal codes or a too wide span): every output of ue5m3_gemm meets the bound against the oracle,
+    whichever kernel computed its tile, and more tiles than CTA pairs are covered by the largest case."""
+    rng = np.random.default_rng(20261125)
+    for case in range(14):
+        Mo = 128 * int(rng.integers(1, 9)) if case else 128 * 40
+        No = 128 * int(rng.integers(1, 7)) if case else 128 * 34
+        Kc = 256 * int(rng.integers(1, 4)) if case else 256
+        ma, mb = int(rng.integers(0, 3)), int(rng.integers(0, 3))
+        dtype = torch.float32 if case % 2 else torch.bfloat16
+        sa = rng.integers(0x48, 0x98, (Mo // 16 if ma == 2 else Mo, Kc // 16), dtype=np.uint8)
+        sb = rng.integers(0x48, 0x98, (No // 16 if mb == 2 else No, Kc // 16), dtype=np.uint8)
+        for s_, n_bad in ((sa, int(rng.integers(0, 4))), (sb, int(rng.integers(0, 3)))):
+            for r in rng.integers(0, s_.shape[0], n_bad):
+                if rng.integers(0, 2):
+                    s_[r, rng.integers(0, s_.shape[1])] = rng.integers(1, 8)          # subnormal code
+                else:
+                    s_[r, 0], s_[r, -1] = 0x09, 0xF0                                  # too wide for any window
+        qa, ap, asc = _operand(rng, Mo, Kc, ma, 0, 0, dec=0.75, scales=sa)
+        qb, bp, bsc = _operand(rng, No, Kc, mb, 0, 0, dec=2.0 ** -9, scales=sb)
+        out = torch.full((Mo, No), float("nan"), dtype=dtype, device=DEV)
+        lib.gemm(lib.FPROP, qa, qb, out=out)
+        torch.cuda.synchronize()
+        assert lib.last_device_status() == 0, case
+        if case == 0:                                   # 20 x 17 = 340 tiles: sampled cells plus one full row and column
+            ci = np.concatenate([rng.integers(0, Mo, 4000), np.full(No, 300), np.arange(Mo)])
+            cj = np.concatenate([rng.integers(0, No, 4000), np.arange(No), np.full(Mo, 700)])
+            y, sabs = oracle.gemm_cells(ap, asc, ma == 2, 0.75, bp, bsc, mb == 2, np.float32(2.0 ** -9), ci, cj)
+            got = out.float().cpu().numpy().astype(np.float64)[ci, cj]
+            tol = 1e-5 * sabs + 1e-30 + np.abs(y) * 2.0 ** -8             # BF16 output: one ulp
+            assert np.all(np.abs(got - y) <= tol), case
+        else:
+            y, sabs = oracle.gemm(ap, asc, ma == 2, 0.75, bp, bsc, mb == 2, np.float32(2.0 ** -9))
+            check_gemm_output(out, y, sabs)
