@@ -185,6 +185,26 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // Rows beyond the operand get zeros.  Source layouts: one row after the other (1D), 16-byte pieces of 128 rows
 // interleaved (1D tiled: piece p of row r at (r / 128 * pieces + p) * 2048 + r % 128 * 16), one row per 16 operand
 // rows (2D).
+// Bytes in pairs of 16-bit lanes (the per-byte SIMD intrinsics are emulated on this architecture, a dozen
+// instructions each; max.u16x2 / min.u16x2 are single instructions).
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("min.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+// two codes in the low bytes of the 16-bit lanes -> the same with 256 in the lanes whose code is 0
+__device__ __forceinline__ uint32_t zero_to_256(uint32_t x) { return x | (((x + 0x00FF00FFu) & 0x01000100u) ^ 0x01000100u); }
+// d subtracted from every non-zero byte of v (every non-zero byte is at least d: no borrow crosses a byte)
+__device__ __forceinline__ uint32_t shift_codes(uint32_t v, uint32_t d) {
+    const uint32_t nz = ((((v & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | v) >> 7) & 0x01010101u;
+    return v - (d & (nz * 0xFFu));
+}
+
 struct PrepareParams {
     const uint8_t* src[2];
     int64_t rows[2];              // operand rows (Mo, No)
@@ -227,34 +247,42 @@ __global__ void __launch_bounds__(512) scale_prepare_kernel(const PrepareParams 
     const int i = warp * 8 + (lane >> 2);
     const int64_t srow = s0 + i;
     const bool have_row = i < nrows && srow < srows;
-    uint32_t m = 0u, iv = 0u;
+    uint32_t m = 0u, iv = 0xFFFFFFFFu;                                   // largest code, smallest non-zero code: two 16-bit lanes each
+    // this thread's pieces of a chunk are 4 pieces apart: a constant stride in global memory (64 bytes, or 4 x 2048 in the
+    // tiled layout) and 16 words in shared memory
+    const int64_t piece_stride = tiled ? 2048 : 16;
     auto load_chunk = [&](int c, bool keep, bool reduce) {
         const int first = c * chunk_pieces, n = min(chunk_pieces, pieces - first);
         if (!have_row) return;
-        uint32_t* mine = rows_smem + i * pitch;
-        for (int pc0 = lane & 3; pc0 < n; pc0 += 32) {                   // eight loads in flight per thread
+        const uint8_t* src_p = piece_ptr(srow, first + (lane & 3));
+        uint32_t* dst = rows_smem + i * pitch + 4 * (lane & 3);
+        for (int pc0 = lane & 3; pc0 < n; pc0 += 32, src_p += 32 * piece_stride, dst += 128) {      // eight loads in flight per thread
             uint4 v[8];
 #pragma unroll
             for (int t = 0; t < 8; ++t)
-                v[t] = pc0 + 4 * t < n ? __ldg(reinterpret_cast<const uint4*>(piece_ptr(srow, first + pc0 + 4 * t))) : make_uint4(0u, 0u, 0u, 0u);
+                v[t] = pc0 + 4 * t < n ? __ldg(reinterpret_cast<const uint4*>(src_p + 4 * t * piece_stride)) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
-                const int pc = pc0 + 4 * t;
                 const uint32_t w[4] = {v[t].x, v[t].y, v[t].z, v[t].w};
+                if (reduce) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (reduce) {
-                        m = __vmaxu4(m, w[j]);
-                        iv = __vmaxu4(iv, ~w[j] & ~__vcmpeq4(w[j], 0u));  // 255 - c, and 0 for c = 0
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t e = w[j] & 0x00FF00FFu, o = (w[j] >> 8) & 0x00FF00FFu;
+                        m = max_u16x2(max_u16x2(m, e), o);
+                        iv = min_u16x2(min_u16x2(iv, zero_to_256(e)), zero_to_256(o));     // smallest non-zero code (256: none)
                     }
-                    if (keep && pc < n) mine[4 * pc + j] = w[j];
+                }
+                if (keep && pc0 + 4 * t < n) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dst[16 * t + j] = w[j];
                 }
             }
         }
     };
     for (int c = 0; c < nchunks; ++c) load_chunk(c, nchunks == 1, true);
-    m = max(max(m & 0xFFu, (m >> 8) & 0xFFu), max((m >> 16) & 0xFFu, m >> 24));
-    iv = max(max(iv & 0xFFu, (iv >> 8) & 0xFFu), max((iv >> 16) & 0xFFu, iv >> 24));
+    m = max(m & 0xFFFFu, m >> 16);
+    iv = min(iv & 0xFFFFu, iv >> 16);
+    iv = iv >= 256u ? 0u : 255u - iv;                                    // 255 - the smallest non-zero code, 0 when there is none
 #pragma unroll
     for (int d = 1; d <= 2; d <<= 1) {
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
@@ -279,20 +307,28 @@ __global__ void __launch_bounds__(512) scale_prepare_kernel(const PrepareParams 
             load_chunk(c, true, false);
             __syncthreads();
         }
-        for (int u = threadIdx.x; u < n * 128; u += blockDim.x) {
-            const int dp = u & 31, j = (u >> 5) & 3, sl = u >> 7;
+        // 512 threads: a thread keeps its lane dp and MMA j and walks the stages four at a time, so its four rows, their
+        // shifts and its position inside a stage are fixed
+        const int dp = threadIdx.x & 31, j = (threadIdx.x >> 5) & 3;
+        uint32_t sh[4];
+        int idx[4];
+        bool have[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int row = 32 * g + dp, ri = two_d ? row >> 4 : row;
+            have[g] = r0 + row < R;
+            sh[g] = shift8[ri];
+            idx[g] = ri * pitch + j;
+        }
+        uint8_t* dst = out + (int64_t)(first + (threadIdx.x >> 7)) * stride_s + j * stride_j + dp * 16;
+        for (int sl = threadIdx.x >> 7; sl < n; sl += 4, dst += 4 * stride_s) {
             uint32_t w[4];
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
-                const int row = 32 * g + dp;
-                w[g] = 0u;
-                if (r0 + row < R) {
-                    const int ri = two_d ? row >> 4 : row;
-                    const uint32_t v = rows_smem[ri * pitch + 4 * sl + j];
-                    w[g] = __vsub4(v, shift8[ri]) & ~__vcmpeq4(v, 0u);    // a code of 0 stays 0
-                }
+                const uint32_t v = have[g] ? rows_smem[idx[g] + 4 * sl] : 0u;
+                w[g] = shift_codes(v, sh[g]);                             // a code of 0 stays 0
             }
-            *reinterpret_cast<uint4*>(out + (int64_t)(first + sl) * stride_s + j * stride_j + dp * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
         }
     }
 }
