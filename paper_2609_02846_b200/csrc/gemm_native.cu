@@ -185,6 +185,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // Rows beyond the operand get zeros.  Source layouts: one row after the other (1D), 16-byte pieces of 128 rows
 // interleaved (1D tiled: piece p of row r at (r / 128 * pieces + p) * 2048 + r % 128 * 16), one row per 16 operand
 // rows (2D).
+// 16 bytes through the read-only path; volatile, so that a batch of them is issued before the first is used
+__device__ __forceinline__ uint4 ldg_nc_16(const uint8_t* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
 // Bytes in pairs of 16-bit lanes (the per-byte SIMD intrinsics are emulated on this architecture, a dozen
 // instructions each; max.u16x2 / min.u16x2 are single instructions).
 __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
@@ -260,7 +266,7 @@ __global__ void __launch_bounds__(512) scale_prepare_kernel(const PrepareParams 
             uint4 v[8];
 #pragma unroll
             for (int t = 0; t < 8; ++t)
-                v[t] = pc0 + 4 * t < n ? __ldg(reinterpret_cast<const uint4*>(src_p + 4 * t * piece_stride)) : make_uint4(0u, 0u, 0u, 0u);
+                v[t] = ldg_nc_16(src_p + (pc0 + 4 * t < n ? 4 * t * piece_stride : 0));    // beyond the chunk: the first piece again (harmless for the extremes, not stored)
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
                 const uint32_t w[4] = {v[t].x, v[t].y, v[t].z, v[t].w};
