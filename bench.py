@@ -553,6 +553,14 @@ def run_ours(args):
         sweep = None
         if world == 1 and not args.no_sweep:
             sweep = quantizer_sweep_cells(dev, peaks)
+        # A region of a few hundred milliseconds holds a handful of samples, and the power-cap flag is not up in every one
+        # of them while the clock is already down; the sustained leg that follows runs the same steps for two seconds.
+        if (clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] < 0.97 * clocks["sm_max_mhz"]
+                and not clocks.get("reasons") and sustained and sustained["clocks"].get("reasons")):
+            clocks["note"] = ("median clock below the maximum with no reason flagged in this region's %d samples; the sustained leg "
+                              "after it (the same steps for %.1f s) records %s at up to %.0f W" % (
+                                  clocks.get("samples", 0), sustained["seconds"], "+".join(sustained["clocks"]["reasons"]),
+                                  sustained["clocks"].get("power_w_max") or 0.0))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
